@@ -1,0 +1,204 @@
+/*
+ * rwkvq -- hybrid scalar/vector-quantized RWKV projection products on NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library.  Every entry point returns a status code; nothing aborts,
+ * throws or traps.  Pointers named *_host are host memory, pointers named *_dev
+ * are device memory owned by the caller (the library never allocates device
+ * memory in any call declared here unless the comment says so).  `stream` is a
+ * cudaStream_t passed as void* (NULL = the legacy default stream).  Kernels are
+ * asynchronous on `stream`; argument errors are detected on the host before any
+ * launch.
+ *
+ * Method references are to RWKVQuant (arXiv 2505.03803): scalar quantization
+ * Section 3.2 Eq. 2, vector quantization Section 3.2 Eq. 3, coarse-to-fine proxy
+ * Section 4.1 Eqs. 5-18, element-wise (token-shift) weights Section 4.2 and
+ * Appendix A.1 Eqs. 20-26.
+ */
+#ifndef RWKVQ_H_
+#define RWKVQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RWKVQ_OK = 0,
+  RWKVQ_EINVAL = 1,       /* NULL pointer, bad enum, bad size */
+  RWKVQ_ESHAPE = 2,       /* shape not supported by the format (see rwkvq_pack) */
+  RWKVQ_EALIGN = 3,       /* a device pointer is not 16-byte aligned */
+  RWKVQ_ENONFINITE = 4,   /* NaN/Inf in the weights */
+  RWKVQ_ENOMEM = 5,       /* host allocation failed, or caller buffer / workspace too small */
+  RWKVQ_ECUDA = 6,        /* a CUDA runtime call failed (see rwkvq_last_cuda_error) */
+  RWKVQ_EUNSUPPORTED = 7, /* valid request this build does not implement */
+  RWKVQ_ETIMEOUT = 8      /* a bounded device-side wait expired (reported by rwkvq_device_status) */
+} rwkvq_status;
+
+/* phi_m of Section 4.1 Eq. 18: 1 = scalar quantization, 0 = vector quantization. */
+typedef enum { RWKVQ_VQ = 0, RWKVQ_SQ = 1 } rwkvq_method;
+
+typedef enum { RWKVQ_F32 = 0, RWKVQ_F16 = 1, RWKVQ_BF16 = 2 } rwkvq_dtype;
+
+/*
+ * Logical (format-independent) codes of one matrix, host memory.
+ *  SQ (Eq. 2):  q[oc*ic] codes in [0, 2^bits-1] row-major; scale/zero: fp16 bit
+ *               patterns, [oc * ic/group], one pair per run of `group` consecutive
+ *               input-dim weights of one row.  Decode: w_hat = s * (q - z).
+ *  VQ (Eq. 3):  q[oc*ic/2] codebook indices row-major (vector = two consecutive
+ *               input-dim weights of one row); codebook: fp16 bit patterns
+ *               [oc/tile][ic/tile][2^bits][2], one codebook per tile x tile block.
+ *               Decode: w_hat[i][2p+e] = C_tile(i,p)[q[i][p]][e].
+ *  mu vectors (oc == 1, VQ): one codebook [2^bits][2], q[ic/2].
+ * Unused members are NULL.
+ */
+typedef struct {
+  uint8_t* q;
+  uint16_t* scale;
+  uint16_t* zero;
+  uint16_t* codebook;
+} rwkvq_codes;
+
+typedef struct {
+  int32_t method;       /* rwkvq_method */
+  int32_t bits;         /* SQ: code bits, 3.  VQ: index bits, 6 (64 entries) or 8 (256 entries) */
+  int32_t group;        /* SQ: 128 */
+  int32_t vec_dim;      /* VQ: 2 */
+  int32_t tile;         /* VQ: 256 (ignored for oc == 1) */
+  int32_t kmeans_iters; /* VQ: Lloyd iterations after k-means++ seeding, e.g. 10 */
+  uint64_t seed;        /* VQ: seed of the library's own generator */
+  const rwkvq_codes* codes_in; /* optional: pre-made logical codes; the quantizer is skipped
+                                  and the codes are packed as given (w_fp16_host may be NULL) */
+} rwkvq_quant_cfg;
+
+/* Host-side description of a packed matrix; travels with the device image. */
+typedef struct {
+  int32_t method, bits, oc, ic, group, vec_dim, tile, entries;
+  int32_t oc_pad, ic_pad;  /* rows padded to 128, columns to 256 inside the image */
+  uint64_t image_bytes;    /* size of the device image, multiple of 256 */
+  uint64_t stream_bytes;   /* bytes a product must read: codes + scales / indices + codebooks */
+} rwkvq_desc;
+
+typedef struct rwkvq_blob rwkvq_blob; /* host-owned packed matrix, opaque */
+
+/*
+ * Quantize (unless cfg->codes_in) and bit-pack one fp16 matrix W[oc][ic] (row-major, rows =
+ * output channels, host memory, fp16 bit patterns).  SQ follows Eq. 2 with s = (max-min)/(2^b-1)
+ * rounded to fp16, integer zero point z = round(-min/s) and round-to-nearest-even; VQ follows
+ * Eq. 3 with a k-means codebook per tile (Section 3.2).  Token-shift vectors (Section 4.2) are
+ * packed with oc = 1, method = RWKVQ_VQ.
+ * Shapes: SQ needs oc % 16 == 0 and ic % 128 == 0; VQ matrices need oc % 256 == 0 and
+ * ic % 256 == 0; vectors need ic % 2 == 0.  Errors: EINVAL, ESHAPE, ENONFINITE, ENOMEM.
+ * On success *out owns host memory until rwkvq_blob_free.
+ */
+rwkvq_status rwkvq_pack(const uint16_t* w_fp16_host, int oc, int ic, const rwkvq_quant_cfg* cfg,
+                        rwkvq_blob** out);
+rwkvq_status rwkvq_blob_desc(const rwkvq_blob* blob, rwkvq_desc* desc_out);
+/* Size of the device image in bytes (multiple of 256; 0 for NULL). */
+size_t rwkvq_blob_nbytes(const rwkvq_blob* blob);
+/* Copy the device image (header + bit-packed payload) into dst_host[n]; the caller then copies
+ * it to a 256-byte-aligned device buffer.  ENOMEM if n is too small. */
+rwkvq_status rwkvq_blob_image(const rwkvq_blob* blob, void* dst_host, size_t n);
+/* Copy the logical codes into caller-allocated arrays (sizes as in rwkvq_codes). */
+rwkvq_status rwkvq_blob_export_codes(const rwkvq_blob* blob, rwkvq_codes* dst_host);
+/* Unpack a host copy of a device image back into logical codes (inverse of the bit packing;
+ * checks magic, version, sizes and CRC).  desc_out may be NULL; dst arrays as in rwkvq_codes. */
+rwkvq_status rwkvq_image_unpack(const void* image_host, size_t n, rwkvq_desc* desc_out,
+                                rwkvq_codes* dst_host);
+void rwkvq_blob_free(rwkvq_blob* blob);
+
+/*
+ * Coarse-to-fine proxy (Section 4.1).  For each of n_mats fp16 matrices resident on the device
+ * computes P_c (Eq. 9) and P_f (Eq. 17, orders 2..K, 2 <= K <= 8) from the sorted-gap
+ * distribution of the flattened weights and applies Eq. 18:
+ * phi = 1 (SQ) iff P_c < tau_c and P_f < tau_f, else 0 (VQ).  A constant matrix yields
+ * P_c = P_f = +inf (VQ).  Pc_host/Pf_host/phi_host: host arrays of n_mats (written after the
+ * call synchronizes `stream`).  workspace_dev: at least rwkvq_proxy_workspace_bytes(n_mats) bytes,
+ * 16-byte aligned; its contents on entry are irrelevant.  Errors: EINVAL, EALIGN, ENOMEM,
+ * ENONFINITE (a NaN/Inf weight was seen), ECUDA.
+ */
+size_t rwkvq_proxy_workspace_bytes(int n_mats);
+rwkvq_status rwkvq_proxy_select(const void* const* w_fp16_dev, const int* oc, const int* ic,
+                                int n_mats, int K, double tau_c, double tau_f, double* Pc_host,
+                                double* Pf_host, int* phi_host, void* workspace_dev,
+                                size_t workspace_bytes, void* stream);
+
+/*
+ * Decode product y[b][i] = sum_j w_hat[i][j] * x_mix[b][j], 1 <= B <= 16 (Appendix A.1, the
+ * W.(...) products), with the token-shift mix x_mix = x + (x_prev - x) (.) mu_hat fused into the
+ * input stage when mu_image_dev != NULL (Eq. 20 with mu_paper = 1 - mu_hat).
+ *  W_desc/W_image_dev: packed matrix and its description.  mu_desc/mu_image_dev: packed vector of
+ *  length ic, or both NULL.  x_fp16_dev, xprev_fp16_dev: [B][ic] fp16 (xprev NULL iff mu NULL).
+ *  y_dev: [B][oc], y_dtype F32 or F16.  workspace_dev: rwkvq_gemv_workspace_bytes() bytes, must
+ *  be zero-filled once before its first use; every call leaves it zero-filled again, so calls
+ *  that share a workspace must not overlap on the device.
+ * Accumulation is fp32.  Errors: EINVAL, ESHAPE, EALIGN, ENOMEM, ECUDA.
+ */
+size_t rwkvq_gemv_workspace_bytes(const rwkvq_desc* W_desc, int B);
+rwkvq_status rwkvq_gemv(const rwkvq_desc* W_desc, const void* W_image_dev, const rwkvq_desc* mu_desc,
+                        const void* mu_image_dev, const void* x_fp16_dev, const void* xprev_fp16_dev,
+                        int B, void* y_dev, int y_dtype, void* workspace_dev, size_t workspace_bytes,
+                        void* stream);
+
+/* One product of a decode step (same meaning as the rwkvq_gemv arguments).  `stage` orders the
+ * step: every product of stage s is complete before any activation of stage s+1 is read. */
+typedef struct {
+  rwkvq_desc W_desc;
+  const void* W_image_dev;
+  rwkvq_desc mu_desc;         /* ignored when mu_image_dev == NULL */
+  const void* mu_image_dev;
+  const void* x_fp16_dev;
+  const void* xprev_fp16_dev;
+  void* y_dev;
+  int32_t stage;
+  int32_t y_dtype;
+} rwkvq_gemv_op;
+
+/*
+ * A whole decode step (all projections of all layers, Appendix A.1) as ONE persistent launch:
+ * packed weights are streamed through shared memory continuously across products and stages
+ * while a grid-wide barrier enforces the stage order.  rwkvq_step_plan builds the schedule on
+ * the host and copies it into plan_dev (rwkvq_step_plan_bytes() bytes, caller-owned); the plan
+ * embeds the pointers of `ops`, so the buffers must stay where they are.  rwkvq_step_run launches
+ * it.  ops must be sorted by stage (non-decreasing).  Errors as rwkvq_gemv plus ETIMEOUT through
+ * rwkvq_device_status.
+ */
+size_t rwkvq_step_plan_bytes(const rwkvq_gemv_op* ops, int n_ops, int B);
+rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* plan_dev,
+                             size_t plan_bytes, void* stream);
+rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream);
+
+/*
+ * Prefill product Y[t][i] = sum_j bf16(w_hat[i][j]) * x_mix[t][j] for M tokens, bf16 x bf16 ->
+ * fp32 on the tensor cores.  x_mix[t] = X[t] + (X[t-1] - X[t]) (.) mu_hat, with X[-1] = xprev0
+ * (zeros if NULL); mu NULL = no mix.  X_bf16_dev: [M][ic]; Y_dev: [M][oc] F32 or BF16.
+ * workspace_dev: rwkvq_prefill_workspace_bytes() bytes (holds x_mix when mu is given).
+ */
+size_t rwkvq_prefill_workspace_bytes(const rwkvq_desc* W_desc, int M, int has_mu);
+rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* W_desc, const void* W_image_dev,
+                                const rwkvq_desc* mu_desc, const void* mu_image_dev,
+                                const void* X_bf16_dev, const void* xprev0_bf16_dev, int M,
+                                void* Y_dev, int y_dtype, void* workspace_dev,
+                                size_t workspace_bytes, void* stream);
+
+/*
+ * Decode the packed matrix to out_dev[oc][ic]: F32 = the exact value s*(q-z) (two IEEE fp32
+ * operations: subtract, then multiply) or the fp16 codebook entry; BF16 = that value rounded to
+ * nearest even.  Uses the same device unpack routines as the products (test surface for
+ * "decoded weights are bit-exact").  For vectors (oc == 1) out_dev has ic elements.
+ */
+rwkvq_status rwkvq_dequant(const rwkvq_desc* W_desc, const void* W_image_dev, void* out_dev,
+                           int dtype, void* stream);
+
+/* Device status word of the last launches on this device: RWKVQ_OK, or ETIMEOUT if a bounded
+ * wait inside a kernel gave up.  Synchronizes `stream`; clears the word. */
+rwkvq_status rwkvq_device_status(void* stream);
+const char* rwkvq_status_str(rwkvq_status s);
+/* Text of the last CUDA error seen by this thread's library calls ("" if none). */
+const char* rwkvq_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RWKVQ_H_ */

@@ -1,0 +1,265 @@
+// Per-record building blocks of the decode products: input staging with the fused token-shift
+// mix (Appendix A.1 Eq. 20), and the record -> tensor-core step routines for both formats.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/rwkvq.h"
+#include "unpack.cuh"
+
+namespace rwkvq {
+
+enum { FMT_SQ3 = 0, FMT_VQ6 = 1, FMT_VQ8 = 2 };
+
+struct GemvArgs {
+  const uint8_t* payload;   // chunks
+  const uint8_t* aux;       // VQ codebooks
+  const uint8_t* mu;        // vector index stream, or nullptr
+  const uint8_t* mu_aux;    // vector codebook
+  const __half* x;
+  const __half* xprev;
+  void* y;
+  float* partial;
+  unsigned* counters;
+  int oc, ic, KT, S, nkt, entries, B, mu_bits, mu_entries, y_dtype;
+};
+
+struct SmemLayout {
+  uint32_t xstride;   // bytes between batch rows of the staged input
+  uint32_t gs_off;    // SQ: per-group sums  float[groups][3][16]
+  uint32_t cb_off;    // VQ: two lane-replicated codebooks
+  uint32_t mucb_off;  // token-shift codebook
+  uint32_t total;
+};
+
+// Staged input rows are nkt*256 fp16 values plus 32 bytes of padding, which makes the 8-byte
+// B-fragment loads of a half-warp (4 batch rows x 4 column quads) hit 16 distinct bank pairs.
+__host__ __device__ inline SmemLayout smem_layout_rt(int fmt, int nkt, int B, int mu_entries, int entries) {
+  SmemLayout L;
+  L.xstride = (uint32_t)nkt * 512u + 32u;
+  uint32_t off = (uint32_t)B * L.xstride;
+  L.gs_off = off;
+  if (fmt == FMT_SQ3) off += (uint32_t)nkt * 2u * 3u * 16u * 4u;
+  off = (off + 127u) & ~127u;
+  L.cb_off = off;
+  if (fmt != FMT_SQ3) off += 2u * (uint32_t)entries * 128u;
+  L.mucb_off = off;
+  off += (uint32_t)mu_entries * 4u;
+  L.total = (off + 15u) & ~15u;
+  return L;
+}
+template <int FMT>
+__host__ __device__ inline SmemLayout smem_layout(int nkt, int B, int mu_entries, int entries) {
+  return smem_layout_rt(FMT, nkt, B, mu_entries, entries);
+}
+
+__device__ __forceinline__ uint32_t vector_index(const uint8_t* stream, int p, int bits) {
+  const uint32_t bitpos = (uint32_t)p * (uint32_t)bits, byte = bitpos >> 3;
+  const uint32_t v = (uint32_t)stream[byte] | ((uint32_t)stream[byte + 1] << 8);
+  return (v >> (bitpos & 7u)) & ((1u << bits) - 1u);
+}
+
+__device__ __forceinline__ void store_y(void* y, int dtype, size_t idx, float v) {
+  if (dtype == RWKVQ_F32) static_cast<float*>(y)[idx] = v;
+  else static_cast<__half*>(y)[idx] = __float2half_rn(v);
+}
+__device__ __forceinline__ void store_w(void* out, int dtype, size_t idx, float v) {
+  if (dtype == RWKVQ_F32) static_cast<float*>(out)[idx] = v;
+  else static_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(v);
+}
+
+// x_mix = x + (x_prev - x) * mu_hat for columns [kt0*256, kt1*256) of every batch row, rounded
+// to fp16 into shared memory (zeros beyond ic); then, for SQ, per 128-column group and batch
+// row the three sums the factored dequantisation needs:
+//    Sx  = sum x,   Bx_h = sum bias_h(col) * x   (h = 0: rows g, 1: rows g+8 of a record)
+// computed from the rounded values the tensor core will see, reduced with warp shuffles.
+template <int FMT>
+__device__ __forceinline__ void stage_input(uint8_t* smem, const SmemLayout& L, const GemvArgs& a, int kt0, int kt1) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  uint32_t* mucb = reinterpret_cast<uint32_t*>(smem + L.mucb_off);
+  if (a.mu) {
+    for (int e = tid; e < a.mu_entries; e += nthr) mucb[e] = reinterpret_cast<const uint32_t*>(a.mu_aux)[e];
+    __syncthreads();
+  }
+  const int npairs = (kt1 - kt0) * 128;
+  for (int p = tid; p < a.B * npairs; p += nthr) {
+    const int b = p / npairs, cp = p - b * npairs;
+    const int col = kt0 * 256 + 2 * cp;
+    __half2 v = __float2half2_rn(0.f);
+    if (col < a.ic) {
+      v = *reinterpret_cast<const __half2*>(a.x + (size_t)b * a.ic + col);
+      if (a.mu) {
+        const float2 xf = __half22float2(v);
+        const float2 pf = __half22float2(*reinterpret_cast<const __half2*>(a.xprev + (size_t)b * a.ic + col));
+        const uint32_t mw = mucb[vector_index(a.mu, col >> 1, a.mu_bits)];
+        const float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw));
+        v = __floats2half2_rn(fmaf(pf.x - xf.x, mf.x, xf.x), fmaf(pf.y - xf.y, mf.y, xf.y));
+      }
+    }
+    *reinterpret_cast<__half2*>(smem + (size_t)b * L.xstride + (size_t)cp * 4) = v;
+  }
+  __syncthreads();
+  if constexpr (FMT == FMT_SQ3) {
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
+    const int ngroups = (kt1 - kt0) * 2;
+    float* gs = reinterpret_cast<float*>(smem + L.gs_off);
+    const int o = (lane * 4) & 63;
+    const float b00 = (float)rwkvq_sq_bias(o, 0), b02 = (float)rwkvq_sq_bias(o + 2, 0);
+    const float b10 = (float)rwkvq_sq_bias(o, 1), b12 = (float)rwkvq_sq_bias(o + 2, 1);
+    for (int task = warp; task < ngroups * a.B; task += nwarps) {
+      const int grp = task / a.B, b = task - grp * a.B;
+      const uint2 raw = *reinterpret_cast<const uint2*>(smem + (size_t)b * L.xstride + (size_t)(grp * 128 + lane * 4) * 2);
+      const float2 x01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+      const float2 x23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+      const float p01 = x01.x + x01.y, p23 = x23.x + x23.y;
+      float sx = p01 + p23;
+      float s0 = fmaf(b00, p01, b02 * p23);
+      float s1 = fmaf(b10, p01, b12 * p23);
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) {
+        sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+        s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, d);
+        s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, d);
+      }
+      if (lane == 0) {
+        gs[(grp * 3 + 0) * 16 + b] = sx;
+        gs[(grp * 3 + 1) * 16 + b] = s0;
+        gs[(grp * 3 + 2) * 16 + b] = s1;
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// B fragment of tensor-core step j of local tile ktl for batch block nb: 8 contiguous bytes.
+__device__ __forceinline__ uint2 x_frag(const uint8_t* smem, const SmemLayout& L, int ktl, int j, int nb, int B, int lane) {
+  const int b = nb * 8 + (lane >> 2);
+  uint2 v = make_uint2(0u, 0u);
+  if (b < B) v = *reinterpret_cast<const uint2*>(smem + (size_t)b * L.xstride + (size_t)(ktl * 256 + 16 * j + 4 * (lane & 3)) * 2);
+  return v;
+}
+
+struct SqRecord {
+  uint4 p0, p1, p2, sz;
+  __device__ __forceinline__ void load(const uint8_t* rec, int lane) {
+    p0 = ldg_stream(rec + lane * 16);
+    p1 = ldg_stream(rec + 512 + lane * 16);
+    p2 = ldg_stream(rec + 1024 + lane * 16);
+    sz = ldg_stream(rec + RWKVQ_SQ_CODE_BYTES + (lane >> 2) * 16);
+  }
+  __device__ __forceinline__ void words(uint32_t (&w)[12]) const {
+    w[0] = p0.x; w[1] = p0.y; w[2] = p0.z; w[3] = p0.w;
+    w[4] = p1.x; w[5] = p1.y; w[6] = p1.z; w[7] = p1.w;
+    w[8] = p2.x; w[9] = p2.y; w[10] = p2.z; w[11] = p2.w;
+  }
+  // k = 2 * row_half + group:  low 16 bits = s, high 16 bits = z (fp16)
+  __device__ __forceinline__ uint32_t sz_word(int k) const { return k == 0 ? sz.x : k == 1 ? sz.y : k == 2 ? sz.z : sz.w; }
+};
+
+// One SQ record (16 rows x 256 columns) against the staged input:
+//   y[b][row] += sum_groups s * ( sum_cols (q+bias) x  -  Bx_h  -  z * Sx )
+// The inner sum is eight m16n8k16 steps per group with fp32 accumulation in the tensor core;
+// the bias each extracted half carries is removed with the precomputed Bx_h.
+template <int NB>
+__device__ __forceinline__ void sq_record_mma(const SqRecord& rec, const uint8_t* smem, const SmemLayout& L, int ktl,
+                                              int B, int lane, float (&acc)[NB][4]) {
+  uint32_t w[12];
+  rec.words(w);
+  const float* gs = reinterpret_cast<const float*>(smem + L.gs_off);
+  const int t = lane & 3;
+#pragma unroll
+  for (int grp = 0; grp < 2; ++grp) {
+    float c[NB][4];
+#pragma unroll
+    for (int n = 0; n < NB; ++n) c[n][0] = c[n][1] = c[n][2] = c[n][3] = 0.f;
+#pragma unroll
+    for (int ti = 0; ti < 2; ++ti) {
+      const int i = 2 * grp + ti;
+      uint32_t r[16];
+      sq_unpack_triple(w[3 * i], w[3 * i + 1], w[3 * i + 2], r);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
+#pragma unroll
+        for (int n = 0; n < NB; ++n) {
+          const uint2 bf = x_frag(smem, L, ktl, 4 * i + m, n, B, lane);
+          mma_16816(c[n], afrag, bf.x, bf.y);
+        }
+      }
+    }
+    const float2 sz0 = __half22float2(*reinterpret_cast<const __half2*>(grp == 0 ? &rec.sz.x : &rec.sz.y));
+    const float2 sz1 = __half22float2(*reinterpret_cast<const __half2*>(grp == 0 ? &rec.sz.z : &rec.sz.w));
+    const float* g0 = gs + (size_t)((ktl * 2 + grp) * 3) * 16;
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      const float2 sx = *reinterpret_cast<const float2*>(g0 + n * 8 + 2 * t);
+      const float2 b0 = *reinterpret_cast<const float2*>(g0 + 16 + n * 8 + 2 * t);
+      const float2 b1 = *reinterpret_cast<const float2*>(g0 + 32 + n * 8 + 2 * t);
+      acc[n][0] = fmaf(sz0.x, fmaf(-sz0.y, sx.x, c[n][0] - b0.x), acc[n][0]);
+      acc[n][1] = fmaf(sz0.x, fmaf(-sz0.y, sx.y, c[n][1] - b0.y), acc[n][1]);
+      acc[n][2] = fmaf(sz1.x, fmaf(-sz1.y, sx.x, c[n][2] - b1.x), acc[n][2]);
+      acc[n][3] = fmaf(sz1.x, fmaf(-sz1.y, sx.y, c[n][3] - b1.y), acc[n][3]);
+    }
+  }
+}
+
+template <int BITS>
+struct VqRecord {
+  static constexpr int NW = 2 * BITS;  // 64 indices of BITS bits = 2*BITS words per lane
+  uint32_t w[NW];
+  __device__ __forceinline__ void load(const uint8_t* rec, int lane) {
+#pragma unroll
+    for (int p = 0; p < NW / 4; ++p) {
+      const uint4 v = ldg_stream(rec + p * 512 + lane * 16);
+      w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+    }
+  }
+};
+
+// Copy one codebook (E half2 entries) into 32 lane-private replicas: entry e of lane l at word
+// e*32 + l, so a lookup by any index pattern is bank-conflict free.
+__device__ __forceinline__ void stage_codebook(uint8_t* dst, const uint32_t* src, int E) {
+  uint32_t* d = reinterpret_cast<uint32_t*>(dst);
+  for (int idx = threadIdx.x; idx < E * 32; idx += blockDim.x) d[idx] = __ldg(src + (idx >> 5));
+}
+
+// One VQ record: every fragment register is one codebook lookup (a 2-D vector is exactly the
+// (even, odd) column pair a fragment register holds).
+template <int BITS, int NB>
+__device__ __forceinline__ void vq_record_mma(const VqRecord<BITS>& rec, const uint32_t* cb_lane, const uint8_t* smem,
+                                              const SmemLayout& L, int ktl, int B, int lane, float (&acc)[NB][4]) {
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    uint32_t afrag[4];
+#pragma unroll
+    for (int R = 0; R < 4; ++R) afrag[R] = cb_lane[vq_index<BITS, VqRecord<BITS>::NW>(rec.w, 4 * j + R) * 32u];
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      const uint2 bf = x_frag(smem, L, ktl, j, n, B, lane);
+      mma_16816(acc[n], afrag, bf.x, bf.y);
+    }
+  }
+}
+
+inline void fill_gemv_args(GemvArgs* a, const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu,
+                           const void* x, const void* xprev, int B, void* y, int y_dtype) {
+  const uint8_t* img = static_cast<const uint8_t*>(W);
+  size_t rb = d->method == RWKVQ_SQ ? RWKVQ_SQ_RECORD_BYTES : rwkvq_vq_record_bytes(d->bits);
+  a->payload = img + RWKVQ_HEADER_BYTES;
+  a->aux = img + RWKVQ_HEADER_BYTES + (size_t)(d->oc_pad / 128) * (d->ic_pad / 256) * 8 * rb;
+  a->mu = nullptr; a->mu_aux = nullptr; a->mu_bits = 0; a->mu_entries = 0;
+  if (mu) {
+    const uint8_t* m = static_cast<const uint8_t*>(mu);
+    a->mu = m + RWKVQ_HEADER_BYTES;
+    a->mu_aux = m + RWKVQ_HEADER_BYTES + ((((size_t)(mud->ic / 2) * mud->bits + 7) / 8 + 15) / 16 * 16);
+    a->mu_bits = mud->bits; a->mu_entries = mud->entries;
+  }
+  a->x = static_cast<const __half*>(x);
+  a->xprev = static_cast<const __half*>(xprev);
+  a->y = y; a->partial = nullptr; a->counters = nullptr;
+  a->oc = d->oc; a->ic = d->ic; a->entries = d->entries; a->B = B; a->y_dtype = y_dtype;
+  a->KT = d->ic_pad / 256; a->S = 1; a->nkt = a->KT;
+}
+
+}  // namespace rwkvq
