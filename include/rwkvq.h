@@ -131,8 +131,9 @@ rwkvq_status rwkvq_proxy_select(const void* const* w_fp16_dev, const int* oc, co
  *  W_desc/W_image_dev: packed matrix and its description.  mu_desc/mu_image_dev: packed vector of
  *  length ic, or both NULL.  x_fp16_dev, xprev_fp16_dev: [B][ic] fp16 (xprev NULL iff mu NULL).
  *  y_dev: [B][oc], y_dtype F32 or F16.  workspace_dev: rwkvq_gemv_workspace_bytes() bytes, must
- *  be zero-filled once before its first use; every call leaves it zero-filled again, so calls
- *  that share a workspace must not overlap on the device.
+ *  be zero-filled once before its first use; later calls may reuse it without clearing (each call
+ *  restores the part that has to be zero), but calls that share a workspace must not overlap on
+ *  the device.
  * Accumulation is fp32.  Errors: EINVAL, ESHAPE, EALIGN, ENOMEM, ECUDA.
  */
 size_t rwkvq_gemv_workspace_bytes(const rwkvq_desc* W_desc, int B);

@@ -1,0 +1,65 @@
+"""GPU parity of the coarse-to-fine proxy (Section 4.1) against the oracle's literal sort-and-diff."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rwkvq_oracle as orc
+from paper_2505_03803_b200 import binding as B
+from paper_2505_03803_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(mats, K=4, tau_c=1.5, tau_f=50.0):
+    dev = [torch.from_numpy(np.ascontiguousarray(m)).cuda() for m in mats]
+    ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(dev)), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xAB)  # contents on entry must not matter
+    return B.rwkvq_proxy_select(dev, K, tau_c, tau_f, ws)
+
+
+def _close(a, b, rel=1e-9):
+    return abs(a - b) <= rel * max(1.0, abs(b))
+
+
+@pytest.mark.parametrize("K", [2, 4, 6, 8])
+def test_proxy_matches_oracle(K):
+    mats = [inputs.gen_weight(0, 512, 512, "gauss"), inputs.gen_weight(1, 256, 768, "student"),
+            inputs.gen_weight(2, 128, 384, "uniform"), inputs.gen_weight(3, 3, 37, "gauss"),
+            (np.arange(4096).reshape(64, 64) % 17 - 8).astype(np.float16)]
+    big = inputs.gen_weight(4, 64, 64, "gauss").copy()
+    big[0, 0], big[5, 7] = np.float16(900.0), np.float16(-40000.0)   # outside the shared-memory window
+    mats.append(big)
+    pc, pf, phi = _run(mats, K=K)
+    for m, a, b, p in zip(mats, pc, pf, phi):
+        ra, rb = orc.proxy(m.astype(np.float64), K=K)
+        assert _close(a, ra) and _close(b, rb, 1e-8), (a, ra, b, rb)
+        assert p == orc.select(ra, rb, 1.5, 50.0)
+
+
+def test_proxy_full_size_matrix_and_threshold_between_clusters():
+    g = inputs.gen_weight(10, 2048, 2048, "gauss")
+    t = inputs.gen_weight(11, 2048, 2048, "student")
+    pc, pf, _ = _run([g, t])
+    rg, rt = orc.proxy(g.astype(np.float64)), orc.proxy(t.astype(np.float64))
+    assert _close(pc[0], rg[0]) and _close(pc[1], rt[0]) and _close(pf[0], rg[1], 1e-8) and _close(pf[1], rt[1], 1e-8)
+    assert pc[0] < pc[1]
+    tau = 0.5 * (pc[0] + pc[1])
+    _, _, phi = _run([g, t], tau_c=tau, tau_f=math.inf)
+    assert list(phi) == [B.RWKVQ_SQ, B.RWKVQ_VQ]
+
+
+def test_proxy_degenerate_and_nonfinite():
+    const = np.full((16, 16), 0.25, np.float16)
+    zeros = np.zeros((8, 8), np.float16)
+    zeros[0, 0] = np.float16(-0.0)
+    pc, pf, phi = _run([const, zeros])
+    assert math.isinf(pc[0]) and math.isinf(pf[0]) and math.isinf(pc[1]) and list(phi) == [0, 0]
+    bad = inputs.gen_weight(0, 16, 16).copy()
+    bad[3, 3] = np.float16(np.nan)
+    with pytest.raises(B.RwkvqError) as e:
+        _run([bad])
+    assert e.value.status == 4
+    with pytest.raises(B.RwkvqError):
+        _run([const], K=9)
