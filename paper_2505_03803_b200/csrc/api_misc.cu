@@ -12,6 +12,13 @@ void set_last_cuda_error(cudaError_t e) {
   strncpy(t_last_error, cudaGetErrorString(e), sizeof(t_last_error) - 1);
   t_last_error[sizeof(t_last_error) - 1] = 0;
 }
+// Device address of the status word for the current device (kernels in other translation units
+// receive it as an argument).
+int* device_status_ptr() {
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+  return static_cast<int*>(p);
+}
 }  // namespace rwkvq
 
 extern "C" {

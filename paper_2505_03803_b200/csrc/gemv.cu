@@ -40,7 +40,12 @@ __global__ void __launch_bounds__(256, 2) gemv_kernel(const GemvArgs a) {
     cur.load(rec, lane);
     for (int kt = kt0; kt < kt1; ++kt) {
       if (kt + 1 < kt1) nxt.load(rec + (size_t)(kt + 1 - kt0) * 8 * RWKVQ_SQ_RECORD_BYTES, lane);
-      sq_record_mma<NB>(cur, smem, L, (kt - kt0), a.B, lane, acc[0]);
+      uint32_t w[12];
+      cur.words(w);
+      XView xv;
+      xv.x = smem + (size_t)(kt - kt0) * 512; xv.xstride = L.xstride; xv.B = a.B; xv.nbp = 16;
+      xv.gs = reinterpret_cast<const float*>(smem + L.gs_off) + (size_t)(kt - kt0) * 2 * 3 * 16;
+      sq_record_mma<NB>(w, cur.sz, xv, lane, acc[0]);
       cur = nxt;
     }
   } else {
@@ -59,7 +64,9 @@ __global__ void __launch_bounds__(256, 2) gemv_kernel(const GemvArgs a) {
         const uint8_t* rec = a.payload + ((size_t)((2 * rb + r) * a.KT + kt) * 8 + warp) * RBYTES;
         VqRecord<BITS> v;
         v.load(rec, lane);
-        vq_record_mma<BITS, NB>(v, cb_lane, smem, L, (kt - kt0), a.B, lane, acc[r]);
+        XView xv;
+        xv.x = smem + (size_t)(kt - kt0) * 512; xv.xstride = L.xstride; xv.B = a.B; xv.nbp = 16; xv.gs = nullptr;
+        vq_record_mma<BITS, NB>(v.w, cb_lane, xv, lane, acc[r]);
       }
     }
   }

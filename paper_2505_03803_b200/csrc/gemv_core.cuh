@@ -132,16 +132,32 @@ __device__ __forceinline__ void stage_input(uint8_t* smem, const SmemLayout& L, 
   }
 }
 
-// B fragment of tensor-core step j of local tile ktl for batch block nb: 8 contiguous bytes.
-__device__ __forceinline__ uint2 x_frag(const uint8_t* smem, const SmemLayout& L, int ktl, int j, int nb, int B, int lane) {
+// View of the staged input for one 256-column tile: `x` points at the tile's first column of
+// batch row 0 (rows are `xstride` bytes apart), `gs` at the sums of the tile's first group, laid
+// out [group][3][nbp] floats (Sx, Bx_0, Bx_1 per batch row).
+struct XView {
+  const uint8_t* x;
+  const float* gs;
+  uint32_t xstride, nbp;
+  int B;
+};
+
+// B fragment of tensor-core step j for batch block nb: 8 contiguous bytes.
+__device__ __forceinline__ uint2 x_frag(const XView& xv, int j, int nb, int lane) {
   const int b = nb * 8 + (lane >> 2);
   uint2 v = make_uint2(0u, 0u);
-  if (b < B) v = *reinterpret_cast<const uint2*>(smem + (size_t)b * L.xstride + (size_t)(ktl * 256 + 16 * j + 4 * (lane & 3)) * 2);
+  if (b < xv.B) v = *reinterpret_cast<const uint2*>(xv.x + (size_t)b * xv.xstride + (size_t)(16 * j + 4 * (lane & 3)) * 2);
   return v;
 }
 
 struct SqRecord {
   uint4 p0, p1, p2, sz;
+  __device__ __forceinline__ void load_shared(const uint8_t* rec, int lane) {
+    p0 = *reinterpret_cast<const uint4*>(rec + lane * 16);
+    p1 = *reinterpret_cast<const uint4*>(rec + 512 + lane * 16);
+    p2 = *reinterpret_cast<const uint4*>(rec + 1024 + lane * 16);
+    sz = *reinterpret_cast<const uint4*>(rec + RWKVQ_SQ_CODE_BYTES + (lane >> 2) * 16);
+  }
   __device__ __forceinline__ void load(const uint8_t* rec, int lane) {
     p0 = ldg_stream(rec + lane * 16);
     p1 = ldg_stream(rec + 512 + lane * 16);
@@ -157,50 +173,61 @@ struct SqRecord {
   __device__ __forceinline__ uint32_t sz_word(int k) const { return k == 0 ? sz.x : k == 1 ? sz.y : k == 2 ? sz.z : sz.w; }
 };
 
-// One SQ record (16 rows x 256 columns) against the staged input:
-//   y[b][row] += sum_groups s * ( sum_cols (q+bias) x  -  Bx_h  -  z * Sx )
-// The inner sum is eight m16n8k16 steps per group with fp32 accumulation in the tensor core;
-// the bias each extracted half carries is removed with the precomputed Bx_h.
+// One 128-column group of an SQ record (16 rows) against the staged input:
+//   y[b][row] += s * ( sum_cols (q+bias) x  -  Bx_h  -  z * Sx )
+// The inner sum is eight m16n8k16 steps with fp32 accumulation in the tensor core; the bias each
+// extracted half carries is removed with the precomputed Bx_h.  `w` holds the group's six words
+// (two triples), `sz_lo` / `sz_hi` the (s, z) fp16 pairs of rows g and g+8; `xv.x` points at the
+// group's first column and `xv.gs` at the group's sums.
 template <int NB>
-__device__ __forceinline__ void sq_record_mma(const SqRecord& rec, const uint8_t* smem, const SmemLayout& L, int ktl,
-                                              int B, int lane, float (&acc)[NB][4]) {
-  uint32_t w[12];
-  rec.words(w);
-  const float* gs = reinterpret_cast<const float*>(smem + L.gs_off);
+__device__ __forceinline__ void sq_group_mma(const uint32_t (&w)[6], uint32_t sz_lo, uint32_t sz_hi, const XView& xv,
+                                             int lane, float (&acc)[NB][4]) {
   const int t = lane & 3;
+  float c[NB][4];
 #pragma unroll
-  for (int grp = 0; grp < 2; ++grp) {
-    float c[NB][4];
+  for (int n = 0; n < NB; ++n) c[n][0] = c[n][1] = c[n][2] = c[n][3] = 0.f;
 #pragma unroll
-    for (int n = 0; n < NB; ++n) c[n][0] = c[n][1] = c[n][2] = c[n][3] = 0.f;
+  for (int ti = 0; ti < 2; ++ti) {
+    uint32_t r[16];
+    sq_unpack_triple(w[3 * ti], w[3 * ti + 1], w[3 * ti + 2], r);
 #pragma unroll
-    for (int ti = 0; ti < 2; ++ti) {
-      const int i = 2 * grp + ti;
-      uint32_t r[16];
-      sq_unpack_triple(w[3 * i], w[3 * i + 1], w[3 * i + 2], r);
+    for (int m = 0; m < 4; ++m) {
+      const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
-#pragma unroll
-        for (int n = 0; n < NB; ++n) {
-          const uint2 bf = x_frag(smem, L, ktl, 4 * i + m, n, B, lane);
-          mma_16816(c[n], afrag, bf.x, bf.y);
-        }
+      for (int n = 0; n < NB; ++n) {
+        const uint2 bf = x_frag(xv, 4 * ti + m, n, lane);
+        mma_16816(c[n], afrag, bf.x, bf.y);
       }
     }
-    const float2 sz0 = __half22float2(*reinterpret_cast<const __half2*>(grp == 0 ? &rec.sz.x : &rec.sz.y));
-    const float2 sz1 = __half22float2(*reinterpret_cast<const __half2*>(grp == 0 ? &rec.sz.z : &rec.sz.w));
-    const float* g0 = gs + (size_t)((ktl * 2 + grp) * 3) * 16;
+  }
+  const float2 sz0 = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
+  const float2 sz1 = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
 #pragma unroll
-    for (int n = 0; n < NB; ++n) {
-      const float2 sx = *reinterpret_cast<const float2*>(g0 + n * 8 + 2 * t);
-      const float2 b0 = *reinterpret_cast<const float2*>(g0 + 16 + n * 8 + 2 * t);
-      const float2 b1 = *reinterpret_cast<const float2*>(g0 + 32 + n * 8 + 2 * t);
-      acc[n][0] = fmaf(sz0.x, fmaf(-sz0.y, sx.x, c[n][0] - b0.x), acc[n][0]);
-      acc[n][1] = fmaf(sz0.x, fmaf(-sz0.y, sx.y, c[n][1] - b0.y), acc[n][1]);
-      acc[n][2] = fmaf(sz1.x, fmaf(-sz1.y, sx.x, c[n][2] - b1.x), acc[n][2]);
-      acc[n][3] = fmaf(sz1.x, fmaf(-sz1.y, sx.y, c[n][3] - b1.y), acc[n][3]);
+  for (int n = 0; n < NB; ++n) {
+    float2 sx = make_float2(0.f, 0.f), b0 = sx, b1 = sx;
+    if (n * 8 + 2 * t < xv.B) {   // nbp is even, so the pair is always inside the table
+      sx = *reinterpret_cast<const float2*>(xv.gs + n * 8 + 2 * t);
+      b0 = *reinterpret_cast<const float2*>(xv.gs + xv.nbp + n * 8 + 2 * t);
+      b1 = *reinterpret_cast<const float2*>(xv.gs + 2 * xv.nbp + n * 8 + 2 * t);
     }
+    acc[n][0] = fmaf(sz0.x, fmaf(-sz0.y, sx.x, c[n][0] - b0.x), acc[n][0]);
+    acc[n][1] = fmaf(sz0.x, fmaf(-sz0.y, sx.y, c[n][1] - b0.y), acc[n][1]);
+    acc[n][2] = fmaf(sz1.x, fmaf(-sz1.y, sx.x, c[n][2] - b1.x), acc[n][2]);
+    acc[n][3] = fmaf(sz1.x, fmaf(-sz1.y, sx.y, c[n][3] - b1.y), acc[n][3]);
+  }
+}
+
+// A whole SQ record (16 rows x 256 columns): its two groups in turn.
+template <int NB>
+__device__ __forceinline__ void sq_record_mma(const uint32_t (&w)[12], const uint4 sz, const XView& xv, int lane,
+                                              float (&acc)[NB][4]) {
+#pragma unroll
+  for (int grp = 0; grp < 2; ++grp) {
+    const uint32_t wg[6] = {w[6 * grp], w[6 * grp + 1], w[6 * grp + 2], w[6 * grp + 3], w[6 * grp + 4], w[6 * grp + 5]};
+    XView gv = xv;
+    gv.x = xv.x + grp * 256;                       // 128 columns of fp16
+    gv.gs = xv.gs + (size_t)(grp * 3) * xv.nbp;
+    sq_group_mma<NB>(wg, grp == 0 ? sz.x : sz.y, grp == 0 ? sz.z : sz.w, gv, lane, acc);
   }
 }
 
@@ -208,6 +235,13 @@ template <int BITS>
 struct VqRecord {
   static constexpr int NW = 2 * BITS;  // 64 indices of BITS bits = 2*BITS words per lane
   uint32_t w[NW];
+  __device__ __forceinline__ void load_shared(const uint8_t* rec, int lane) {
+#pragma unroll
+    for (int p = 0; p < NW / 4; ++p) {
+      const uint4 v = *reinterpret_cast<const uint4*>(rec + p * 512 + lane * 16);
+      w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+    }
+  }
   __device__ __forceinline__ void load(const uint8_t* rec, int lane) {
 #pragma unroll
     for (int p = 0; p < NW / 4; ++p) {
@@ -226,17 +260,17 @@ __device__ __forceinline__ void stage_codebook(uint8_t* dst, const uint32_t* src
 
 // One VQ record: every fragment register is one codebook lookup (a 2-D vector is exactly the
 // (even, odd) column pair a fragment register holds).
-template <int BITS, int NB>
-__device__ __forceinline__ void vq_record_mma(const VqRecord<BITS>& rec, const uint32_t* cb_lane, const uint8_t* smem,
-                                              const SmemLayout& L, int ktl, int B, int lane, float (&acc)[NB][4]) {
+template <int BITS, int NB, int JBEG = 0, int JEND = 16>
+__device__ __forceinline__ void vq_record_mma(const uint32_t (&w)[2 * BITS], const uint32_t* cb_lane, const XView& xv,
+                                              int lane, float (&acc)[NB][4]) {
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
+  for (int j = JBEG; j < JEND; ++j) {
     uint32_t afrag[4];
 #pragma unroll
-    for (int R = 0; R < 4; ++R) afrag[R] = cb_lane[vq_index<BITS, VqRecord<BITS>::NW>(rec.w, 4 * j + R) * 32u];
+    for (int R = 0; R < 4; ++R) afrag[R] = cb_lane[vq_index<BITS, 2 * BITS>(w, 4 * j + R) * 32u];
 #pragma unroll
     for (int n = 0; n < NB; ++n) {
-      const uint2 bf = x_frag(smem, L, ktl, j, n, B, lane);
+      const uint2 bf = x_frag(xv, j, n, lane);
       mma_16816(acc[n], afrag, bf.x, bf.y);
     }
   }

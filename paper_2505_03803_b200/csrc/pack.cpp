@@ -48,6 +48,15 @@ uint16_t double_to_half(double d) {
   return sign | (uint16_t)(((exp + 15) << 10) + (m - 1024));
 }
 
+const float* half_table() {
+  static float* table = [] {
+    float* t = new float[65536];
+    for (uint32_t i = 0; i < 65536; ++i) t[i] = (float)half_to_double((uint16_t)i);
+    return t;
+  }();
+  return table;
+}
+
 uint32_t crc32_of(const uint8_t* p, size_t n) {
   static uint32_t table[256];
   static bool init = false;
@@ -186,6 +195,48 @@ inline uint32_t get_bits(const uint8_t* base, size_t bitpos, int nbits) {
 // Byte offset, inside a record, of word `widx` of lane L (planes of 512 bytes).
 inline size_t lane_word_off(int L, int widx) { return (size_t)(widx >> 2) * 512 + (size_t)L * 16 + (size_t)(widx & 3) * 4; }
 
+// Fast path of the packer: builds the three words of each triple directly.
+void sq_record_pack_fast(uint8_t* rec, const uint8_t* q, int ic, int oc, int r0, int c0) {
+  for (int L = 0; L < 32; ++L) {
+    const int g = L >> 2, t = L & 3;
+    for (int i = 0; i < 4; ++i) {
+      uint32_t w3[3] = {0u, 0u, 0u};
+      for (int e = 0; e < 16; ++e) {
+        const int m = e >> 2, R = e & 3;
+        const int row = r0 + g + 8 * (R & 1);
+        const int col = c0 + 64 * i + 16 * m + 4 * t + 2 * (R >> 1);
+        uint32_t lo = 0, hi = 0;
+        if (row < oc && col < ic) { lo = q[(size_t)row * ic + col]; hi = q[(size_t)row * ic + col + 1]; }
+        const uint32_t pair = lo | (hi << 16);
+        if (e < 15) {
+          w3[e / 5] |= pair << (3 * (e % 5));
+        } else {
+          for (int b = 0; b < 3; ++b) w3[b] |= ((pair >> b) & 0x00010001u) << 15;
+        }
+      }
+      for (int wd = 0; wd < 3; ++wd) std::memcpy(rec + lane_word_off(L, 3 * i + wd), &w3[wd], 4);
+    }
+  }
+}
+
+void vq_record_pack_fast(uint8_t* rec, const uint8_t* idx, int bits, int half_ic, int r0, int p0) {
+  const int nw = 2 * bits;
+  for (int L = 0; L < 32; ++L) {
+    const int g = L >> 2, t = L & 3;
+    uint32_t words[17] = {0};
+    for (int n = 0; n < 64; ++n) {
+      const int j = n >> 2, R = n & 3;
+      const int row = r0 + g + 8 * (R & 1);
+      const int pair = p0 + 8 * j + 2 * t + (R >> 1);
+      const uint32_t v = idx[(size_t)row * half_ic + pair];
+      const int bitpos = bits * n, wi = bitpos >> 5, sh = bitpos & 31;
+      words[wi] |= v << sh;
+      if (sh + bits > 32) words[wi + 1] |= v >> (32 - sh);
+    }
+    for (int wi = 0; wi < nw; ++wi) std::memcpy(rec + lane_word_off(L, wi), &words[wi], 4);
+  }
+}
+
 // Visit every (row, column) of an SQ record with the place its code lives.
 // pack == true writes codes from q into rec; pack == false reads them back.
 void sq_record_codes(uint8_t* rec, uint8_t* q, int ic, int oc, int r0, int c0, bool pack) {
@@ -298,7 +349,7 @@ void build_image(rwkvq_blob* b) {
         for (int rt = 0; rt < 8; ++rt) {
           uint8_t* rec = img + h.off_payload + ((size_t)(mb * KT + kt) * 8 + rt) * RWKVQ_SQ_RECORD_BYTES;
           int r0 = mb * 128 + rt * 16, c0 = kt * 256;
-          sq_record_codes(rec, b->q.data(), d.ic, d.oc, r0, c0, true);
+          sq_record_pack_fast(rec, b->q.data(), d.ic, d.oc, r0, c0);
           uint16_t* sz = reinterpret_cast<uint16_t*>(rec + RWKVQ_SQ_CODE_BYTES);
           for (int g = 0; g < 8; ++g)
             for (int k = 0; k < 4; ++k) {
@@ -320,7 +371,7 @@ void build_image(rwkvq_blob* b) {
       for (int kt = 0; kt < KT; ++kt)
         for (int rt = 0; rt < 8; ++rt) {
           uint8_t* rec = img + h.off_payload + ((size_t)(mb * KT + kt) * 8 + rt) * rb;
-          vq_record_codes(rec, b->q.data(), d.bits, d.ic / 2, mb * 128 + rt * 16, kt * 128, true);
+          vq_record_pack_fast(rec, b->q.data(), d.bits, d.ic / 2, mb * 128 + rt * 16, kt * 128);
         }
     std::memcpy(img + h.off_aux, b->codebook.data(), h.aux_bytes);
   } else {
@@ -377,12 +428,13 @@ rwkvq_status rwkvq_pack(const uint16_t* w, int oc, int ic, const rwkvq_quant_cfg
         std::memcpy(b->zero.data(), c->zero, ng * 2);
       } else {
         const int gpr = ic / 128;
+        const float* ht = half_table();
 #pragma omp parallel for schedule(static)
         for (long long gi = 0; gi < (long long)ng; ++gi) {
           size_t row = gi / gpr, grp = gi % gpr;
           double tmp[128];
           const uint16_t* src = w + row * ic + grp * 128;
-          for (int i = 0; i < 128; ++i) tmp[i] = half_to_double(src[i]);
+          for (int i = 0; i < 128; ++i) tmp[i] = (double)ht[src[i]];
           sq_encode_group(tmp, 128, 7, b->q.data() + row * ic + grp * 128, &b->scale[gi], &b->zero[gi]);
         }
       }
@@ -402,6 +454,7 @@ rwkvq_status rwkvq_pack(const uint16_t* w, int oc, int ic, const rwkvq_quant_cfg
         kmeans2d(vx.data(), vy.data(), ic / 2, d.entries, cfg->kmeans_iters, rng, b->codebook.data(), b->q.data());
       } else {
         const int TR = oc / 256, TC = ic / 256;
+        const float* ht = half_table();
 #pragma omp parallel for collapse(2) schedule(dynamic)
         for (int tr = 0; tr < TR; ++tr)
           for (int tc = 0; tc < TC; ++tc) {
@@ -410,8 +463,8 @@ rwkvq_status rwkvq_pack(const uint16_t* w, int oc, int ic, const rwkvq_quant_cfg
             for (int r = 0; r < 256; ++r)
               for (int p = 0; p < 128; ++p) {
                 const uint16_t* src = w + (size_t)(tr * 256 + r) * ic + tc * 256 + 2 * p;
-                vx[r * 128 + p] = (float)half_to_double(src[0]);
-                vy[r * 128 + p] = (float)half_to_double(src[1]);
+                vx[r * 128 + p] = ht[src[0]];
+                vy[r * 128 + p] = ht[src[1]];
               }
             SplitMix64 rng(cfg->seed * 0x9E3779B97F4A7C15ull + (uint64_t)(tr * TC + tc) + 1);
             kmeans2d(vx.data(), vy.data(), 256 * 128, d.entries, cfg->kmeans_iters, rng,

@@ -1,0 +1,176 @@
+"""Synthetic RWKV-6-shaped projection stacks: seeded weights -> proxy selection -> packed images on
+the device, plus the activation buffers of one decode step.
+
+Only marshalling lives here: the selection runs in rwkvq_proxy_select, quantization and packing in
+rwkvq_pack, the products in rwkvq_gemv / rwkvq_step_run.
+"""
+from __future__ import annotations
+
+import math
+import time
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs
+
+
+def largest_gap_threshold(pc: np.ndarray) -> float:
+    """Threshold in the middle of the widest gap between sorted finite P_c values: separates the
+    two clusters a stack of Gaussian and heavy-tailed matrices produces.  With fewer than two
+    distinct values everything is kept below the threshold."""
+    v = np.sort(np.asarray(pc, dtype=np.float64))
+    v = v[np.isfinite(v)]
+    if v.size < 2 or v[-1] == v[0]:
+        return math.inf
+    gaps = v[1:] - v[:-1]
+    i = int(np.argmax(gaps))
+    return float(0.5 * (v[i] + v[i + 1]))
+
+
+class MatrixEntry:
+    __slots__ = ("layer", "name", "oc", "ic", "kind", "seed", "stage", "has_mu", "method", "pc", "pf",
+                 "desc", "image", "mu_desc", "mu_image", "x", "xprev", "y")
+
+
+class Stack:
+    """All projection matrices of `layers` RWKV-6 blocks of width d and channel-mix width h.
+
+    Per matrix the weight distribution is N(0, 0.02) or Student-t(3)*0.01 by a seeded coin; the
+    SQ/VQ method comes from rwkvq_proxy_select with tau_c at the widest gap of the measured P_c and
+    tau_f = +inf; SQ is 3-bit group-128, VQ uses 2-D vectors with `entries` codebook entries per
+    256x256 tile.  The four time-mix input projections and the channel-mix key projection get a
+    VQ-coded token-shift vector.  `distinct_layers` > 0 draws weights for that many layers only and
+    reuses their values (in separate device buffers) for the remaining layers, to shorten set-up of
+    the large stacks.
+    """
+
+    def __init__(self, d: int, h: int, layers: int, entries: int, batch: int, n_outliers: int = 8,
+                 heavy_fraction: float = 0.1, tag: str = "stack", device: str = "cuda",
+                 distinct_layers: int = 0, force_method: int | None = None, kmeans_iters: int = 10,
+                 verbose: bool = False):
+        self.d, self.h, self.layers, self.entries, self.batch = d, h, layers, entries, batch
+        self.tag, self.device = tag, device
+        self.vq_bits = 6 if entries == 64 else 8
+        self.ops: list[MatrixEntry] = []
+        self.setup_seconds = {}
+        t0 = time.time()
+        shapes = inputs.layer_shapes(d, h)
+        n_src = layers if distinct_layers <= 0 else min(layers, distinct_layers)
+        self.n_src = n_src
+        # pass 1: weights of the source layers, P_c / P_f on the device
+        host_w = {}
+        for l in range(n_src):
+            mats = []
+            for (name, oc, ic, has_mu, stage) in shapes:
+                seed = inputs.seed_of(tag, l, name)
+                kind = inputs.weight_kind(seed, heavy_fraction)
+                w = inputs.gen_weight(seed, oc, ic, kind)
+                host_w[(l, name)] = (w, kind, seed)
+                mats.append(torch.from_numpy(w).to(device))
+            ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(mats)), dtype=torch.uint8, device=device)
+            pc, pf, _ = B.rwkvq_proxy_select(mats, 4, math.inf, math.inf, ws)
+            for (name, *_), a, b in zip(shapes, pc, pf):
+                host_w[(l, name)] += (float(a), float(b))
+            del mats, ws
+        self.setup_seconds["generate+proxy"] = time.time() - t0
+        t0 = time.time()
+        all_pc = np.array([v[3] for v in host_w.values()])
+        self.tau_c = largest_gap_threshold(all_pc)
+        self.tau_f = math.inf
+        # pass 2: selection (Eq. 18 inside the library), quantize + pack, upload
+        packed = {}
+        for l in range(n_src):
+            mats = [torch.from_numpy(host_w[(l, name)][0]).to(device) for (name, *_r) in shapes]
+            ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(mats)), dtype=torch.uint8, device=device)
+            _, _, phi = B.rwkvq_proxy_select(mats, 4, self.tau_c, self.tau_f, ws)
+            del mats, ws
+            for (name, oc, ic, has_mu, stage), p in zip(shapes, phi):
+                w, kind, seed, pc_v, pf_v = host_w[(l, name)]
+                method = int(p) if force_method is None else force_method
+                if method == B.RWKVQ_SQ:
+                    blob = B.rwkvq_pack(w, oc, ic, B.RWKVQ_SQ, 3)
+                else:
+                    blob = B.rwkvq_pack(w, oc, ic, B.RWKVQ_VQ, self.vq_bits, kmeans_iters=kmeans_iters, seed=seed)
+                mu_blob = None
+                if has_mu:
+                    mu = inputs.gen_mu(seed ^ 0xABCD, ic)
+                    mu_blob = B.rwkvq_pack(mu.reshape(1, -1), 1, ic, B.RWKVQ_VQ, self.vq_bits,
+                                           kmeans_iters=kmeans_iters, seed=seed + 1)
+                packed[(l, name)] = (blob, mu_blob, kind, seed, method, pc_v, pf_v)
+                if verbose:
+                    print(f"layer {l} {name}: {kind} pc={pc_v:.3f} -> {'SQ' if method else 'VQ'}", flush=True)
+            for (name, *_r) in shapes:
+                host_w.pop((l, name))
+        self.setup_seconds["select+pack"] = time.time() - t0
+        t0 = time.time()
+        for l in range(layers):
+            src = l % n_src
+            for (name, oc, ic, has_mu, stage) in shapes:
+                blob, mu_blob, kind, seed, method, pc_v, pf_v = packed[(src, name)]
+                e = MatrixEntry()
+                e.layer, e.name, e.oc, e.ic, e.kind, e.seed = l, name, oc, ic, kind, seed
+                e.stage, e.has_mu, e.method, e.pc, e.pf = 4 * l + stage, has_mu, method, pc_v, pf_v
+                e.desc, e.image = blob.desc, blob.to_device(device)
+                e.mu_desc, e.mu_image = (mu_blob.desc, mu_blob.to_device(device)) if has_mu else (None, None)
+                act_seed = inputs.seed_of(tag, "act", l, name)
+                if has_mu:
+                    x, xp = inputs.gen_activation_pair(act_seed, batch, ic, n_outliers)
+                    e.xprev = torch.from_numpy(xp.astype(np.float16)).to(device)
+                else:
+                    x = inputs.gen_activation(act_seed, batch, ic, n_outliers)
+                    e.xprev = None
+                e.x = torch.from_numpy(x.astype(np.float16)).to(device)
+                e.y = torch.zeros((batch, oc), dtype=torch.float32, device=device)
+                self.ops.append(e)
+        self.ops.sort(key=lambda o: o.stage)
+        self.setup_seconds["upload"] = time.time() - t0
+        self._packed = packed  # keeps the host blobs (logical codes) for parity checks
+        self.n_weights = sum(o.oc * o.ic for o in self.ops)
+        self.stream_bytes = sum(int(o.desc.stream_bytes) + (int(o.mu_desc.stream_bytes) if o.has_mu else 0)
+                                for o in self.ops)
+        self.act_bytes = sum(batch * o.ic * 2 * (2 if o.has_mu else 1) + batch * o.oc * 4 for o in self.ops)
+        self.n_sq = sum(1 for o in self.ops if o.method == B.RWKVQ_SQ)
+        self.n_stages = len({o.stage for o in self.ops})
+        ws_bytes = max(B.rwkvq_gemv_workspace_bytes(o.desc, batch) for o in self.ops)
+        self.workspace = torch.zeros(max(ws_bytes, 256), dtype=torch.uint8, device=device)
+        self._plan = None
+
+    def host_codes(self, op: MatrixEntry):
+        """Logical codes (numpy) of a matrix and of its mu vector, exported by the packer."""
+        blob, mu_blob, *_ = self._packed[(op.layer % self.n_src, op.name)]
+        return blob.export_codes(), (mu_blob.export_codes() if mu_blob is not None else None)
+
+    # ---- one decode step ----------------------------------------------------------------------
+    def run_ops(self, stream=None):
+        """One rwkvq_gemv launch per product, in stage order."""
+        for o in self.ops:
+            B.rwkvq_gemv(o.desc, o.image, o.mu_desc, o.mu_image, o.x, o.xprev, self.batch, o.y,
+                         self.workspace, stream)
+        return len(self.ops)
+
+    def plan_step(self):
+        entries = [dict(desc=o.desc, W=o.image, mu_desc=o.mu_desc, mu=o.mu_image, x=o.x, xprev=o.xprev,
+                        y=o.y, stage=o.stage) for o in self.ops]
+        ops = B.make_ops(entries)
+        nbytes = B.rwkvq_step_plan_bytes(ops, self.batch)
+        if nbytes == 0:
+            raise RuntimeError("rwkvq_step_plan_bytes returned 0 (plan rejected)")
+        self._plan = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+        B.rwkvq_step_plan(ops, self.batch, self._plan)
+        torch.cuda.synchronize()
+
+    def run_step(self, stream=None):
+        """The whole step as one persistent launch (rwkvq_step_run)."""
+        if self._plan is None:
+            self.plan_step()
+        B.rwkvq_step_run(self._plan, stream)
+        return 1
+
+
+def from_name(name: str, batch: int | None = None, **kw) -> Stack:
+    spec = inputs.STACKS[name]
+    b = spec["batches"][0] if batch is None else batch
+    return Stack(spec["d"], spec["h"], kw.pop("layers", spec["layers"]), spec["entries"], b,
+                 n_outliers=spec["outliers"], tag=name, **kw)

@@ -1,0 +1,97 @@
+"""GPU parity of the whole-step persistent launch (rwkvq_step_plan / rwkvq_step_run) against the
+oracle, product by product."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_03803_b200 import binding as B
+from paper_2505_03803_b200 import inputs
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _build_ops(d, h, layers, Bn, bits, seed, all_method=None):
+    """Logical codes drawn at random (valid by construction), packed by the library."""
+    ops = []
+    k = 0
+    for l in range(layers):
+        for (name, oc, ic, has_mu, stage) in inputs.layer_shapes(d, h):
+            k += 1
+            use_sq = (k % 3 != 0) if all_method is None else (all_method == B.RWKVQ_SQ)
+            W = H.pack_sq(H.random_sq_codes(seed + k, oc, ic)) if use_sq else H.pack_vq(H.random_vq_codes(seed + k, oc, ic, bits), bits)
+            mu = H.pack_mu(H.random_mu_codes(seed + 100 + k, ic, bits), bits) if has_mu else None
+            x, xp = inputs.gen_activation_pair(seed + 200 + k, Bn, ic, n_outliers=4)
+            x16, xp16 = x.astype(np.float16), xp.astype(np.float16)
+            e = dict(W=W, mu=mu, x16=x16, xp16=xp16, stage=4 * l + stage,
+                     xd=torch.from_numpy(x16).cuda(), xpd=torch.from_numpy(xp16).cuda() if has_mu else None,
+                     y=torch.full((Bn, oc), float("nan"), dtype=torch.float32, device="cuda"))
+            ops.append(e)
+    ops.sort(key=lambda e: e["stage"])
+    return ops
+
+
+def _plan(ops, Bn):
+    arr = B.make_ops([dict(desc=e["W"].desc, W=e["W"].dev, mu_desc=None if e["mu"] is None else e["mu"].desc,
+                           mu=None if e["mu"] is None else e["mu"].dev, x=e["xd"], xprev=e["xpd"], y=e["y"],
+                           stage=e["stage"]) for e in ops])
+    n = B.rwkvq_step_plan_bytes(arr, Bn)
+    assert n > 0
+    plan = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    B.rwkvq_step_plan(arr, Bn, plan)
+    return plan
+
+
+def _check(ops, Bn):
+    worst = 0.0
+    for e in ops:
+        y = e["y"].double().cpu().numpy()
+        ref, tol = H.reference(e["W"], e["mu"], e["x16"], e["xp16"])
+        err = np.abs(y - ref)
+        assert np.isfinite(y).all()
+        ratio = float((err / tol).max())
+        worst = max(worst, ratio)
+        assert (err <= tol).all(), f"stage {e['stage']}: max err/tol = {ratio}"
+    return worst
+
+
+@pytest.mark.parametrize("Bn,bits", [(1, 6), (8, 6), (16, 8), (3, 8)])
+def test_step_matches_oracle_small_stack(Bn, bits):
+    ops = _build_ops(512, 1280, 2, Bn, bits, seed=10 * Bn + bits)   # h = 5 column tiles: odd tile count
+    plan = _plan(ops, Bn)
+    for rep in range(3):          # outputs are cleared and recomputed on every run
+        B.rwkvq_step_run(plan)
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        _check(ops, Bn)
+
+
+@pytest.mark.parametrize("method", [B.RWKVQ_SQ, B.RWKVQ_VQ])
+def test_step_matches_oracle_1p6b_layer(method):
+    ops = _build_ops(2048, 7168, 1, 1, 6, seed=77, all_method=method)
+    plan = _plan(ops, 1)
+    B.rwkvq_step_run(plan)
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 0
+    _check(ops, 1)
+
+
+def test_step_agrees_with_single_product_calls():
+    ops = _build_ops(512, 1280, 1, 8, 6, seed=5)
+    plan = _plan(ops, 8)
+    B.rwkvq_step_run(plan)
+    torch.cuda.synchronize()
+    for e in ops:
+        y1 = H.run_gemv(e["W"], e["mu"], e["x16"], e["xp16"])
+        _, tol = H.reference(e["W"], e["mu"], e["x16"], e["xp16"])
+        assert (np.abs(e["y"].double().cpu().numpy() - y1) <= tol).all()
+
+
+def test_step_rejects_bad_plans():
+    ops = _build_ops(512, 1280, 1, 1, 6, seed=6)
+    plan = _plan(ops, 1)
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_step_run(plan[256:])         # not the buffer a plan was written to
+    arr = B.make_ops([dict(desc=e["W"].desc, W=e["W"].dev, mu_desc=None, mu=None, x=e["xd"], xprev=None,
+                           y=e["y"].half(), stage=e["stage"]) for e in ops[:1]])
+    assert B.rwkvq_step_plan_bytes(arr, 1) == 0   # fp16 outputs are not supported by the step launch
