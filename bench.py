@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Decode-throughput benchmark of the hybrid SQ/VQ projection stack.
+
+One step = one decode pass over every projection of every layer of a seeded synthetic
+RWKV-6-shaped stack (time-mix R/K/V/G/O, channel-mix K/R/V, the five token-shift mixes fused),
+issued as one persistent launch (rwkvq_step_run).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_1p6b|c3_7b|c4_14b] [--batch B]
+  python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
+replica of the same stack (the path has no exchange step); the value is the tokens all ranks
+processed divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_1p6b", choices=["c2_1p6b", "c3_7b", "c4_14b"])
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--distinct-layers", type=int, default=4,
+                    help="draw and quantize weights for this many layers and reuse their values, in "
+                         "separate device buffers, for the others (0 = every layer distinct)")
+    ap.add_argument("--force-method", default=None, choices=[None, "sq", "vq"],
+                    help="pack every matrix with one format instead of the proxy's choice")
+    ap.add_argument("--mode", default="step", choices=["step", "ops"],
+                    help="step = one persistent launch per step; ops = one rwkvq_gemv launch per product")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args(argv)
+
+
+def workload_name(spec_name, batch):
+    from paper_2505_03803_b200 import inputs
+    sp = inputs.STACKS[spec_name]
+    return (f"{spec_name}: RWKV-6-shaped stack d={sp['d']} h={sp['h']} L={sp['layers']}, 8 projections + 5 fused "
+            f"token-shift mixes per layer, hybrid SQ(3-bit g128)/VQ(2-D, {sp['entries']} entries) by proxy, "
+            f"decode batch {batch}")
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for (t, r) in self.rows if (t0 is None or t >= t0) and (t1 is None or t <= t1 + 0.2)]
+        if not rows:
+            rows = [r for (_, r) in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# rank aggregation (host logic; also exercised on CPU with the gloo backend)
+# ---------------------------------------------------------------------------------------------
+def aggregate_over_ranks(local_ms: float, local_units: float, dist=None):
+    """(max over ranks of the elapsed milliseconds, sum over ranks of the units processed)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(local_ms), float(local_units)
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([local_units], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle leg
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(spec_name: str, batch: int, rows_fraction: float = 1.0):
+    """Seeded logical codes and activations of ONE layer of the workload (random valid codes; the
+    matrix that the seeded coin makes heavy-tailed is VQ-coded, the others SQ), optionally cut to
+    the first `rows_fraction` of each matrix's rows (whole 256-row tiles)."""
+    from paper_2505_03803_b200 import inputs
+    sp = inputs.STACKS[spec_name]
+    bits = 6 if sp["entries"] == 64 else 8
+    items = []
+    for (name, oc, ic, has_mu, stage) in inputs.layer_shapes(sp["d"], sp["h"]):
+        seed = inputs.seed_of(spec_name, 0, name)
+        roc = max(256, int(oc * rows_fraction) // 256 * 256)
+        if inputs.weight_kind(seed) == "gauss":
+            codes, method = inputs.random_sq_codes(seed, roc, ic), "sq"
+        else:
+            codes, method = inputs.random_vq_codes(seed, roc, ic, bits), "vq"
+        mu = inputs.random_mu_codes(seed + 1, ic, bits) if has_mu else None
+        if has_mu:
+            x, xp = inputs.gen_activation_pair(seed + 2, batch, ic, sp["outliers"])
+            xp = xp.astype(np.float16)
+        else:
+            x, xp = inputs.gen_activation(seed + 2, batch, ic, sp["outliers"]), None
+        items.append(dict(method=method, codes=codes, mu=mu, x=x.astype(np.float16), xp=xp, oc=roc, ic=ic))
+    return items, sp
+
+
+def oracle_step(items):
+    """The oracle's dequantize-and-multiply over the sample, as it stands (fp64)."""
+    from oracle import rwkvq_oracle as orc
+    out = []
+    for it in items:
+        c = it["codes"]
+        w_hat = orc.sq_decode(c["q"], c["scale"], c["zero"]) if it["method"] == "sq" else orc.vq_decode(c["codebook"], c["q"])
+        x = it["x"].astype(np.float64)
+        if it["mu"] is not None:
+            x = orc.token_shift(x, it["xp"].astype(np.float64), orc.mu_decode(it["mu"]["codebook"], it["mu"]["q"]))
+        out.append(orc.gemv(w_hat, x))
+    return out
+
+
+def cpu_threads():
+    try:
+        import threadpoolctl
+        n = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(spec_name, batch, budget_s=12.0, rows_fraction=1.0, steps=None, warmup=0):
+    """Times the oracle on one layer (or a row slice of it) and scales to the whole stack."""
+    items, sp = oracle_sample(spec_name, batch, rows_fraction)
+    sample_weights = sum(it["oc"] * it["ic"] for it in items)
+    from paper_2505_03803_b200 import inputs
+    total_weights = sum(oc * ic for (_, oc, ic, _, _) in inputs.layer_shapes(sp["d"], sp["h"])) * sp["layers"]
+    for _ in range(warmup):
+        oracle_step(items)
+    times = []
+    t_start = time.time()
+    while True:
+        t0 = time.perf_counter()
+        oracle_step(items)
+        times.append(time.perf_counter() - t0)
+        if steps is not None:
+            if len(times) >= steps:
+                break
+        elif time.time() - t_start >= budget_s or len(times) >= 50:
+            break
+    per_step = sum(times) / len(times)
+    full_step_s = per_step * total_weights / sample_weights
+    return dict(value=batch / full_step_s, per_sample_s=per_step, n=len(times), sample_weights=sample_weights,
+                total_weights=total_weights, full_step_s=full_step_s)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2505_03803_b200 import inputs
+    sp = inputs.STACKS[args.workload]
+    batch = args.batch or sp["batches"][0]
+    K = args.steps if args.steps is not None else 5
+    W = args.warmup if args.warmup is not None else 1
+    # size the per-step sample from a probe so that the whole run stays near two minutes
+    probe = time_oracle(args.workload, batch, steps=1, rows_fraction=0.125)
+    full_layer_s = probe["per_sample_s"] * 8.0
+    frac = min(1.0, max(0.125, 120.0 / max(1e-9, full_layer_s * (K + W))))
+    frac = max(0.125, int(frac * 8) / 8.0)
+    r = time_oracle(args.workload, batch, steps=K, warmup=W, rows_fraction=frac)
+    cores = cpu_threads()
+    sample = (f"per step: the oracle's decode + token shift + fp64 product over the first {frac:g} of the rows of "
+              f"each of the 8 matrices of one layer ({r['sample_weights']} of {r['total_weights']} weights), "
+              f"time scaled to the whole stack by weight count")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+        "warmup": W, "ms_per_step": r["full_step_s"] * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload, batch), "batch": batch},
+        "cpu_baseline": {"value": r["value"], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU leg
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_03803_b200 import binding as B
+    from paper_2505_03803_b200 import build as build_mod
+    from paper_2505_03803_b200 import inputs, stack as stack_mod
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; this benchmark has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build_mod.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+
+    sp = inputs.STACKS[args.workload]
+    batch = args.batch or sp["batches"][0]
+    force = None if args.force_method is None else (B.RWKVQ_SQ if args.force_method == "sq" else B.RWKVQ_VQ)
+    t_setup = time.time()
+    st = stack_mod.Stack(sp["d"], sp["h"], sp["layers"], sp["entries"], batch, n_outliers=sp["outliers"],
+                         tag=args.workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force)
+    if args.mode == "step":
+        st.plan_step()
+    setup_s = time.time() - t_setup
+    run = st.run_step if args.mode == "step" else st.run_ops
+    launches_per_step = 1 if args.mode == "step" else len(st.ops)
+
+    est_ms = max(0.05, st.stream_bytes / 4.0e9)    # ms per step at 4 TB/s: only sizes the default step count
+    K = args.steps if args.steps is not None else int(min(2000, max(20, 4000.0 / est_ms)))
+    W = args.warmup if args.warmup is not None else 5
+    W = max(W, 3)
+
+    stream = torch.cuda.current_stream()
+    for _ in range(W):
+        run(stream)
+    torch.cuda.synchronize()
+    if B.rwkvq_device_status() != 0:
+        raise SystemExit("bench.py: a device-side wait timed out during warm-up")
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    time.sleep(0.3)
+
+    # ---- device-resident timing: K steps, one event per step boundary
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    ev[0].record(stream)
+    for i in range(K):
+        run(stream)
+        ev[i + 1].record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t1 = time.time()
+    total_ms = ev[0].elapsed_time(ev[K])
+    per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) / launches_per_step for i in range(K)]
+    status = B.rwkvq_device_status()
+
+    # ---- end to end: activations from pinned host memory, results back to the host, every step
+    e2e_ms = None
+    if args.mode == "step":
+        for _ in range(3):
+            st.run_step_host(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(K):
+            st.run_step_host(stream)
+            stream.synchronize()          # the caller reads the step's outputs before the next step
+        b.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        e2e_ms = a.elapsed_time(b)
+    t2 = time.time()
+    clocks = sampler.stop(t0, t2)
+    if status != 0:
+        raise SystemExit("bench.py: a device-side wait timed out during the timed region")
+
+    max_ms, tokens = aggregate_over_ranks(total_ms, float(batch * K), dist if world > 1 else None)
+    value = tokens / (max_ms * 1e-3)
+    e2e = None
+    if e2e_ms is not None:
+        m2, tok2 = aggregate_over_ranks(e2e_ms, float(batch * K), dist if world > 1 else None)
+        e2e = {"value": tok2 / (m2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(st.act_host.numel()),
+               "d2h_bytes_per_step": int(st.y_host.numel())}
+
+    peak, peak_kind = measured_hbm_peak()
+    alg_bytes = st.stream_bytes + st.act_bytes
+    avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
+    achieved = alg_bytes / launches_per_step / (avg_launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "step_kernel" if args.mode == "step" else "gemv_kernel",
+                "algorithmic_bytes_per_launch": alg_bytes / launches_per_step,
+                "launch_ms_avg": avg_launch_ms, "launch_ms_median": statistics.median(per_launch_ms),
+                "launch_ms_min": min(per_launch_ms), "frac_of_8TBs_nominal": achieved / 8000.0}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        r = time_oracle(args.workload, batch, budget_s=12.0)
+        cpu = {"value": r["value"], "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+               "sample": (f"the oracle's decode + token shift + fp64 product over the 8 matrices of one layer "
+                          f"({r['sample_weights']} of {r['total_weights']} weights), {r['n']} repetitions, "
+                          f"{r['per_sample_s']:.3f} s each, scaled to {sp['layers']} layers")}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": max_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload, batch), "batch": batch, "mode": args.mode,
+                   "matrices": len(st.ops), "sq_matrices": st.n_sq, "stages": st.n_stages,
+                   "weights": st.n_weights, "packed_bytes_per_step": st.stream_bytes,
+                   "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src,
+                   "l2": "inputs larger than L2: every step streams the whole packed stack once",
+                   "replicas": "independent replica per GPU, no exchange step" if world > 1 else "single GPU",
+                   "not_included": "WKV recurrence, norms, gates, embedding and head are not part of the workload",
+                   "tau_c": st.tau_c, "setup_s": round(setup_s, 1)},
+        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": K * launches_per_step,
+        "hbm_gbs": achieved,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -169,6 +169,16 @@ size_t rwkvq_step_plan_bytes(const rwkvq_gemv_op* ops, int n_ops, int B);
 rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* plan_dev,
                              size_t plan_bytes, void* stream);
 rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream);
+/*
+ * The same step for callers whose activations live in host memory: copies act_bytes from act_host
+ * to act_dev (the device buffer the plan's x / x_prev pointers lie in), runs the step, and copies
+ * y_bytes from y_dev (the buffer the plan's outputs lie in) to y_host, all asynchronously on
+ * `stream` in that order; the caller synchronizes the stream before reading y_host.  Host buffers
+ * should be page-locked, otherwise the copies serialize with the host.  A size of 0 skips that copy.
+ */
+rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const void* act_host,
+                                 void* act_dev, size_t act_bytes, const void* y_dev, void* y_host,
+                                 size_t y_bytes, void* stream);
 
 /*
  * Prefill product Y[t][i] = sum_j bf16(w_hat[i][j]) * x_mix[t][j] for M tokens, bf16 x bf16 ->

@@ -58,6 +58,7 @@ EXPORTS = [
     "rwkvq_pack", "rwkvq_blob_desc", "rwkvq_blob_nbytes", "rwkvq_blob_image", "rwkvq_blob_export_codes",
     "rwkvq_image_unpack", "rwkvq_blob_free", "rwkvq_proxy_workspace_bytes", "rwkvq_proxy_select",
     "rwkvq_gemv_workspace_bytes", "rwkvq_gemv", "rwkvq_step_plan_bytes", "rwkvq_step_plan", "rwkvq_step_run",
+    "rwkvq_step_run_host",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
 ]
@@ -104,6 +105,7 @@ def lib() -> C.CDLL:
         L.rwkvq_step_plan_bytes.restype = sz
         L.rwkvq_step_plan.argtypes = [C.POINTER(GemvOp), i32, i32, vp, sz, vp]
         L.rwkvq_step_run.argtypes = [vp, sz, vp]
+        L.rwkvq_step_run_host.argtypes = [vp, sz, vp, vp, sz, vp, vp, sz, vp]
     if hasattr(L, "rwkvq_gemm_prefill"):
         L.rwkvq_prefill_workspace_bytes.argtypes = [C.POINTER(Desc), i32, i32]
         L.rwkvq_prefill_workspace_bytes.restype = sz
@@ -316,6 +318,15 @@ def rwkvq_step_plan(ops, B: int, plan, stream=None):
 
 def rwkvq_step_run(plan, stream=None):
     _check(lib().rwkvq_step_run(_dev_ptr(plan), plan.numel(), _stream_ptr(stream)), "rwkvq_step_run")
+
+
+def rwkvq_step_run_host(plan, act_host, act_dev, y_dev, y_host, stream=None):
+    """rwkvq_step_run_host: act_host / y_host are (pinned) host uint8 tensors, act_dev / y_dev the
+    device buffers the plan's activations and outputs lie in."""
+    _check(lib().rwkvq_step_run_host(_dev_ptr(plan), plan.numel(), C.c_void_p(act_host.data_ptr()),
+                                     _dev_ptr(act_dev), act_host.numel(), _dev_ptr(y_dev),
+                                     C.c_void_p(y_host.data_ptr()), y_host.numel(), _stream_ptr(stream)),
+           "rwkvq_step_run_host")
 
 
 def rwkvq_prefill_workspace_bytes(desc: Desc, M: int, has_mu: bool) -> int:

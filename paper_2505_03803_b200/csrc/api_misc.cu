@@ -2,12 +2,16 @@
 #include <cuda_runtime.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "../../include/rwkvq.h"
 #include "host_util.h"
 
 namespace rwkvq {
 __device__ int g_device_status = 0;
 static thread_local char t_last_error[256] = "";
+static std::atomic<unsigned> g_abort_epoch{0};
+unsigned abort_epoch() { return g_abort_epoch.load(); }
 void set_last_cuda_error(cudaError_t e) {
   strncpy(t_last_error, cudaGetErrorString(e), sizeof(t_last_error) - 1);
   t_last_error[sizeof(t_last_error) - 1] = 0;
@@ -31,6 +35,7 @@ rwkvq_status rwkvq_device_status(void* stream) {
   if (e == cudaSuccess) e = cudaMemcpyToSymbolAsync(rwkvq::g_device_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return rwkvq::cuda_status(e);
+  if (v != 0) rwkvq::g_abort_epoch.fetch_add(1);
   return v == 0 ? RWKVQ_OK : (rwkvq_status)v;
 }
 }

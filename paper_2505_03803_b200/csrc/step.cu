@@ -31,6 +31,7 @@
 namespace rwkvq {
 
 int* device_status_ptr();  // api_misc.cu
+unsigned abort_epoch();     // api_misc.cu: bumped whenever rwkvq_device_status reports a failed wait
 
 enum { UF_FLUSH = 1, UF_STAGE_END = 2, UF_NEW_XSEG = 4, UF_END_XSEG = 8, UF_SPLIT = 16 };
 // bits 16..31 of a unit's flags: index of the stage barrier a UF_STAGE_END unit arrives at
@@ -69,7 +70,8 @@ struct StepArgs {
   const StepXSeg* xsegs;
   const uint32_t* unit_off;   // [P+1]
   const uint32_t* xseg_off;   // [P+1]
-  unsigned* counter;          // stage barriers: arrivals at barrier k in counter[k]
+  unsigned* counter;          // stage barriers: arrivals at barrier k, summed over all runs, in counter[k]
+  unsigned target;            // arrivals that open a barrier in this run: run number * CTAs (mod 2^32)
   unsigned n_ctas;
   int* status;
   int B, n_slots;
@@ -222,7 +224,7 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       // barrier has its own arrival counter, so a CTA without work may run ahead and arrive at
       // later barriers without releasing this one early.
       uint32_t it = 0;
-      while (ld_acquire_gpu(a.counter + (sg.barrier - 1u)) < a.n_ctas) {
+      while ((int)(ld_acquire_gpu(a.counter + (sg.barrier - 1u)) - a.target) < 0) {
         if (++it >= kPollLimit || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
         __nanosleep(20);
       }
@@ -465,6 +467,8 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
 
 struct PlanInfo {
   int P, B, NB, n_slots;
+  unsigned runs;        // launches since the counters were last zero
+  unsigned abort_epoch; // value of the abort epoch when the counters were last known good
   uint32_t slot_bytes, replica_bytes, smem_bytes;
   size_t off_unit_off, off_xseg_off, off_units, off_xsegs, off_counter, total_bytes;
   uint32_t n_units, n_xsegs, n_barriers;
@@ -752,6 +756,8 @@ rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* p
   cudaError_t e = cudaMemcpyAsync(plan_dev, image.data(), image.size(), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);   // `image` is a pageable temporary
   if (e != cudaSuccess) return cuda_status(e);
+  info.runs = 0;
+  info.abort_epoch = abort_epoch();   // the image just copied holds zeroed counters
   std::lock_guard<std::mutex> lock(g_plan_mutex);
   g_plans[plan_dev] = info;
   return RWKVQ_OK;
@@ -760,13 +766,19 @@ rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* p
 rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream) {
   if (!plan_dev) return RWKVQ_EINVAL;
   PlanInfo info;
+  bool clear_counters = false;
   {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     auto it = g_plans.find(plan_dev);
     if (it == g_plans.end()) return RWKVQ_EINVAL;   // not a plan written by rwkvq_step_plan in this process
+    if (plan_bytes < it->second.total_bytes) return RWKVQ_ENOMEM;
+    // The arrival counters only ever grow: run r opens a barrier at r * CTAs arrivals, so a launch
+    // needs no clearing pass.  A run that gave up leaves them short; start over after one.
+    const unsigned epoch = abort_epoch();
+    if (it->second.abort_epoch != epoch) { it->second.abort_epoch = epoch; it->second.runs = 0; clear_counters = true; }
+    it->second.runs += 1;
     info = it->second;
   }
-  if (plan_bytes < info.total_bytes) return RWKVQ_ENOMEM;
   const uint8_t* p = static_cast<const uint8_t*>(plan_dev);
   StepArgs a;
   a.units = reinterpret_cast<const StepUnit*>(p + info.off_units);
@@ -779,15 +791,41 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
   a.B = info.B; a.n_slots = info.n_slots; a.slot_bytes = info.slot_bytes; a.replica_bytes = info.replica_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   a.n_ctas = (unsigned)info.P;
-  cudaError_t e = cudaMemsetAsync(a.counter, 0, round_up_sz((size_t)info.n_barriers * 4, 256), s);
-  if (e != cudaSuccess) return cuda_status(e);
+  a.target = info.runs * (unsigned)info.P;
+  cudaError_t e = cudaSuccess;
+  if (clear_counters) {
+    e = cudaMemsetAsync(a.counter, 0, round_up_sz((size_t)info.n_barriers * 4, 256), s);
+    if (e != cudaSuccess) return cuda_status(e);
+  }
   const void* fn = info.NB == 1 ? (const void*)step_kernel<1> : (const void*)step_kernel<2>;
   e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)info.smem_bytes);
   if (e != cudaSuccess) return cuda_status(e);
   void* params[] = {&a};
   // Cooperative launch: all CTAs must be resident at once because they meet at the stage barrier.
   e = cudaLaunchCooperativeKernel(fn, dim3(info.P), dim3(kThreads), params, info.smem_bytes, s);
+  if (e != cudaSuccess) {   // this run will never arrive: have the next one clear the counters
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    auto it = g_plans.find(plan_dev);
+    if (it != g_plans.end()) it->second.abort_epoch = abort_epoch() - 1u;
+  }
   return cuda_status(e);
+}
+
+rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const void* act_host, void* act_dev,
+                                 size_t act_bytes, const void* y_dev, void* y_host, size_t y_bytes, void* stream) {
+  if ((act_bytes && (!act_host || !act_dev)) || (y_bytes && (!y_dev || !y_host))) return RWKVQ_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (act_bytes) {
+    cudaError_t e = cudaMemcpyAsync(act_dev, act_host, act_bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_status(e);
+  }
+  rwkvq_status st = rwkvq_step_run(plan_dev, plan_bytes, stream);
+  if (st != RWKVQ_OK) return st;
+  if (y_bytes) {
+    cudaError_t e = cudaMemcpyAsync(y_host, y_dev, y_bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_status(e);
+  }
+  return RWKVQ_OK;
 }
 
 }  // extern "C"

@@ -97,6 +97,34 @@ def gen_activation_pair(seed: int, batch: int, ic: int, n_outliers: int = 8, sca
     return x, xp
 
 
+def random_sq_codes(seed: int, oc: int, ic: int, group: int = 128, bits: int = 3) -> dict:
+    """Valid logical SQ codes drawn at random (no quantizer involved): codes uniform in
+    [0, 2^bits), fp16 scales in [0.005, 0.025), integer zero points in [0, 2^bits)."""
+    rng = np.random.default_rng(seed)
+    q = rng.integers(0, 1 << bits, size=(oc, ic), dtype=np.uint8)
+    s = (rng.random((oc, ic // group)) * 0.02 + 0.005).astype(np.float16)
+    z = rng.integers(0, 1 << bits, size=(oc, ic // group)).astype(np.float16)
+    return dict(q=q, scale=s, zero=z)
+
+
+def random_vq_codes(seed: int, oc: int, ic: int, bits: int, tile: int = 256) -> dict:
+    """Valid logical VQ codes drawn at random: indices uniform in [0, 2^bits), one fp16 codebook
+    of N(0, 0.02) 2-vectors per tile x tile block."""
+    rng = np.random.default_rng(seed)
+    E = 1 << bits
+    idx = rng.integers(0, E, size=(oc, ic // 2), dtype=np.uint8)
+    cb = (rng.standard_normal((oc // tile, ic // tile, E, 2)) * 0.02).astype(np.float16)
+    return dict(q=idx, codebook=cb)
+
+
+def random_mu_codes(seed: int, ic: int, bits: int = 6) -> dict:
+    """Valid logical codes of a token-shift vector: indices uniform, codebook uniform in (0,1)."""
+    rng = np.random.default_rng(seed)
+    E = 1 << bits
+    return dict(q=rng.integers(0, E, size=(ic // 2,), dtype=np.uint8),
+                codebook=rng.random((E, 2)).astype(np.float16))
+
+
 def to_bf16_bits(a: np.ndarray) -> np.ndarray:
     """Round float32 to bf16 (nearest even) and return the uint16 bit patterns.
     Pure number-format conversion (no method arithmetic)."""

@@ -31,7 +31,7 @@ def largest_gap_threshold(pc: np.ndarray) -> float:
 
 class MatrixEntry:
     __slots__ = ("layer", "name", "oc", "ic", "kind", "seed", "stage", "has_mu", "method", "pc", "pf",
-                 "desc", "image", "mu_desc", "mu_image", "x", "xprev", "y")
+                 "desc", "image", "mu_desc", "mu_image", "x", "xprev", "y", "act_off")
 
 
 class Stack:
@@ -105,25 +105,53 @@ class Stack:
                 host_w.pop((l, name))
         self.setup_seconds["select+pack"] = time.time() - t0
         t0 = time.time()
+        # Activations of every product live in one device arena and the outputs in another, so a
+        # step's inputs arrive in one host-to-device copy and its results leave in one copy back.
+        def _al(n):
+            return (n + 255) // 256 * 256
+        act_off, y_off, slots = 0, 0, []
+        for l in range(layers):
+            for (name, oc, ic, has_mu, stage) in shapes:
+                xo = act_off
+                act_off += _al(batch * ic * 2)
+                po = None
+                if has_mu:
+                    po = act_off
+                    act_off += _al(batch * ic * 2)
+                slots.append((xo, po, y_off))
+                y_off += _al(batch * oc * 4)
+        self.act_host = torch.empty(act_off, dtype=torch.uint8).pin_memory() if device != "cpu" else torch.empty(act_off, dtype=torch.uint8)
+        self.act_arena = torch.empty(act_off, dtype=torch.uint8, device=device)
+        self.y_arena = torch.zeros(y_off, dtype=torch.uint8, device=device)
+        self.y_host = torch.empty(y_off, dtype=torch.uint8).pin_memory() if device != "cpu" else torch.empty(y_off, dtype=torch.uint8)
+        act_np = self.act_host.numpy()
+        k = 0
         for l in range(layers):
             src = l % n_src
             for (name, oc, ic, has_mu, stage) in shapes:
                 blob, mu_blob, kind, seed, method, pc_v, pf_v = packed[(src, name)]
+                xo, po, yo = slots[k]
+                k += 1
                 e = MatrixEntry()
                 e.layer, e.name, e.oc, e.ic, e.kind, e.seed = l, name, oc, ic, kind, seed
                 e.stage, e.has_mu, e.method, e.pc, e.pf = 4 * l + stage, has_mu, method, pc_v, pf_v
                 e.desc, e.image = blob.desc, blob.to_device(device)
                 e.mu_desc, e.mu_image = (mu_blob.desc, mu_blob.to_device(device)) if has_mu else (None, None)
                 act_seed = inputs.seed_of(tag, "act", l, name)
+                nb = batch * ic * 2
                 if has_mu:
                     x, xp = inputs.gen_activation_pair(act_seed, batch, ic, n_outliers)
-                    e.xprev = torch.from_numpy(xp.astype(np.float16)).to(device)
+                    act_np[po:po + nb] = xp.astype(np.float16).reshape(-1).view(np.uint8)
+                    e.xprev = self.act_arena[po:po + nb].view(torch.float16).view(batch, ic)
                 else:
                     x = inputs.gen_activation(act_seed, batch, ic, n_outliers)
                     e.xprev = None
-                e.x = torch.from_numpy(x.astype(np.float16)).to(device)
-                e.y = torch.zeros((batch, oc), dtype=torch.float32, device=device)
+                act_np[xo:xo + nb] = x.astype(np.float16).reshape(-1).view(np.uint8)
+                e.x = self.act_arena[xo:xo + nb].view(torch.float16).view(batch, ic)
+                e.y = self.y_arena[yo:yo + batch * oc * 4].view(torch.float32).view(batch, oc)
+                e.act_off = (xo, po, yo)
                 self.ops.append(e)
+        self.act_arena.copy_(self.act_host)
         self.ops.sort(key=lambda o: o.stage)
         self.setup_seconds["upload"] = time.time() - t0
         self._packed = packed  # keeps the host blobs (logical codes) for parity checks
@@ -166,6 +194,14 @@ class Stack:
         if self._plan is None:
             self.plan_step()
         B.rwkvq_step_run(self._plan, stream)
+        return 1
+
+    def run_step_host(self, stream=None):
+        """The step with its activations read from and its outputs written to pinned host memory
+        (rwkvq_step_run_host); the caller synchronizes before reading self.y_host."""
+        if self._plan is None:
+            self.plan_step()
+        B.rwkvq_step_run_host(self._plan, self.act_host, self.act_arena, self.y_arena, self.y_host, stream)
         return 1
 
 

@@ -8,26 +8,9 @@ from paper_2505_03803_b200 import binding as B
 from paper_2505_03803_b200 import inputs
 
 
-def random_sq_codes(seed, oc, ic):
-    rng = np.random.default_rng(seed)
-    q = rng.integers(0, 8, size=(oc, ic), dtype=np.uint8)
-    s = (rng.random((oc, ic // 128)) * 0.02 + 0.005).astype(np.float16)
-    z = rng.integers(0, 8, size=(oc, ic // 128)).astype(np.float16)
-    return dict(q=q, scale=s, zero=z)
-
-
-def random_vq_codes(seed, oc, ic, bits):
-    rng = np.random.default_rng(seed)
-    E = 1 << bits
-    idx = rng.integers(0, E, size=(oc, ic // 2), dtype=np.uint8)
-    cb = (rng.standard_normal((oc // 256, ic // 256, E, 2)) * 0.02).astype(np.float16)
-    return dict(q=idx, codebook=cb)
-
-
-def random_mu_codes(seed, ic, bits=6):
-    rng = np.random.default_rng(seed)
-    E = 1 << bits
-    return dict(q=rng.integers(0, E, size=(ic // 2,), dtype=np.uint8), codebook=rng.random((E, 2)).astype(np.float16))
+random_sq_codes = inputs.random_sq_codes
+random_vq_codes = inputs.random_vq_codes
+random_mu_codes = inputs.random_mu_codes
 
 
 def decode(codes, method):
