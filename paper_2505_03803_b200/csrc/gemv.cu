@@ -42,10 +42,9 @@ __global__ void __launch_bounds__(256, 2) gemv_kernel(const GemvArgs a) {
       if (kt + 1 < kt1) nxt.load(rec + (size_t)(kt + 1 - kt0) * 8 * RWKVQ_SQ_RECORD_BYTES, lane);
       uint32_t w[12];
       cur.words(w);
-      XView xv;
-      xv.x = smem + (size_t)(kt - kt0) * 512; xv.xstride = L.xstride; xv.B = a.B; xv.nbp = 16;
-      xv.gs = reinterpret_cast<const float*>(smem + L.gs_off) + (size_t)(kt - kt0) * 2 * 3 * 16;
-      sq_record_mma<NB>(w, cur.sz, xv, lane, acc[0]);
+      const XLane xl = make_xlane(smem + (size_t)(kt - kt0) * 512, L.xstride,
+                                  reinterpret_cast<const float*>(smem + L.gs_off) + (size_t)(kt - kt0) * 2 * 3 * 16, 16, a.B, lane);
+      sq_record_mma<NB>(w, cur.sz, xl, acc[0]);
       cur = nxt;
     }
   } else {
@@ -64,9 +63,8 @@ __global__ void __launch_bounds__(256, 2) gemv_kernel(const GemvArgs a) {
         const uint8_t* rec = a.payload + ((size_t)((2 * rb + r) * a.KT + kt) * 8 + warp) * RBYTES;
         VqRecord<BITS> v;
         v.load(rec, lane);
-        XView xv;
-        xv.x = smem + (size_t)(kt - kt0) * 512; xv.xstride = L.xstride; xv.B = a.B; xv.nbp = 16; xv.gs = nullptr;
-        vq_record_mma<BITS, NB>(v.w, cb_lane, xv, lane, acc[r]);
+        const XLane xl = make_xlane(smem + (size_t)(kt - kt0) * 512, L.xstride, nullptr, 16, a.B, lane);
+        vq_record_mma<BITS, NB>(v.w, cb_lane, xl, acc[r]);
       }
     }
   }

@@ -132,22 +132,29 @@ __device__ __forceinline__ void stage_input(uint8_t* smem, const SmemLayout& L, 
   }
 }
 
-// View of the staged input for one 256-column tile: `x` points at the tile's first column of
-// batch row 0 (rows are `xstride` bytes apart), `gs` at the sums of the tile's first group, laid
-// out [group][3][nbp] floats (Sx, Bx_0, Bx_1 per batch row).
-struct XView {
-  const uint8_t* x;
-  const float* gs;
-  uint32_t xstride, nbp;
-  int B;
+// Per-lane view of the staged input for one 256-column tile.  Lane (g, t) of a warp reads, for
+// tensor-core step j and batch block n, the 8 bytes x_mix[8n + g][16j + 4t .. +3]; `x[n]` points at
+// step 0 of that row, so a fragment is one 64-bit load at a compile-time offset.  Batch rows beyond
+// B are clamped to row B-1: the tensor core then computes values for batch columns that do not
+// exist, which are never stored.  `gs` points at the sums (Sx, Bx_0, Bx_1) of the tile's first group
+// for batch columns 2t, 2t+1; the three rows are `gstride` bytes apart and groups 3*gstride.
+struct XLane {
+  const uint8_t* x[2];
+  const uint8_t* gs;
+  uint32_t gstride;
 };
 
-// B fragment of tensor-core step j for batch block nb: 8 contiguous bytes.
-__device__ __forceinline__ uint2 x_frag(const XView& xv, int j, int nb, int lane) {
-  const int b = nb * 8 + (lane >> 2);
-  uint2 v = make_uint2(0u, 0u);
-  if (b < xv.B) v = *reinterpret_cast<const uint2*>(xv.x + (size_t)b * xv.xstride + (size_t)(16 * j + 4 * (lane & 3)) * 2);
-  return v;
+// xtile: first column of the tile in batch row 0; rows `xstride` bytes apart.  gs_tile: sums of the
+// tile's first group, laid out [group][3][nbp] floats.
+__device__ __forceinline__ XLane make_xlane(const uint8_t* xtile, uint32_t xstride, const float* gs_tile, uint32_t nbp,
+                                            int B, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  XLane xl;
+  xl.x[0] = xtile + (size_t)min(g, B - 1) * xstride + t * 8;
+  xl.x[1] = xtile + (size_t)min(8 + g, B - 1) * xstride + t * 8;
+  xl.gs = reinterpret_cast<const uint8_t*>(gs_tile) + t * 8;
+  xl.gstride = nbp * 4u;
+  return xl;
 }
 
 struct SqRecord {
@@ -177,12 +184,11 @@ struct SqRecord {
 //   y[b][row] += s * ( sum_cols (q+bias) x  -  Bx_h  -  z * Sx )
 // The inner sum is eight m16n8k16 steps with fp32 accumulation in the tensor core; the bias each
 // extracted half carries is removed with the precomputed Bx_h.  `w` holds the group's six words
-// (two triples), `sz_lo` / `sz_hi` the (s, z) fp16 pairs of rows g and g+8; `xv.x` points at the
-// group's first column and `xv.gs` at the group's sums.
-template <int NB>
-__device__ __forceinline__ void sq_group_mma(const uint32_t (&w)[6], uint32_t sz_lo, uint32_t sz_hi, const XView& xv,
-                                             int lane, float (&acc)[NB][4]) {
-  const int t = lane & 3;
+// (two triples), `sz_lo` / `sz_hi` the (s, z) fp16 pairs of rows g and g+8.  GRP selects the
+// 128-column half of the tile `xl` describes.
+template <int NB, int GRP>
+__device__ __forceinline__ void sq_group_mma(const uint32_t (&w)[6], uint32_t sz_lo, uint32_t sz_hi, const XLane& xl,
+                                             float (&acc)[NB][4]) {
   float c[NB][4];
 #pragma unroll
   for (int n = 0; n < NB; ++n) c[n][0] = c[n][1] = c[n][2] = c[n][3] = 0.f;
@@ -195,21 +201,19 @@ __device__ __forceinline__ void sq_group_mma(const uint32_t (&w)[6], uint32_t sz
       const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
 #pragma unroll
       for (int n = 0; n < NB; ++n) {
-        const uint2 bf = x_frag(xv, 4 * ti + m, n, lane);
+        const uint2 bf = *reinterpret_cast<const uint2*>(xl.x[n] + GRP * 256 + (4 * ti + m) * 32);
         mma_16816(c[n], afrag, bf.x, bf.y);
       }
     }
   }
   const float2 sz0 = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));
   const float2 sz1 = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));
+  const uint8_t* gsp = xl.gs + (size_t)(GRP * 3) * xl.gstride;
 #pragma unroll
   for (int n = 0; n < NB; ++n) {
-    float2 sx = make_float2(0.f, 0.f), b0 = sx, b1 = sx;
-    if (n * 8 + 2 * t < xv.B) {   // nbp is even, so the pair is always inside the table
-      sx = *reinterpret_cast<const float2*>(xv.gs + n * 8 + 2 * t);
-      b0 = *reinterpret_cast<const float2*>(xv.gs + xv.nbp + n * 8 + 2 * t);
-      b1 = *reinterpret_cast<const float2*>(xv.gs + 2 * xv.nbp + n * 8 + 2 * t);
-    }
+    const float2 sx = *reinterpret_cast<const float2*>(gsp + n * 32);
+    const float2 b0 = *reinterpret_cast<const float2*>(gsp + xl.gstride + n * 32);
+    const float2 b1 = *reinterpret_cast<const float2*>(gsp + 2 * xl.gstride + n * 32);
     acc[n][0] = fmaf(sz0.x, fmaf(-sz0.y, sx.x, c[n][0] - b0.x), acc[n][0]);
     acc[n][1] = fmaf(sz0.x, fmaf(-sz0.y, sx.y, c[n][1] - b0.y), acc[n][1]);
     acc[n][2] = fmaf(sz1.x, fmaf(-sz1.y, sx.x, c[n][2] - b1.x), acc[n][2]);
@@ -219,16 +223,12 @@ __device__ __forceinline__ void sq_group_mma(const uint32_t (&w)[6], uint32_t sz
 
 // A whole SQ record (16 rows x 256 columns): its two groups in turn.
 template <int NB>
-__device__ __forceinline__ void sq_record_mma(const uint32_t (&w)[12], const uint4 sz, const XView& xv, int lane,
+__device__ __forceinline__ void sq_record_mma(const uint32_t (&w)[12], const uint4 sz, const XLane& xl,
                                               float (&acc)[NB][4]) {
-#pragma unroll
-  for (int grp = 0; grp < 2; ++grp) {
-    const uint32_t wg[6] = {w[6 * grp], w[6 * grp + 1], w[6 * grp + 2], w[6 * grp + 3], w[6 * grp + 4], w[6 * grp + 5]};
-    XView gv = xv;
-    gv.x = xv.x + grp * 256;                       // 128 columns of fp16
-    gv.gs = xv.gs + (size_t)(grp * 3) * xv.nbp;
-    sq_group_mma<NB>(wg, grp == 0 ? sz.x : sz.y, grp == 0 ? sz.z : sz.w, gv, lane, acc);
-  }
+  const uint32_t w0[6] = {w[0], w[1], w[2], w[3], w[4], w[5]};
+  const uint32_t w1[6] = {w[6], w[7], w[8], w[9], w[10], w[11]};
+  sq_group_mma<NB, 0>(w0, sz.x, sz.z, xl, acc);
+  sq_group_mma<NB, 1>(w1, sz.y, sz.w, xl, acc);
 }
 
 template <int BITS>
@@ -261,8 +261,8 @@ __device__ __forceinline__ void stage_codebook(uint8_t* dst, const uint32_t* src
 // One VQ record: every fragment register is one codebook lookup (a 2-D vector is exactly the
 // (even, odd) column pair a fragment register holds).
 template <int BITS, int NB, int JBEG = 0, int JEND = 16>
-__device__ __forceinline__ void vq_record_mma(const uint32_t (&w)[2 * BITS], const uint32_t* cb_lane, const XView& xv,
-                                              int lane, float (&acc)[NB][4]) {
+__device__ __forceinline__ void vq_record_mma(const uint32_t (&w)[2 * BITS], const uint32_t* cb_lane, const XLane& xl,
+                                              float (&acc)[NB][4]) {
 #pragma unroll
   for (int j = JBEG; j < JEND; ++j) {
     uint32_t afrag[4];
@@ -270,7 +270,7 @@ __device__ __forceinline__ void vq_record_mma(const uint32_t (&w)[2 * BITS], con
     for (int R = 0; R < 4; ++R) afrag[R] = cb_lane[vq_index<BITS, 2 * BITS>(w, 4 * j + R) * 32u];
 #pragma unroll
     for (int n = 0; n < NB; ++n) {
-      const uint2 bf = x_frag(xv, j, n, lane);
+      const uint2 bf = *reinterpret_cast<const uint2*>(xl.x[n] + j * 32);
       mma_16816(acc[n], afrag, bf.x, bf.y);
     }
   }

@@ -53,7 +53,10 @@ static_assert(sizeof(StepUnit) == 128, "unit descriptor size");
 
 struct StepXSeg {            // 64 bytes
   uint64_t x, xprev, mu, mu_aux;
-  uint32_t ic, col0, ncols, mu_bits, mu_entries, sums, barrier, xstride;   // barrier: index + 1 of the stage barrier to pass first
+  uint32_t ic, col0, ncols;
+  uint16_t mu_bits, mu_entries;
+  uint32_t sums, barrier, xstride;   // barrier: index + 1 of the stage barrier to pass first
+  uint32_t mu_off;                   // offset of the decoded mu row inside the buffer
 };
 static_assert(sizeof(StepXSeg) == 64, "segment descriptor size");
 
@@ -126,9 +129,16 @@ __device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred) {
                : "=r"(r) : "r"((uint32_t)pred), "r"(id), "r"(nthreads) : "memory");
   return r != 0;
 }
-__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+// Packed weights are read exactly once per step: they are marked evict-first so that streaming
+// them does not push the activations, the plan and the outputs out of L2.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
@@ -155,6 +165,7 @@ __device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint
   const uint4* base = reinterpret_cast<const uint4*>(a.units);
   const uint32_t n = u1 - u0;
   volatile int* abortp = &ctrl->abort_flag;
+  const uint64_t policy = policy_evict_first();
   uint4 next = make_uint4(0, 0, 0, 0);
   if ((uint32_t)(lane >> 3) < n) next = __ldg(base + (size_t)(u0 + (lane >> 3)) * 8 + (lane & 7));
   uint32_t issued = 0;
@@ -188,9 +199,9 @@ __device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint
         } else {
           mbar_arrive_expect_tx(full, tx);
           uint8_t* data = sl + 128;
-          if (by0) bulk_g2s(data, reinterpret_cast<const void*>(((uint64_t)s0h << 32) | s0l), by0, full);
-          if (by1) bulk_g2s(data + by0, reinterpret_cast<const void*>(((uint64_t)s1h << 32) | s1l), by1, full);
-          if (cbb) bulk_g2s(data + by0 + by1, reinterpret_cast<const void*>(((uint64_t)cbh << 32) | cbl), cbb, full);
+          if (by0) bulk_g2s(data, reinterpret_cast<const void*>(((uint64_t)s0h << 32) | s0l), by0, full, policy);
+          if (by1) bulk_g2s(data + by0, reinterpret_cast<const void*>(((uint64_t)s1h << 32) | s1l), by1, full, policy);
+          if (cbb) bulk_g2s(data + by0 + by1, reinterpret_cast<const void*>(((uint64_t)cbh << 32) | cbl), cbb, full, policy);
         }
       }
       ++issued;
@@ -209,16 +220,74 @@ __device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint
 }
 
 // Stagers: x_mix and, for SQ, the per-group sums of the segment, into buffer (segment index & 1).
+// Everything that does not depend on the previous stage -- the decoded token-shift vector mu_hat
+// and the previous token's activations -- is put into shared memory BEFORE the stage barrier, so
+// that only one round of vector loads of x, the mix and the sums remain behind it.
+// A thread owns 8 consecutive columns (16 bytes) of one batch row; a half-warp owns one
+// 128-column group, whose three sums it reduces with shuffles.
+__device__ __forceinline__ uint32_t mix2(uint32_t xr, uint32_t pr, uint32_t mr) {
+  const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xr));
+  const float2 pf = __half22float2(*reinterpret_cast<const __half2*>(&pr));
+  const float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mr));
+  const __half2 v = __floats2half2_rn(fmaf(pf.x - xf.x, mf.x, xf.x), fmaf(pf.y - xf.y, mf.y, xf.y));
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ float pair_sum(uint32_t r) {
+  const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r));
+  return f.x + f.y;
+}
+
+constexpr int kStageUnroll = 4;
+
 __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_t* xbufs, uint32_t* mucb,
                             uint32_t s0, uint32_t s1) {
   const int stid = threadIdx.x - kConsumerThreads;
-  const int lane = stid & 31, warp = stid >> 5;
+  const int lane = stid & 31;
   volatile int* abortp = &ctrl->abort_flag;
   for (uint32_t si = s0; si < s1; ++si) {
     const uint32_t li = si - s0;
     const int buf = (int)(li & 1u);
     const StepXSeg sg = *reinterpret_cast<const StepXSeg*>(reinterpret_cast<const uint8_t*>(a.xsegs) + (size_t)si * 64);
     bool ok = mbar_wait_warp(&ctrl->xempty[buf], ((li >> 1) & 1u) ^ 1u, abortp, a.status);
+    uint8_t* xb = xbufs + (size_t)buf * kXBufBytes;
+    const uint8_t* mu = reinterpret_cast<const uint8_t*>(sg.mu);
+    const __half* x = reinterpret_cast<const __half*>(sg.x);
+    const __half* xp = reinterpret_cast<const __half*>(sg.xprev);
+    const int nvr = (int)sg.ncols >> 3;            // 16-byte vectors per batch row
+    const int total = a.B * nvr;
+    const int nbp = (a.B + 1) & ~1;
+    uint8_t* murow = xb + sg.mu_off;
+    if (ok && mu) {
+      for (int e = stid; e < (int)sg.mu_entries; e += kStagerThreads) mucb[e] = __ldg(reinterpret_cast<const uint32_t*>(sg.mu_aux) + e);
+      named_bar_sync(4, kStagerThreads);
+      const int bits = (int)sg.mu_bits;
+      const uint32_t mask = (1u << bits) - 1u;
+      for (int c8 = stid; c8 < nvr; c8 += kStagerThreads) {
+        const int col = (int)sg.col0 + 8 * c8;
+        uint4 m = make_uint4(0u, 0u, 0u, 0u);
+        if (col < (int)sg.ic) {
+          // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
+          const uint32_t byte = (uint32_t)(col >> 1) * (uint32_t)bits >> 3;
+          const uint32_t* w = reinterpret_cast<const uint32_t*>(mu) + (byte >> 2);
+          const uint32_t sh = (byte & 3u) * 8u;
+          const uint32_t lo = __ldg(w);
+          const uint32_t hi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+          const uint32_t f = __funnelshift_r(lo, hi, sh);
+          m.x = mucb[f & mask];
+          m.y = mucb[(f >> bits) & mask];
+          m.z = mucb[(f >> (2 * bits)) & mask];
+          m.w = mucb[(f >> (3 * bits)) & mask];
+        }
+        *reinterpret_cast<uint4*>(murow + (size_t)c8 * 16) = m;
+      }
+      for (int v = stid; v < total; v += kStagerThreads) {
+        const int b = v / nvr, c8 = v - b * nvr;
+        const int col = (int)sg.col0 + 8 * c8;
+        uint4 r = make_uint4(0u, 0u, 0u, 0u);
+        if (col < (int)sg.ic) r = __ldg(reinterpret_cast<const uint4*>(xp + (size_t)b * sg.ic + col));
+        *reinterpret_cast<uint4*>(xb + (size_t)b * sg.xstride + (size_t)c8 * 16) = r;
+      }
+    }
     if (ok && sg.barrier && stid == 0) {
       // grid-wide stage barrier: every CTA has finished (and published) the previous stage.  Each
       // barrier has its own arrival counter, so a CTA without work may run ahead and arrive at
@@ -226,64 +295,54 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       uint32_t it = 0;
       while ((int)(ld_acquire_gpu(a.counter + (sg.barrier - 1u)) - a.target) < 0) {
         if (++it >= kPollLimit || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
-        __nanosleep(20);
       }
     }
     if (!named_bar_and(4, kStagerThreads, ok)) return;   // all stager threads leave together
-    uint8_t* xb = xbufs + (size_t)buf * kXBufBytes;
-    const uint8_t* mu = reinterpret_cast<const uint8_t*>(sg.mu);
-    if (mu) {
-      for (int e = stid; e < (int)sg.mu_entries; e += kStagerThreads) mucb[e] = __ldg(reinterpret_cast<const uint32_t*>(sg.mu_aux) + e);
-      named_bar_sync(4, kStagerThreads);
-    }
-    const __half* x = reinterpret_cast<const __half*>(sg.x);
-    const __half* xp = reinterpret_cast<const __half*>(sg.xprev);
-    const int npairs = (int)sg.ncols / 2;
-    for (int p = stid; p < a.B * npairs; p += kStagerThreads) {
-      const int b = p / npairs, cp = p - b * npairs;
-      const int col = (int)sg.col0 + 2 * cp;
-      uint32_t raw = 0u;
-      if (col < (int)sg.ic) {
-        raw = __ldcg(reinterpret_cast<const unsigned*>(x + (size_t)b * sg.ic + col));
-        if (mu) {
-          const uint32_t rawp = __ldcg(reinterpret_cast<const unsigned*>(xp + (size_t)b * sg.ic + col));
-          const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&raw));
-          const float2 pf = __half22float2(*reinterpret_cast<const __half2*>(&rawp));
-          const uint32_t mw = mucb[vector_index(mu, col >> 1, (int)sg.mu_bits)];
-          const float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw));
-          const __half2 v = __floats2half2_rn(fmaf(pf.x - xf.x, mf.x, xf.x), fmaf(pf.y - xf.y, mf.y, xf.y));
-          raw = *reinterpret_cast<const uint32_t*>(&v);
+    float* gs = reinterpret_cast<float*>(xb + (size_t)a.B * sg.xstride);
+    for (int v0 = stid; v0 < total; v0 += kStagerThreads * kStageUnroll) {
+      uint4 raw[kStageUnroll];
+#pragma unroll
+      for (int u = 0; u < kStageUnroll; ++u) {
+        const int v = v0 + u * kStagerThreads;
+        raw[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (v < total) {
+          const int b = v / nvr, c8 = v - b * nvr;
+          const int col = (int)sg.col0 + 8 * c8;
+          if (col < (int)sg.ic) raw[u] = __ldcg(reinterpret_cast<const uint4*>(x + (size_t)b * sg.ic + col));
         }
       }
-      *reinterpret_cast<uint32_t*>(xb + (size_t)b * sg.xstride + (size_t)cp * 4) = raw;
-    }
-    named_bar_sync(4, kStagerThreads);
-    if (sg.sums) {
-      const int ngroups = (int)sg.ncols / 128;
-      const int nbp = (a.B + 1) & ~1;
-      float* gs = reinterpret_cast<float*>(xb + (size_t)a.B * sg.xstride);
-      const int o = (lane * 4) & 63;
-      const float b00 = (float)rwkvq_sq_bias(o, 0), b02 = (float)rwkvq_sq_bias(o + 2, 0);
-      const float b10 = (float)rwkvq_sq_bias(o, 1), b12 = (float)rwkvq_sq_bias(o + 2, 1);
-      for (int task = warp; task < ngroups * a.B; task += kStagerWarps) {
-        const int grp = task / a.B, b = task - grp * a.B;
-        const uint2 raw = *reinterpret_cast<const uint2*>(xb + (size_t)b * sg.xstride + (size_t)(grp * 128 + lane * 4) * 2);
-        const float2 x01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-        const float2 x23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
-        const float p01 = x01.x + x01.y, p23 = x23.x + x23.y;
-        float sx = p01 + p23;
-        float t0 = fmaf(b00, p01, b02 * p23);
-        float t1 = fmaf(b10, p01, b12 * p23);
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-          sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
-          t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
-          t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+      for (int u = 0; u < kStageUnroll; ++u) {
+        const int v = v0 + u * kStagerThreads;
+        if (v >= total) break;                      // warp-uniform: total is a multiple of 32
+        const int b = v / nvr, c8 = v - b * nvr;
+        uint4 r = raw[u];
+        uint8_t* dst = xb + (size_t)b * sg.xstride + (size_t)c8 * 16;
+        if (mu) {
+          const uint4 pr = *reinterpret_cast<const uint4*>(dst);          // this thread's own earlier store
+          const uint4 mr = *reinterpret_cast<const uint4*>(murow + (size_t)c8 * 16);
+          r.x = mix2(r.x, pr.x, mr.x); r.y = mix2(r.y, pr.y, mr.y);
+          r.z = mix2(r.z, pr.z, mr.z); r.w = mix2(r.w, pr.w, mr.w);
         }
-        if (lane == 0) {
-          gs[(grp * 3 + 0) * nbp + b] = sx;
-          gs[(grp * 3 + 1) * nbp + b] = t0;
-          gs[(grp * 3 + 2) * nbp + b] = t1;
+        *reinterpret_cast<uint4*>(dst) = r;
+        if (sg.sums) {
+          const int o = (8 * c8) & 63;
+          const float pa = pair_sum(r.x) + pair_sum(r.z), pb = pair_sum(r.y) + pair_sum(r.w);
+          float sx = pa + pb;
+          float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
+          float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
+#pragma unroll
+          for (int d = 8; d > 0; d >>= 1) {
+            sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+            t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
+            t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+          }
+          if ((lane & 15) == 0) {
+            const int grp = c8 >> 4;
+            gs[(grp * 3 + 0) * nbp + b] = sx;
+            gs[(grp * 3 + 1) * nbp + b] = t0;
+            gs[(grp * 3 + 2) * nbp + b] = t1;
+          }
         }
       }
     }
@@ -326,8 +385,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
     }
     const uint8_t* data = sl + 128;
     const uint8_t* xb = xbufs + (size_t)xcur * kXBufBytes;
-    XView xv;
-    xv.xstride = u->xstride; xv.nbp = u->nbp; xv.B = a.B;
+    const uint32_t xstride = u->xstride, nbp = u->nbp;
     if (dead) {
       if (fmt == UFMT_VQ6 || fmt == UFMT_VQ8) { named_bar_sync(1, kConsumerThreads); named_bar_sync(1, kConsumerThreads); }
     } else if (fmt == UFMT_SQ) {
@@ -339,9 +397,8 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
         uint32_t w[12];
         r.words(w);
         const uint32_t col = u->xcol0 + (uint32_t)half * 256u;
-        xv.x = xb + (size_t)col * 2;
-        xv.gs = gs0 + (size_t)(col >> 7) * 3 * xv.nbp;
-        sq_record_mma<NB>(w, r.sz, xv, lane, acc);
+        const XLane xl = make_xlane(xb + (size_t)col * 2, xstride, gs0 + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
+        sq_record_mma<NB>(w, r.sz, xl, acc);
       } else {
         // single chunk: the two halves take one 128-column group each
         const uint8_t* rp = data + (size_t)rec * RWKVQ_SQ_RECORD_BYTES;
@@ -353,9 +410,8 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
         }
         const uint4 sz = *reinterpret_cast<const uint4*>(rp + RWKVQ_SQ_CODE_BYTES + g * 16);
         const uint32_t col = u->xcol0 + (uint32_t)half * 128u;
-        xv.x = xb + (size_t)col * 2;
-        xv.gs = gs0 + (size_t)(col >> 7) * 3 * xv.nbp;
-        sq_group_mma<NB>(w, half == 0 ? sz.x : sz.y, half == 0 ? sz.z : sz.w, xv, lane, acc);
+        const XLane xl = make_xlane(xb + (size_t)col * 2, xstride, gs0 + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
+        sq_group_mma<NB, 0>(w, half == 0 ? sz.x : sz.y, half == 0 ? sz.z : sz.w, xl, acc);
       }
     } else if (fmt == UFMT_VQ6 || fmt == UFMT_VQ8) {
       // replicate the tile's codebook for conflict-free lookups (all consumer warps take part)
@@ -368,30 +424,29 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
       }
       named_bar_sync(1, kConsumerThreads);
       const uint32_t* cb_lane = reinterpret_cast<const uint32_t*>(replicas) + lane;
-      xv.x = xb + (size_t)u->xcol0 * 2;
-      xv.gs = nullptr;
+      const XLane xl = make_xlane(xb + (size_t)u->xcol0 * 2, xstride, nullptr, nbp, a.B, lane);
       if (!(flags & UF_SPLIT)) {
         // warp (rec, half): record `rec` of chunk `half` (chunk B = the next 128 rows, same columns)
         if (fmt == UFMT_VQ6) {
           VqRecord<6> r;
           r.load_shared(data + (size_t)half * by0 + (size_t)rec * 1536, lane);
-          vq_record_mma<6, NB>(r.w, cb_lane, xv, lane, acc);
+          vq_record_mma<6, NB>(r.w, cb_lane, xl, acc);
         } else {
           VqRecord<8> r;
           r.load_shared(data + (size_t)half * by0 + (size_t)rec * 2048, lane);
-          vq_record_mma<8, NB>(r.w, cb_lane, xv, lane, acc);
+          vq_record_mma<8, NB>(r.w, cb_lane, xl, acc);
         }
       } else {
         if (fmt == UFMT_VQ6) {
           VqRecord<6> r;
           r.load_shared(data + (size_t)rec * 1536, lane);
-          if (half == 0) vq_record_mma<6, NB, 0, 8>(r.w, cb_lane, xv, lane, acc);
-          else vq_record_mma<6, NB, 8, 16>(r.w, cb_lane, xv, lane, acc);
+          if (half == 0) vq_record_mma<6, NB, 0, 8>(r.w, cb_lane, xl, acc);
+          else vq_record_mma<6, NB, 8, 16>(r.w, cb_lane, xl, acc);
         } else {
           VqRecord<8> r;
           r.load_shared(data + (size_t)rec * 2048, lane);
-          if (half == 0) vq_record_mma<8, NB, 0, 8>(r.w, cb_lane, xv, lane, acc);
-          else vq_record_mma<8, NB, 8, 16>(r.w, cb_lane, xv, lane, acc);
+          if (half == 0) vq_record_mma<8, NB, 0, 8>(r.w, cb_lane, xl, acc);
+          else vq_record_mma<8, NB, 8, 16>(r.w, cb_lane, xl, acc);
         }
       }
     }
@@ -428,7 +483,8 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
         float* z = reinterpret_cast<float*>(zp[k]);
         for (uint32_t e = threadIdx.x; e < (dead ? 0u : zc[k]); e += kConsumerThreads) z[e] = 0.f;
       }
-      __threadfence();
+      // The named barrier orders every consumer thread's stores and reductions before thread 0's
+      // fence, which is cumulative: one fence publishes the whole CTA's share of the stage.
       named_bar_sync(2, kConsumerThreads);
       if (threadIdx.x == 0) { __threadfence(); atomicAdd(a.counter + (flags >> 16), 1u); }
     }
@@ -483,10 +539,16 @@ struct HostUnit {
   uint32_t bytes;
 };
 
-static uint32_t xseg_bytes(int B, int ncols, bool sums) {
+// Shared-memory footprint of an input segment: B rows of x_mix, the per-group sums (SQ) and one
+// row of decoded mu_hat (products with a token shift).
+static uint32_t xseg_mu_off(int B, int ncols, bool sums) {
   uint32_t xstride = (uint32_t)ncols * 2u + 32u;
   uint32_t nbp = (uint32_t)((B + 1) & ~1);
-  return (uint32_t)B * xstride + (sums ? (uint32_t)(ncols / 128) * 3u * nbp * 4u : 0u);
+  uint32_t off = (uint32_t)B * xstride + (sums ? (uint32_t)(ncols / 128) * 3u * nbp * 4u : 0u);
+  return (off + 15u) & ~15u;
+}
+static uint32_t xseg_bytes(int B, int ncols, bool sums, bool has_mu) {
+  return xseg_mu_off(B, ncols, sums) + (has_mu ? (uint32_t)ncols * 2u : 0u);
 }
 
 static rwkvq_status validate_ops(const rwkvq_gemv_op* ops, int n_ops, int B) {
@@ -664,29 +726,31 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       if (L[i].u.fmt == UFMT_EMPTY) { ++i; continue; }
       const int op = L[i].op;
       const bool sums = ops[op].W_desc.method == RWKVQ_SQ;
+      const bool has_mu = ops[op].mu_image_dev != nullptr;
       int kmin = L[i].kt, kmax = L[i].kt + L[i].ntiles;
       size_t j = i + 1, last = i;
       while (j < n) {
         if (L[j].u.fmt == UFMT_EMPTY) { if (L[j].stage != L[i].stage) break; ++j; continue; }
         if (L[j].op != op || L[j].stage != L[i].stage) break;
         const int nmin = std::min(kmin, L[j].kt), nmax = std::max(kmax, L[j].kt + L[j].ntiles);
-        if (xseg_bytes(B, (nmax - nmin) * 256, sums) > kXBufBytes) break;
+        if (xseg_bytes(B, (nmax - nmin) * 256, sums, has_mu) > kXBufBytes) break;
         kmin = nmin; kmax = nmax; last = j; ++j;
       }
       const int ncols = (kmax - kmin) * 256;
-      if (xseg_bytes(B, ncols, sums) > kXBufBytes) return RWKVQ_EUNSUPPORTED;
+      if (xseg_bytes(B, ncols, sums, has_mu) > kXBufBytes) return RWKVQ_EUNSUPPORTED;
       StepXSeg sg{};
       const rwkvq_gemv_op& o = ops[op];
       sg.x = (uint64_t)(uintptr_t)o.x_fp16_dev;
       sg.ic = (uint32_t)o.W_desc.ic; sg.col0 = (uint32_t)kmin * 256u; sg.ncols = (uint32_t)ncols;
       sg.sums = sums ? 1u : 0u; sg.xstride = (uint32_t)ncols * 2u + 32u;
+      sg.mu_off = xseg_mu_off(B, ncols, sums);
       sg.barrier = (uint32_t)L[i].stage + 1u;   // stage s reads its inputs after barrier s
       if (o.mu_image_dev) {
         const uint8_t* m = static_cast<const uint8_t*>(o.mu_image_dev);
         sg.xprev = (uint64_t)(uintptr_t)o.xprev_fp16_dev;
         sg.mu = (uint64_t)(uintptr_t)(m + RWKVQ_HEADER_BYTES);
         sg.mu_aux = (uint64_t)(uintptr_t)(m + vector_aux_offset(&o.mu_desc));
-        sg.mu_bits = (uint32_t)o.mu_desc.bits; sg.mu_entries = (uint32_t)o.mu_desc.entries;
+        sg.mu_bits = (uint16_t)o.mu_desc.bits; sg.mu_entries = (uint16_t)o.mu_desc.entries;
       }
       all_segs.push_back(sg);
       bool first = true;
