@@ -231,6 +231,71 @@ __device__ __forceinline__ void sq_record_mma(const uint32_t (&w)[12], const uin
   sq_group_mma<NB, 1>(w1, sz.y, sz.w, xl, acc);
 }
 
+// Two SQ records that cover the same 128 columns (rows r and r + 128 of a 256-row tile): every
+// input fragment is loaded once and used by both.  `wa` / `wb`: the group's six words of each
+// record; sza / szb: the records' (s, z) words {row g group 0, row g group 1, row g+8 group 0,
+// row g+8 group 1}.  has_b == false skips the second record (warp-uniform).
+template <int NB, int GRP>
+__device__ __forceinline__ void sq_group_mma2(const uint32_t (&wa)[6], const uint32_t (&wb)[6], const uint4 sza,
+                                              const uint4 szb, bool has_b, const XLane& xl, float (&acca)[NB][4],
+                                              float (&accb)[NB][4]) {
+  float ca[NB][4], cb[NB][4];
+#pragma unroll
+  for (int n = 0; n < NB; ++n) {
+    ca[n][0] = ca[n][1] = ca[n][2] = ca[n][3] = 0.f;
+    cb[n][0] = cb[n][1] = cb[n][2] = cb[n][3] = 0.f;
+  }
+#pragma unroll
+  for (int ti = 0; ti < 2; ++ti) {
+    uint2 bf[4][NB];
+#pragma unroll
+    for (int m = 0; m < 4; ++m)
+#pragma unroll
+      for (int n = 0; n < NB; ++n) bf[m][n] = *reinterpret_cast<const uint2*>(xl.x[n] + GRP * 256 + (4 * ti + m) * 32);
+    {
+      uint32_t r[16];
+      sq_unpack_triple(wa[3 * ti], wa[3 * ti + 1], wa[3 * ti + 2], r);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
+#pragma unroll
+        for (int n = 0; n < NB; ++n) mma_16816(ca[n], afrag, bf[m][n].x, bf[m][n].y);
+      }
+    }
+    if (has_b) {
+      uint32_t r[16];
+      sq_unpack_triple(wb[3 * ti], wb[3 * ti + 1], wb[3 * ti + 2], r);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
+#pragma unroll
+        for (int n = 0; n < NB; ++n) mma_16816(cb[n], afrag, bf[m][n].x, bf[m][n].y);
+      }
+    }
+  }
+  const uint32_t a_lo = GRP == 0 ? sza.x : sza.y, a_hi = GRP == 0 ? sza.z : sza.w;
+  const uint32_t b_lo = GRP == 0 ? szb.x : szb.y, b_hi = GRP == 0 ? szb.z : szb.w;
+  const float2 sa0 = __half22float2(*reinterpret_cast<const __half2*>(&a_lo));
+  const float2 sa1 = __half22float2(*reinterpret_cast<const __half2*>(&a_hi));
+  const float2 sb0 = __half22float2(*reinterpret_cast<const __half2*>(&b_lo));
+  const float2 sb1 = __half22float2(*reinterpret_cast<const __half2*>(&b_hi));
+  const uint8_t* gsp = xl.gs + (size_t)(GRP * 3) * xl.gstride;
+#pragma unroll
+  for (int n = 0; n < NB; ++n) {
+    const float2 sx = *reinterpret_cast<const float2*>(gsp + n * 32);
+    const float2 b0 = *reinterpret_cast<const float2*>(gsp + xl.gstride + n * 32);
+    const float2 b1 = *reinterpret_cast<const float2*>(gsp + 2 * xl.gstride + n * 32);
+    acca[n][0] = fmaf(sa0.x, fmaf(-sa0.y, sx.x, ca[n][0] - b0.x), acca[n][0]);
+    acca[n][1] = fmaf(sa0.x, fmaf(-sa0.y, sx.y, ca[n][1] - b0.y), acca[n][1]);
+    acca[n][2] = fmaf(sa1.x, fmaf(-sa1.y, sx.x, ca[n][2] - b1.x), acca[n][2]);
+    acca[n][3] = fmaf(sa1.x, fmaf(-sa1.y, sx.y, ca[n][3] - b1.y), acca[n][3]);
+    accb[n][0] = fmaf(sb0.x, fmaf(-sb0.y, sx.x, cb[n][0] - b0.x), accb[n][0]);
+    accb[n][1] = fmaf(sb0.x, fmaf(-sb0.y, sx.y, cb[n][1] - b0.y), accb[n][1]);
+    accb[n][2] = fmaf(sb1.x, fmaf(-sb1.y, sx.x, cb[n][2] - b1.x), accb[n][2]);
+    accb[n][3] = fmaf(sb1.x, fmaf(-sb1.y, sx.y, cb[n][3] - b1.y), accb[n][3]);
+  }
+}
+
 template <int BITS>
 struct VqRecord {
   static constexpr int NW = 2 * BITS;  // 64 indices of BITS bits = 2*BITS words per lane
@@ -272,6 +337,49 @@ __device__ __forceinline__ void vq_record_mma(const uint32_t (&w)[2 * BITS], con
     for (int n = 0; n < NB; ++n) {
       const uint2 bf = *reinterpret_cast<const uint2*>(xl.x[n] + j * 32);
       mma_16816(acc[n], afrag, bf.x, bf.y);
+    }
+  }
+}
+
+// Words [HALF * BITS, (HALF + 1) * BITS) of a lane's VQ stream (the indices of eight tensor-core
+// steps) from a record in shared memory; the other entries of `w` are left untouched.
+template <int BITS, int HALF>
+__device__ __forceinline__ void vq_half_words(const uint8_t* rec, int lane, uint32_t (&w)[2 * BITS]) {
+  if constexpr (BITS == 8) {
+    const uint4 p = *reinterpret_cast<const uint4*>(rec + (2 * HALF) * 512 + lane * 16);
+    const uint4 q = *reinterpret_cast<const uint4*>(rec + (2 * HALF + 1) * 512 + lane * 16);
+    w[8 * HALF + 0] = p.x; w[8 * HALF + 1] = p.y; w[8 * HALF + 2] = p.z; w[8 * HALF + 3] = p.w;
+    w[8 * HALF + 4] = q.x; w[8 * HALF + 5] = q.y; w[8 * HALF + 6] = q.z; w[8 * HALF + 7] = q.w;
+  } else if constexpr (HALF == 0) {
+    const uint4 p = *reinterpret_cast<const uint4*>(rec + lane * 16);
+    const uint2 q = *reinterpret_cast<const uint2*>(rec + 512 + lane * 16);
+    w[0] = p.x; w[1] = p.y; w[2] = p.z; w[3] = p.w; w[4] = q.x; w[5] = q.y;
+  } else {
+    const uint2 p = *reinterpret_cast<const uint2*>(rec + 512 + lane * 16 + 8);
+    const uint4 q = *reinterpret_cast<const uint4*>(rec + 1024 + lane * 16);
+    w[6] = p.x; w[7] = p.y; w[8] = q.x; w[9] = q.y; w[10] = q.z; w[11] = q.w;
+  }
+}
+
+// Eight tensor-core steps (HALF of the tile's columns) of two VQ records of one tile (rows r and
+// r + 128, same columns, same codebook): shared input fragments, eight lookups per step.
+template <int BITS, int NB, int HALF>
+__device__ __forceinline__ void vq_half_mma2(const uint32_t (&wa)[2 * BITS], const uint32_t (&wb)[2 * BITS],
+                                             const uint32_t* cb_lane, const XLane& xl, float (&acca)[NB][4],
+                                             float (&accb)[NB][4]) {
+#pragma unroll
+  for (int j = 8 * HALF; j < 8 * HALF + 8; ++j) {
+    uint32_t fa[4], fb[4];
+#pragma unroll
+    for (int R = 0; R < 4; ++R) {
+      fa[R] = cb_lane[vq_index<BITS, 2 * BITS>(wa, 4 * j + R) * 32u];
+      fb[R] = cb_lane[vq_index<BITS, 2 * BITS>(wb, 4 * j + R) * 32u];
+    }
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      const uint2 bf = *reinterpret_cast<const uint2*>(xl.x[n] + j * 32);
+      mma_16816(acca[n], fa, bf.x, bf.y);
+      mma_16816(accb[n], fb, bf.x, bf.y);
     }
   }
 }

@@ -5,21 +5,28 @@
 // 7B-class layer is only a few microseconds of HBM time.  Launching one kernel per projection
 // leaves the memory system idle between launches, so the step is ONE kernel with one CTA per SM:
 //
-//   * a producer thread streams packed chunks from HBM into a ring of shared-memory slots with
+//   * a producer warp streams packed weights from HBM into a ring of shared-memory slots with
 //     bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts).  Weights never depend
 //     on activations, so the stream runs ahead across products and across stage boundaries;
-//   * four stager warps build the fp16 input x_mix = x + (x_prev - x) (.) mu_hat (Appendix A.1
-//     Eq. 20) for the next run of chunks into one of two shared-memory buffers, after waiting on
-//     the grid-wide stage barrier when the run opens a new stage;
-//   * sixteen consumer warps turn records into m16n8k16 tensor-core steps (gemv_core.cuh),
-//     accumulate along K in registers and add their partial sums into y with fp32 atomics.
+//   * three stager warps build the fp16 input x_mix = x + (x_prev - x) (.) mu_hat (Appendix A.1
+//     Eq. 20) of the next run of units in one of two shared-memory buffers.  What does not depend
+//     on the previous stage (mu_hat, x_prev) is prepared before the grid-wide stage barrier; the
+//     stagers also clear the next stage's outputs and post this CTA's arrival at the barrier;
+//   * sixteen consumer warps in two groups of eight.  A unit is a 256-row x 256-column tile (two
+//     128-row chunks of the packed image); the groups take the CTA's units alternately, so one
+//     group computes while the other waits, flushes or synchronises.  Warp w of a group owns rows
+//     16w..16w+15 of both chunks and runs the m16n8k16 tensor-core steps of gemv_core.cuh with
+//     every input fragment shared by the two records.  Partial sums go to y with fp32 atomics at
+//     the end of a run along K.
 //
-// The host plans the step once: every stage's chunks are cut into units (two chunks = sixteen
-// records, one per consumer warp), dealt to the CTAs in contiguous byte-balanced ranges, and
-// written as a per-CTA list of 128-byte unit descriptors plus a list of input segments.
+// The host plans the step once: every stage's units are dealt to the CTAs in contiguous,
+// byte-balanced ranges cut at one eighth of a unit (one warp's records), and written as a per-CTA
+// list of 128-byte unit descriptors plus a list of 64-byte input events (segments and barrier
+// arrivals).
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstring>
 #include <mutex>
 #include <unordered_map>
 #include <vector>
@@ -33,51 +40,70 @@ namespace rwkvq {
 int* device_status_ptr();  // api_misc.cu
 unsigned abort_epoch();     // api_misc.cu: bumped whenever rwkvq_device_status reports a failed wait
 
-enum { UF_FLUSH = 1, UF_STAGE_END = 2, UF_NEW_XSEG = 4, UF_END_XSEG = 8, UF_SPLIT = 16 };
-// bits 16..31 of a unit's flags: index of the stage barrier a UF_STAGE_END unit arrives at
-enum { UFMT_SQ = 0, UFMT_VQ6 = 1, UFMT_VQ8 = 2, UFMT_EMPTY = 3 };
+enum { UF_FLUSH = 1, UF_VQ = 2, UF_BITS8 = 4 };
 
-struct StepUnit {            // 128 bytes; the first 48 bytes are all the producer needs
-  uint64_t src0, src1;       // global addresses of chunk A / chunk B (0 = absent)
+struct StepUnit {            // 128 bytes, copied into the slot header by the producer
+  uint64_t src0, src1;       // global addresses of the first copied record of chunk A / chunk B (0 = absent)
   uint64_t cb_src;           // VQ: codebook of the tile
-  uint32_t bytes0, bytes1;
-  uint32_t cb_bytes, flags, fmt, xcol0;   // xcol0: column of the unit's first tile inside the x segment
+  uint32_t bytes0, bytes1;   // bytes copied from each chunk: (w1 - w0) records
+  uint32_t cb_bytes;
+  uint32_t off0;             // w0 * record bytes: where the copied records sit inside a chunk
+  uint32_t flags;            // UF_* | w0 << 8 | w1 << 12: warps w0 <= w < w1 of the group have a record
+  uint32_t seg;              // number, within this CTA, of the input segment the unit reads
+  uint32_t stage;            // stage number (0-based)
+  uint32_t xcol0;            // column of the unit's tile inside the segment
   uint32_t row0, oc;         // first output row of chunk A; rows of the product
   uint64_t y;                // float y[B][oc]
-  uint32_t xstride, gs_off;  // geometry of the x segment: bytes between batch rows, offset of the sums
+  uint32_t xstride, gs_off;  // geometry of the segment: bytes between batch rows, offset of the sums
   uint32_t nbp, entries;
-  uint64_t zptr[4];          // float ranges to clear before this CTA arrives at the stage barrier
-  uint32_t zcount[4];
+  uint32_t chunk_bytes;      // distance between chunk A and chunk B inside the slot
+  uint32_t rec_bytes;
+  uint32_t ev_index;         // position of the unit's segment in this CTA's event list
+  uint32_t between_mask;     // events between the group's previous segment and this one, oldest in bit 0:
+                             // 1 = barrier arrival, 0 = segment of the other group (valid for up to 32 events)
+  uint32_t after_count;      // set on a group's last unit of a stage: events after its segment up to and
+  uint32_t after_mask;       // including the stage's barrier arrival, to be passed right after the unit
+  uint32_t pad[4];
 };
 static_assert(sizeof(StepUnit) == 128, "unit descriptor size");
 
-struct StepXSeg {            // 64 bytes
-  uint64_t x, xprev, mu, mu_aux;
-  uint32_t ic, col0, ncols;
-  uint16_t mu_bits, mu_entries;
-  uint32_t sums, barrier, xstride;   // barrier: index + 1 of the stage barrier to pass first
-  uint32_t mu_off;                   // offset of the decoded mu row inside the buffer
-};
-static_assert(sizeof(StepXSeg) == 64, "segment descriptor size");
+enum { EV_SEGMENT = 0, EV_ARRIVE = 1 };
 
-constexpr int kConsumerWarps = 16, kStagerWarps = 4;
+struct StepEvent {           // 64 bytes
+  union {
+    struct { uint64_t x, xprev, mu, mu_aux; } seg;
+    struct { uint64_t zptr[4]; } arr;          // float ranges to clear before arriving
+  };
+  union {
+    struct { uint32_t ic, col0, ncols; uint16_t mu_bits, mu_entries; } segd;
+    struct { uint32_t zcount[4]; } arrd;
+  };
+  uint32_t kind;             // EV_SEGMENT / EV_ARRIVE
+  uint32_t barrier;          // segment: index + 1 of the stage barrier to pass first; arrival: index of the barrier
+  uint32_t xstride_sums;     // segment: xstride | sums << 31
+  uint16_t mu_off16;         // segment: offset / 16 of the decoded mu row inside the buffer
+  uint16_t reserved;
+};
+static_assert(sizeof(StepEvent) == 64, "event descriptor size");
+
+constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGroups, kStagerWarps = 3;
 constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
+constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
 constexpr int kMaxSlots = 12;
-constexpr uint32_t kCtrlBytes = 1024, kXBufBytes = 32768, kMuScratch = 1024;
+constexpr uint32_t kCtrlBytes = 1024, kXBufBytes = 24576, kMuScratch = 1024;
 constexpr uint32_t kSmemLimit = 232448;  // 227 KB
-constexpr uint32_t kPollLimit = 1u << 24;
+constexpr uint32_t kPollLimit = 1u << 22;
 
 struct StepArgs {
   const StepUnit* units;
-  const StepXSeg* xsegs;
+  const StepEvent* events;
   const uint32_t* unit_off;   // [P+1]
-  const uint32_t* xseg_off;   // [P+1]
+  const uint32_t* event_off;  // [P+1]
   unsigned* counter;          // stage barriers: arrivals at barrier k, summed over all runs, in counter[k]
   unsigned target;            // arrivals that open a barrier in this run: run number * CTAs (mod 2^32)
-  unsigned n_ctas;
   int* status;
-  int B, n_slots;
+  int B, n_slots, n_stages;
   uint32_t slot_bytes, replica_bytes;
 };
 
@@ -92,11 +118,13 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// The hint lets the hardware park the thread for up to that many nanoseconds (it is woken when
+// the phase completes), so that waiting warps do not compete for issue slots with computing ones.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(2000u) : "memory");
   return ok != 0;
 }
 // Bounded wait by one thread: gives up (and raises the CTA-wide abort flag) after kPollLimit polls
@@ -104,23 +132,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait_one(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   for (uint32_t it = 0; it < kPollLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;
+    if ((it & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
   atomicExch(status, (int)RWKVQ_ETIMEOUT);
   return false;
 }
-// Warp-collective bounded wait: lane 0 polls, the verdict is warp-uniform; on success every lane
-// observes the completed phase itself so that the data the barrier guards is visible to it.
+// Warp-collective bounded wait: every lane polls (so that each lane itself observes the completed
+// phase and with it the data the barrier guards); the verdict is made warp-uniform.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = mbar_wait_one(bar, parity, abort_flag, status) ? 1 : 0;
-  ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-  if (ok) {
-    for (uint32_t it = 0; it < (1u << 20); ++it)
-      if (mbar_try_wait(bar, parity)) break;
-  }
-  return ok != 0;
+  const bool ok = mbar_wait_one(bar, parity, abort_flag, status);
+  return __all_sync(0xFFFFFFFFu, ok);
 }
 // Named barrier over `nthreads` threads that also ANDs a predicate: a uniform verdict for a role.
 __device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred) {
@@ -148,12 +170,35 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ void smem_add_release(uint32_t* p, uint32_t v) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t smem_ld_acquire(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+// Bounded wait until a shared-memory counter reaches `target`.
+__device__ __forceinline__ bool wait_count(const uint32_t* p, uint32_t target, volatile int* abort_flag, int* status) {
+  for (uint32_t it = 0; it < (kPollLimit << 4); ++it) {
+    if (smem_ld_acquire(p) >= target) return true;
+    if ((it & 255u) == 255u && *abort_flag) return false;
+    __nanosleep(32);
+  }
+  *abort_flag = 1;
+  atomicExch(status, (int)RWKVQ_ETIMEOUT);
+  return false;
+}
 
 struct Ctrl {
   uint64_t full[kMaxSlots], empty[kMaxSlots];
   uint64_t xfull[2], xempty[2];
+  uint32_t cdone;            // stage completions reported by consumer warps: 16 per finished stage.  A
+                             // plain counter, not an mbarrier: consumers of a CTA without work in the
+                             // coming stages may run any number of stages ahead of the stagers.
   int abort_flag;
 };
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 
 // ---- roles -------------------------------------------------------------------------------------
 
@@ -184,12 +229,13 @@ __device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint
       good = __shfl_sync(0xFFFFFFFFu, good, 0);
       if (!good) { ok = false; break; }
       if ((lane >> 3) == k) *reinterpret_cast<uint4*>(sl + (lane & 7) * 16) = cur;
-      // fields for lane 0: words of the first three 16-byte pieces of descriptor k
+      // fields for lane 0, by 16-byte piece of descriptor k
       const uint32_t s0l = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k), s0h = __shfl_sync(0xFFFFFFFFu, cur.y, 8 * k);
       const uint32_t s1l = __shfl_sync(0xFFFFFFFFu, cur.z, 8 * k), s1h = __shfl_sync(0xFFFFFFFFu, cur.w, 8 * k);
       const uint32_t cbl = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k + 1), cbh = __shfl_sync(0xFFFFFFFFu, cur.y, 8 * k + 1);
       const uint32_t by0 = __shfl_sync(0xFFFFFFFFu, cur.z, 8 * k + 1), by1 = __shfl_sync(0xFFFFFFFFu, cur.w, 8 * k + 1);
-      const uint32_t cbb = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k + 2);
+      const uint32_t cbb = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k + 2), off0 = __shfl_sync(0xFFFFFFFFu, cur.y, 8 * k + 2);
+      const uint32_t chb = __shfl_sync(0xFFFFFFFFu, cur.z, 8 * k + 5);
       __syncwarp();
       if (lane == 0) {
         const uint32_t tx = by0 + by1 + cbb;
@@ -199,9 +245,9 @@ __device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint
         } else {
           mbar_arrive_expect_tx(full, tx);
           uint8_t* data = sl + 128;
-          if (by0) bulk_g2s(data, reinterpret_cast<const void*>(((uint64_t)s0h << 32) | s0l), by0, full, policy);
-          if (by1) bulk_g2s(data + by0, reinterpret_cast<const void*>(((uint64_t)s1h << 32) | s1l), by1, full, policy);
-          if (cbb) bulk_g2s(data + by0 + by1, reinterpret_cast<const void*>(((uint64_t)cbh << 32) | cbl), cbb, full, policy);
+          if (by0) bulk_g2s(data + off0, reinterpret_cast<const void*>(((uint64_t)s0h << 32) | s0l), by0, full, policy);
+          if (by1) bulk_g2s(data + chb + off0, reinterpret_cast<const void*>(((uint64_t)s1h << 32) | s1l), by1, full, policy);
+          if (cbb) bulk_g2s(data + 2 * chb, reinterpret_cast<const void*>(((uint64_t)cbh << 32) | cbl), cbb, full, policy);
         }
       }
       ++issued;
@@ -219,12 +265,6 @@ __device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint
   }
 }
 
-// Stagers: x_mix and, for SQ, the per-group sums of the segment, into buffer (segment index & 1).
-// Everything that does not depend on the previous stage -- the decoded token-shift vector mu_hat
-// and the previous token's activations -- is put into shared memory BEFORE the stage barrier, so
-// that only one round of vector loads of x, the mix and the sums remain behind it.
-// A thread owns 8 consecutive columns (16 bytes) of one batch row; a half-warp owns one
-// 128-column group, whose three sums it reduces with shuffles.
 __device__ __forceinline__ uint32_t mix2(uint32_t xr, uint32_t pr, uint32_t mr) {
   const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xr));
   const float2 pf = __half22float2(*reinterpret_cast<const __half2*>(&pr));
@@ -239,33 +279,74 @@ __device__ __forceinline__ float pair_sum(uint32_t r) {
 
 constexpr int kStageUnroll = 4;
 
+// Stagers walk the CTA's event list.
+//  EV_ARRIVE: clear this CTA's slice of the next stage's outputs, then (deferred until the next
+//    segment's barrier-independent preparation is done) wait for the consumer warps to finish
+//    the stage, publish with one cumulative fence and add this CTA's arrival to the grid barrier.
+//  EV_SEGMENT: x_mix and, for SQ, the per-group sums of the segment, into buffer (segment number
+//    & 1).  The decoded token-shift vector mu_hat and the previous token's activations go to
+//    shared memory BEFORE the stage barrier, so that only one round of vector loads of x, the
+//    mix and the sums remain behind it.  A thread owns 8 consecutive columns (16 bytes) of one
+//    batch row; a half-warp owns one 128-column group, whose three sums it reduces with shuffles.
 __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_t* xbufs, uint32_t* mucb,
-                            uint32_t s0, uint32_t s1) {
+                            uint32_t e0, uint32_t e1) {
   const int stid = threadIdx.x - kConsumerThreads;
   const int lane = stid & 31;
   volatile int* abortp = &ctrl->abort_flag;
-  for (uint32_t si = s0; si < s1; ++si) {
-    const uint32_t li = si - s0;
-    const int buf = (int)(li & 1u);
-    const StepXSeg sg = *reinterpret_cast<const StepXSeg*>(reinterpret_cast<const uint8_t*>(a.xsegs) + (size_t)si * 64);
-    bool ok = mbar_wait_warp(&ctrl->xempty[buf], ((li >> 1) & 1u) ^ 1u, abortp, a.status);
+  uint32_t nseg = 0;          // segments staged so far
+  uint32_t narrive = 0;       // arrivals posted so far
+  int pending = -1;           // barrier index of an arrival not yet posted
+  bool ok = true;
+  // posts the pending arrival (thread 0 acts; the others only keep count)
+  auto post_arrival = [&]() {
+    if (pending < 0) return;
+    if (stid == 0 && ok) {
+      // barrier 0 (the clearing pass) has no consumer work before it; barrier j closes stage j - 1,
+      // which all sixteen consumer warps must have reported, like every stage before it
+      if (pending > 0) ok = wait_count(&ctrl->cdone, (uint32_t)kConsumerWarps * narrive, abortp, a.status);
+      if (ok) { __threadfence(); atomicAdd(a.counter + pending, 1u); }
+    }
+    ++narrive;
+    pending = -1;
+  };
+  for (uint32_t ei = e0; ei < e1; ++ei) {
+    const StepEvent ev = *reinterpret_cast<const StepEvent*>(reinterpret_cast<const uint8_t*>(a.events) + (size_t)ei * 64);
+    if (ev.kind == EV_ARRIVE) {
+      post_arrival();                         // an earlier arrival with no segment in between
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float* z = reinterpret_cast<float*>(ev.arr.zptr[k]);
+        for (uint32_t e = stid; e < ev.arrd.zcount[k]; e += kStagerThreads) z[e] = 0.f;
+      }
+      // the clearing stores of every stager thread must precede thread 0's fence
+      ok = named_bar_and(4, kStagerThreads, ok);
+      pending = (int)ev.barrier;
+      if (!ok) break;
+      continue;
+    }
+    const int buf = (int)(nseg & 1u);
+    // uniform verdict over all stager threads: the named barriers below must be reached by all or none
+    ok = named_bar_and(7, kStagerThreads, mbar_wait_warp(&ctrl->xempty[buf], ((nseg >> 1) & 1u) ^ 1u, abortp, a.status) && ok);
     uint8_t* xb = xbufs + (size_t)buf * kXBufBytes;
-    const uint8_t* mu = reinterpret_cast<const uint8_t*>(sg.mu);
-    const __half* x = reinterpret_cast<const __half*>(sg.x);
-    const __half* xp = reinterpret_cast<const __half*>(sg.xprev);
-    const int nvr = (int)sg.ncols >> 3;            // 16-byte vectors per batch row
+    const uint8_t* mu = reinterpret_cast<const uint8_t*>(ev.seg.mu);
+    const __half* x = reinterpret_cast<const __half*>(ev.seg.x);
+    const __half* xp = reinterpret_cast<const __half*>(ev.seg.xprev);
+    const int ic = (int)ev.segd.ic, col0 = (int)ev.segd.col0;
+    const uint32_t xstride = ev.xstride_sums & 0x7FFFFFFFu;
+    const bool sums = (ev.xstride_sums >> 31) != 0;
+    const int nvr = (int)ev.segd.ncols >> 3;            // 16-byte vectors per batch row
     const int total = a.B * nvr;
     const int nbp = (a.B + 1) & ~1;
-    uint8_t* murow = xb + sg.mu_off;
+    uint8_t* murow = xb + (size_t)ev.mu_off16 * 16;
     if (ok && mu) {
-      for (int e = stid; e < (int)sg.mu_entries; e += kStagerThreads) mucb[e] = __ldg(reinterpret_cast<const uint32_t*>(sg.mu_aux) + e);
-      named_bar_sync(4, kStagerThreads);
-      const int bits = (int)sg.mu_bits;
+      for (int e = stid; e < (int)ev.segd.mu_entries; e += kStagerThreads) mucb[e] = __ldg(reinterpret_cast<const uint32_t*>(ev.seg.mu_aux) + e);
+      named_bar_sync(5, kStagerThreads);
+      const int bits = (int)ev.segd.mu_bits;
       const uint32_t mask = (1u << bits) - 1u;
       for (int c8 = stid; c8 < nvr; c8 += kStagerThreads) {
-        const int col = (int)sg.col0 + 8 * c8;
+        const int col = col0 + 8 * c8;
         uint4 m = make_uint4(0u, 0u, 0u, 0u);
-        if (col < (int)sg.ic) {
+        if (col < ic) {
           // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
           const uint32_t byte = (uint32_t)(col >> 1) * (uint32_t)bits >> 3;
           const uint32_t* w = reinterpret_cast<const uint32_t*>(mu) + (byte >> 2);
@@ -282,212 +363,274 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       }
       for (int v = stid; v < total; v += kStagerThreads) {
         const int b = v / nvr, c8 = v - b * nvr;
-        const int col = (int)sg.col0 + 8 * c8;
+        const int col = col0 + 8 * c8;
         uint4 r = make_uint4(0u, 0u, 0u, 0u);
-        if (col < (int)sg.ic) r = __ldg(reinterpret_cast<const uint4*>(xp + (size_t)b * sg.ic + col));
-        *reinterpret_cast<uint4*>(xb + (size_t)b * sg.xstride + (size_t)c8 * 16) = r;
+        if (col < ic) r = __ldg(reinterpret_cast<const uint4*>(xp + (size_t)b * ic + col));
+        *reinterpret_cast<uint4*>(xb + (size_t)b * xstride + (size_t)c8 * 16) = r;
       }
     }
-    if (ok && sg.barrier && stid == 0) {
+    post_arrival();
+    if (ok && ev.barrier && stid == 0) {
       // grid-wide stage barrier: every CTA has finished (and published) the previous stage.  Each
       // barrier has its own arrival counter, so a CTA without work may run ahead and arrive at
       // later barriers without releasing this one early.
       uint32_t it = 0;
-      while ((int)(ld_acquire_gpu(a.counter + (sg.barrier - 1u)) - a.target) < 0) {
-        if (++it >= kPollLimit || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
+      while ((int)(ld_acquire_gpu(a.counter + (ev.barrier - 1u)) - a.target) < 0) {
+        if (++it >= (kPollLimit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
       }
     }
-    if (!named_bar_and(4, kStagerThreads, ok)) return;   // all stager threads leave together
-    float* gs = reinterpret_cast<float*>(xb + (size_t)a.B * sg.xstride);
-    for (int v0 = stid; v0 < total; v0 += kStagerThreads * kStageUnroll) {
-      uint4 raw[kStageUnroll];
+    ok = named_bar_and(6, kStagerThreads, ok);   // uniform verdict; orders the mu row before its readers
+    if (ok) {
+      float* gs = reinterpret_cast<float*>(xb + (size_t)a.B * xstride);
+      for (int v0 = stid; v0 < total; v0 += kStagerThreads * kStageUnroll) {
+        uint4 raw[kStageUnroll];
 #pragma unroll
-      for (int u = 0; u < kStageUnroll; ++u) {
-        const int v = v0 + u * kStagerThreads;
-        raw[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (v < total) {
-          const int b = v / nvr, c8 = v - b * nvr;
-          const int col = (int)sg.col0 + 8 * c8;
-          if (col < (int)sg.ic) raw[u] = __ldcg(reinterpret_cast<const uint4*>(x + (size_t)b * sg.ic + col));
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < kStageUnroll; ++u) {
-        const int v = v0 + u * kStagerThreads;
-        if (v >= total) break;                      // warp-uniform: total is a multiple of 32
-        const int b = v / nvr, c8 = v - b * nvr;
-        uint4 r = raw[u];
-        uint8_t* dst = xb + (size_t)b * sg.xstride + (size_t)c8 * 16;
-        if (mu) {
-          const uint4 pr = *reinterpret_cast<const uint4*>(dst);          // this thread's own earlier store
-          const uint4 mr = *reinterpret_cast<const uint4*>(murow + (size_t)c8 * 16);
-          r.x = mix2(r.x, pr.x, mr.x); r.y = mix2(r.y, pr.y, mr.y);
-          r.z = mix2(r.z, pr.z, mr.z); r.w = mix2(r.w, pr.w, mr.w);
-        }
-        *reinterpret_cast<uint4*>(dst) = r;
-        if (sg.sums) {
-          const int o = (8 * c8) & 63;
-          const float pa = pair_sum(r.x) + pair_sum(r.z), pb = pair_sum(r.y) + pair_sum(r.w);
-          float sx = pa + pb;
-          float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
-          float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
-#pragma unroll
-          for (int d = 8; d > 0; d >>= 1) {
-            sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
-            t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
-            t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+        for (int u = 0; u < kStageUnroll; ++u) {
+          const int v = v0 + u * kStagerThreads;
+          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (v < total) {
+            const int b = v / nvr, c8 = v - b * nvr;
+            const int col = col0 + 8 * c8;
+            if (col < ic) raw[u] = __ldcg(reinterpret_cast<const uint4*>(x + (size_t)b * ic + col));
           }
-          if ((lane & 15) == 0) {
-            const int grp = c8 >> 4;
-            gs[(grp * 3 + 0) * nbp + b] = sx;
-            gs[(grp * 3 + 1) * nbp + b] = t0;
-            gs[(grp * 3 + 2) * nbp + b] = t1;
+        }
+#pragma unroll
+        for (int u = 0; u < kStageUnroll; ++u) {
+          const int v = v0 + u * kStagerThreads;
+          if (v >= total) break;                      // warp-uniform: total is a multiple of 32
+          const int b = v / nvr, c8 = v - b * nvr;
+          uint4 r = raw[u];
+          uint8_t* dst = xb + (size_t)b * xstride + (size_t)c8 * 16;
+          if (mu) {
+            const uint4 pr = *reinterpret_cast<const uint4*>(dst);          // this thread's own earlier store
+            const uint4 mr = *reinterpret_cast<const uint4*>(murow + (size_t)c8 * 16);
+            r.x = mix2(r.x, pr.x, mr.x); r.y = mix2(r.y, pr.y, mr.y);
+            r.z = mix2(r.z, pr.z, mr.z); r.w = mix2(r.w, pr.w, mr.w);
+          }
+          *reinterpret_cast<uint4*>(dst) = r;
+          if (sums) {
+            const int o = (8 * c8) & 63;
+            const float pa = pair_sum(r.x) + pair_sum(r.z), pb = pair_sum(r.y) + pair_sum(r.w);
+            float sx = pa + pb;
+            float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
+            float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
+#pragma unroll
+            for (int d = 8; d > 0; d >>= 1) {
+              sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+              t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
+              t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+            }
+            if ((lane & 15) == 0) {
+              const int grp = c8 >> 4;
+              gs[(grp * 3 + 0) * nbp + b] = sx;
+              gs[(grp * 3 + 1) * nbp + b] = t0;
+              gs[(grp * 3 + 2) * nbp + b] = t1;
+            }
           }
         }
       }
     }
     __syncwarp();
+    // A stager that gave up still arrives, so that no consumer is left waiting on this barrier;
+    // the consumers stop at the abort flag.
     if (lane == 0) mbar_arrive(&ctrl->xfull[buf]);
+    ++nseg;
+    if (!ok) break;
+  }
+  if (ok) post_arrival();
+}
+
+// Six words of one 128-column group of the record of lane `lane` (planes of 512 bytes, 16 bytes
+// per lane): group 0 = words 0..5, group 1 = words 6..11.
+template <int GRP>
+__device__ __forceinline__ void sq_group_words(const uint8_t* rec, int lane, uint32_t (&w)[6]) {
+  if constexpr (GRP == 0) {
+    const uint4 p0 = *reinterpret_cast<const uint4*>(rec + lane * 16);
+    const uint2 p1 = *reinterpret_cast<const uint2*>(rec + 512 + lane * 16);
+    w[0] = p0.x; w[1] = p0.y; w[2] = p0.z; w[3] = p0.w; w[4] = p1.x; w[5] = p1.y;
+  } else {
+    const uint2 p1 = *reinterpret_cast<const uint2*>(rec + 512 + lane * 16 + 8);
+    const uint4 p2 = *reinterpret_cast<const uint4*>(rec + 1024 + lane * 16);
+    w[0] = p1.x; w[1] = p1.y; w[2] = p2.x; w[3] = p2.y; w[4] = p2.z; w[5] = p2.w;
   }
 }
 
+// Consumer warp `w` of group `grp`: units grp, grp + 2, ... of the CTA's list.
 template <int NB>
 __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, const uint8_t* xbufs, uint8_t* replicas,
-                              uint32_t unit_base, uint32_t n_units) {
+                              uint32_t unit_base, uint32_t n_units, uint32_t ev_base, uint32_t n_events) {
   bool dead = false;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int rec = warp & 7, half = warp >> 3;
+  const int grp = warp >> 3, w = warp & 7;
   const int g = lane >> 2, t = lane & 3;
   volatile int* abortp = &ctrl->abort_flag;
-  float acc[NB][4];
+  float acca[NB][4], accb[NB][4];
 #pragma unroll
-  for (int n = 0; n < NB; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-  int xcur = 1;
-  uint32_t xuse = 0;  // segments acquired so far
-  for (uint32_t i = 0; i < n_units; ++i) {
+  for (int n = 0; n < NB; ++n)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) acca[n][k] = accb[n][k] = 0.f;
+  // Every consumer warp walks the CTA's event list in order -- it reports each stage it leaves and
+  // passes through each input segment, used or not -- so that the phases of the shared barriers
+  // advance in step for all sixteen warps.
+  int held = -1;              // input segment this warp currently holds
+  uint32_t seg_next = 0;      // number of segment events passed so far
+  uint32_t cur_ev = 0;        // last event processed (event 0 is the clearing arrival: nothing to do)
+  // Report the current stage as finished: the warp's reductions into y are ordered before the
+  // count by the warp barrier and the release.
+  auto arrive_stage = [&]() {
+    __syncwarp();
+    if (lane == 0 && !dead) smem_add_release(&ctrl->cdone, 1u);
+  };
+  auto release_held = [&]() {
+    __syncwarp();
+    if (held >= 0 && lane == 0 && !dead) mbar_arrive(&ctrl->xempty[held & 1]);
+    held = -1;
+  };
+  auto pass_segment = [&]() {   // a segment this warp does not use: observe it, hand it back
+    const uint32_t q = seg_next++;
+    if (!dead && !mbar_wait_warp(&ctrl->xfull[q & 1u], (q >> 1) & 1u, abortp, a.status)) dead = true;
+    __syncwarp();
+    if (lane == 0 && !dead) mbar_arrive(&ctrl->xempty[q & 1u]);
+  };
+  // Events (cur_ev, upto) in order; `mask` describes them when there are at most 32 and the planner
+  // could say so, otherwise (and for the tail of the list) the kinds are read from the plan, 32 at
+  // a time.
+  auto pass_events = [&](uint32_t upto, uint32_t mask, bool mask_valid) {
+    if (cur_ev + 1u >= upto) return;
+    release_held();
+    while (cur_ev + 1u < upto && !dead) {
+      const uint32_t first = cur_ev + 1u;
+      const uint32_t cnt = min(32u, upto - first);
+      uint32_t m = mask;
+      if (!mask_valid) {
+        bool arr = false;
+        if ((uint32_t)lane < cnt) {
+          const uint2 kb = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint8_t*>(a.events) + (size_t)(ev_base + first + lane) * 64 + 48));
+          arr = kb.x == EV_ARRIVE && kb.y > 0u;
+        }
+        m = __ballot_sync(0xFFFFFFFFu, arr);
+      }
+      for (uint32_t j = 0; j < cnt && !dead; ++j) {
+        if ((m >> j) & 1u) arrive_stage(); else pass_segment();
+      }
+      cur_ev += cnt;
+      mask_valid = false;
+    }
+  };
+  uint8_t* rep = replicas + (size_t)grp * a.replica_bytes;
+  for (uint32_t i = (uint32_t)grp; i < n_units; i += kGroups) {
     const int slot = (int)(i % (uint32_t)a.n_slots);
     const uint32_t round = i / (uint32_t)a.n_slots;
-    // A warp that gave up keeps walking the list (named barriers and arrivals still happen, so no
-    // other warp is left waiting for it) but touches neither the slots nor global memory.
-    if (!dead && !mbar_wait_warp(&ctrl->full[slot], round & 1u, abortp, a.status)) dead = true;
     const uint8_t* sl = smem + kCtrlBytes + (size_t)slot * a.slot_bytes;
     const StepUnit* u = reinterpret_cast<const StepUnit*>(sl);
-    uint32_t flags = u->flags, fmt = u->fmt;
-    const uint32_t by0 = u->bytes0, by1 = u->bytes1;
-    if (dead) {   // the header may not have landed: take the barrier-relevant bits from the plan itself
-      const StepUnit* gu = a.units + unit_base + i;
-      flags = gu->flags; fmt = gu->fmt;
+    if (!dead && !mbar_wait_warp(&ctrl->full[slot], round & 1u, abortp, a.status)) dead = true;
+    if (!dead && u->ev_index != cur_ev) {
+      const uint32_t target = u->ev_index;
+      pass_events(target, u->between_mask, target - cur_ev - 1u <= 32u);
+      if (!dead) {
+        release_held();
+        const uint32_t q = seg_next++;
+        held = (int)q;
+        cur_ev = target;
+        if (!mbar_wait_warp(&ctrl->xfull[q & 1u], (q >> 1) & 1u, abortp, a.status)) dead = true;
+      }
     }
-    if (flags & UF_NEW_XSEG) {
-      xcur = (int)(xuse & 1u);
-      if (!dead && !mbar_wait_warp(&ctrl->xfull[xcur], (xuse >> 1) & 1u, abortp, a.status)) dead = true;
-      ++xuse;
-    }
-    const uint8_t* data = sl + 128;
-    const uint8_t* xb = xbufs + (size_t)xcur * kXBufBytes;
-    const uint32_t xstride = u->xstride, nbp = u->nbp;
     if (dead) {
-      if (fmt == UFMT_VQ6 || fmt == UFMT_VQ8) { named_bar_sync(1, kConsumerThreads); named_bar_sync(1, kConsumerThreads); }
-    } else if (fmt == UFMT_SQ) {
-      const float* gs0 = reinterpret_cast<const float*>(xb + u->gs_off);
-      if (!(flags & UF_SPLIT)) {
-        // warp (rec, half): record `rec` of chunk `half` (chunk B = the next 256 columns)
-        SqRecord r;
-        r.load_shared(data + (size_t)half * by0 + (size_t)rec * RWKVQ_SQ_RECORD_BYTES, lane);
-        uint32_t w[12];
-        r.words(w);
-        const uint32_t col = u->xcol0 + (uint32_t)half * 256u;
-        const XLane xl = make_xlane(xb + (size_t)col * 2, xstride, gs0 + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
-        sq_record_mma<NB>(w, r.sz, xl, acc);
-      } else {
-        // single chunk: the two halves take one 128-column group each
-        const uint8_t* rp = data + (size_t)rec * RWKVQ_SQ_RECORD_BYTES;
-        uint32_t w[6];
-#pragma unroll
-        for (int k = 0; k < 6; ++k) {
-          const int widx = 6 * half + k;
-          w[k] = *reinterpret_cast<const uint32_t*>(rp + (widx >> 2) * 512 + lane * 16 + (widx & 3) * 4);
-        }
-        const uint4 sz = *reinterpret_cast<const uint4*>(rp + RWKVQ_SQ_CODE_BYTES + g * 16);
-        const uint32_t col = u->xcol0 + (uint32_t)half * 128u;
-        const XLane xl = make_xlane(xb + (size_t)col * 2, xstride, gs0 + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
-        sq_group_mma<NB, 0>(w, half == 0 ? sz.x : sz.y, half == 0 ? sz.z : sz.w, xl, acc);
-      }
-    } else if (fmt == UFMT_VQ6 || fmt == UFMT_VQ8) {
-      // replicate the tile's codebook for conflict-free lookups (all consumer warps take part)
-      const uint32_t E = u->entries;
-      named_bar_sync(1, kConsumerThreads);          // previous unit's lookups are done
-      {
-        const uint32_t* cbraw = reinterpret_cast<const uint32_t*>(data + by0 + by1);
-        uint32_t* rep = reinterpret_cast<uint32_t*>(replicas);
-        for (uint32_t idx = threadIdx.x; idx < E * 32u; idx += kConsumerThreads) rep[idx] = cbraw[idx >> 5];
-      }
-      named_bar_sync(1, kConsumerThreads);
-      const uint32_t* cb_lane = reinterpret_cast<const uint32_t*>(replicas) + lane;
-      const XLane xl = make_xlane(xb + (size_t)u->xcol0 * 2, xstride, nullptr, nbp, a.B, lane);
-      if (!(flags & UF_SPLIT)) {
-        // warp (rec, half): record `rec` of chunk `half` (chunk B = the next 128 rows, same columns)
-        if (fmt == UFMT_VQ6) {
-          VqRecord<6> r;
-          r.load_shared(data + (size_t)half * by0 + (size_t)rec * 1536, lane);
-          vq_record_mma<6, NB>(r.w, cb_lane, xl, acc);
-        } else {
-          VqRecord<8> r;
-          r.load_shared(data + (size_t)half * by0 + (size_t)rec * 2048, lane);
-          vq_record_mma<8, NB>(r.w, cb_lane, xl, acc);
-        }
-      } else {
-        if (fmt == UFMT_VQ6) {
-          VqRecord<6> r;
-          r.load_shared(data + (size_t)rec * 1536, lane);
-          if (half == 0) vq_record_mma<6, NB, 0, 8>(r.w, cb_lane, xl, acc);
-          else vq_record_mma<6, NB, 8, 16>(r.w, cb_lane, xl, acc);
-        } else {
-          VqRecord<8> r;
-          r.load_shared(data + (size_t)rec * 2048, lane);
-          if (half == 0) vq_record_mma<8, NB, 0, 8>(r.w, cb_lane, xl, acc);
-          else vq_record_mma<8, NB, 8, 16>(r.w, cb_lane, xl, acc);
-        }
-      }
+      // A warp that gave up keeps walking the list only to keep the group's named barriers whole
+      // (the other warps stop at their next bounded wait); it touches neither slots nor outputs.
+      if (a.units[unit_base + i].flags & UF_VQ) { named_bar_sync(1 + grp, kGroupThreads); named_bar_sync(1 + grp, kGroupThreads); }
+      continue;
     }
-    // everything this warp needs from the slot is in registers now, except flags read above
-    const uint32_t oc = u->oc;
-    const uint32_t row0 = u->row0 + ((fmt != UFMT_SQ && !(flags & UF_SPLIT)) ? (uint32_t)half * 128u : 0u);
+    const uint32_t flags = u->flags;
+    const uint32_t by1 = u->bytes1;
+    const uint32_t after_count = u->after_count, after_mask = u->after_mask;
+    const uint8_t* data = sl + 128;
+    const uint8_t* xb = xbufs + (size_t)(held & 1) * kXBufBytes;
+    const uint32_t xstride = u->xstride, nbp = u->nbp, chb = u->chunk_bytes, rb = u->rec_bytes;
+    const uint32_t w0 = (flags >> 8) & 15u, w1 = (flags >> 12) & 15u;
+    const bool active = (uint32_t)w >= w0 && (uint32_t)w < w1;
+    const bool has_b = by1 != 0u;
+    const uint32_t oc = u->oc, row0 = u->row0;
     float* y = reinterpret_cast<float*>(u->y);
-    uint64_t zp[4] = {0, 0, 0, 0};
-    uint32_t zc[4] = {0, 0, 0, 0};
-    if ((flags & UF_STAGE_END) && !dead) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) { zp[k] = u->zptr[k]; zc[k] = u->zcount[k]; }
+    const uint8_t* ra = data + (size_t)w * rb;
+    const uint8_t* rbp = data + chb + (size_t)w * rb;
+    if (!(flags & UF_VQ)) {
+      const uint32_t col = u->xcol0;
+      const XLane xl = make_xlane(xb + (size_t)col * 2, xstride,
+                                  reinterpret_cast<const float*>(xb + u->gs_off) + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
+      uint32_t wa[6], wb[6];
+      uint4 sza = make_uint4(0, 0, 0, 0), szb = sza;
+      if (active) {
+        sq_group_words<0>(ra, lane, wa);
+        sza = *reinterpret_cast<const uint4*>(ra + RWKVQ_SQ_CODE_BYTES + g * 16);
+        if (has_b) {
+          sq_group_words<0>(rbp, lane, wb);
+          szb = *reinterpret_cast<const uint4*>(rbp + RWKVQ_SQ_CODE_BYTES + g * 16);
+        }
+        sq_group_mma2<NB, 0>(wa, wb, sza, szb, has_b, xl, acca, accb);
+        sq_group_words<1>(ra, lane, wa);
+        if (has_b) sq_group_words<1>(rbp, lane, wb);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl->empty[slot]);     // the rest of the records is in registers: free the slot
+      if (active) sq_group_mma2<NB, 1>(wa, wb, sza, szb, has_b, xl, acca, accb);
+    } else {
+      // replicate the tile's codebook for conflict-free lookups (the eight warps of the group)
+      const uint32_t E = u->entries;
+      named_bar_sync(1 + grp, kGroupThreads);          // the group's previous lookups are done
+      {
+        const uint32_t* cbraw = reinterpret_cast<const uint32_t*>(data + 2 * chb);
+        uint32_t* rp = reinterpret_cast<uint32_t*>(rep);
+        for (uint32_t idx = (uint32_t)(w * 32 + lane); idx < E * 32u; idx += kGroupThreads) rp[idx] = cbraw[idx >> 5];
+      }
+      named_bar_sync(1 + grp, kGroupThreads);
+      const uint32_t* cb_lane = reinterpret_cast<const uint32_t*>(rep) + lane;
+      const XLane xl = make_xlane(xb + (size_t)u->xcol0 * 2, xstride, nullptr, nbp, a.B, lane);
+      if (flags & UF_BITS8) {
+        uint32_t va[16], vb[16];
+        if (active) {
+          vq_half_words<8, 0>(ra, lane, va); vq_half_words<8, 0>(rbp, lane, vb);
+          vq_half_mma2<8, NB, 0>(va, vb, cb_lane, xl, acca, accb);
+          vq_half_words<8, 1>(ra, lane, va); vq_half_words<8, 1>(rbp, lane, vb);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
+        if (active) vq_half_mma2<8, NB, 1>(va, vb, cb_lane, xl, acca, accb);
+      } else {
+        uint32_t va[12], vb[12];
+        if (active) {
+          vq_half_words<6, 0>(ra, lane, va); vq_half_words<6, 0>(rbp, lane, vb);
+          vq_half_mma2<6, NB, 0>(va, vb, cb_lane, xl, acca, accb);
+          vq_half_words<6, 1>(ra, lane, va); vq_half_words<6, 1>(rbp, lane, vb);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
+        if (active) vq_half_mma2<6, NB, 1>(va, vb, cb_lane, xl, acca, accb);
+      }
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
-    if ((flags & UF_FLUSH) && !dead) {
+    if (flags & UF_FLUSH) {
+      if (active) {
+#pragma unroll
+        for (int n = 0; n < NB; ++n)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t row = row0 + (uint32_t)w * 16u + (uint32_t)g + 8u * (uint32_t)(k >> 1);
+            const int b = n * 8 + 2 * t + (k & 1);
+            if (b < a.B && row < oc) atomicAdd(y + (size_t)b * oc + row, acca[n][k]);
+            if (b < a.B && has_b && row + 128u < oc) atomicAdd(y + (size_t)b * oc + row + 128u, accb[n][k]);
+          }
+      }
 #pragma unroll
       for (int n = 0; n < NB; ++n)
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint32_t row = row0 + (uint32_t)rec * 16u + (uint32_t)g + 8u * (uint32_t)(k >> 1);
-          const int b = n * 8 + 2 * t + (k & 1);
-          if (b < a.B && row < oc) atomicAdd(y + (size_t)b * oc + row, acc[n][k]);
-          acc[n][k] = 0.f;
-        }
+        for (int k = 0; k < 4; ++k) acca[n][k] = accb[n][k] = 0.f;
     }
-    if (flags & UF_END_XSEG) {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ctrl->xempty[xcur]);
-    }
-    if (flags & UF_STAGE_END) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        float* z = reinterpret_cast<float*>(zp[k]);
-        for (uint32_t e = threadIdx.x; e < (dead ? 0u : zc[k]); e += kConsumerThreads) z[e] = 0.f;
-      }
-      // The named barrier orders every consumer thread's stores and reductions before thread 0's
-      // fence, which is cumulative: one fence publishes the whole CTA's share of the stage.
-      named_bar_sync(2, kConsumerThreads);
-      if (threadIdx.x == 0) { __threadfence(); atomicAdd(a.counter + (flags >> 16), 1u); }
-    }
+    // the group's last unit of the stage: report the stage as finished without waiting for the next unit
+    if (after_count) pass_events(cur_ev + after_count + 1u, after_mask, true);
+  }
+  if (!dead) {
+    release_held();
+    pass_events(n_events, 0u, false);     // the rest of the list: later stages this warp has no unit in
   }
 }
 
@@ -499,35 +642,34 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   uint32_t* mucb = reinterpret_cast<uint32_t*>(xbufs + 2 * kXBufBytes);
   uint8_t* replicas = reinterpret_cast<uint8_t*>(mucb) + kMuScratch;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < a.n_slots; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], kConsumerWarps); }
+    for (int s = 0; s < a.n_slots; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], kGroupWarps); }
     for (int b = 0; b < 2; ++b) { mbar_init(&ctrl->xfull[b], kStagerWarps); mbar_init(&ctrl->xempty[b], kConsumerWarps); }
+    ctrl->cdone = 0u;
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   const uint32_t u0 = a.unit_off[blockIdx.x], u1 = a.unit_off[blockIdx.x + 1];
-  const uint32_t s0 = a.xseg_off[blockIdx.x], s1 = a.xseg_off[blockIdx.x + 1];
-  StepArgs la = a;
-  la.units = a.units;  // descriptors are indexed globally
+  const uint32_t e0 = a.event_off[blockIdx.x], e1 = a.event_off[blockIdx.x + 1];
   const int warp = threadIdx.x >> 5;
   if (warp < kConsumerWarps) {
-    consumer_role<NB>(la, smem, ctrl, xbufs, replicas, u0, u1 - u0);
+    consumer_role<NB>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
   } else if (warp < kConsumerWarps + kStagerWarps) {
-    stager_role(la, smem, ctrl, xbufs, mucb, s0, s1);
+    stager_role(a, smem, ctrl, xbufs, mucb, e0, e1);
   } else {
-    producer_role(la, smem, ctrl, u0, u1);
+    producer_role(a, smem, ctrl, u0, u1);
   }
 }
 
 // ---- host planner --------------------------------------------------------------------------------
 
 struct PlanInfo {
-  int P, B, NB, n_slots;
+  int P, B, NB, n_slots, n_stages;
   unsigned runs;        // launches since the counters were last zero
   unsigned abort_epoch; // value of the abort epoch when the counters were last known good
   uint32_t slot_bytes, replica_bytes, smem_bytes;
-  size_t off_unit_off, off_xseg_off, off_units, off_xsegs, off_counter, total_bytes;
-  uint32_t n_units, n_xsegs, n_barriers;
+  size_t off_unit_off, off_event_off, off_units, off_events, off_counter, total_bytes;
+  uint32_t n_units, n_events, n_barriers;
 };
 
 static std::mutex g_plan_mutex;
@@ -535,8 +677,7 @@ static std::unordered_map<const void*, PlanInfo> g_plans;
 
 struct HostUnit {
   StepUnit u;
-  int op, rowkey, kt, ntiles, stage;
-  uint32_t bytes;
+  int op, tr, kt, stage, w0, w1;
 };
 
 // Shared-memory footprint of an input segment: B rows of x_mix, the per-group sums (SQ) and one
@@ -544,7 +685,8 @@ struct HostUnit {
 static uint32_t xseg_mu_off(int B, int ncols, bool sums) {
   uint32_t xstride = (uint32_t)ncols * 2u + 32u;
   uint32_t nbp = (uint32_t)((B + 1) & ~1);
-  uint32_t off = (uint32_t)B * xstride + (sums ? (uint32_t)(ncols / 128) * 3u * nbp * 4u : 0u);
+  // 64 bytes of slack: lanes of batch columns that do not exist read (and discard) sums past the table
+  uint32_t off = (uint32_t)B * xstride + (sums ? (uint32_t)(ncols / 128) * 3u * nbp * 4u + 64u : 0u);
   return (off + 15u) & ~15u;
 }
 static uint32_t xseg_bytes(int B, int ncols, bool sums, bool has_mu) {
@@ -587,8 +729,8 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   if (has_vq6) data_max = std::max(data_max, 2u * 8u * 1536u + 256u);
   if (has_vq8) data_max = std::max(data_max, 2u * 8u * 2048u + 1024u);
   info->slot_bytes = (128u + data_max + 127u) & ~127u;
-  info->replica_bytes = has_vq8 ? 256u * 128u : has_vq6 ? 64u * 128u : 0u;
-  const uint32_t fixed = kCtrlBytes + 2u * kXBufBytes + kMuScratch + info->replica_bytes;
+  info->replica_bytes = has_vq8 ? 256u * 128u : has_vq6 ? 64u * 128u : 0u;   // per consumer group
+  const uint32_t fixed = kCtrlBytes + 2u * kXBufBytes + kMuScratch + (uint32_t)kGroups * info->replica_bytes;
   int ns = (int)((kSmemLimit - fixed) / info->slot_bytes);
   if (ns > kMaxSlots) ns = kMaxSlots;
   if (ns < 2) return RWKVQ_EUNSUPPORTED;
@@ -597,7 +739,6 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   info->P = P; info->B = B; info->NB = B <= 8 ? 1 : 2;
   const uint32_t nbp = (uint32_t)((B + 1) & ~1);
 
-  // stages in order of appearance
   std::vector<std::pair<int, int>> stage_ranges;  // [first op, last op) per distinct stage value
   for (int i = 0; i < n_ops;) {
     int j = i;
@@ -606,45 +747,38 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     i = j;
   }
   const int n_stages = (int)stage_ranges.size();
+  info->n_stages = n_stages;
   info->n_barriers = (uint32_t)n_stages + 1;
-  if (info->n_barriers > 65535u) return RWKVQ_EUNSUPPORTED;
 
   std::vector<std::vector<HostUnit>> cta_units(P);
-  auto zero_ranges_for = [&](int stage_idx, int c, std::vector<std::pair<uint64_t, uint32_t>>* ranges) {
-    // CTA c's slice of the concatenated outputs of stage `stage_idx`
-    ranges->clear();
-    if (stage_idx >= n_stages) return;
-    uint64_t total = 0;
-    for (int o = stage_ranges[stage_idx].first; o < stage_ranges[stage_idx].second; ++o) total += (uint64_t)B * ops[o].W_desc.oc;
-    const uint64_t lo = total * (uint64_t)c / P, hi = total * (uint64_t)(c + 1) / P;
-    uint64_t base = 0;
-    for (int o = stage_ranges[stage_idx].first; o < stage_ranges[stage_idx].second; ++o) {
-      const uint64_t n = (uint64_t)B * ops[o].W_desc.oc;
-      const uint64_t a0 = std::max(lo, base), a1 = std::min(hi, base + n);
-      if (a1 > a0) ranges->push_back({(uint64_t)(uintptr_t)ops[o].y_dev + (a0 - base) * 4, (uint32_t)(a1 - a0)});
-      base += n;
-    }
-  };
+  std::vector<std::vector<StepEvent>> cta_arrivals(P);      // arrival events, one per barrier
   bool too_many_ranges = false;
-  auto push_stage_end = [&](int c, int next_stage_idx, int stage_tag) {
-    // attach the stage end (and the clearing of the next stage's outputs) to CTA c's list: to its
-    // last unit of this stage, or to an empty unit if it has none
-    std::vector<std::pair<uint64_t, uint32_t>> ranges;
-    zero_ranges_for(next_stage_idx, c, &ranges);
-    if (ranges.size() > 4) { too_many_ranges = true; return; }
-    std::vector<HostUnit>& L = cta_units[c];
-    if (L.empty() || L.back().stage != stage_tag) {
-      HostUnit h{};
-      h.u.fmt = UFMT_EMPTY; h.stage = stage_tag; h.op = -1; h.rowkey = -1;
-      L.push_back(h);
+  auto make_arrival = [&](int c, int stage_idx_to_clear, int barrier) {
+    StepEvent ev;
+    std::memset(&ev, 0, sizeof(ev));
+    ev.kind = EV_ARRIVE; ev.barrier = (uint32_t)barrier;
+    if (stage_idx_to_clear < n_stages) {
+      uint64_t total = 0;
+      for (int o = stage_ranges[stage_idx_to_clear].first; o < stage_ranges[stage_idx_to_clear].second; ++o)
+        total += (uint64_t)B * ops[o].W_desc.oc;
+      const uint64_t lo = total * (uint64_t)c / P, hi = total * (uint64_t)(c + 1) / P;
+      uint64_t base = 0;
+      int k = 0;
+      for (int o = stage_ranges[stage_idx_to_clear].first; o < stage_ranges[stage_idx_to_clear].second; ++o) {
+        const uint64_t n = (uint64_t)B * ops[o].W_desc.oc;
+        const uint64_t a0 = std::max(lo, base), a1 = std::min(hi, base + n);
+        if (a1 > a0) {
+          if (k >= 4) { too_many_ranges = true; break; }
+          ev.arr.zptr[k] = (uint64_t)(uintptr_t)ops[o].y_dev + (a0 - base) * 4;
+          ev.arrd.zcount[k] = (uint32_t)(a1 - a0);
+          ++k;
+        }
+        base += n;
+      }
     }
-    HostUnit& last = L.back();
-    last.u.flags |= UF_STAGE_END | ((uint32_t)(stage_tag + 1) << 16);   // barrier 0 = the clearing pass
-    for (size_t k = 0; k < ranges.size(); ++k) { last.u.zptr[k] = ranges[k].first; last.u.zcount[k] = ranges[k].second; }
+    cta_arrivals[c].push_back(ev);
   };
-
-  // barrier #0: clear the outputs of the first stage
-  for (int c = 0; c < P; ++c) push_stage_end(c, 0, -1);
+  for (int c = 0; c < P; ++c) make_arrival(c, 0, 0);   // barrier 0: the first stage's outputs are clear
 
   for (int s = 0; s < n_stages; ++s) {
     std::vector<HostUnit> units;
@@ -652,139 +786,170 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       const rwkvq_desc& d = ops[o].W_desc;
       const uint8_t* img = static_cast<const uint8_t*>(ops[o].W_image_dev);
       const uint8_t* payload = img + RWKVQ_HEADER_BYTES;
-      const int KT = d.ic_pad / 256;
-      if (d.method == RWKVQ_SQ) {
-        const int MB = d.oc_pad / 128;
-        const uint32_t cb = 8u * RWKVQ_SQ_RECORD_BYTES;
-        for (int rb = 0; rb < MB; ++rb)
-          for (int kt = 0; kt < KT; kt += 2) {
-            HostUnit h{};
-            h.u.fmt = UFMT_SQ;
-            h.u.src0 = (uint64_t)(uintptr_t)(payload + (size_t)(rb * KT + kt) * cb);
-            h.u.bytes0 = cb;
-            if (kt + 1 < KT) { h.u.src1 = h.u.src0 + cb; h.u.bytes1 = cb; h.ntiles = 2; }
-            else { h.u.flags |= UF_SPLIT; h.ntiles = 1; }
-            h.u.row0 = (uint32_t)rb * 128u; h.u.oc = (uint32_t)d.oc; h.u.y = (uint64_t)(uintptr_t)ops[o].y_dev;
-            h.op = o; h.rowkey = rb; h.kt = kt; h.stage = s; h.bytes = h.u.bytes0 + h.u.bytes1;
-            units.push_back(h);
-          }
-      } else {
-        const int TR = d.oc / 256;
-        const uint32_t rbytes = rwkvq_vq_record_bytes(d.bits), cb = 8u * rbytes;
-        const uint8_t* aux = img + matrix_aux_offset(&d);
-        for (int tr = 0; tr < TR; ++tr)
-          for (int kt = 0; kt < KT; ++kt) {
-            HostUnit h{};
-            h.u.fmt = d.bits == 6 ? UFMT_VQ6 : UFMT_VQ8;
-            h.u.src0 = (uint64_t)(uintptr_t)(payload + (size_t)((2 * tr) * KT + kt) * cb);
-            h.u.src1 = (uint64_t)(uintptr_t)(payload + (size_t)((2 * tr + 1) * KT + kt) * cb);
-            h.u.bytes0 = cb; h.u.bytes1 = cb;
+      const int KT = d.ic_pad / 256, MB = d.oc_pad / 128;
+      const bool vq = d.method != RWKVQ_SQ;
+      const uint32_t rb = vq ? rwkvq_vq_record_bytes(d.bits) : (uint32_t)RWKVQ_SQ_RECORD_BYTES;
+      const uint32_t cb = 8u * rb;
+      const uint8_t* aux = vq ? img + matrix_aux_offset(&d) : nullptr;
+      for (int tr = 0; tr < (MB + 1) / 2; ++tr)
+        for (int kt = 0; kt < KT; ++kt) {
+          HostUnit h;
+          std::memset(&h, 0, sizeof(h));
+          h.u.flags = vq ? (UF_VQ | (d.bits == 8 ? UF_BITS8 : 0)) : 0;
+          h.u.src0 = (uint64_t)(uintptr_t)(payload + (size_t)((2 * tr) * KT + kt) * cb);
+          h.u.bytes0 = cb;
+          if (2 * tr + 1 < MB) { h.u.src1 = (uint64_t)(uintptr_t)(payload + (size_t)((2 * tr + 1) * KT + kt) * cb); h.u.bytes1 = cb; }
+          if (vq) {
             h.u.cb_src = (uint64_t)(uintptr_t)(aux + (size_t)(tr * KT + kt) * d.entries * 4);
             h.u.cb_bytes = (uint32_t)d.entries * 4u; h.u.entries = (uint32_t)d.entries;
-            h.u.row0 = (uint32_t)tr * 256u; h.u.oc = (uint32_t)d.oc; h.u.y = (uint64_t)(uintptr_t)ops[o].y_dev;
-            h.op = o; h.rowkey = tr; h.kt = kt; h.ntiles = 1; h.stage = s;
-            h.bytes = h.u.bytes0 + h.u.bytes1 + h.u.cb_bytes;
-            units.push_back(h);
           }
-      }
+          h.u.chunk_bytes = cb; h.u.rec_bytes = rb;
+          h.u.row0 = (uint32_t)tr * 256u; h.u.oc = (uint32_t)d.oc; h.u.y = (uint64_t)(uintptr_t)ops[o].y_dev;
+          h.u.stage = (uint32_t)s;
+          h.op = o; h.tr = tr; h.kt = kt; h.stage = s;
+          units.push_back(h);
+        }
     }
-    // contiguous, byte-balanced ranges: unit -> CTA by the position of its midpoint
+    // contiguous, byte-balanced ranges cut at one eighth of a unit (the records of one warp)
     uint64_t total = 0;
-    for (const HostUnit& h : units) total += h.bytes;
+    for (const HostUnit& h : units) total += h.u.bytes0 + h.u.bytes1;
     uint64_t run = 0;
-    for (const HostUnit& h : units) {
-      const uint64_t mid = run + h.bytes / 2;
+    auto cta_of = [&](uint64_t mid) {
       int c = (int)((mid * (uint64_t)P) / (total ? total : 1));
-      if (c >= P) c = P - 1;
-      cta_units[c].push_back(h);
-      run += h.bytes;
+      return c >= P ? P - 1 : c;
+    };
+    for (const HostUnit& h : units) {
+      const uint64_t e8 = (h.u.bytes0 + h.u.bytes1) / 8;
+      int w = 0;
+      while (w < 8) {
+        const int c = cta_of(run + (uint64_t)w * e8 + e8 / 2);
+        int w1 = w + 1;
+        while (w1 < 8 && cta_of(run + (uint64_t)w1 * e8 + e8 / 2) == c) ++w1;
+        HostUnit part = h;
+        part.w0 = w; part.w1 = w1;
+        const uint32_t rb = h.u.rec_bytes;
+        part.u.off0 = (uint32_t)w * rb;
+        part.u.src0 = h.u.src0 + (uint64_t)w * rb;
+        part.u.bytes0 = (uint32_t)(w1 - w) * rb;
+        if (h.u.bytes1) { part.u.src1 = h.u.src1 + (uint64_t)w * rb; part.u.bytes1 = (uint32_t)(w1 - w) * rb; }
+        part.u.flags |= ((uint32_t)w << 8) | ((uint32_t)w1 << 12);
+        cta_units[c].push_back(part);
+        w = w1;
+      }
+      run += h.u.bytes0 + h.u.bytes1;
     }
-    for (int c = 0; c < P; ++c) push_stage_end(c, s + 1, s);
+    for (int c = 0; c < P; ++c) make_arrival(c, s + 1, s + 1);
   }
+  if (too_many_ranges) return RWKVQ_EUNSUPPORTED;   // a CTA's slice of a stage's outputs may touch at most four products
 
-  // flush flags, x segments
-  std::vector<uint32_t> unit_off(P + 1, 0), xseg_off(P + 1, 0);
+  std::vector<uint32_t> unit_off(P + 1, 0), event_off(P + 1, 0);
   std::vector<StepUnit> all_units;
-  std::vector<StepXSeg> all_segs;
+  std::vector<StepEvent> all_events;
   for (int c = 0; c < P; ++c) {
     std::vector<HostUnit>& L = cta_units[c];
     unit_off[c] = (uint32_t)all_units.size();
-    xseg_off[c] = (uint32_t)all_segs.size();
+    event_off[c] = (uint32_t)all_events.size();
     const size_t n = L.size();
+    // a group accumulates along K in registers while its consecutive units stay on the same rows
     for (size_t i = 0; i < n; ++i) {
-      if (L[i].u.fmt == UFMT_EMPTY) continue;
-      // next real unit of the same stage
-      size_t j = i + 1;
-      while (j < n && L[j].u.fmt == UFMT_EMPTY && L[j].stage == L[i].stage) ++j;
-      const bool same_run = j < n && L[j].u.fmt != UFMT_EMPTY && L[j].stage == L[i].stage && L[j].op == L[i].op &&
-                            L[j].rowkey == L[i].rowkey;
+      const size_t j = i + kGroups;
+      const bool same_run = j < n && L[j].stage == L[i].stage && L[j].op == L[i].op && L[j].tr == L[i].tr &&
+                            L[j].w0 == L[i].w0 && L[j].w1 == L[i].w1;
       if (!same_run) L[i].u.flags |= UF_FLUSH;
     }
-    // segments: maximal runs of real units of one product whose column span fits the buffer
+    all_events.push_back(cta_arrivals[c][0]);
+    uint32_t seg_no = 0;
     size_t i = 0;
-    while (i < n) {
-      if (L[i].u.fmt == UFMT_EMPTY) { ++i; continue; }
-      const int op = L[i].op;
-      const bool sums = ops[op].W_desc.method == RWKVQ_SQ;
-      const bool has_mu = ops[op].mu_image_dev != nullptr;
-      int kmin = L[i].kt, kmax = L[i].kt + L[i].ntiles;
-      size_t j = i + 1, last = i;
-      while (j < n) {
-        if (L[j].u.fmt == UFMT_EMPTY) { if (L[j].stage != L[i].stage) break; ++j; continue; }
-        if (L[j].op != op || L[j].stage != L[i].stage) break;
-        const int nmin = std::min(kmin, L[j].kt), nmax = std::max(kmax, L[j].kt + L[j].ntiles);
-        if (xseg_bytes(B, (nmax - nmin) * 256, sums, has_mu) > kXBufBytes) break;
-        kmin = nmin; kmax = nmax; last = j; ++j;
+    for (int s = 0; s < n_stages; ++s) {
+      // segments: maximal runs of units of one product whose column span fits the buffer
+      while (i < n && L[i].stage == s) {
+        const int op = L[i].op;
+        const bool sums = ops[op].W_desc.method == RWKVQ_SQ;
+        const bool has_mu = ops[op].mu_image_dev != nullptr;
+        int kmin = L[i].kt, kmax = L[i].kt + 1;
+        size_t j = i + 1, last = i;
+        while (j < n && L[j].op == op && L[j].stage == s) {
+          const int nmin = std::min(kmin, L[j].kt), nmax = std::max(kmax, L[j].kt + 1);
+          if (xseg_bytes(B, (nmax - nmin) * 256, sums, has_mu) > kXBufBytes) break;
+          kmin = nmin; kmax = nmax; last = j; ++j;
+        }
+        const int ncols = (kmax - kmin) * 256;
+        if (xseg_bytes(B, ncols, sums, has_mu) > kXBufBytes) return RWKVQ_EUNSUPPORTED;
+        StepEvent ev;
+        std::memset(&ev, 0, sizeof(ev));
+        const rwkvq_gemv_op& o = ops[op];
+        ev.kind = EV_SEGMENT;
+        ev.seg.x = (uint64_t)(uintptr_t)o.x_fp16_dev;
+        ev.segd.ic = (uint32_t)o.W_desc.ic; ev.segd.col0 = (uint32_t)kmin * 256u; ev.segd.ncols = (uint32_t)ncols;
+        const uint32_t xstride = (uint32_t)ncols * 2u + 32u;
+        ev.xstride_sums = xstride | (sums ? 0x80000000u : 0u);
+        ev.mu_off16 = (uint16_t)(xseg_mu_off(B, ncols, sums) / 16u);
+        ev.barrier = (uint32_t)s + 1u;   // stage s reads its inputs after barrier s
+        if (has_mu) {
+          const uint8_t* m = static_cast<const uint8_t*>(o.mu_image_dev);
+          ev.seg.xprev = (uint64_t)(uintptr_t)o.xprev_fp16_dev;
+          ev.seg.mu = (uint64_t)(uintptr_t)(m + RWKVQ_HEADER_BYTES);
+          ev.seg.mu_aux = (uint64_t)(uintptr_t)(m + vector_aux_offset(&o.mu_desc));
+          ev.segd.mu_bits = (uint16_t)o.mu_desc.bits; ev.segd.mu_entries = (uint16_t)o.mu_desc.entries;
+        }
+        for (size_t k = i; k <= last; ++k) {
+          L[k].u.seg = seg_no;
+          L[k].u.ev_index = (uint32_t)(all_events.size() - event_off[c]);
+          L[k].u.xcol0 = (uint32_t)(L[k].kt - kmin) * 256u;
+          L[k].u.xstride = xstride; L[k].u.gs_off = (uint32_t)B * xstride; L[k].u.nbp = nbp;
+        }
+        all_events.push_back(ev);
+        ++seg_no;
+        i = last + 1;
       }
-      const int ncols = (kmax - kmin) * 256;
-      if (xseg_bytes(B, ncols, sums, has_mu) > kXBufBytes) return RWKVQ_EUNSUPPORTED;
-      StepXSeg sg{};
-      const rwkvq_gemv_op& o = ops[op];
-      sg.x = (uint64_t)(uintptr_t)o.x_fp16_dev;
-      sg.ic = (uint32_t)o.W_desc.ic; sg.col0 = (uint32_t)kmin * 256u; sg.ncols = (uint32_t)ncols;
-      sg.sums = sums ? 1u : 0u; sg.xstride = (uint32_t)ncols * 2u + 32u;
-      sg.mu_off = xseg_mu_off(B, ncols, sums);
-      sg.barrier = (uint32_t)L[i].stage + 1u;   // stage s reads its inputs after barrier s
-      if (o.mu_image_dev) {
-        const uint8_t* m = static_cast<const uint8_t*>(o.mu_image_dev);
-        sg.xprev = (uint64_t)(uintptr_t)o.xprev_fp16_dev;
-        sg.mu = (uint64_t)(uintptr_t)(m + RWKVQ_HEADER_BYTES);
-        sg.mu_aux = (uint64_t)(uintptr_t)(m + vector_aux_offset(&o.mu_desc));
-        sg.mu_bits = (uint16_t)o.mu_desc.bits; sg.mu_entries = (uint16_t)o.mu_desc.entries;
+      all_events.push_back(cta_arrivals[c][s + 1]);
+    }
+    // what each group has to pass between its consecutive segments, and after its last unit of a stage
+    uint32_t prev_ev[kGroups] = {0, 0};
+    const StepEvent* evs = all_events.data() + event_off[c];
+    const uint32_t n_ev = (uint32_t)(all_events.size() - event_off[c]);
+    std::vector<uint32_t> arr_idx(n_stages, 0);
+    for (uint32_t e = 0; e < n_ev; ++e)
+      if (evs[e].kind == EV_ARRIVE && evs[e].barrier > 0u) arr_idx[evs[e].barrier - 1u] = e;
+    auto mask_of = [&](uint32_t first, uint32_t last_excl) {
+      uint32_t mask = 0;
+      for (uint32_t e = first; e < last_excl; ++e)
+        if (evs[e].kind == EV_ARRIVE && evs[e].barrier > 0u) mask |= 1u << (e - first);
+      return mask;
+    };
+    for (size_t k = 0; k < n; ++k) {
+      const int gidx = (int)(k % kGroups);
+      const uint32_t target = L[k].u.ev_index;
+      L[k].u.between_mask = (target > prev_ev[gidx] && target - prev_ev[gidx] - 1u <= 32u) ? mask_of(prev_ev[gidx] + 1u, target) : 0u;
+      prev_ev[gidx] = target;
+      const bool last_of_stage = k + kGroups >= n || L[k + kGroups].stage != L[k].stage;
+      const uint32_t arr = arr_idx[L[k].stage];
+      if (last_of_stage && arr > target && arr - target <= 32u) {
+        L[k].u.after_count = arr - target;
+        L[k].u.after_mask = mask_of(target + 1u, arr + 1u);
+        prev_ev[gidx] = arr;
       }
-      all_segs.push_back(sg);
-      bool first = true;
-      for (size_t k = i; k <= last; ++k) {
-        if (L[k].u.fmt == UFMT_EMPTY) continue;
-        if (first) { L[k].u.flags |= UF_NEW_XSEG; first = false; }
-        L[k].u.xcol0 = (uint32_t)(L[k].kt - kmin) * 256u;
-        L[k].u.xstride = sg.xstride; L[k].u.gs_off = (uint32_t)B * sg.xstride; L[k].u.nbp = nbp;
-      }
-      L[last].u.flags |= UF_END_XSEG;
-      i = last + 1;
     }
     for (size_t k = 0; k < n; ++k) all_units.push_back(L[k].u);
   }
   unit_off[P] = (uint32_t)all_units.size();
-  xseg_off[P] = (uint32_t)all_segs.size();
-  // A CTA's slice of a stage's outputs may touch at most four products (descriptor space).
-  if (too_many_ranges) return RWKVQ_EUNSUPPORTED;
+  event_off[P] = (uint32_t)all_events.size();
 
   info->n_units = (uint32_t)all_units.size();
-  info->n_xsegs = (uint32_t)all_segs.size();
+  info->n_events = (uint32_t)all_events.size();
   size_t off = 256;
   info->off_unit_off = off; off += round_up_sz((size_t)(P + 1) * 4, 256);
-  info->off_xseg_off = off; off += round_up_sz((size_t)(P + 1) * 4, 256);
-  info->off_units = off; off += round_up_sz(all_units.size() * sizeof(StepUnit), 256);
-  info->off_xsegs = off; off += round_up_sz(std::max<size_t>(1, all_segs.size()) * sizeof(StepXSeg), 256);
+  info->off_event_off = off; off += round_up_sz((size_t)(P + 1) * 4, 256);
+  info->off_units = off; off += round_up_sz(std::max<size_t>(1, all_units.size()) * sizeof(StepUnit), 256);
+  info->off_events = off; off += round_up_sz(all_events.size() * sizeof(StepEvent), 256);
   info->off_counter = off; off += round_up_sz((size_t)info->n_barriers * 4, 256);
   info->total_bytes = off;
   if (out) {
     out->assign(off, 0);
     memcpy(out->data() + info->off_unit_off, unit_off.data(), (size_t)(P + 1) * 4);
-    memcpy(out->data() + info->off_xseg_off, xseg_off.data(), (size_t)(P + 1) * 4);
-    memcpy(out->data() + info->off_units, all_units.data(), all_units.size() * sizeof(StepUnit));
-    if (!all_segs.empty()) memcpy(out->data() + info->off_xsegs, all_segs.data(), all_segs.size() * sizeof(StepXSeg));
+    memcpy(out->data() + info->off_event_off, event_off.data(), (size_t)(P + 1) * 4);
+    if (!all_units.empty()) memcpy(out->data() + info->off_units, all_units.data(), all_units.size() * sizeof(StepUnit));
+    memcpy(out->data() + info->off_events, all_events.data(), all_events.size() * sizeof(StepEvent));
   }
   return RWKVQ_OK;
 }
@@ -846,15 +1011,15 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
   const uint8_t* p = static_cast<const uint8_t*>(plan_dev);
   StepArgs a;
   a.units = reinterpret_cast<const StepUnit*>(p + info.off_units);
-  a.xsegs = reinterpret_cast<const StepXSeg*>(p + info.off_xsegs);
+  a.events = reinterpret_cast<const StepEvent*>(p + info.off_events);
   a.unit_off = reinterpret_cast<const uint32_t*>(p + info.off_unit_off);
-  a.xseg_off = reinterpret_cast<const uint32_t*>(p + info.off_xseg_off);
+  a.event_off = reinterpret_cast<const uint32_t*>(p + info.off_event_off);
   a.counter = reinterpret_cast<unsigned*>(const_cast<uint8_t*>(p) + info.off_counter);
   a.status = device_status_ptr();
   if (!a.status) return RWKVQ_ECUDA;
-  a.B = info.B; a.n_slots = info.n_slots; a.slot_bytes = info.slot_bytes; a.replica_bytes = info.replica_bytes;
+  a.B = info.B; a.n_slots = info.n_slots; a.n_stages = info.n_stages;
+  a.slot_bytes = info.slot_bytes; a.replica_bytes = info.replica_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  a.n_ctas = (unsigned)info.P;
   a.target = info.runs * (unsigned)info.P;
   cudaError_t e = cudaSuccess;
   if (clear_counters) {
