@@ -1,0 +1,120 @@
+"""GPU parity of the prefill product (rwkvq_gemm_prefill: dequantise to bf16 tiles, tcgen05 MMA, fp32
+accumulation) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rwkvq_oracle as orc
+from paper_2505_03803_b200 import binding as B
+from paper_2505_03803_b200 import inputs
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _bf16(a32):
+    """float32 array -> (float32 array holding the bf16-rounded values, torch bf16 device tensor)."""
+    bits = inputs.to_bf16_bits(a32)
+    vals = inputs.bf16_bits_to_f32(bits)
+    return vals, torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _run(W, mu, X_dev, xprev0_dev, M, y_dtype=torch.float32):
+    Y = torch.full((M, W.oc), float("nan"), dtype=y_dtype, device="cuda")
+    nbytes = B.rwkvq_prefill_workspace_bytes(W.desc, M, mu is not None)
+    assert nbytes > 0
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ws.fill_(0xCD)       # contents on entry must not matter
+    B.rwkvq_gemm_prefill(W.desc, W.dev, None if mu is None else mu.desc, None if mu is None else mu.dev,
+                         X_dev, xprev0_dev, M, Y, ws)
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 0
+    return Y
+
+
+def _reference(W, mu, Xv, xprev0v):
+    X64 = Xv.astype(np.float64)
+    if mu is None:
+        xm = X64
+    else:
+        prev = orc.prefill_prev(X64, None if xprev0v is None else xprev0v.astype(np.float64))
+        xm = orc.token_shift(X64, prev, mu.w_hat)
+    return xm
+
+
+def _check(W, mu, M, seed, with_prev0=True, y_dtype=torch.float32, sample_tokens=None):
+    x = inputs.gen_activation(seed, M, W.ic, n_outliers=8)
+    Xv, Xd = _bf16(x)
+    p0v, p0d = (None, None)
+    if mu is not None and with_prev0:
+        p0v, p0d = _bf16(inputs.gen_activation(seed + 1, 1, W.ic, n_outliers=8))
+        p0v = p0v.reshape(-1)
+        p0d = p0d.reshape(-1)
+    Y = _run(W, mu, Xd, p0d, M, y_dtype).float().cpu().numpy().astype(np.float64)
+    xm = _reference(W, mu, Xv, p0v)
+    rows = np.arange(M) if sample_tokens is None else np.asarray(sample_tokens)
+    ref = orc.gemv(W.w_hat, xm[rows])
+    tol = orc.tolerance(W.w_hat, xm[rows])
+    if y_dtype == torch.bfloat16:
+        tol = tol + np.abs(ref) * 2.0 ** -8
+    err = np.abs(Y[rows] - ref)
+    assert np.isfinite(Y).all()
+    ratio = float((err / np.maximum(tol, 1e-300)).max())
+    assert (err <= tol).all(), f"max err/tol = {ratio}"
+    return ratio
+
+
+@pytest.mark.parametrize("fmt", ["sq", "vq6", "vq8"])
+@pytest.mark.parametrize("M", [1, 77, 256, 300])
+def test_prefill_small_matches_oracle(fmt, M):
+    oc, ic = 256, 512
+    W = (H.pack_sq(H.random_sq_codes(M + 3, oc, ic)) if fmt == "sq"
+         else H.pack_vq(H.random_vq_codes(M + 5, oc, ic, 6 if fmt == "vq6" else 8), 6 if fmt == "vq6" else 8))
+    mu = H.pack_mu(H.random_mu_codes(M + 7, ic))
+    _check(W, mu, M, seed=M)
+    _check(W, None, M, seed=M + 1)
+    _check(W, mu, M, seed=M + 2, with_prev0=False)
+
+
+def test_prefill_identity_probe_returns_bf16_rounded_decoded_weights():
+    # X = I (bf16 ones are exact), no mix: Y[t][i] = bf16_rne(w_hat[i][t]) exactly (adding zeros is exact)
+    for W in (H.pack_sq(H.random_sq_codes(11, 384, 512)), H.pack_vq(H.random_vq_codes(12, 256, 512, 6), 6),
+              H.pack_vq(H.random_vq_codes(13, 256, 512, 8), 8)):
+        M = W.ic
+        eye = np.eye(M, dtype=np.float32)
+        _, Xd = _bf16(eye)
+        Y = _run(W, None, Xd, None, M).cpu().numpy()
+        assert np.array_equal(Y, orc.bf16_rne(W.w_hat).T)
+
+
+def test_prefill_odd_shapes_and_bf16_output():
+    W = H.pack_sq(H.random_sq_codes(21, 48, 384))        # rows and columns padded inside the image
+    _check(W, H.pack_mu(H.random_mu_codes(22, 384)), 130, seed=23)
+    W = H.pack_sq(H.random_sq_codes(24, 256, 1024))
+    _check(W, None, 513, seed=25, y_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("fmt", ["sq", "vq6"])
+def test_prefill_7b_shape_sampled(fmt):
+    oc, ic, M = 4096, 4096, 2048
+    W = H.pack_sq(H.random_sq_codes(31, oc, ic)) if fmt == "sq" else H.pack_vq(H.random_vq_codes(32, oc, ic, 6), 6)
+    mu = H.pack_mu(H.random_mu_codes(33, ic))
+    toks = [0, 1, 255, 256, 257, 1023, 1024, 2046, 2047]
+    _check(W, mu, M, seed=34, sample_tokens=toks)
+
+
+def test_prefill_argument_errors():
+    W = H.pack_sq(H.random_sq_codes(41, 128, 256))
+    X = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
+    Y = torch.zeros((4, 128), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(B.rwkvq_prefill_workspace_bytes(W.desc, 4, False), dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.RwkvqError) as e:
+        B.rwkvq_gemm_prefill(W.desc, W.dev, None, None, X, None, 4, Y, ws[:1024])
+    assert e.value.status == 5
+    with pytest.raises(B.RwkvqError) as e:
+        B.rwkvq_gemm_prefill(W.desc, W.dev, None, None, X, None, 0, Y, ws)
+    assert e.value.status == 1
+    mu = H.pack_mu(H.random_mu_codes(42, 512))
+    with pytest.raises(B.RwkvqError) as e:
+        B.rwkvq_gemm_prefill(W.desc, W.dev, mu.desc, mu.dev, X, None, 4, Y, ws)
+    assert e.value.status == 2
