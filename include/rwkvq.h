@@ -142,6 +142,25 @@ rwkvq_status rwkvq_gemv(const rwkvq_desc* W_desc, const void* W_image_dev, const
                         int B, void* y_dev, int y_dtype, void* workspace_dev, size_t workspace_bytes,
                         void* stream);
 
+/*
+ * rwkvq_gemv without a workspace argument, for callers that must not allocate device memory:
+ * code running where cudaMalloc is forbidden or unavailable (inside a pre-sized memory pool, in a
+ * real-time or embedded serving loop, in a plug-in that is only handed its inputs and outputs).
+ * The paper has no counterpart; this is a convenience of this library.  Inputs and outputs are
+ * the caller's, exactly as for rwkvq_gemv; the split-K scratch is a fixed array of
+ * rwkvq_gemv_static_max_scratch_bytes() (8 MiB) inside the library, held by every GPU that loads
+ * it until the process exits.  A product whose scratch would be larger is refused with
+ * RWKVQ_ENOMEM (use rwkvq_gemv with your own workspace).  The call allocates nothing, on host or
+ * device.  The first call on each device looks up the array's device address (that device must be
+ * current) and should therefore be made before any stream capture begins.  All calls share the
+ * one array: calls that overlap on the same GPU (different streams) race on it and give wrong
+ * results; issue them on one stream or separate them with events.
+ */
+size_t rwkvq_gemv_static_max_scratch_bytes(void);
+rwkvq_status rwkvq_gemv_static(const rwkvq_desc* W_desc, const void* W_image_dev, const rwkvq_desc* mu_desc,
+                               const void* mu_image_dev, const void* x_fp16_dev, const void* xprev_fp16_dev,
+                               int B, void* y_dev, int y_dtype, void* stream);
+
 /* One product of a decode step (same meaning as the rwkvq_gemv arguments).  `stage` orders the
  * step: every product of stage s is complete before any activation of stage s+1 is read. */
 typedef struct {

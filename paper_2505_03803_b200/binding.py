@@ -57,7 +57,7 @@ class GemvOp(C.Structure):
 EXPORTS = [
     "rwkvq_pack", "rwkvq_blob_desc", "rwkvq_blob_nbytes", "rwkvq_blob_image", "rwkvq_blob_export_codes",
     "rwkvq_image_unpack", "rwkvq_blob_free", "rwkvq_proxy_workspace_bytes", "rwkvq_proxy_select",
-    "rwkvq_gemv_workspace_bytes", "rwkvq_gemv", "rwkvq_step_plan_bytes", "rwkvq_step_plan", "rwkvq_step_run",
+    "rwkvq_gemv_workspace_bytes", "rwkvq_gemv", "rwkvq_gemv_static", "rwkvq_gemv_static_max_scratch_bytes", "rwkvq_step_plan_bytes", "rwkvq_step_plan", "rwkvq_step_run",
     "rwkvq_step_run_host",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
@@ -93,6 +93,9 @@ def lib() -> C.CDLL:
         L.rwkvq_gemv_workspace_bytes.argtypes = [C.POINTER(Desc), i32]
         L.rwkvq_gemv_workspace_bytes.restype = sz
         L.rwkvq_gemv.argtypes = [C.POINTER(Desc), vp, C.POINTER(Desc), vp, vp, vp, i32, vp, i32, vp, sz, vp]
+        L.rwkvq_gemv_static.argtypes = [C.POINTER(Desc), vp, C.POINTER(Desc), vp, vp, vp, i32, vp, i32, vp]
+        L.rwkvq_gemv_static_max_scratch_bytes.argtypes = []
+        L.rwkvq_gemv_static_max_scratch_bytes.restype = sz
         L.rwkvq_dequant.argtypes = [C.POINTER(Desc), vp, vp, i32, vp]
         L.rwkvq_device_status.argtypes = [vp]
     if hasattr(L, "rwkvq_proxy_select"):
@@ -248,6 +251,19 @@ def rwkvq_gemv(desc: Desc, W_image, mu_desc, mu_image, x, xprev, B: int, y, work
                             _dev_ptr(mu_image), _dev_ptr(x), _dev_ptr(xprev), B, _dev_ptr(y), y_dtype,
                             _dev_ptr(workspace), workspace.numel() * workspace.element_size(),
                             _stream_ptr(stream)), "rwkvq_gemv")
+
+
+def rwkvq_gemv_static_max_scratch_bytes() -> int:
+    return int(lib().rwkvq_gemv_static_max_scratch_bytes())
+
+
+def rwkvq_gemv_static(desc: Desc, W_image, mu_desc, mu_image, x, xprev, B: int, y, stream=None):
+    """rwkvq_gemv_static: same product as rwkvq_gemv, scratch inside the library (no workspace)."""
+    import torch
+    y_dtype = RWKVQ_F32 if y.dtype == torch.float32 else RWKVQ_F16
+    _check(lib().rwkvq_gemv_static(C.byref(desc), _dev_ptr(W_image), None if mu_desc is None else C.byref(mu_desc),
+                                   _dev_ptr(mu_image), _dev_ptr(x), _dev_ptr(xprev), B, _dev_ptr(y), y_dtype,
+                                   _stream_ptr(stream)), "rwkvq_gemv_static")
 
 
 def rwkvq_dequant(desc: Desc, W_image, out, stream=None):

@@ -279,6 +279,40 @@ rwkvq_status rwkvq_gemv(const rwkvq_desc* d, const void* W, const rwkvq_desc* mu
   return cuda_status(e);
 }
 
+// ---------------------------------------------------------------------------------------------
+// rwkvq_gemv for callers that cannot allocate device memory: the split-K scratch lives in a
+// file-scope device array.  In host code the array's name is only a handle; its device address
+// is looked up once per device (with that device current) and cached.
+// ---------------------------------------------------------------------------------------------
+#define RWKVQ_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[RWKVQ_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_addr[64] = {nullptr};
+
+size_t rwkvq_gemv_static_max_scratch_bytes(void) { return RWKVQ_STATIC_SCRATCH_BYTES; }
+
+rwkvq_status rwkvq_gemv_static(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu,
+                               const void* x, const void* xprev, int B, void* y, int y_dtype, void* stream) {
+  if (!d) return RWKVQ_EINVAL;
+  GemvPlan p;
+  rwkvq_status st = plan_gemv(d, B, mu != nullptr, (mu && mud) ? mud->entries : 0, &p);
+  if (st != RWKVQ_OK) return st;
+  if (p.ws_bytes > RWKVQ_STATIC_SCRATCH_BYTES) return RWKVQ_ENOMEM;   // this product needs more scratch than the built-in array holds
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_status(e);
+  if (dev < 0 || dev >= 64) return RWKVQ_EUNSUPPORTED;
+  void* ws = g_static_scratch_addr[dev];
+  if (!ws) {
+    e = cudaGetSymbolAddress(&ws, g_static_scratch);
+    if (e != cudaSuccess) return cuda_status(e);
+    g_static_scratch_addr[dev] = ws;
+  }
+  // The array keeps whatever the previous call left: the arrival counters must start at zero.
+  e = cudaMemsetAsync(ws, 0, p.counters_bytes, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_status(e);
+  return rwkvq_gemv(d, W, mud, mu, x, xprev, B, y, y_dtype, ws, RWKVQ_STATIC_SCRATCH_BYTES, stream);
+}
+
 rwkvq_status rwkvq_dequant(const rwkvq_desc* d, const void* W, void* out, int dtype, void* stream) {
   if (!d || !W || !out) return RWKVQ_EINVAL;
   if (dtype != RWKVQ_F32 && dtype != RWKVQ_BF16) return RWKVQ_EINVAL;
