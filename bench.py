@@ -50,6 +50,7 @@ def parse_args(argv=None):
     ap.add_argument("--mode", default="step", choices=["step", "ops"],
                     help="step = one persistent launch per step; ops = one rwkvq_gemv launch per product")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the prefill leg (one 7B-class layer, M = 2048)")
     return ap.parse_args(argv)
 
 
@@ -249,6 +250,67 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------
+# prefill leg: one 7B-class layer, M = 2048 tokens, through rwkvq_gemm_prefill
+# ---------------------------------------------------------------------------------------------
+def measured_bf16_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def prefill_leg(reps: int = 10, M: int = 2048):
+    """All eight projections of one 7B-class layer (d = 4096, h = 14336) over M tokens: random valid
+    logical codes (the time does not depend on the code values), SQ for the matrices the seeded coin
+    makes Gaussian and VQ-64 for the heavy-tailed ones, token-shift mix on R, K, V, G and cm_k.
+    Returns TFLOP/s over the layer (2*M*oc*ic per matrix) and the fraction of the measured bf16 peak."""
+    import torch
+    from paper_2505_03803_b200 import binding as B
+    from paper_2505_03803_b200 import inputs
+    sp = inputs.STACKS["c3_7b"]
+    mats = []
+    for (name, oc, ic, has_mu, stage) in inputs.layer_shapes(sp["d"], sp["h"]):
+        seed = inputs.seed_of("c5_prefill", name)
+        if inputs.weight_kind(seed) == "gauss":
+            blob = B.rwkvq_pack(None, oc, ic, B.RWKVQ_SQ, 3, codes=inputs.random_sq_codes(seed, oc, ic))
+        else:
+            blob = B.rwkvq_pack(None, oc, ic, B.RWKVQ_VQ, 6, codes=inputs.random_vq_codes(seed, oc, ic, 6))
+        mu = B.rwkvq_pack(None, 1, ic, B.RWKVQ_VQ, 6, codes=inputs.random_mu_codes(seed + 1, ic)) if has_mu else None
+        x = inputs.gen_activation(seed + 2, M, ic, sp["outliers"])
+        X = torch.from_numpy(inputs.to_bf16_bits(x).view(np.int16)).cuda().view(torch.bfloat16)
+        Y = torch.empty((M, oc), dtype=torch.float32, device="cuda")
+        ws = torch.empty(B.rwkvq_prefill_workspace_bytes(blob.desc, M, has_mu), dtype=torch.uint8, device="cuda")
+        mats.append((blob.desc, blob.to_device(), mu.desc if mu else None, mu.to_device() if mu else None, X, Y, ws, oc, ic))
+
+    def layer():
+        for (d, W, md, m, X, Y, ws, oc, ic) in mats:
+            B.rwkvq_gemm_prefill(d, W, md, m, X, None, M, Y, ws)
+    for _ in range(3):
+        layer()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        layer()
+    e1.record()
+    torch.cuda.synchronize()
+    if B.rwkvq_device_status() != 0:
+        raise SystemExit("bench.py: a device-side wait timed out in the prefill leg")
+    ms = e0.elapsed_time(e1) / reps
+    flops = sum(2.0 * M * oc * ic for (*_r, oc, ic) in mats)
+    tf = flops / (ms * 1e-3) / 1e12
+    peak, kind = measured_bf16_peak()
+    return {"workload": f"one 7B-class layer (8 projections, d=4096 h=14336), M={M} tokens, hybrid SQ/VQ-64, bf16 x bf16 -> fp32",
+            "ms_per_layer": ms, "flop_per_layer": flops, "launches_per_layer": 2 * len(mats), "sq_matrices":
+            sum(1 for m in mats if m[0].method == B.RWKVQ_SQ),
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                         "traffic": None, "peak_kind": f"of {kind} (burst)", "kernel": "prefill_kernel",
+                         "frac_of_2250_nominal": tf / 2250.0}}
+
+
+# ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -369,6 +431,10 @@ def run_ours(args):
             dist.destroy_process_group()
         return 0
 
+    prefill = None
+    if world == 1 and not args.no_prefill:
+        prefill = prefill_leg()
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         r = time_oracle(args.workload, batch, budget_s=12.0)
@@ -391,7 +457,7 @@ def run_ours(args):
                    "tau_c": st.tau_c, "setup_s": round(setup_s, 1)},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": K * launches_per_step,
-        "hbm_gbs": achieved,
+        "hbm_gbs": achieved, "prefill": prefill,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
