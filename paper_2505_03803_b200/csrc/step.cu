@@ -170,6 +170,9 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ void red_release_gpu(unsigned* p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void smem_add_release(uint32_t* p, uint32_t v) {
   asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
@@ -304,7 +307,7 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       // barrier 0 (the clearing pass) has no consumer work before it; barrier j closes stage j - 1,
       // which all sixteen consumer warps must have reported, like every stage before it
       if (pending > 0) ok = wait_count(&ctrl->cdone, (uint32_t)kConsumerWarps * narrive, abortp, a.status);
-      if (ok) { __threadfence(); atomicAdd(a.counter + pending, 1u); }
+      if (ok) red_release_gpu(a.counter + pending, 1u);
     }
     ++narrive;
     pending = -1;
@@ -475,9 +478,11 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
   int held = -1;              // input segment this warp currently holds
   uint32_t seg_next = 0;      // number of segment events passed so far
   uint32_t cur_ev = 0;        // last event processed (event 0 is the clearing arrival: nothing to do)
-  // Report the current stage as finished: the warp's reductions into y are ordered before the
-  // count by the warp barrier and the release.
+  // Report the current stage as finished.  Every lane first makes its own reductions into y
+  // visible GPU-wide (all lanes and warps wait in parallel), so that the stager's single arrival
+  // at the grid barrier has nothing left to wait for.
   auto arrive_stage = [&]() {
+    __threadfence();
     __syncwarp();
     if (lane == 0 && !dead) smem_add_release(&ctrl->cdone, 1u);
   };
@@ -868,10 +873,16 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         const bool has_mu = ops[op].mu_image_dev != nullptr;
         int kmin = L[i].kt, kmax = L[i].kt + 1;
         size_t j = i + 1, last = i;
+        // A segment is a contiguous run of column tiles (a range that wraps from the end of one row
+        // pair to the start of the next starts a new segment), small enough that staging it is about
+        // one round of loads per stager thread.
+        const int max_tiles = std::max(1, 12 / B);
         while (j < n && L[j].op == op && L[j].stage == s) {
-          const int nmin = std::min(kmin, L[j].kt), nmax = std::max(kmax, L[j].kt + 1);
-          if (xseg_bytes(B, (nmax - nmin) * 256, sums, has_mu) > kXBufBytes) break;
-          kmin = nmin; kmax = nmax; last = j; ++j;
+          if (L[j].kt < kmin || L[j].kt > kmax) break;
+          const int nmax = std::max(kmax, L[j].kt + 1);
+          if (nmax - kmin > max_tiles) break;
+          if (xseg_bytes(B, (nmax - kmin) * 256, sums, has_mu) > kXBufBytes) break;
+          kmax = nmax; last = j; ++j;
         }
         const int ncols = (kmax - kmin) * 256;
         if (xseg_bytes(B, ncols, sums, has_mu) > kXBufBytes) return RWKVQ_EUNSUPPORTED;
