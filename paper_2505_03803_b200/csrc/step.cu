@@ -874,13 +874,10 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         int kmin = L[i].kt, kmax = L[i].kt + 1;
         size_t j = i + 1, last = i;
         // A segment is a contiguous run of column tiles (a range that wraps from the end of one row
-        // pair to the start of the next starts a new segment), small enough that staging it is about
-        // one round of loads per stager thread.
-        const int max_tiles = std::max(1, 12 / B);
+        // pair to the start of the next starts a new segment) that fits the buffer.
         while (j < n && L[j].op == op && L[j].stage == s) {
           if (L[j].kt < kmin || L[j].kt > kmax) break;
           const int nmax = std::max(kmax, L[j].kt + 1);
-          if (nmax - kmin > max_tiles) break;
           if (xseg_bytes(B, (nmax - kmin) * 256, sums, has_mu) > kXBufBytes) break;
           kmax = nmax; last = j; ++j;
         }
