@@ -9,7 +9,8 @@
 // tokens:
 //   * a producer warp streams packed chunks (13-17 KB per 256 columns) and activation tiles
 //     (32 KB per 64 columns) into shared-memory rings with cp.async.bulk + mbarrier transactions;
-//   * eight dequantisation warps, one per 16-row record, turn 64 columns at a time into bf16 with
+//   * sixteen dequantisation warps (two groups of eight, one warp per 16-row record, alternating
+//     64-column blocks) turn packed codes into bf16 with
 //     the shared unpack routines, exactly bf16_rne(s * (q - z)) or bf16_rne(codebook entry), and
 //     store them in the K-major 128-byte-swizzled layout; a proxy fence hands them to the tensor core;
 //   * one thread issues tcgen05.mma (A = weights 128 x 16, B = activations 256 x 16, fp32
@@ -43,7 +44,7 @@ constexpr uint32_t kPackedSlot = 8 * 2048 + 1024;             // largest chunk (
 constexpr int kPackedSlots = 2;
 constexpr uint32_t kCtrlBytes = 1024;
 constexpr uint32_t kSmemBytes = kCtrlBytes + kStages * kStageBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
-constexpr int kDequantWarps = 8, kEpilogueWarps = 4;
+constexpr int kRecordWarps = 8, kDequantGroups = 2, kDequantWarps = kRecordWarps * kDequantGroups, kEpilogueWarps = 4;
 constexpr int kThreads = 32 * (2 + kDequantWarps + kEpilogueWarps);
 constexpr uint32_t kPollLimit = 1u << 22;
 constexpr uint32_t kTmemCols = 512;
@@ -220,10 +221,11 @@ __device__ __forceinline__ void sq_store_triple(const uint32_t (&r)[16], uint32_
 #pragma unroll
       for (int p = 0; p < 2; ++p) {
         const int e = 4 * m + 2 * p + h;
-        const float bias = (float)(1024 >> rwkvq_sq_pos(e));
-        const float2 qb = __half22float2(*reinterpret_cast<const __half2*>(&r[e]));
-        const float v0 = __fmul_rn(s, __fsub_rn(qb.x - bias, z));
-        const float v1 = __fmul_rn(s, __fsub_rn(qb.y - bias, z));
+        // (q + bias) - bias is exact in fp16: both are integers below 2048
+        const __half2 bias2 = __float2half2_rn((float)(1024 >> rwkvq_sq_pos(e)));
+        const float2 qf = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&r[e]), bias2));
+        const float v0 = __fmul_rn(s, __fsub_rn(qf.x, z));
+        const float v1 = __fmul_rn(s, __fsub_rn(qf.y, z));
         out[p] = pack_bf16(v0, v1);
       }
       const uint32_t off = sw128_offset((uint32_t)(row_base + g + 8 * h), (uint32_t)(16 * m + 4 * t));
@@ -272,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
   volatile int* abortp = &ctrl->abort_flag;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPackedSlots; ++s) { mbar_init(&ctrl->wfull[s], 1); mbar_init(&ctrl->wempty[s], kDequantWarps); }
-    for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->wready[s], kDequantWarps); mbar_init(&ctrl->sempty[s], 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->wready[s], kRecordWarps); mbar_init(&ctrl->sempty[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->accfull[s], 1); mbar_init(&ctrl->accempty[s], kEpilogueWarps); }
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -342,7 +344,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
     }
   } else if (warp < 2 + kDequantWarps) {
     // ---- dequantisation: warp dw owns record dw (rows 16 dw .. 16 dw + 15 of the chunk) --------------
-    const int dw = warp - 2, g = lane >> 2;
+    // two groups of eight warps take the 64-column blocks alternately, so that one group's unpacking
+    // overlaps the other's stores and barrier traffic
+    const int dw = (warp - 2) & 7, dg = (warp - 2) >> 3, g = lane >> 2;
     uint32_t kt_iter = 0, kb_iter = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x) {
@@ -365,6 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
 #pragma unroll
         for (int q = 0; q < 4; ++q, ++kb_iter) {
           const int st = (int)(kb_iter % kStages);
+          if ((q & 1) != dg) continue;          // the other group's block (blocks per tile are a multiple of four)
           if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->sempty[st], ((kb_iter / kStages) & 1u) ^ 1u, abortp, a.status));
           if (ok) {
             uint8_t* wtile = stages + (size_t)st * kStageBytes + kXTileBytes;
