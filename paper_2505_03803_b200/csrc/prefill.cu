@@ -36,14 +36,13 @@ int* device_status_ptr();  // api_misc.cu
 namespace pf {
 
 constexpr int kTileTokens = 256, kTileRows = 128, kKBlock = 64;
-constexpr int kStages = 3;
+constexpr int kXStages = 3, kWStages = 5;   // activation tiles (32 KB) and dequantised weight tiles (16 KB) have rings of their own
 constexpr uint32_t kXTileBytes = kTileTokens * kKBlock * 2;   // 32 KB: activations of one stage
 constexpr uint32_t kWTileBytes = kTileRows * kKBlock * 2;     // 16 KB: dequantised weights of one stage
-constexpr uint32_t kStageBytes = kXTileBytes + kWTileBytes;
 constexpr uint32_t kPackedSlot = 8 * 2048 + 1024;             // largest chunk (VQ, 8-bit) + its codebook
 constexpr int kPackedSlots = 2;
 constexpr uint32_t kCtrlBytes = 1024;
-constexpr uint32_t kSmemBytes = kCtrlBytes + kStages * kStageBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
+constexpr uint32_t kSmemBytes = kCtrlBytes + kXStages * kXTileBytes + kWStages * kWTileBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
 constexpr int kRecordWarps = 8, kDequantGroups = 2, kDequantWarps = kRecordWarps * kDequantGroups, kEpilogueWarps = 4;
 constexpr int kThreads = 32 * (2 + kDequantWarps + kEpilogueWarps);
 constexpr uint32_t kPollLimit = 1u << 22;
@@ -192,7 +191,7 @@ enum { PF_SQ3 = 0, PF_VQ6 = 1, PF_VQ8 = 2 };
 
 struct Ctrl {
   uint64_t wfull[kPackedSlots], wempty[kPackedSlots];
-  uint64_t xfull[kStages], wready[kStages], sempty[kStages];
+  uint64_t xfull[kXStages], xempty[kXStages], wready[kWStages], wfree[kWStages];
   uint64_t accfull[2], accempty[2];
   uint32_t tmem_base;
   int abort_flag;
@@ -268,13 +267,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
   // operand tiles need 1024-byte alignment (8 rows of 128 bytes per swizzle group)
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
-  uint8_t* stages = smem + kCtrlBytes;                       // [kStages][X tile 32 KB | W tile 16 KB]
-  uint8_t* packed = stages + kStages * kStageBytes;          // [kPackedSlots][chunk | codebook]
+  uint8_t* xring = smem + kCtrlBytes;                        // [kXStages] activation tiles
+  uint8_t* wring = xring + kXStages * kXTileBytes;           // [kWStages] dequantised weight tiles
+  uint8_t* packed = wring + kWStages * kWTileBytes;          // [kPackedSlots][chunk | codebook]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abortp = &ctrl->abort_flag;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPackedSlots; ++s) { mbar_init(&ctrl->wfull[s], 1); mbar_init(&ctrl->wempty[s], kDequantWarps); }
-    for (int s = 0; s < kStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->wready[s], kRecordWarps); mbar_init(&ctrl->sempty[s], 1); }
+    for (int s = 0; s < kXStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->xempty[s], 1); }
+    for (int s = 0; s < kWStages; ++s) { mbar_init(&ctrl->wready[s], kRecordWarps); mbar_init(&ctrl->wfree[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->accfull[s], 1); mbar_init(&ctrl->accempty[s], kEpilogueWarps); }
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -301,17 +302,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
           bulk_g2s(dst, a.payload + (size_t)(mb * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->wfull[slot]);
           if (a.cb_bytes) bulk_g2s(dst + a.chunk_bytes, a.aux + (size_t)((mb >> 1) * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->wfull[slot]);
           for (int q = 0; q < 4 && ok; ++q, ++kb_iter) {
-            const int st = (int)(kb_iter % kStages);
-            ok = mbar_wait(&ctrl->sempty[st], ((kb_iter / kStages) & 1u) ^ 1u, abortp, a.status);
+            const int st = (int)(kb_iter % kXStages);
+            ok = mbar_wait(&ctrl->xempty[st], ((kb_iter / kXStages) & 1u) ^ 1u, abortp, a.status);
             if (!ok) break;
             mbar_arrive_expect_tx(&ctrl->xfull[st], kXTileBytes);
-            bulk_g2s(stages + (size_t)st * kStageBytes, a.xtiles + ((size_t)mt * a.KB + (kt * 4 + q)) * kXTileBytes, kXTileBytes, &ctrl->xfull[st]);
+            bulk_g2s(xring + (size_t)st * kXTileBytes, a.xtiles + ((size_t)mt * a.KB + (kt * 4 + q)) * kXTileBytes, kXTileBytes, &ctrl->xfull[st]);
           }
         }
       }
       // do not leave while copies issued by this thread may still be landing
-      for (uint32_t i = (kb_iter > kStages ? kb_iter - kStages : 0); i < kb_iter; ++i)
-        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->xfull[i % kStages], (i / kStages) & 1u)) break;
+      for (uint32_t i = (kb_iter > kXStages ? kb_iter - kXStages : 0); i < kb_iter; ++i)
+        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->xfull[i % kXStages], (i / kXStages) & 1u)) break;
       for (uint32_t i = (kt_iter > kPackedSlots ? kt_iter - kPackedSlots : 0); i < kt_iter; ++i)
         for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->wfull[i % kPackedSlots], (i / kPackedSlots) & 1u)) break;
     }
@@ -328,16 +329,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + set * (uint32_t)kTileTokens;
         for (int kb = 0; kb < a.KB && ok; ++kb, ++kb_iter) {
-          const int st = (int)(kb_iter % kStages);
-          const uint32_t ph = (kb_iter / kStages) & 1u;
-          ok = mbar_wait(&ctrl->xfull[st], ph, abortp, a.status) && mbar_wait(&ctrl->wready[st], ph, abortp, a.status);
+          const int xst = (int)(kb_iter % kXStages), wst = (int)(kb_iter % kWStages);
+          ok = mbar_wait(&ctrl->xfull[xst], (kb_iter / kXStages) & 1u, abortp, a.status) &&
+               mbar_wait(&ctrl->wready[wst], (kb_iter / kWStages) & 1u, abortp, a.status);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t xs = smem_u32(stages + (size_t)st * kStageBytes), ws = xs + kXTileBytes;
+          const uint32_t xs = smem_u32(xring + (size_t)xst * kXTileBytes), ws = smem_u32(wring + (size_t)wst * kWTileBytes);
 #pragma unroll
           for (int k = 0; k < kKBlock / 16; ++k)
             umma_bf16(tmem_d, smem_desc_sw128(ws + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(&ctrl->sempty[st]);     // the stage is free once these products have read it
+          umma_commit(&ctrl->xempty[xst]);    // both tiles are free once these products have read them
+          umma_commit(&ctrl->wfree[wst]);
         }
         if (ok) umma_commit(&ctrl->accfull[set]);
       }
@@ -368,11 +370,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
         if (a.fmt == PF_SQ3) sz = *reinterpret_cast<const uint4*>(rec + RWKVQ_SQ_CODE_BYTES + g * 16);
 #pragma unroll
         for (int q = 0; q < 4; ++q, ++kb_iter) {
-          const int st = (int)(kb_iter % kStages);
+          const int st = (int)(kb_iter % kWStages);
           if ((q & 1) != dg) continue;          // the other group's block (blocks per tile are a multiple of four)
-          if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->sempty[st], ((kb_iter / kStages) & 1u) ^ 1u, abortp, a.status));
+          if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfree[st], ((kb_iter / kWStages) & 1u) ^ 1u, abortp, a.status));
           if (ok) {
-            uint8_t* wtile = stages + (size_t)st * kStageBytes + kXTileBytes;
+            uint8_t* wtile = wring + (size_t)st * kWTileBytes;
             if (a.fmt == PF_SQ3) {
               uint32_t r[16];
               sq_unpack_triple(w[3 * q], w[3 * q + 1], w[3 * q + 2], r);
