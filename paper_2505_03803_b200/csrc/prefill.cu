@@ -5,18 +5,18 @@
 // writes the result tile by tile in the shared-memory operand layout of the tensor core (tiles of
 // 256 tokens x 64 columns, 128-byte rows, 128-byte swizzle), so that the main kernel fetches an
 // operand tile with ONE bulk asynchronous copy.  (2) The main kernel is persistent, one CTA per
-// SM, each looping over output tiles of 128 weight rows (one chunk of the packed image) x 256
-// tokens:
-//   * a producer warp streams packed chunks (13-17 KB per 256 columns) and activation tiles
-//     (32 KB per 64 columns) into shared-memory rings with cp.async.bulk + mbarrier transactions;
-//   * sixteen dequantisation warps (two groups of eight, one warp per 16-row record, alternating
-//     64-column blocks) turn packed codes into bf16 with
+// SM, each looping over output tiles of 256 weight rows (two chunks of the packed image) x 256
+// tokens, so that one activation tile feeds two products:
+//   * a producer warp streams packed chunk pairs (27-34 KB per 256 columns) and activation tiles
+//     (32 KB per 64 columns) into shared memory with cp.async.bulk + mbarrier transactions;
+//   * sixteen dequantisation warps (one group of eight per row half, one warp per 16-row record)
+//     turn packed codes into bf16 with
 //     the shared unpack routines, exactly bf16_rne(s * (q - z)) or bf16_rne(codebook entry), and
 //     store them in the K-major 128-byte-swizzled layout; a proxy fence hands them to the tensor core;
 //   * one thread issues tcgen05.mma (A = weights 128 x 16, B = activations 256 x 16, fp32
-//     accumulators in tensor memory, two accumulator sets) and commits to mbarriers;
-//   * four epilogue warps read an accumulator set with tcgen05.ld (lane = weight row, so a warp
-//     writes 32 consecutive outputs of one token) while the next tile's products run.
+//     accumulators in tensor memory, one of 256 columns per row half) and commits to mbarriers;
+//   * four epilogue warps read the accumulators with tcgen05.ld (lane = weight row, so a warp
+//     writes 32 consecutive outputs of one token) while the next tile's operands stream in.
 // Every wait is bounded; a wait that gives up raises the device status word and all roles leave
 // through the common exit, where tensor memory is freed.
 #include <cuda_bf16.h>
@@ -36,13 +36,13 @@ int* device_status_ptr();  // api_misc.cu
 namespace pf {
 
 constexpr int kTileTokens = 256, kTileRows = 128, kKBlock = 64;
-constexpr int kXStages = 3, kWStages = 5;   // activation tiles (32 KB) and dequantised weight tiles (16 KB) have rings of their own
+constexpr int kXStages = 3, kWStages = 2;   // rings: activation tiles (32 KB); dequantised weight tiles (16 KB), one ring per row half
 constexpr uint32_t kXTileBytes = kTileTokens * kKBlock * 2;   // 32 KB: activations of one stage
 constexpr uint32_t kWTileBytes = kTileRows * kKBlock * 2;     // 16 KB: dequantised weights of one stage
-constexpr uint32_t kPackedSlot = 8 * 2048 + 1024;             // largest chunk (VQ, 8-bit) + its codebook
-constexpr int kPackedSlots = 2;
+constexpr uint32_t kPackedSlot = 2 * 8 * 2048 + 1024;         // two largest chunks (VQ, 8-bit) + their codebook
+constexpr int kPackedSlots = 1;
 constexpr uint32_t kCtrlBytes = 1024;
-constexpr uint32_t kSmemBytes = kCtrlBytes + kXStages * kXTileBytes + kWStages * kWTileBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
+constexpr uint32_t kSmemBytes = kCtrlBytes + kXStages * kXTileBytes + 2 * kWStages * kWTileBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
 constexpr int kRecordWarps = 8, kDequantGroups = 2, kDequantWarps = kRecordWarps * kDequantGroups, kEpilogueWarps = 4;
 constexpr int kThreads = 32 * (2 + kDequantWarps + kEpilogueWarps);
 constexpr uint32_t kPollLimit = 1u << 22;
@@ -191,8 +191,8 @@ enum { PF_SQ3 = 0, PF_VQ6 = 1, PF_VQ8 = 2 };
 
 struct Ctrl {
   uint64_t wfull[kPackedSlots], wempty[kPackedSlots];
-  uint64_t xfull[kXStages], xempty[kXStages], wready[kWStages], wfree[kWStages];
-  uint64_t accfull[2], accempty[2];
+  uint64_t xfull[kXStages], xempty[kXStages], wready[2][kWStages], wfree[2][kWStages];
+  uint64_t accfull, accempty;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -268,15 +268,16 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
   uint8_t* xring = smem + kCtrlBytes;                        // [kXStages] activation tiles
-  uint8_t* wring = xring + kXStages * kXTileBytes;           // [kWStages] dequantised weight tiles
-  uint8_t* packed = wring + kWStages * kWTileBytes;          // [kPackedSlots][chunk | codebook]
+  uint8_t* wring = xring + kXStages * kXTileBytes;           // [2 row halves][kWStages] dequantised weight tiles
+  uint8_t* packed = wring + 2 * kWStages * kWTileBytes;      // [chunk A | chunk B | codebook]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abortp = &ctrl->abort_flag;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPackedSlots; ++s) { mbar_init(&ctrl->wfull[s], 1); mbar_init(&ctrl->wempty[s], kDequantWarps); }
     for (int s = 0; s < kXStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->xempty[s], 1); }
-    for (int s = 0; s < kWStages; ++s) { mbar_init(&ctrl->wready[s], kRecordWarps); mbar_init(&ctrl->wfree[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->accfull[s], 1); mbar_init(&ctrl->accempty[s], kEpilogueWarps); }
+    for (int h = 0; h < 2; ++h)
+      for (int s = 0; s < kWStages; ++s) { mbar_init(&ctrl->wready[h][s], kRecordWarps); mbar_init(&ctrl->wfree[h][s], 1); }
+    mbar_init(&ctrl->accfull, 1); mbar_init(&ctrl->accempty, kEpilogueWarps);
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -285,6 +286,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctrl->tmem_base;
+  // A tile is 256 weight rows (row pair tr: chunks 2 tr and 2 tr + 1 of the image) x 256 tokens: one
+  // activation tile feeds two products, which halves the activation traffic from L2 per FLOP.
+  // The last row pair of a matrix with an odd number of chunks has only its first half.
 
   if (warp == 0) {
     // ---- producer ------------------------------------------------------------------------------
@@ -292,15 +296,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
       uint32_t kt_iter = 0, kb_iter = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x) {
-        const int mb = tile / a.MT, mt = tile % a.MT;
+        const int tr = tile / a.MT, mt = tile % a.MT;
+        const bool has_b = 2 * tr + 1 < a.MB;
         for (int kt = 0; kt < a.KT && ok; ++kt, ++kt_iter) {
-          const int slot = (int)(kt_iter % kPackedSlots);
-          ok = mbar_wait(&ctrl->wempty[slot], ((kt_iter / kPackedSlots) & 1u) ^ 1u, abortp, a.status);
+          ok = mbar_wait(&ctrl->wempty[0], (kt_iter & 1u) ^ 1u, abortp, a.status);
           if (!ok) break;
-          uint8_t* dst = packed + (size_t)slot * kPackedSlot;
-          mbar_arrive_expect_tx(&ctrl->wfull[slot], a.chunk_bytes + a.cb_bytes);
-          bulk_g2s(dst, a.payload + (size_t)(mb * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->wfull[slot]);
-          if (a.cb_bytes) bulk_g2s(dst + a.chunk_bytes, a.aux + (size_t)((mb >> 1) * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->wfull[slot]);
+          mbar_arrive_expect_tx(&ctrl->wfull[0], a.chunk_bytes * (has_b ? 2u : 1u) + a.cb_bytes);
+          bulk_g2s(packed, a.payload + (size_t)((2 * tr) * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->wfull[0]);
+          if (has_b) bulk_g2s(packed + a.chunk_bytes, a.payload + (size_t)((2 * tr + 1) * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->wfull[0]);
+          if (a.cb_bytes) bulk_g2s(packed + 2 * a.chunk_bytes, a.aux + (size_t)(tr * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->wfull[0]);
           for (int q = 0; q < 4 && ok; ++q, ++kb_iter) {
             const int st = (int)(kb_iter % kXStages);
             ok = mbar_wait(&ctrl->xempty[st], ((kb_iter / kXStages) & 1u) ^ 1u, abortp, a.status);
@@ -313,119 +317,139 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
       // do not leave while copies issued by this thread may still be landing
       for (uint32_t i = (kb_iter > kXStages ? kb_iter - kXStages : 0); i < kb_iter; ++i)
         for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->xfull[i % kXStages], (i / kXStages) & 1u)) break;
-      for (uint32_t i = (kt_iter > kPackedSlots ? kt_iter - kPackedSlots : 0); i < kt_iter; ++i)
-        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->wfull[i % kPackedSlots], (i / kPackedSlots) & 1u)) break;
+      if (kt_iter > 0)
+        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->wfull[0], (kt_iter - 1u) & 1u)) break;
     }
   } else if (warp == 1) {
     // ---- tensor-core issue -----------------------------------------------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16(kTileRows, kTileTokens);
-      uint32_t kb_iter = 0, tile_iter = 0;
+      uint32_t kb_iter = 0, kb_b = 0, tile_iter = 0;     // kb_b counts the blocks of tiles that have a second half
       bool ok = true;
       for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x, ++tile_iter) {
-        const uint32_t set = tile_iter & 1u;
-        ok = mbar_wait(&ctrl->accempty[set], ((tile_iter >> 1) & 1u) ^ 1u, abortp, a.status);
+        const int tr = tile / a.MT;
+        const bool has_b = 2 * tr + 1 < a.MB;
+        ok = mbar_wait(&ctrl->accempty, (tile_iter & 1u) ^ 1u, abortp, a.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tmem_d = tmem_base + set * (uint32_t)kTileTokens;
         for (int kb = 0; kb < a.KB && ok; ++kb, ++kb_iter) {
-          const int xst = (int)(kb_iter % kXStages), wst = (int)(kb_iter % kWStages);
+          const int xst = (int)(kb_iter % kXStages), sa = (int)(kb_iter % kWStages);
           ok = mbar_wait(&ctrl->xfull[xst], (kb_iter / kXStages) & 1u, abortp, a.status) &&
-               mbar_wait(&ctrl->wready[wst], (kb_iter / kWStages) & 1u, abortp, a.status);
+               mbar_wait(&ctrl->wready[0][sa], (kb_iter / kWStages) & 1u, abortp, a.status);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t xs = smem_u32(xring + (size_t)xst * kXTileBytes), ws = smem_u32(wring + (size_t)wst * kWTileBytes);
+          const uint32_t xs = smem_u32(xring + (size_t)xst * kXTileBytes);
+          const uint32_t wa = smem_u32(wring + (size_t)sa * kWTileBytes);
 #pragma unroll
           for (int k = 0; k < kKBlock / 16; ++k)
-            umma_bf16(tmem_d, smem_desc_sw128(ws + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(&ctrl->xempty[xst]);    // both tiles are free once these products have read them
-          umma_commit(&ctrl->wfree[wst]);
+            umma_bf16(tmem_base, smem_desc_sw128(wa + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(&ctrl->wfree[0][sa]);
+          if (has_b) {
+            const int sb = (int)(kb_b % kWStages);
+            ok = mbar_wait(&ctrl->wready[1][sb], (kb_b / kWStages) & 1u, abortp, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t wb = smem_u32(wring + (size_t)(kWStages + sb) * kWTileBytes);
+#pragma unroll
+            for (int k = 0; k < kKBlock / 16; ++k)
+              umma_bf16(tmem_base + (uint32_t)kTileTokens, smem_desc_sw128(wb + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            umma_commit(&ctrl->wfree[1][sb]);
+            ++kb_b;
+          }
+          umma_commit(&ctrl->xempty[xst]);    // the activation tile is free once both products have read it
         }
-        if (ok) umma_commit(&ctrl->accfull[set]);
+        if (ok) umma_commit(&ctrl->accfull);
       }
     }
   } else if (warp < 2 + kDequantWarps) {
-    // ---- dequantisation: warp dw owns record dw (rows 16 dw .. 16 dw + 15 of the chunk) --------------
-    // two groups of eight warps take the 64-column blocks alternately, so that one group's unpacking
-    // overlaps the other's stores and barrier traffic
+    // ---- dequantisation: group dg takes row half dg of the tile, warp dw its record dw (16 rows) ----
     const int dw = (warp - 2) & 7, dg = (warp - 2) >> 3, g = lane >> 2;
-    uint32_t kt_iter = 0, kb_iter = 0;
+    uint32_t kt_iter = 0, kbm = 0;      // kbm: 64-column blocks this group has produced
     bool ok = true;
     for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x) {
+      const int tr = tile / a.MT;
+      const bool mine = dg == 0 || 2 * tr + 1 < a.MB;     // the second half may be absent
       for (int kt = 0; kt < a.KT && ok; ++kt, ++kt_iter) {
-        const int slot = (int)(kt_iter % kPackedSlots);
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfull[slot], (kt_iter / kPackedSlots) & 1u, abortp, a.status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfull[0], kt_iter & 1u, abortp, a.status));
         if (!ok) break;
-        const uint8_t* rec = packed + (size_t)slot * kPackedSlot + (size_t)dw * a.rec_bytes;
-        const uint32_t* cb = reinterpret_cast<const uint32_t*>(packed + (size_t)slot * kPackedSlot + a.chunk_bytes);
+        const uint8_t* rec = packed + (size_t)dg * a.chunk_bytes + (size_t)dw * a.rec_bytes;
+        const uint32_t* cb = reinterpret_cast<const uint32_t*>(packed + 2 * a.chunk_bytes);
         uint32_t w[16];
         uint4 sz = make_uint4(0, 0, 0, 0);
         const int nplanes = a.fmt == PF_VQ8 ? 4 : 3;
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
           uint4 v = make_uint4(0, 0, 0, 0);
-          if (p < nplanes) v = *reinterpret_cast<const uint4*>(rec + p * 512 + lane * 16);
+          if (mine && p < nplanes) v = *reinterpret_cast<const uint4*>(rec + p * 512 + lane * 16);
           w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
         }
-        if (a.fmt == PF_SQ3) sz = *reinterpret_cast<const uint4*>(rec + RWKVQ_SQ_CODE_BYTES + g * 16);
+        if (mine && a.fmt == PF_SQ3) sz = *reinterpret_cast<const uint4*>(rec + RWKVQ_SQ_CODE_BYTES + g * 16);
+        // SQ needs nothing more from the packed slot (the codes are in registers): free it now so
+        // that the next 256 columns stream in while these are expanded.  VQ still reads the codebook.
+        const bool early = a.fmt == PF_SQ3;
+        __syncwarp();
+        if (early && lane == 0) mbar_arrive(&ctrl->wempty[0]);
+        if (mine) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q, ++kb_iter) {
-          const int st = (int)(kb_iter % kWStages);
-          if ((q & 1) != dg) continue;          // the other group's block (blocks per tile are a multiple of four)
-          if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfree[st], ((kb_iter / kWStages) & 1u) ^ 1u, abortp, a.status));
-          if (ok) {
-            uint8_t* wtile = wring + (size_t)st * kWTileBytes;
-            if (a.fmt == PF_SQ3) {
-              uint32_t r[16];
-              sq_unpack_triple(w[3 * q], w[3 * q + 1], w[3 * q + 2], r);
-              sq_store_triple(r, q < 2 ? sz.x : sz.y, q < 2 ? sz.z : sz.w, wtile, dw * 16, lane);
-            } else if (a.fmt == PF_VQ6) {
-              const uint32_t (&w6)[12] = *reinterpret_cast<const uint32_t (*)[12]>(&w[0]);
-              vq_store_block<6>(w6, q, cb, wtile, dw * 16, lane);
-            } else {
-              vq_store_block<8>(w, q, cb, wtile, dw * 16, lane);
+          for (int q = 0; q < 4; ++q, ++kbm) {
+            const int st = (int)(kbm % kWStages);
+            if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfree[dg][st], ((kbm / kWStages) & 1u) ^ 1u, abortp, a.status));
+            if (ok) {
+              uint8_t* wtile = wring + (size_t)(dg * kWStages + st) * kWTileBytes;
+              if (a.fmt == PF_SQ3) {
+                uint32_t r[16];
+                sq_unpack_triple(w[3 * q], w[3 * q + 1], w[3 * q + 2], r);
+                sq_store_triple(r, q < 2 ? sz.x : sz.y, q < 2 ? sz.z : sz.w, wtile, dw * 16, lane);
+              } else if (a.fmt == PF_VQ6) {
+                const uint32_t (&w6)[12] = *reinterpret_cast<const uint32_t (*)[12]>(&w[0]);
+                vq_store_block<6>(w6, q, cb, wtile, dw * 16, lane);
+              } else {
+                vq_store_block<8>(w, q, cb, wtile, dw * 16, lane);
+              }
+              // generic-proxy stores -> visible to the tensor core (async proxy)
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&ctrl->wready[dg][st]);
             }
-            // generic-proxy stores -> visible to the tensor core (async proxy)
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctrl->wready[st]);
           }
         }
         __syncwarp();
-        if (ok && lane == 0) mbar_arrive(&ctrl->wempty[slot]);
+        if (!early && ok && lane == 0) mbar_arrive(&ctrl->wempty[0]);
       }
     }
   } else {
-    // ---- epilogue: warp quarter qd reads lanes 32 qd .. 32 qd + 31 (weight rows) of an accumulator set ----
+    // ---- epilogue: warp quarter qd reads lanes 32 qd .. 32 qd + 31 (weight rows) of both accumulators ----
     const int qd = warp & 3;
     uint32_t tile_iter = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x, ++tile_iter) {
-      const int mb = tile / a.MT, mt = tile % a.MT;
-      const uint32_t set = tile_iter & 1u;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->accfull[set], (tile_iter >> 1) & 1u, abortp, a.status));
+      const int tr = tile / a.MT, mt = tile % a.MT;
+      const int halves = 2 * tr + 1 < a.MB ? 2 : 1;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->accfull, tile_iter & 1u, abortp, a.status));
       if (!ok) break;
       tc_fence_after();
-      const int row = mb * kTileRows + qd * 32 + lane;
       const int t0 = mt * kTileTokens;
+      for (int h = 0; h < halves; ++h) {
+        const int row = (2 * tr + h) * kTileRows + qd * 32 + lane;
 #pragma unroll 1
-      for (int cc = 0; cc < kTileTokens / 32; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tmem_base + set * (uint32_t)kTileTokens + (uint32_t)cc * 32u + ((uint32_t)(qd * 32) << 16), r);
-        if (row < a.oc) {
+        for (int cc = 0; cc < kTileTokens / 32; ++cc) {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + (uint32_t)(h * kTileTokens + cc * 32) + ((uint32_t)(qd * 32) << 16), r);
+          if (row < a.oc) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int t = t0 + cc * 32 + c;
-            if (t < a.M) {
-              if (a.y_dtype == RWKVQ_F32) static_cast<float*>(a.Y)[(size_t)t * a.oc + row] = __uint_as_float(r[c]);
-              else static_cast<__nv_bfloat16*>(a.Y)[(size_t)t * a.oc + row] = __float2bfloat16_rn(__uint_as_float(r[c]));
+            for (int c = 0; c < 32; ++c) {
+              const int t = t0 + cc * 32 + c;
+              if (t < a.M) {
+                if (a.y_dtype == RWKVQ_F32) static_cast<float*>(a.Y)[(size_t)t * a.oc + row] = __uint_as_float(r[c]);
+                else static_cast<__nv_bfloat16*>(a.Y)[(size_t)t * a.oc + row] = __float2bfloat16_rn(__uint_as_float(r[c]));
+              }
             }
           }
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&ctrl->accempty[set]);
+      if (lane == 0) mbar_arrive(&ctrl->accempty);
     }
   }
   // common exit: every role's loops are bounded, so all threads arrive here
@@ -479,7 +503,7 @@ rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* d, const void* W, const rwkvq_
   a.oc = d->oc; a.ic = d->ic; a.M = M;
   a.KT = d->ic_pad / 256; a.KB = a.KT * 4; a.MB = d->oc_pad / 128;
   a.MT = (M + pf::kTileTokens - 1) / pf::kTileTokens;
-  a.n_tiles = a.MB * a.MT;
+  a.n_tiles = ((a.MB + 1) / 2) * a.MT;
   a.fmt = d->method == RWKVQ_SQ ? pf::PF_SQ3 : (d->bits == 6 ? pf::PF_VQ6 : pf::PF_VQ8);
   a.entries = d->entries; a.y_dtype = y_dtype;
   a.rec_bytes = d->method == RWKVQ_SQ ? (uint32_t)RWKVQ_SQ_RECORD_BYTES : rwkvq_vq_record_bytes(d->bits);
