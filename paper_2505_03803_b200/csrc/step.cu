@@ -458,6 +458,31 @@ __device__ __forceinline__ void sq_group_words(const uint8_t* rec, int lane, uin
   }
 }
 
+// One 128-column group of the two records of a warp.  With one batch block (B <= 8) the input
+// fragments are loaded once and shared by both records; with two blocks that costs more
+// registers than a thread has, so the records are taken one after the other.
+template <int NB, int GRP>
+__device__ __forceinline__ void sq_pair(const uint32_t (&wa)[6], const uint32_t (&wb)[6], const uint4 sza, const uint4 szb,
+                                        bool has_b, const XLane& xl, float (&acca)[NB][4], float (&accb)[NB][4]) {
+  if constexpr (NB == 1) {
+    sq_group_mma2<NB, GRP>(wa, wb, sza, szb, has_b, xl, acca, accb);
+  } else {
+    sq_group_mma<NB, GRP>(wa, GRP == 0 ? sza.x : sza.y, GRP == 0 ? sza.z : sza.w, xl, acca);
+    if (has_b) sq_group_mma<NB, GRP>(wb, GRP == 0 ? szb.x : szb.y, GRP == 0 ? szb.z : szb.w, xl, accb);
+  }
+}
+
+template <int BITS, int NB, int HALF>
+__device__ __forceinline__ void vq_pair(const uint32_t (&wa)[2 * BITS], const uint32_t (&wb)[2 * BITS], const uint32_t* cb_lane,
+                                        const XLane& xl, float (&acca)[NB][4], float (&accb)[NB][4]) {
+  if constexpr (NB == 1) {
+    vq_half_mma2<BITS, NB, HALF>(wa, wb, cb_lane, xl, acca, accb);
+  } else {
+    vq_record_mma<BITS, NB, 8 * HALF, 8 * HALF + 8>(wa, cb_lane, xl, acca);
+    vq_record_mma<BITS, NB, 8 * HALF, 8 * HALF + 8>(wb, cb_lane, xl, accb);
+  }
+}
+
 // Consumer warp `w` of group `grp`: units grp, grp + 2, ... of the CTA's list.
 template <int NB>
 __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, const uint8_t* xbufs, uint8_t* replicas,
@@ -572,13 +597,13 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
           sq_group_words<0>(rbp, lane, wb);
           szb = *reinterpret_cast<const uint4*>(rbp + RWKVQ_SQ_CODE_BYTES + g * 16);
         }
-        sq_group_mma2<NB, 0>(wa, wb, sza, szb, has_b, xl, acca, accb);
+        sq_pair<NB, 0>(wa, wb, sza, szb, has_b, xl, acca, accb);
         sq_group_words<1>(ra, lane, wa);
         if (has_b) sq_group_words<1>(rbp, lane, wb);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctrl->empty[slot]);     // the rest of the records is in registers: free the slot
-      if (active) sq_group_mma2<NB, 1>(wa, wb, sza, szb, has_b, xl, acca, accb);
+      if (active) sq_pair<NB, 1>(wa, wb, sza, szb, has_b, xl, acca, accb);
     } else {
       // replicate the tile's codebook for conflict-free lookups (the eight warps of the group)
       const uint32_t E = u->entries;
@@ -595,22 +620,22 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
         uint32_t va[16], vb[16];
         if (active) {
           vq_half_words<8, 0>(ra, lane, va); vq_half_words<8, 0>(rbp, lane, vb);
-          vq_half_mma2<8, NB, 0>(va, vb, cb_lane, xl, acca, accb);
+          vq_pair<8, NB, 0>(va, vb, cb_lane, xl, acca, accb);
           vq_half_words<8, 1>(ra, lane, va); vq_half_words<8, 1>(rbp, lane, vb);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
-        if (active) vq_half_mma2<8, NB, 1>(va, vb, cb_lane, xl, acca, accb);
+        if (active) vq_pair<8, NB, 1>(va, vb, cb_lane, xl, acca, accb);
       } else {
         uint32_t va[12], vb[12];
         if (active) {
           vq_half_words<6, 0>(ra, lane, va); vq_half_words<6, 0>(rbp, lane, vb);
-          vq_half_mma2<6, NB, 0>(va, vb, cb_lane, xl, acca, accb);
+          vq_pair<6, NB, 0>(va, vb, cb_lane, xl, acca, accb);
           vq_half_words<6, 1>(ra, lane, va); vq_half_words<6, 1>(rbp, lane, vb);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
-        if (active) vq_half_mma2<6, NB, 1>(va, vb, cb_lane, xl, acca, accb);
+        if (active) vq_pair<6, NB, 1>(va, vb, cb_lane, xl, acca, accb);
       }
     }
     if (flags & UF_FLUSH) {
