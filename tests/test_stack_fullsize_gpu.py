@@ -1,0 +1,50 @@
+"""Parity at the full sizes of the benchmark workloads, in the launch configuration bench.py times
+(one rwkvq_step_run over the whole stack): sampled products are compared with the fp64 oracle
+computed from the logical codes the packer exported."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rwkvq_oracle as orc
+from paper_2505_03803_b200 import binding as B
+from paper_2505_03803_b200 import stack as stack_mod
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_product(st, op):
+    codes, mu_codes = st.host_codes(op)
+    if op.method == B.RWKVQ_SQ:
+        w_hat = orc.sq_decode(codes["q"], codes["scale"], codes["zero"])
+    else:
+        w_hat = orc.vq_decode(codes["codebook"], codes["q"])
+    x = op.x.cpu().numpy().astype(np.float64)
+    if op.has_mu:
+        mu_hat = orc.mu_decode(mu_codes["codebook"], mu_codes["q"])
+        x = orc.token_shift(x, op.xprev.cpu().numpy().astype(np.float64), mu_hat)
+    return orc.gemv(w_hat, x), orc.tolerance(w_hat, x)
+
+
+@pytest.mark.parametrize("name,batch", [("c2_1p6b", 1), ("c3_7b", 8), ("c4_14b", 16)])
+def test_whole_step_at_benchmark_size_matches_oracle_on_sampled_products(name, batch):
+    st = stack_mod.from_name(name, batch=batch, distinct_layers=1, kmeans_iters=2)
+    st.plan_step()
+    for _ in range(2):                      # a second run must reproduce the first (outputs are cleared in the kernel)
+        st.run_step()
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 0
+    n = len(st.ops)
+    picks = sorted({0, 1, 4, 5, 7, n // 2, n // 2 + 3, n - 8, n - 3, n - 1})
+    kinds = set()
+    for i in picks:
+        op = st.ops[i]
+        kinds.add((op.name, op.method))
+        ref, tol = _oracle_product(st, op)
+        y = op.y.double().cpu().numpy()
+        assert np.isfinite(y).all()
+        err = np.abs(y - ref)
+        assert (err <= tol).all(), f"{name} op {i} ({op.name}, layer {op.layer}): max err/tol {float((err / tol).max())}"
+    assert len(kinds) >= 4
+    # every output of every product was written (none left at its cleared value by accident): spot-check norms
+    for op in st.ops[:: max(1, n // 16)]:
+        assert float(op.y.abs().sum()) > 0.0
