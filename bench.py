@@ -29,6 +29,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
+# profiles/step_kernel_c2_1p6b_b1.md.  Valid only for that workload and for the kernel as it was
+# when the counters were taken: set an entry to None when step.cu changes.
+NCU_TRAFFIC_BYTES = {("c2_1p6b", 1, "step", None, 4): 542_899_712}
+
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -421,7 +426,8 @@ def run_ours(args):
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
     achieved = alg_bytes / launches_per_step / (avg_launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "step_kernel" if args.mode == "step" else "gemv_kernel",
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, batch, args.mode, args.force_method, args.distinct_layers)),
+                "peak_kind": f"of {peak_kind}", "kernel": "step_kernel" if args.mode == "step" else "gemv_kernel",
                 "algorithmic_bytes_per_launch": alg_bytes / launches_per_step,
                 "launch_ms_avg": avg_launch_ms, "launch_ms_median": statistics.median(per_launch_ms),
                 "launch_ms_min": min(per_launch_ms), "frac_of_8TBs_nominal": achieved / 8000.0}
