@@ -71,12 +71,17 @@ enum { EV_SEGMENT = 0, EV_ARRIVE = 1 };
 
 struct StepEvent {           // 64 bytes
   union {
+    // segment.  Mixed in the CTA: x, xprev, mu, mu_aux as given by the caller.  Copied from the
+    // stage's pre-pass (StepArgs::mix): x = first byte of the segment in the pre-pass rows,
+    // xprev = first byte of its sums, mu = 0.
     struct { uint64_t x, xprev, mu, mu_aux; } seg;
-    struct { uint64_t zptr[4]; } arr;          // float ranges to clear before arriving
+    // arrival: float ranges to clear before arriving; then this CTA's share of the stage's
+    // pre-pass: groups [grp_lo, grp_hi) of the stage's (product, batch row, 128-column group) list
+    struct { uint64_t zptr[3]; uint32_t grp_lo, grp_hi; } arr;
   };
   union {
-    struct { uint32_t ic, col0, ncols; uint16_t mu_bits, mu_entries; } segd;
-    struct { uint32_t zcount[4]; } arrd;
+    struct { uint32_t ic, col0, ncols; uint16_t mu_bits, mu_entries; } segd;   // copied segments: ic = bytes between rows
+    struct { uint32_t zcount[3]; uint16_t op_first, op_count; } arrd;          // products of the stage the pre-pass covers
   };
   uint32_t kind;             // EV_SEGMENT / EV_ARRIVE
   uint32_t barrier;          // segment: index + 1 of the stage barrier to pass first; arrival: index of the barrier
@@ -85,6 +90,15 @@ struct StepEvent {           // 64 bytes
   uint16_t reserved;
 };
 static_assert(sizeof(StepEvent) == 64, "event descriptor size");
+
+// One product's share of a stage's pre-pass: where its inputs are and where x_mix (fp16 rows of
+// ic_pad columns, zero beyond ic) and the per-group sums ([group][3][nbp] floats) go.
+struct StepMixOp {           // 64 bytes
+  uint64_t x, xprev, mu, mu_aux, dst_x, dst_sums;
+  uint32_t ic, ic_pad;
+  uint16_t mu_bits, mu_entries, sums, pad;
+};
+static_assert(sizeof(StepMixOp) == 64, "pre-pass descriptor size");
 
 constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGroups, kStagerWarps = 3;
 constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
@@ -105,6 +119,12 @@ struct StepArgs {
   int* status;
   int B, n_slots, n_stages;
   uint32_t slot_bytes, replica_bytes;
+  // Larger batches: x_mix and the sums of a stage are computed ONCE by all CTAs together after the
+  // stage barrier (instead of by every CTA that reads a column), published through a second
+  // barrier per stage (counter[n_stages + 1 + s]), and fetched into the segment buffers with bulk copies.
+  int mix;
+  const StepMixOp* mixops;    // dst_x / dst_sums are offsets into `scratch`
+  uint8_t* scratch;
 };
 
 // ---- mbarrier / bulk-copy wrappers ------------------------------------------------------------
@@ -161,6 +181,10 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_plain(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
@@ -282,6 +306,67 @@ __device__ __forceinline__ float pair_sum(uint32_t r) {
 
 constexpr int kStageUnroll = 4;
 
+// This CTA's share of a stage's pre-pass.  A half-warp takes one (product, batch row, 128-column
+// group) at a time: it loads x (and x_prev, and decodes mu_hat), mixes, rounds to fp16, stores the
+// 128 values to the product's pre-pass rows and reduces the three sums of the group with shuffles.
+__device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
+  const int lane = stid & 31, l16 = lane & 15;
+  const uint32_t lo = ev.arr.grp_lo, hi = ev.arr.grp_hi;
+  const StepMixOp* ops = a.mixops + ev.arrd.op_first;
+  const int n_ops = (int)ev.arrd.op_count;
+  const int nbp = (a.B + 1) & ~1;
+  for (uint32_t g0 = lo + 2u * (uint32_t)(stid >> 5); g0 < hi; g0 += 2u * (uint32_t)kStagerWarps) {
+    const uint32_t gi = g0 + (uint32_t)(lane >> 4);
+    const bool valid = gi < hi;
+    uint32_t r = valid ? gi : lo;
+    int k = 0;
+    uint32_t icp = __ldg(&ops[0].ic_pad);
+    while (k + 1 < n_ops && r >= (uint32_t)a.B * (icp >> 7)) { r -= (uint32_t)a.B * (icp >> 7); ++k; icp = __ldg(&ops[k].ic_pad); }
+    const StepMixOp op = ops[k];
+    const uint32_t ng = op.ic_pad >> 7;
+    const int b = (int)(r / ng), grp = (int)(r % ng);
+    const int col = grp * 128 + l16 * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (col < (int)op.ic) {
+      v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + (size_t)b * op.ic + col));
+      if (op.mu) {
+        const uint4 pr = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.xprev) + (size_t)b * op.ic + col));
+        const uint32_t bits = op.mu_bits, mask = (1u << bits) - 1u;
+        // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
+        const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(op.mu) + (byte >> 2);
+        const uint32_t sh = (byte & 3u) * 8u;
+        const uint32_t wlo = __ldg(w);
+        const uint32_t whi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+        const uint32_t f = __funnelshift_r(wlo, whi, sh);
+        const uint32_t* cb = reinterpret_cast<const uint32_t*>(op.mu_aux);
+        v.x = mix2(v.x, pr.x, __ldg(cb + (f & mask)));
+        v.y = mix2(v.y, pr.y, __ldg(cb + ((f >> bits) & mask)));
+        v.z = mix2(v.z, pr.z, __ldg(cb + ((f >> (2 * bits)) & mask)));
+        v.w = mix2(v.w, pr.w, __ldg(cb + ((f >> (3 * bits)) & mask)));
+      }
+    }
+    if (valid) *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(a.scratch + op.dst_x) + (size_t)b * op.ic_pad + col) = v;
+    const int o = (8 * l16) & 63;
+    const float pa = pair_sum(v.x) + pair_sum(v.z), pb = pair_sum(v.y) + pair_sum(v.w);
+    float sx = pa + pb;
+    float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
+    float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
+#pragma unroll
+    for (int d = 8; d > 0; d >>= 1) {
+      sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+      t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
+      t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+    }
+    if (valid && l16 == 0 && op.sums) {
+      float* gs = reinterpret_cast<float*>(a.scratch + op.dst_sums);
+      gs[(grp * 3 + 0) * nbp + b] = sx;
+      gs[(grp * 3 + 1) * nbp + b] = t0;
+      gs[(grp * 3 + 2) * nbp + b] = t1;
+    }
+  }
+}
+
 // Stagers walk the CTA's event list.
 //  EV_ARRIVE: clear this CTA's slice of the next stage's outputs, then (deferred until the next
 //    segment's barrier-independent preparation is done) wait for the consumer warps to finish
@@ -291,6 +376,7 @@ constexpr int kStageUnroll = 4;
 //    shared memory BEFORE the stage barrier, so that only one round of vector loads of x, the
 //    mix and the sums remain behind it.  A thread owns 8 consecutive columns (16 bytes) of one
 //    batch row; a half-warp owns one 128-column group, whose three sums it reduces with shuffles.
+template <bool MIX>
 __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_t* xbufs, uint32_t* mucb,
                             uint32_t e0, uint32_t e1) {
   const int stid = threadIdx.x - kConsumerThreads;
@@ -299,6 +385,7 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
   uint32_t nseg = 0;          // segments staged so far
   uint32_t narrive = 0;       // arrivals posted so far
   int pending = -1;           // barrier index of an arrival not yet posted
+  uint32_t passed2 = 0xFFFFFFFFu;   // second-stage barrier this CTA has already passed
   bool ok = true;
   // posts the pending arrival (thread 0 acts; the others only keep count)
   auto post_arrival = [&]() {
@@ -317,7 +404,7 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
     if (ev.kind == EV_ARRIVE) {
       post_arrival();                         // an earlier arrival with no segment in between
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
+      for (int k = 0; k < 3; ++k) {
         float* z = reinterpret_cast<float*>(ev.arr.zptr[k]);
         for (uint32_t e = stid; e < ev.arrd.zcount[k]; e += kStagerThreads) z[e] = 0.f;
       }
@@ -325,12 +412,61 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       ok = named_bar_and(4, kStagerThreads, ok);
       pending = (int)ev.barrier;
       if (!ok) break;
+      if constexpr (MIX) {
+        // no preparation to overlap: arrive now, then, once the barrier opens, do this CTA's share
+        // of the new stage's pre-pass and publish it through the stage's second barrier
+        post_arrival();
+        if (ev.barrier < (uint32_t)a.n_stages) {
+          if (ok && stid == 0) {
+            uint32_t it = 0;
+            while ((int)(ld_acquire_gpu(a.counter + ev.barrier) - a.target) < 0) {
+              if (++it >= (kPollLimit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
+            }
+          }
+          ok = named_bar_and(6, kStagerThreads, ok);   // thread 0's acquire precedes every thread's loads of x
+          if (!ok) break;
+          mix_slice(a, ev, stid);
+          named_bar_sync(4, kStagerThreads);           // every thread's pre-pass stores precede thread 0's release
+          if (stid == 0) red_release_gpu(a.counter + (uint32_t)a.n_stages + 1u + ev.barrier, 1u);
+        }
+      }
       continue;
     }
     const int buf = (int)(nseg & 1u);
     // uniform verdict over all stager threads: the named barriers below must be reached by all or none
     ok = named_bar_and(7, kStagerThreads, mbar_wait_warp(&ctrl->xempty[buf], ((nseg >> 1) & 1u) ^ 1u, abortp, a.status) && ok);
     uint8_t* xb = xbufs + (size_t)buf * kXBufBytes;
+    if constexpr (MIX) {
+      // The segment is a rectangle of the stage's pre-pass output: pass the stage's second barrier
+      // (once per stage), then fetch B rows and the block of sums with bulk copies.
+      const uint32_t b2 = (uint32_t)a.n_stages + ev.barrier;      // counter of the second barrier of stage ev.barrier - 1
+      if (ok && stid == 0 && b2 != passed2) {
+        uint32_t it = 0;
+        while ((int)(ld_acquire_gpu(a.counter + b2) - a.target) < 0) {
+          if (++it >= (kPollLimit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
+        }
+      }
+      passed2 = b2;
+      ok = named_bar_and(6, kStagerThreads, ok);
+      if (ok && stid < 32) {
+        const uint32_t xstride = ev.xstride_sums & 0x7FFFFFFFu;
+        const uint32_t row_bytes = ev.segd.ncols * 2u;
+        const uint32_t sums_bytes = (ev.xstride_sums >> 31) ? (ev.segd.ncols >> 7) * 3u * (uint32_t)((a.B + 1) & ~1) * 4u : 0u;
+        // what other CTAs wrote with ordinary stores is read below by the copy engine
+        asm volatile("fence.proxy.async;" ::: "memory");
+        if (lane == 0) mbar_arrive_expect_tx(&ctrl->xfull[buf], (uint32_t)a.B * row_bytes + sums_bytes);
+        __syncwarp();
+        if (lane < a.B)
+          bulk_g2s_plain(xb + (size_t)lane * xstride, a.scratch + ev.seg.x + (size_t)lane * ev.segd.ic, row_bytes, &ctrl->xfull[buf]);
+        else if (lane == a.B && sums_bytes)
+          bulk_g2s_plain(xb + (size_t)a.B * xstride, a.scratch + ev.seg.xprev, sums_bytes, &ctrl->xfull[buf]);
+      } else if (lane == 0) {
+        mbar_arrive(&ctrl->xfull[buf]);      // the other stager warps (and everyone after a failure) only arrive
+      }
+      ++nseg;
+      if (!ok) break;
+      continue;
+    }
     const uint8_t* mu = reinterpret_cast<const uint8_t*>(ev.seg.mu);
     const __half* x = reinterpret_cast<const __half*>(ev.seg.x);
     const __half* xp = reinterpret_cast<const __half*>(ev.seg.xprev);
@@ -664,7 +800,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
   }
 }
 
-template <int NB>
+template <int NB, bool MIX>
 __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
@@ -685,7 +821,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   if (warp < kConsumerWarps) {
     consumer_role<NB>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
   } else if (warp < kConsumerWarps + kStagerWarps) {
-    stager_role(a, smem, ctrl, xbufs, mucb, e0, e1);
+    stager_role<MIX>(a, smem, ctrl, xbufs, mucb, e0, e1);
   } else {
     producer_role(a, smem, ctrl, u0, u1);
   }
@@ -694,11 +830,11 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
 // ---- host planner --------------------------------------------------------------------------------
 
 struct PlanInfo {
-  int P, B, NB, n_slots, n_stages;
+  int P, B, NB, n_slots, n_stages, mix;
   unsigned runs;        // launches since the counters were last zero
   unsigned abort_epoch; // value of the abort epoch when the counters were last known good
   uint32_t slot_bytes, replica_bytes, smem_bytes;
-  size_t off_unit_off, off_event_off, off_units, off_events, off_counter, total_bytes;
+  size_t off_unit_off, off_event_off, off_units, off_events, off_counter, off_mixops, off_scratch, total_bytes;
   uint32_t n_units, n_events, n_barriers;
 };
 
@@ -767,6 +903,8 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   info->n_slots = ns;
   info->smem_bytes = fixed + (uint32_t)ns * info->slot_bytes;
   info->P = P; info->B = B; info->NB = B <= 8 ? 1 : 2;
+  const bool mix = B >= 4;     // see StepArgs::mix
+  info->mix = mix ? 1 : 0;
   const uint32_t nbp = (uint32_t)((B + 1) & ~1);
 
   std::vector<std::pair<int, int>> stage_ranges;  // [first op, last op) per distinct stage value
@@ -778,7 +916,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   }
   const int n_stages = (int)stage_ranges.size();
   info->n_stages = n_stages;
-  info->n_barriers = (uint32_t)n_stages + 1;
+  info->n_barriers = ((uint32_t)n_stages + 1) * (mix ? 2u : 1u);   // the pre-pass has a barrier of its own per stage
 
   std::vector<std::vector<HostUnit>> cta_units(P);
   std::vector<std::vector<StepEvent>> cta_arrivals(P);      // arrival events, one per barrier
@@ -798,13 +936,21 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         const uint64_t n = (uint64_t)B * ops[o].W_desc.oc;
         const uint64_t a0 = std::max(lo, base), a1 = std::min(hi, base + n);
         if (a1 > a0) {
-          if (k >= 4) { too_many_ranges = true; break; }
+          if (k >= 3) { too_many_ranges = true; break; }
           ev.arr.zptr[k] = (uint64_t)(uintptr_t)ops[o].y_dev + (a0 - base) * 4;
           ev.arrd.zcount[k] = (uint32_t)(a1 - a0);
           ++k;
         }
         base += n;
       }
+    }
+    if (mix && barrier < n_stages) {
+      // this CTA's share of the pre-pass of stage `barrier`
+      uint64_t G = 0;
+      for (int o = stage_ranges[barrier].first; o < stage_ranges[barrier].second; ++o) G += (uint64_t)B * (ops[o].W_desc.ic_pad / 128);
+      ev.arr.grp_lo = (uint32_t)(G * (uint64_t)c / P); ev.arr.grp_hi = (uint32_t)(G * (uint64_t)(c + 1) / P);
+      ev.arrd.op_first = (uint16_t)stage_ranges[barrier].first;
+      ev.arrd.op_count = (uint16_t)(stage_ranges[barrier].second - stage_ranges[barrier].first);
     }
     cta_arrivals[c].push_back(ev);
   };
@@ -870,8 +1016,37 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     }
     for (int c = 0; c < P; ++c) make_arrival(c, s + 1, s + 1);
   }
-  if (too_many_ranges) return RWKVQ_EUNSUPPORTED;   // a CTA's slice of a stage's outputs may touch at most four products
+  if (too_many_ranges) return RWKVQ_EUNSUPPORTED;   // a CTA's slice of a stage's outputs may touch at most three products
 
+  // pre-pass outputs: one region, reused by every stage (a stage's pre-pass starts only after the
+  // previous stage, and with it every copy out of the region, has finished everywhere)
+  std::vector<uint64_t> mix_x_off(n_ops, 0), mix_sums_off(n_ops, 0);
+  std::vector<StepMixOp> mixops(mix ? n_ops : 0);
+  uint64_t scratch_bytes = 0;
+  if (mix) {
+    for (int st_i = 0; st_i < n_stages; ++st_i) {
+      uint64_t off = 0;
+      for (int o = stage_ranges[st_i].first; o < stage_ranges[st_i].second; ++o) {
+        const rwkvq_gemv_op& op = ops[o];
+        mix_x_off[o] = off; off += round_up_sz((size_t)B * op.W_desc.ic_pad * 2, 256);
+        mix_sums_off[o] = off; off += round_up_sz((size_t)(op.W_desc.ic_pad / 128) * 3 * nbp * 4, 256);
+        StepMixOp& m = mixops[o];
+        std::memset(&m, 0, sizeof(m));
+        m.x = (uint64_t)(uintptr_t)op.x_fp16_dev;
+        if (op.mu_image_dev) {
+          const uint8_t* mi = static_cast<const uint8_t*>(op.mu_image_dev);
+          m.xprev = (uint64_t)(uintptr_t)op.xprev_fp16_dev;
+          m.mu = (uint64_t)(uintptr_t)(mi + RWKVQ_HEADER_BYTES);
+          m.mu_aux = (uint64_t)(uintptr_t)(mi + vector_aux_offset(&op.mu_desc));
+          m.mu_bits = (uint16_t)op.mu_desc.bits; m.mu_entries = (uint16_t)op.mu_desc.entries;
+        }
+        m.dst_x = mix_x_off[o]; m.dst_sums = mix_sums_off[o];
+        m.ic = (uint32_t)op.W_desc.ic; m.ic_pad = (uint32_t)op.W_desc.ic_pad;
+        m.sums = op.W_desc.method == RWKVQ_SQ ? 1 : 0;
+      }
+      scratch_bytes = std::max(scratch_bytes, off);
+    }
+  }
   std::vector<uint32_t> unit_off(P + 1, 0), event_off(P + 1, 0);
   std::vector<StepUnit> all_units;
   std::vector<StepEvent> all_events;
@@ -895,7 +1070,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       while (i < n && L[i].stage == s) {
         const int op = L[i].op;
         const bool sums = ops[op].W_desc.method == RWKVQ_SQ;
-        const bool has_mu = ops[op].mu_image_dev != nullptr;
+        const bool has_mu = !mix && ops[op].mu_image_dev != nullptr;   // copied segments carry no mu row
         int kmin = L[i].kt, kmax = L[i].kt + 1;
         size_t j = i + 1, last = i;
         // A segment is a contiguous run of column tiles (a range that wraps from the end of one row
@@ -918,7 +1093,11 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         ev.xstride_sums = xstride | (sums ? 0x80000000u : 0u);
         ev.mu_off16 = (uint16_t)(xseg_mu_off(B, ncols, sums) / 16u);
         ev.barrier = (uint32_t)s + 1u;   // stage s reads its inputs after barrier s
-        if (has_mu) {
+        if (mix) {
+          ev.seg.x = mix_x_off[op] + (uint64_t)kmin * 512u;
+          ev.seg.xprev = mix_sums_off[op] + (uint64_t)(kmin * 2) * 3u * nbp * 4u;
+          ev.segd.ic = (uint32_t)o.W_desc.ic_pad * 2u;
+        } else if (has_mu) {
           const uint8_t* m = static_cast<const uint8_t*>(o.mu_image_dev);
           ev.seg.xprev = (uint64_t)(uintptr_t)o.xprev_fp16_dev;
           ev.seg.mu = (uint64_t)(uintptr_t)(m + RWKVQ_HEADER_BYTES);
@@ -976,6 +1155,8 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   info->off_units = off; off += round_up_sz(std::max<size_t>(1, all_units.size()) * sizeof(StepUnit), 256);
   info->off_events = off; off += round_up_sz(all_events.size() * sizeof(StepEvent), 256);
   info->off_counter = off; off += round_up_sz((size_t)info->n_barriers * 4, 256);
+  info->off_mixops = off; off += round_up_sz(mixops.size() * sizeof(StepMixOp), 256);
+  info->off_scratch = off; off += round_up_sz((size_t)scratch_bytes, 256);
   info->total_bytes = off;
   if (out) {
     out->assign(off, 0);
@@ -983,6 +1164,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     memcpy(out->data() + info->off_event_off, event_off.data(), (size_t)(P + 1) * 4);
     if (!all_units.empty()) memcpy(out->data() + info->off_units, all_units.data(), all_units.size() * sizeof(StepUnit));
     memcpy(out->data() + info->off_events, all_events.data(), all_events.size() * sizeof(StepEvent));
+    if (!mixops.empty()) memcpy(out->data() + info->off_mixops, mixops.data(), mixops.size() * sizeof(StepMixOp));
   }
   return RWKVQ_OK;
 }
@@ -1051,6 +1233,8 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
   a.status = device_status_ptr();
   if (!a.status) return RWKVQ_ECUDA;
   a.B = info.B; a.n_slots = info.n_slots; a.n_stages = info.n_stages;
+  a.mix = info.mix; a.mixops = reinterpret_cast<const StepMixOp*>(p + info.off_mixops);
+  a.scratch = const_cast<uint8_t*>(p) + info.off_scratch;
   a.slot_bytes = info.slot_bytes; a.replica_bytes = info.replica_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   a.target = info.runs * (unsigned)info.P;
@@ -1059,7 +1243,8 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
     e = cudaMemsetAsync(a.counter, 0, round_up_sz((size_t)info.n_barriers * 4, 256), s);
     if (e != cudaSuccess) return cuda_status(e);
   }
-  const void* fn = info.NB == 1 ? (const void*)step_kernel<1> : (const void*)step_kernel<2>;
+  // batches of 4 and more use the stage pre-pass (StepArgs::mix)
+  const void* fn = !info.mix ? (const void*)step_kernel<1, false> : info.NB == 1 ? (const void*)step_kernel<1, true> : (const void*)step_kernel<2, true>;
   e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)info.smem_bytes);
   if (e != cudaSuccess) return cuda_status(e);
   void* params[] = {&a};
