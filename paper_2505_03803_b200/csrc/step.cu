@@ -105,7 +105,11 @@ constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWa
 constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
 constexpr int kMaxSlots = 12;
-constexpr uint32_t kCtrlBytes = 1024, kXBufBytes = 24576, kMuScratch = 1024;
+constexpr uint32_t kCtrlBytes = 1024, kXBufTotal = 49152, kMuScratch = 1024;
+// Input-segment buffers: two of 24 KB when the CTA mixes its own inputs (the segment carries a mu row and
+// is prepared ahead), four of 12 KB when segments are copied from the stage's pre-pass.
+// (up to 8 batch rows; larger batches keep two buffers, a 256-column tile of 16 rows being 9 KB).
+template <bool MIX, int NB> struct XBufs { static constexpr uint32_t kCount = (MIX && NB == 1) ? 4u : 2u, kBytes = kXBufTotal / kCount; };
 constexpr uint32_t kSmemLimit = 232448;  // 227 KB
 constexpr uint32_t kPollLimit = 1u << 22;
 
@@ -219,7 +223,7 @@ __device__ __forceinline__ bool wait_count(const uint32_t* p, uint32_t target, v
 
 struct Ctrl {
   uint64_t full[kMaxSlots], empty[kMaxSlots];
-  uint64_t xfull[2], xempty[2];
+  uint64_t xfull[4], xempty[4];
   uint32_t cdone;            // stage completions reported by consumer warps: 16 per finished stage.  A
                              // plain counter, not an mbarrier: consumers of a CTA without work in the
                              // coming stages may run any number of stages ahead of the stagers.
@@ -376,7 +380,7 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
 //    shared memory BEFORE the stage barrier, so that only one round of vector loads of x, the
 //    mix and the sums remain behind it.  A thread owns 8 consecutive columns (16 bytes) of one
 //    batch row; a half-warp owns one 128-column group, whose three sums it reduces with shuffles.
-template <bool MIX>
+template <bool MIX, int NB>
 __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_t* xbufs, uint32_t* mucb,
                             uint32_t e0, uint32_t e1) {
   const int stid = threadIdx.x - kConsumerThreads;
@@ -432,10 +436,10 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       }
       continue;
     }
-    const int buf = (int)(nseg & 1u);
+    const int buf = (int)(nseg % XBufs<MIX, NB>::kCount);
     // uniform verdict over all stager threads: the named barriers below must be reached by all or none
-    ok = named_bar_and(7, kStagerThreads, mbar_wait_warp(&ctrl->xempty[buf], ((nseg >> 1) & 1u) ^ 1u, abortp, a.status) && ok);
-    uint8_t* xb = xbufs + (size_t)buf * kXBufBytes;
+    ok = named_bar_and(7, kStagerThreads, mbar_wait_warp(&ctrl->xempty[buf], ((nseg / XBufs<MIX, NB>::kCount) & 1u) ^ 1u, abortp, a.status) && ok);
+    uint8_t* xb = xbufs + (size_t)buf * XBufs<MIX, NB>::kBytes;
     if constexpr (MIX) {
       // The segment is a rectangle of the stage's pre-pass output: pass the stage's second barrier
       // (once per stage), then fetch B rows and the block of sums with bulk copies.
@@ -620,7 +624,7 @@ __device__ __forceinline__ void vq_pair(const uint32_t (&wa)[2 * BITS], const ui
 }
 
 // Consumer warp `w` of group `grp`: units grp, grp + 2, ... of the CTA's list.
-template <int NB>
+template <int NB, bool MIX>
 __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, const uint8_t* xbufs, uint8_t* replicas,
                               uint32_t unit_base, uint32_t n_units, uint32_t ev_base, uint32_t n_events) {
   bool dead = false;
@@ -649,14 +653,14 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
   };
   auto release_held = [&]() {
     __syncwarp();
-    if (held >= 0 && lane == 0 && !dead) mbar_arrive(&ctrl->xempty[held & 1]);
+    if (held >= 0 && lane == 0 && !dead) mbar_arrive(&ctrl->xempty[(uint32_t)held % XBufs<MIX, NB>::kCount]);
     held = -1;
   };
   auto pass_segment = [&]() {   // a segment this warp does not use: observe it, hand it back
     const uint32_t q = seg_next++;
-    if (!dead && !mbar_wait_warp(&ctrl->xfull[q & 1u], (q >> 1) & 1u, abortp, a.status)) dead = true;
+    if (!dead && !mbar_wait_warp(&ctrl->xfull[q % XBufs<MIX, NB>::kCount], (q / XBufs<MIX, NB>::kCount) & 1u, abortp, a.status)) dead = true;
     __syncwarp();
-    if (lane == 0 && !dead) mbar_arrive(&ctrl->xempty[q & 1u]);
+    if (lane == 0 && !dead) mbar_arrive(&ctrl->xempty[q % XBufs<MIX, NB>::kCount]);
   };
   // Events (cur_ev, upto) in order; `mask` describes them when there are at most 32 and the planner
   // could say so, otherwise (and for the tail of the list) the kinds are read from the plan, 32 at
@@ -698,7 +702,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
         const uint32_t q = seg_next++;
         held = (int)q;
         cur_ev = target;
-        if (!mbar_wait_warp(&ctrl->xfull[q & 1u], (q >> 1) & 1u, abortp, a.status)) dead = true;
+        if (!mbar_wait_warp(&ctrl->xfull[q % XBufs<MIX, NB>::kCount], (q / XBufs<MIX, NB>::kCount) & 1u, abortp, a.status)) dead = true;
       }
     }
     if (dead) {
@@ -711,7 +715,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
     const uint32_t by1 = u->bytes1;
     const uint32_t after_count = u->after_count, after_mask = u->after_mask;
     const uint8_t* data = sl + 128;
-    const uint8_t* xb = xbufs + (size_t)(held & 1) * kXBufBytes;
+    const uint8_t* xb = xbufs + (size_t)((uint32_t)held % XBufs<MIX, NB>::kCount) * XBufs<MIX, NB>::kBytes;
     const uint32_t xstride = u->xstride, nbp = u->nbp, chb = u->chunk_bytes, rb = u->rec_bytes;
     const uint32_t w0 = (flags >> 8) & 15u, w1 = (flags >> 12) & 15u;
     const bool active = (uint32_t)w >= w0 && (uint32_t)w < w1;
@@ -805,11 +809,11 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
   uint8_t* xbufs = smem + kCtrlBytes + (size_t)a.n_slots * a.slot_bytes;
-  uint32_t* mucb = reinterpret_cast<uint32_t*>(xbufs + 2 * kXBufBytes);
+  uint32_t* mucb = reinterpret_cast<uint32_t*>(xbufs + kXBufTotal);
   uint8_t* replicas = reinterpret_cast<uint8_t*>(mucb) + kMuScratch;
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.n_slots; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], kGroupWarps); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&ctrl->xfull[b], kStagerWarps); mbar_init(&ctrl->xempty[b], kConsumerWarps); }
+    for (int b = 0; b < 4; ++b) { mbar_init(&ctrl->xfull[b], kStagerWarps); mbar_init(&ctrl->xempty[b], kConsumerWarps); }
     ctrl->cdone = 0u;
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -819,9 +823,9 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   const uint32_t e0 = a.event_off[blockIdx.x], e1 = a.event_off[blockIdx.x + 1];
   const int warp = threadIdx.x >> 5;
   if (warp < kConsumerWarps) {
-    consumer_role<NB>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
+    consumer_role<NB, MIX>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
   } else if (warp < kConsumerWarps + kStagerWarps) {
-    stager_role<MIX>(a, smem, ctrl, xbufs, mucb, e0, e1);
+    stager_role<MIX, NB>(a, smem, ctrl, xbufs, mucb, e0, e1);
   } else {
     producer_role(a, smem, ctrl, u0, u1);
   }
@@ -896,7 +900,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   if (has_vq8) data_max = std::max(data_max, 2u * 8u * 2048u + 1024u);
   info->slot_bytes = (128u + data_max + 127u) & ~127u;
   info->replica_bytes = has_vq8 ? 256u * 128u : has_vq6 ? 64u * 128u : 0u;   // per consumer group
-  const uint32_t fixed = kCtrlBytes + 2u * kXBufBytes + kMuScratch + (uint32_t)kGroups * info->replica_bytes;
+  const uint32_t fixed = kCtrlBytes + kXBufTotal + kMuScratch + (uint32_t)kGroups * info->replica_bytes;
   int ns = (int)((kSmemLimit - fixed) / info->slot_bytes);
   if (ns > kMaxSlots) ns = kMaxSlots;
   if (ns < 2) return RWKVQ_EUNSUPPORTED;
@@ -904,6 +908,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   info->smem_bytes = fixed + (uint32_t)ns * info->slot_bytes;
   info->P = P; info->B = B; info->NB = B <= 8 ? 1 : 2;
   const bool mix = B >= 4;     // see StepArgs::mix
+  const uint32_t xbuf_bytes = mix && B <= 8 ? XBufs<true, 1>::kBytes : XBufs<false, 1>::kBytes;
   info->mix = mix ? 1 : 0;
   const uint32_t nbp = (uint32_t)((B + 1) & ~1);
 
@@ -1078,11 +1083,11 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         while (j < n && L[j].op == op && L[j].stage == s) {
           if (L[j].kt < kmin || L[j].kt > kmax) break;
           const int nmax = std::max(kmax, L[j].kt + 1);
-          if (xseg_bytes(B, (nmax - kmin) * 256, sums, has_mu) > kXBufBytes) break;
+          if (xseg_bytes(B, (nmax - kmin) * 256, sums, has_mu) > xbuf_bytes) break;
           kmax = nmax; last = j; ++j;
         }
         const int ncols = (kmax - kmin) * 256;
-        if (xseg_bytes(B, ncols, sums, has_mu) > kXBufBytes) return RWKVQ_EUNSUPPORTED;
+        if (xseg_bytes(B, ncols, sums, has_mu) > xbuf_bytes) return RWKVQ_EUNSUPPORTED;
         StepEvent ev;
         std::memset(&ev, 0, sizeof(ev));
         const rwkvq_gemv_op& o = ops[op];
