@@ -18,7 +18,8 @@ Passages followed (RWKVQuant, arXiv 2505.03803):
   * fine proxy P_f                       -- Section 4.1, Eqs. 10-17
   * selection rule phi                   -- Section 4.1, Eq. 18
   * token shift mix and projections      -- Appendix A.1, Eqs. 20-22, 24-26
-  * weighted loss for element-wise mu    -- Section 4.2, Eq. 19 (only the decode of mu is used here)
+  * weighted loss for element-wise mu    -- Section 4.2, Eq. 19 (weighted k-means; representative X by
+                                            percentile clipping before the mean)
 
 Pin status: every function here is pinned by tests/test_oracle_pins.py to
 closed forms, invariants or brute force, except `vq_kmeans` codebook *values*
@@ -109,10 +110,14 @@ def sq_decode(q: np.ndarray, s: np.ndarray, z: np.ndarray, group: int = 128) -> 
 # --------------------------------------------------------------------------
 
 
-def _nearest(vecs: np.ndarray, centres: np.ndarray) -> np.ndarray:
-    """argmin_j ||v_i - C_j||^2 (Eq. 3); ties resolve to the lowest index."""
-    d2 = ((vecs[:, None, :] - centres[None, :, :]) ** 2).sum(axis=2)
-    return np.argmin(d2, axis=1)
+def _nearest(vecs: np.ndarray, centres: np.ndarray, weights: np.ndarray | None = None) -> np.ndarray:
+    """argmin_j ||v_i - C_j||^2 (Eq. 3); ties resolve to the lowest index.  With
+    per-element weights X_ij^2 the distance is the term of Eq. 19 that vector i
+    contributes, sum_d X_id^2 (v_id - C_jd)^2."""
+    sq = (vecs[:, None, :] - centres[None, :, :]) ** 2
+    if weights is not None:
+        sq = weights[:, None, :] * sq
+    return np.argmin(sq.sum(axis=2), axis=1)
 
 
 def kmeans_tile(vecs: np.ndarray, entries: int, iters: int, rng: np.random.Generator,
@@ -126,10 +131,17 @@ def kmeans_tile(vecs: np.ndarray, entries: int, iters: int, rng: np.random.Gener
     move each centre to the (optionally weighted) mean of its members; an empty
     cluster keeps its previous centre.  Centres are then rounded to fp16 and the
     final assignment is taken against the rounded centres.
+
+    With `weights` (X^2 of Section 4.2, one per vector or one per element) both
+    Lloyd half-steps minimise the loss of Eq. 19: vectors go to the centre with
+    the smallest weighted distance and a centre moves, per dimension, to the
+    weighted mean of its members (a dimension whose member weights sum to zero
+    keeps its value).  Seeding ignores the weights.
     """
     v = np.asarray(vecs, dtype=np.float64)
     n, d = v.shape
     wt = np.ones((n, 1)) if weights is None else np.asarray(weights, dtype=np.float64).reshape(n, -1)
+    wa = None if weights is None else np.broadcast_to(wt, (n, d))
     centres = np.empty((entries, d))
     centres[0] = v[rng.integers(n)]
     dist = ((v - centres[0]) ** 2).sum(axis=1)
@@ -144,7 +156,7 @@ def kmeans_tile(vecs: np.ndarray, entries: int, iters: int, rng: np.random.Gener
         dist = np.minimum(dist, ((v - centres[e]) ** 2).sum(axis=1))
     losses = []
     for _ in range(iters):
-        idx = _nearest(v, centres)
+        idx = _nearest(v, centres, wa)
         if return_losses:
             losses.append(float((wt * (v - centres[idx]) ** 2).sum()))
         for dd in range(d):
@@ -154,7 +166,7 @@ def kmeans_tile(vecs: np.ndarray, entries: int, iters: int, rng: np.random.Gener
             upd = den > 0
             centres[upd, dd] = num[upd] / den[upd]
     cb16 = centres.astype(np.float16)
-    idx = _nearest(v, cb16.astype(np.float64))
+    idx = _nearest(v, cb16.astype(np.float64), wa)
     if return_losses:
         losses.append(float((wt * (v - cb16.astype(np.float64)[idx]) ** 2).sum()))
         return cb16, idx, losses
@@ -208,6 +220,19 @@ def mu_encode(mu16: np.ndarray, entries: int = 64, iters: int = 10, seed: int = 
     wts = None if act_sq is None else np.asarray(act_sq, dtype=np.float64).reshape(-1, 2)
     cb, ix = kmeans_tile(mu, entries, iters, rng, weights=wts)
     return cb, ix.astype(np.uint8 if entries <= 256 else np.uint16)
+
+
+def representative_activation(samples: np.ndarray, pct: float) -> np.ndarray:
+    """Representative X of a batch of calibration activations (Section 4.2):
+    every position's samples are first limited to the range between their
+    pct-th and (100 - pct)-th percentiles (percentiles by linear interpolation
+    between order statistics), then averaged.  samples: [S, n]; returns [n]
+    float64.  pct = 0 is the plain mean the paper calls outlier-prone."""
+    x = np.asarray(samples, dtype=np.float64)
+    assert x.ndim == 2 and 0.0 <= pct < 50.0
+    lo = np.percentile(x, pct, axis=0)
+    hi = np.percentile(x, 100.0 - pct, axis=0)
+    return np.clip(x, lo[None, :], hi[None, :]).mean(axis=0)
 
 
 def mu_decode(cb: np.ndarray, idx: np.ndarray) -> np.ndarray:

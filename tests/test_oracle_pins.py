@@ -172,6 +172,67 @@ def test_weighted_kmeans_minimises_weighted_loss():
     assert np.allclose(cb.astype(np.float64)[0], [0.75, 0.75])
 
 
+def test_weighted_kmeans_both_half_steps_lower_eq19():
+    # Eq. 19: with element weights X^2 spanning six decades, assignment by weighted distance and
+    # weighted means never raise the loss; the final assignment is the brute-force weighted argmin.
+    rng = np.random.default_rng(11)
+    vecs = rng.uniform(0.0, 1.0, (400, 2)).astype(np.float16).astype(np.float64)
+    wts = 10.0 ** rng.uniform(-3.0, 3.0, (400, 2))
+    cb, ix, losses = orc.kmeans_tile(vecs, 8, 10, np.random.default_rng(2), weights=wts, return_losses=True)
+    body = losses[:-1]
+    assert all(b <= a * (1 + 1e-12) for a, b in zip(body, body[1:]))
+    assert body[-1] < body[0]
+    c = cb.astype(np.float64)
+    for i in range(len(vecs)):
+        d = [wts[i, 0] * (vecs[i, 0] - c[e, 0]) ** 2 + wts[i, 1] * (vecs[i, 1] - c[e, 1]) ** 2 for e in range(8)]
+        assert ix[i] == d.index(min(d))
+    # an unweighted assignment is a different (worse or equal) answer under Eq. 19
+    ix_plain = orc._nearest(vecs, c)
+    loss_w = float((wts * (vecs - c[ix]) ** 2).sum())
+    loss_p = float((wts * (vecs - c[ix_plain]) ** 2).sum())
+    assert loss_w <= loss_p and not np.array_equal(ix, ix_plain)
+
+
+def test_weighted_kmeans_zero_weight_elements_do_not_move_centres():
+    # vectors whose weights are zero contribute nothing to Eq. 19: the single centre sits on the
+    # weighted members' mean however far the unweighted ones are.
+    vecs = np.array([[0.25, 0.5]] * 4 + [[100.0, -100.0]] * 4)
+    wts = np.array([[2.0, 2.0]] * 4 + [[0.0, 0.0]] * 4)
+    cb, _ = orc.kmeans_tile(vecs, 1, 2, np.random.default_rng(0), weights=wts)
+    assert np.array_equal(cb.astype(np.float64)[0], [0.25, 0.5])
+
+
+def test_representative_activation_hand_worked():
+    # Section 4.2.  Four samples 0, 1, 2, 10 of one position, pct = 25: the percentiles by linear
+    # interpolation sit at positions 0.75 and 2.25 of the sorted samples, i.e. 0.75 and
+    # 2 + 0.25 * 8 = 4; the limited samples 0.75, 1, 2, 4 average to 1.9375 (plain mean 3.25).
+    x = np.array([[2.0], [10.0], [0.0], [1.0]])
+    assert orc.representative_activation(x, 25.0)[0] == 1.9375
+    assert orc.representative_activation(x, 0.0)[0] == 3.25
+    # 101 samples 0..99 and one outlier 10000, pct = 10: limits are the order statistics 10 and
+    # 90, the limited samples sum to 10*10 + (10+...+90) + 10*90 = 5050, mean 50 (plain mean 148.02).
+    col = np.concatenate([np.arange(100.0), [10000.0]])
+    rep = orc.representative_activation(np.random.default_rng(0).permutation(col)[:, None], 10.0)
+    assert abs(rep[0] - 50.0) < 1e-12
+    assert abs(orc.representative_activation(col[:, None], 0.0)[0] - 14950.0 / 101.0) < 1e-12
+
+
+def test_representative_activation_matches_winsorised_mean_on_order_statistics():
+    # Where the percentiles fall exactly on order statistics the clipped mean is the winsorised
+    # mean of a statistics library.
+    from scipy.stats.mstats import winsorize
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((101, 7))
+    x[rng.integers(0, 101, 5), rng.integers(0, 7, 5)] *= 50.0
+    rep = orc.representative_activation(x, 10.0)
+    for j in range(7):
+        ref = float(np.asarray(winsorize(x[:, j], limits=(0.1, 0.1))).mean())
+        assert abs(rep[j] - ref) < 1e-12
+    # constant positions stay put; each position is treated on its own
+    y = np.tile(np.array([[1.5, -2.0]]), (9, 1))
+    assert np.array_equal(orc.representative_activation(y, 5.0), [1.5, -2.0])
+
+
 def test_mu_roundtrip_shapes():
     mu = np.linspace(0.0, 1.0, 512).astype(np.float16)
     cb, ix = orc.mu_encode(mu, entries=64, iters=10, seed=0)
