@@ -221,6 +221,49 @@ rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* W_desc, const void* W_image_de
 rwkvq_status rwkvq_dequant(const rwkvq_desc* W_desc, const void* W_image_dev, void* out_dev,
                            int dtype, void* stream);
 
+/*
+ * Description (padded sizes, image_bytes, stream_bytes) of the image that rwkvq_pack and
+ * rwkvq_quantize_dev produce for an oc x ic matrix (or a vector, oc == 1 with method VQ) under
+ * `cfg`; only method, bits, group, vec_dim and tile of cfg are read.  Errors as rwkvq_pack.
+ */
+rwkvq_status rwkvq_desc_for(const rwkvq_quant_cfg* cfg, int oc, int ic, rwkvq_desc* desc_out);
+
+/*
+ * The quantizers of rwkvq_pack as device kernels: W[oc][ic] fp16 in device memory is quantized
+ * and written as a packed image straight into image_dev (256-byte aligned, at least
+ * desc.image_bytes of rwkvq_desc_for), ready for every product call above.
+ *  SQ (Eq. 2): codes, scales and zero points are identical to rwkvq_pack's (same rounding rules),
+ *      bit for bit.
+ *  VQ (Eq. 3): one thread block per 256 x 256 tile (or per vector) runs k-means++ seeding and
+ *      cfg->kmeans_iters Lloyd iterations in fp32 with exact integer cluster sums, rounds the
+ *      centres to fp16 and takes the final assignment in fp64 against the rounded centres (lowest
+ *      index wins ties).  Random draws come from the library's generator seeded with cfg->seed and
+ *      the tile number; results are reproducible but differ from rwkvq_pack's codebooks.
+ *  elem_weight_dev (vectors only, else NULL): fp32 [ic], the X^2 of Section 4.2 Eq. 19 for each
+ *      element of mu.  Vectors are then assigned by the weighted distance and centres move to the
+ *      weighted means (fp64, fixed order), which is the weighted k-means of Section 4.2.
+ *  cfg->codes_in must be NULL.  The image carries no checksum (rwkvq_image_unpack accepts that).
+ *  workspace_dev: rwkvq_quantize_workspace_bytes() bytes, 16-byte aligned, contents irrelevant.
+ * The call synchronizes `stream` before it returns (it reads back a flag word).  Errors: EINVAL,
+ * ESHAPE, EUNSUPPORTED, EALIGN, ENOMEM (image or workspace too small), ENONFINITE, ECUDA.
+ */
+size_t rwkvq_quantize_workspace_bytes(void);
+rwkvq_status rwkvq_quantize_dev(const void* w_fp16_dev, int oc, int ic, const rwkvq_quant_cfg* cfg,
+                                const float* elem_weight_dev, void* image_dev, size_t image_bytes,
+                                rwkvq_desc* desc_out, void* workspace_dev, size_t workspace_bytes,
+                                void* stream);
+
+/*
+ * Representative X of a batch of calibration activations (Section 4.2): for each of the n
+ * positions, the n_samples values samples_dev[s][j] (fp32, row-major [n_samples][n],
+ * 2 <= n_samples <= 1024) are limited to the range between their pct-th and (100 - pct)-th
+ * percentiles (linear interpolation between order statistics, 0 <= pct < 50) and averaged in
+ * fp64.  rep_dev[j] receives the mean, rep_sq_dev[j] its square (the weight of Eq. 19); either
+ * may be NULL.  Asynchronous on `stream`.  Errors: EINVAL, ECUDA.
+ */
+rwkvq_status rwkvq_calib_representative(const float* samples_dev, int n_samples, int n, double pct,
+                                        float* rep_dev, float* rep_sq_dev, void* stream);
+
 /* Device status word of the last launches on this device: RWKVQ_OK, or ETIMEOUT if a bounded
  * wait inside a kernel gave up.  Synchronizes `stream`; clears the word. */
 rwkvq_status rwkvq_device_status(void* stream);

@@ -61,6 +61,7 @@ EXPORTS = [
     "rwkvq_step_run_host",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
+    "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
 ]
 
 _lib = None
@@ -113,6 +114,12 @@ def lib() -> C.CDLL:
         L.rwkvq_prefill_workspace_bytes.argtypes = [C.POINTER(Desc), i32, i32]
         L.rwkvq_prefill_workspace_bytes.restype = sz
         L.rwkvq_gemm_prefill.argtypes = [C.POINTER(Desc), vp, C.POINTER(Desc), vp, vp, vp, i32, vp, i32, vp, sz, vp]
+    if hasattr(L, "rwkvq_quantize_dev"):
+        L.rwkvq_desc_for.argtypes = [C.POINTER(QuantCfg), i32, i32, C.POINTER(Desc)]
+        L.rwkvq_quantize_workspace_bytes.argtypes = []
+        L.rwkvq_quantize_workspace_bytes.restype = sz
+        L.rwkvq_quantize_dev.argtypes = [vp, i32, i32, C.POINTER(QuantCfg), vp, vp, sz, C.POINTER(Desc), vp, sz, vp]
+        L.rwkvq_calib_representative.argtypes = [vp, i32, i32, dbl, vp, vp, vp]
     _lib = L
     return L
 
@@ -358,3 +365,38 @@ def rwkvq_gemm_prefill(desc: Desc, W_image, mu_desc, mu_image, X, xprev0, M: int
                                     _dev_ptr(workspace),
                                     0 if workspace is None else workspace.numel() * workspace.element_size(),
                                     _stream_ptr(stream)), "rwkvq_gemm_prefill")
+
+
+def rwkvq_desc_for(oc: int, ic: int, method: int, bits: int, *, group: int = 128, vec_dim: int = 2,
+                   tile: int = 256) -> Desc:
+    cfg = QuantCfg(method=method, bits=bits, group=group, vec_dim=vec_dim, tile=tile, kmeans_iters=0, seed=0,
+                   codes_in=None)
+    d = Desc()
+    _check(lib().rwkvq_desc_for(C.byref(cfg), oc, ic, C.byref(d)), "rwkvq_desc_for")
+    return d
+
+
+def rwkvq_quantize_workspace_bytes() -> int:
+    return int(lib().rwkvq_quantize_workspace_bytes())
+
+
+def rwkvq_quantize_dev(w, oc: int, ic: int, method: int, bits: int, image, workspace, *, elem_weight=None,
+                       group: int = 128, vec_dim: int = 2, tile: int = 256, kmeans_iters: int = 10, seed: int = 0,
+                       stream=None) -> Desc:
+    """rwkvq_quantize_dev.  `w`: float16 CUDA tensor [oc, ic]; `image`: uint8 CUDA tensor that receives
+    the packed image; `elem_weight`: float32 CUDA tensor [ic] (vectors only) or None."""
+    cfg = QuantCfg(method=method, bits=bits, group=group, vec_dim=vec_dim, tile=tile, kmeans_iters=kmeans_iters,
+                   seed=seed, codes_in=None)
+    d = Desc()
+    _check(lib().rwkvq_quantize_dev(_dev_ptr(w), oc, ic, C.byref(cfg), _dev_ptr(elem_weight), _dev_ptr(image),
+                                    image.numel() * image.element_size(), C.byref(d), _dev_ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+           "rwkvq_quantize_dev")
+    return d
+
+
+def rwkvq_calib_representative(samples, pct: float, rep=None, rep_sq=None, stream=None):
+    """rwkvq_calib_representative.  `samples`: float32 CUDA tensor [n_samples, n]."""
+    S, n = samples.shape
+    _check(lib().rwkvq_calib_representative(_dev_ptr(samples), S, n, float(pct), _dev_ptr(rep), _dev_ptr(rep_sq),
+                                            _stream_ptr(stream)), "rwkvq_calib_representative")

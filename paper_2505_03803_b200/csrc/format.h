@@ -68,6 +68,8 @@ struct rwkvq_image_header {
 static_assert(sizeof(rwkvq_image_header) == RWKVQ_HEADER_BYTES, "header size");
 #endif
 
+#define RWKVQ_IMAGE_FLAG_NO_CRC 1u /* reserved1 bit 0: the image was written on the device, crc32 is not set */
+
 #if defined(__CUDACC__)
 #define RWKVQ_HD __host__ __device__ inline
 #else
@@ -87,3 +89,33 @@ RWKVQ_HD int rwkvq_sq_bias(int o, int h) {
   return 1024 >> rwkvq_sq_pos(4 * m + R);
 }
 RWKVQ_HD uint32_t rwkvq_vq_record_bytes(int bits) { return 64u * 32u * (uint32_t)bits / 8u; }
+
+#ifdef __cplusplus
+// Header of the image of a matrix (or vector) with these logical sizes; crc32 is left 0.
+inline void rwkvq_fill_header(rwkvq_image_header* h, int method, int bits, int oc, int ic, int oc_pad, int ic_pad,
+                              int group, int vec_dim, int tile, int entries, bool is_vector,
+                              uint64_t image_bytes, uint64_t stream_bytes) {
+  *h = rwkvq_image_header{};
+  h->magic = RWKVQ_MAGIC; h->version = RWKVQ_VERSION;
+  h->method = (uint32_t)method; h->bits = (uint32_t)bits; h->oc = (uint32_t)oc; h->ic = (uint32_t)ic;
+  h->oc_pad = (uint32_t)oc_pad; h->ic_pad = (uint32_t)ic_pad;
+  h->group = (uint32_t)group; h->vec_dim = (uint32_t)vec_dim; h->tile = (uint32_t)tile; h->entries = (uint32_t)entries;
+  h->is_vector = is_vector ? 1u : 0u;
+  h->off_payload = RWKVQ_HEADER_BYTES;
+  h->image_bytes = image_bytes; h->stream_bytes = stream_bytes;
+  if (method == 1) {            // SQ
+    h->record_bytes = RWKVQ_SQ_RECORD_BYTES; h->chunk_bytes = 8 * RWKVQ_SQ_RECORD_BYTES;
+    h->payload_bytes = (uint64_t)(oc_pad / 128) * (uint64_t)(ic_pad / 256) * h->chunk_bytes;
+    h->aux_bytes = 0;
+  } else if (!is_vector) {      // VQ matrix
+    h->record_bytes = rwkvq_vq_record_bytes(bits); h->chunk_bytes = 8 * h->record_bytes;
+    h->payload_bytes = (uint64_t)(oc / 128) * (uint64_t)(ic / 256) * h->chunk_bytes;
+    h->aux_bytes = (uint64_t)(oc / 256) * (uint64_t)(ic / 256) * (uint64_t)entries * 4;
+  } else {                      // VQ vector
+    h->record_bytes = 0; h->chunk_bytes = 0;
+    h->payload_bytes = ((((uint64_t)(ic / 2) * (uint64_t)bits + 7) / 8) + 15) / 16 * 16;
+    h->aux_bytes = (uint64_t)entries * 4;
+  }
+  h->off_aux = h->off_payload + h->payload_bytes;
+}
+#endif

@@ -330,19 +330,11 @@ void build_image(rwkvq_blob* b) {
   const rwkvq_desc& d = b->desc;
   b->image.assign(d.image_bytes, 0);
   rwkvq_image_header h;
-  std::memset(&h, 0, sizeof(h));
-  h.magic = RWKVQ_MAGIC; h.version = RWKVQ_VERSION;
-  h.method = d.method; h.bits = d.bits; h.oc = d.oc; h.ic = d.ic; h.oc_pad = d.oc_pad; h.ic_pad = d.ic_pad;
-  h.group = d.group; h.vec_dim = d.vec_dim; h.tile = d.tile; h.entries = d.entries;
-  h.is_vector = b->is_vector;
-  h.off_payload = RWKVQ_HEADER_BYTES;
-  h.image_bytes = d.image_bytes; h.stream_bytes = d.stream_bytes;
+  rwkvq_fill_header(&h, d.method, d.bits, d.oc, d.ic, d.oc_pad, d.ic_pad, d.group, d.vec_dim, d.tile, d.entries,
+                    b->is_vector, d.image_bytes, d.stream_bytes);
   uint8_t* img = b->image.data();
   if (d.method == RWKVQ_SQ) {
-    h.record_bytes = RWKVQ_SQ_RECORD_BYTES; h.chunk_bytes = 8 * RWKVQ_SQ_RECORD_BYTES;
     int MB = d.oc_pad / 128, KT = d.ic_pad / 256, ng = d.ic / 128;
-    h.payload_bytes = (uint64_t)MB * KT * h.chunk_bytes;
-    h.off_aux = h.off_payload + h.payload_bytes; h.aux_bytes = 0;
 #pragma omp parallel for collapse(2) schedule(static)
     for (int mb = 0; mb < MB; ++mb)
       for (int kt = 0; kt < KT; ++kt)
@@ -361,11 +353,7 @@ void build_image(rwkvq_blob* b) {
         }
   } else if (!b->is_vector) {
     uint32_t rb = rwkvq_vq_record_bytes(d.bits);
-    h.record_bytes = rb; h.chunk_bytes = 8 * rb;
     int MB = d.oc / 128, KT = d.ic / 256;
-    h.payload_bytes = (uint64_t)MB * KT * h.chunk_bytes;
-    h.off_aux = h.off_payload + h.payload_bytes;
-    h.aux_bytes = (uint64_t)(d.oc / 256) * KT * d.entries * 4;
 #pragma omp parallel for collapse(2) schedule(static)
     for (int mb = 0; mb < MB; ++mb)
       for (int kt = 0; kt < KT; ++kt)
@@ -375,10 +363,6 @@ void build_image(rwkvq_blob* b) {
         }
     std::memcpy(img + h.off_aux, b->codebook.data(), h.aux_bytes);
   } else {
-    h.record_bytes = 0; h.chunk_bytes = 0;
-    h.payload_bytes = round_up(((size_t)(d.ic / 2) * d.bits + 7) / 8, 16);
-    h.off_aux = h.off_payload + h.payload_bytes;
-    h.aux_bytes = (uint64_t)d.entries * 4;
     for (int p = 0; p < d.ic / 2; ++p) put_bits(img + h.off_payload, (size_t)p * d.bits, b->q[p], d.bits);
     std::memcpy(img + h.off_aux, b->codebook.data(), h.aux_bytes);
   }
@@ -483,6 +467,14 @@ rwkvq_status rwkvq_pack(const uint16_t* w, int oc, int ic, const rwkvq_quant_cfg
   return RWKVQ_OK;
 }
 
+rwkvq_status rwkvq_desc_for(const rwkvq_quant_cfg* cfg, int oc, int ic, rwkvq_desc* desc_out) {
+  if (!cfg || !desc_out) return RWKVQ_EINVAL;
+  rwkvq_status st = fill_desc(desc_out, cfg->method, cfg->bits, oc, ic, cfg->group, cfg->tile,
+                              cfg->method == RWKVQ_VQ && oc == 1);
+  if (st == RWKVQ_OK && cfg->method == RWKVQ_VQ && cfg->vec_dim != 2) st = RWKVQ_EUNSUPPORTED;
+  return st;
+}
+
 rwkvq_status rwkvq_blob_desc(const rwkvq_blob* b, rwkvq_desc* d) {
   if (!b || !d) return RWKVQ_EINVAL;
   *d = b->desc;
@@ -519,7 +511,15 @@ rwkvq_status rwkvq_image_unpack(const void* image, size_t n, rwkvq_desc* desc_ou
   if (st != RWKVQ_OK) return st;
   if (d.image_bytes != h.image_bytes || n < d.image_bytes) return RWKVQ_EINVAL;
   const uint8_t* img = static_cast<const uint8_t*>(image);
-  if (crc32_of(img + RWKVQ_HEADER_BYTES, d.image_bytes - RWKVQ_HEADER_BYTES) != h.crc32) return RWKVQ_EINVAL;
+  if (!(h.reserved1 & RWKVQ_IMAGE_FLAG_NO_CRC) &&
+      crc32_of(img + RWKVQ_HEADER_BYTES, d.image_bytes - RWKVQ_HEADER_BYTES) != h.crc32) return RWKVQ_EINVAL;
+  {  // offsets come from the logical sizes, never from the header bytes
+    rwkvq_image_header ref;
+    rwkvq_fill_header(&ref, d.method, d.bits, d.oc, d.ic, d.oc_pad, d.ic_pad, d.group, d.vec_dim, d.tile, d.entries,
+                      h.is_vector != 0, d.image_bytes, d.stream_bytes);
+    if (ref.off_payload != h.off_payload || ref.off_aux != h.off_aux || ref.aux_bytes != h.aux_bytes ||
+        ref.off_aux + ref.aux_bytes > d.image_bytes) return RWKVQ_EINVAL;
+  }
   if (desc_out) *desc_out = d;
   if (!dst) return RWKVQ_OK;
   if (!dst->q) return RWKVQ_EINVAL;

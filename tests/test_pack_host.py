@@ -241,3 +241,15 @@ def test_error_paths():
     with pytest.raises(B.RwkvqError):
         B.rwkvq_image_unpack(broken)
     assert B.lib().rwkvq_status_str(8) == b"device-side wait timed out"
+
+
+def test_desc_for_matches_the_packer():
+    for method, bits, oc, ic in ((B.RWKVQ_SQ, 3, 272, 384), (B.RWKVQ_VQ, 6, 256, 512), (B.RWKVQ_VQ, 8, 512, 256),
+                                 (B.RWKVQ_VQ, 6, 1, 514)):
+        w = np.zeros((oc, ic), dtype=np.float16)
+        blob = B.rwkvq_pack(w, oc, ic, method, bits, kmeans_iters=1)
+        d, e = B.rwkvq_desc_for(oc, ic, method, bits), blob.desc
+        for f, _ in B.Desc._fields_:
+            assert getattr(d, f) == getattr(e, f), f
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_desc_for(100, 384, B.RWKVQ_SQ, 3)
