@@ -56,6 +56,9 @@ def parse_args(argv=None):
                     help="step = one persistent launch per step; ops = one rwkvq_gemv launch per product")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill leg (one 7B-class layer, M = 2048)")
+    ap.add_argument("--quantizer", default="host", choices=["host", "device"],
+                    help="where the stack's weights are quantized and packed: rwkvq_pack or rwkvq_quantize_dev")
+    ap.add_argument("--no-quantize", action="store_true", help="skip the device-quantizer leg (one 7B-class layer)")
     return ap.parse_args(argv)
 
 
@@ -315,6 +318,57 @@ def prefill_leg(reps: int = 10, M: int = 2048):
                          "frac_of_2250_nominal": tf / 2250.0}}
 
 
+def quantize_leg(reps: int = 5):
+    """The device quantizers on one 7B-class layer: every projection scalar-quantized (Eq. 2) from fp16
+    weights resident on the device, timed over the layer, and one 4096 x 4096 matrix vector-quantized
+    (Eq. 3, 256 tiles, 64 entries, 10 Lloyd iterations).  The scalar quantizer reads 2 bytes and writes
+    0.40625 bytes per weight: an HBM-bound kernel."""
+    import torch
+    from paper_2505_03803_b200 import binding as B
+    from paper_2505_03803_b200 import inputs
+    sp = inputs.STACKS["c3_7b"]
+    gen = torch.Generator(device="cuda").manual_seed(1234)
+    ws = torch.empty(B.rwkvq_quantize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    mats = []
+    for (name, oc, ic, has_mu, stage) in inputs.layer_shapes(sp["d"], sp["h"]):
+        w = (torch.randn((oc, ic), generator=gen, device="cuda") * 0.02).to(torch.float16)
+        d = B.rwkvq_desc_for(oc, ic, B.RWKVQ_SQ, 3)
+        mats.append((w, oc, ic, torch.empty(int(d.image_bytes), dtype=torch.uint8, device="cuda")))
+
+    def layer():
+        for (w, oc, ic, img) in mats:
+            B.rwkvq_quantize_dev(w, oc, ic, B.RWKVQ_SQ, 3, img, ws)
+    layer()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        layer()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    weights = sum(oc * ic for (_w, oc, ic, _i) in mats)
+    nbytes = sum(2 * oc * ic + img.numel() for (_w, oc, ic, img) in mats)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    peak, kind = measured_hbm_peak()
+    w, oc, ic, _ = mats[0]
+    dv = B.rwkvq_desc_for(oc, ic, B.RWKVQ_VQ, 6)
+    imgv = torch.empty(int(dv.image_bytes), dtype=torch.uint8, device="cuda")
+    B.rwkvq_quantize_dev(w, oc, ic, B.RWKVQ_VQ, 6, imgv, ws)
+    torch.cuda.synchronize()
+    e0.record()
+    B.rwkvq_quantize_dev(w, oc, ic, B.RWKVQ_VQ, 6, imgv, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    vq_ms = e0.elapsed_time(e1)
+    return {"workload": "one 7B-class layer (8 projections, d=4096 h=14336), fp16 weights on the device -> packed images",
+            "sq_ms_per_layer": ms, "sq_weights_per_s": weights / (ms * 1e-3), "launches_per_layer": 2 * len(mats),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                         "peak_kind": f"of {kind}", "kernel": "sq_quantize_kernel", "algorithmic_bytes_per_layer": nbytes},
+            "vq": {"matrix": f"{oc}x{ic}, 64 entries, 10 Lloyd iterations", "ms": vq_ms, "tiles": (oc // 256) * (ic // 256),
+                   "weights_per_s": oc * ic / (vq_ms * 1e-3)}}
+
+
 # ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
@@ -344,7 +398,8 @@ def run_ours(args):
     force = None if args.force_method is None else (B.RWKVQ_SQ if args.force_method == "sq" else B.RWKVQ_VQ)
     t_setup = time.time()
     st = stack_mod.Stack(sp["d"], sp["h"], sp["layers"], sp["entries"], batch, n_outliers=sp["outliers"],
-                         tag=args.workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force)
+                         tag=args.workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force,
+                         quantizer=args.quantizer)
     if args.mode == "step":
         st.plan_step()
     setup_s = time.time() - t_setup
@@ -440,6 +495,9 @@ def run_ours(args):
     prefill = None
     if world == 1 and not args.no_prefill:
         prefill = prefill_leg()
+    quantize = None
+    if world == 1 and not args.no_quantize:
+        quantize = quantize_leg()
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -456,14 +514,14 @@ def run_ours(args):
         "config": {"workload": workload_name(args.workload, batch), "batch": batch, "mode": args.mode,
                    "matrices": len(st.ops), "sq_matrices": st.n_sq, "stages": st.n_stages,
                    "weights": st.n_weights, "packed_bytes_per_step": st.stream_bytes,
-                   "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src,
+                   "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src, "quantizer": st.quantizer,
                    "l2": "inputs larger than L2: every step streams the whole packed stack once",
                    "replicas": "independent replica per GPU, no exchange step" if world > 1 else "single GPU",
                    "not_included": "WKV recurrence, norms, gates, embedding and head are not part of the workload",
                    "tau_c": st.tau_c, "setup_s": round(setup_s, 1)},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": K * launches_per_step,
-        "hbm_gbs": achieved, "prefill": prefill,
+        "hbm_gbs": achieved, "prefill": prefill, "quantize": quantize,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

@@ -19,19 +19,26 @@ constexpr int kFlagNonFinite = 1;
 // ---- scalar quantizer ------------------------------------------------------------------------
 //
 // One warp per record (16 rows x 256 columns), one block of eight warps per chunk.  Pass 1 finds
-// each (row, group) minimum and maximum with shuffles (lanes 0..15 hold group 0, lanes 16..31
-// group 1, eight columns each); lane r + 16 h then derives (s, z) of (row r, group h) in fp64 exactly
-// as Eq. 2 prescribes.  Pass 2 codes the sixteen rows from the values still held in registers.
-// The per-weight division runs in fp32: w and s are fp16 numbers, so a quotient of magnitude up to
-// 8.5 that is not exactly a tie lies at least 2^-12 away from one and IEEE fp32 division rounds it
-// to the same integer as exact arithmetic would; larger quotients saturate the 3-bit code either way.
+// each (row, group) minimum and maximum with packed fp16 min/max and shuffles (lanes 0..15 hold
+// group 0, lanes 16..31 group 1, eight columns each); lane r + 16 h then derives (s, z) of
+// (row r, group h) in fp64 exactly as Eq. 2 prescribes.
+//
+// The codes need no division.  q = clamp(round(w / s) + z, 0, 7) counts the k in 1..7 with
+// round(w / s) >= k - z, and round(x) >= m (ties to even) holds iff x > m - 1/2, or x = m - 1/2
+// with m even.  (m - 1/2) * s is exact in fp32 (4 bits times 11 bits), so each k has an exact
+// fp16 threshold T_k -- the smallest fp16 number that is >= (or >) that product -- and
+// q = #{k : w >= T_k}, seven packed fp16 comparisons for two weights.  Pass 2 reads the rows
+// again (from cache) and counts.
 constexpr int kSqRowStride = 256 + 16;   // bytes per row of the code staging area: conflict-free lane reads
 
 __device__ __forceinline__ float h2f_bits(uint32_t h) { return __half2float(__ushort_as_half((unsigned short)h)); }
+__device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<__half2*>(&v); }
+__device__ __forceinline__ uint32_t as_u32(__half2 v) { return *reinterpret_cast<uint32_t*>(&v); }
 
-__global__ void __launch_bounds__(256) sq_quantize_kernel(const uint16_t* __restrict__ w, int oc, int ic, int KT,
-                                                          uint8_t* __restrict__ payload, int* __restrict__ flags) {
+__global__ void __launch_bounds__(256, 3) sq_quantize_kernel(const uint16_t* __restrict__ w, int oc, int ic, int KT,
+                                                             uint8_t* __restrict__ payload, int* __restrict__ flags) {
   __shared__ __align__(16) uint8_t codes_all[8][16 * kSqRowStride];
+  __shared__ __align__(16) uint32_t thr_all[8][2][16][8];     // [warp][group][row][k]: (T_k, T_k) as half2, k = 1..7 in 0..6
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int mb = blockIdx.x / KT, kt = blockIdx.x % KT;
   const int r0 = mb * 128 + warp * 16, c0 = kt * 256;
@@ -39,76 +46,91 @@ __global__ void __launch_bounds__(256) sq_quantize_kernel(const uint16_t* __rest
   const int half = lane >> 4;
   const int col = c0 + 8 * lane;
   const bool col_in = col < ic;            // ic is a multiple of 128: a whole group is inside or outside
-  uint4 raw[16];
+  const uint16_t* src = w + (size_t)r0 * ic + col;
   float my_mn = 0.f, my_mx = 0.f;
-  bool bad = false;
-#pragma unroll
+  uint32_t bad = 0u;
+#pragma unroll 4
   for (int r = 0; r < 16; ++r) {
-    const int row = r0 + r;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (col_in && row < oc) v = __ldg(reinterpret_cast<const uint4*>(w + (size_t)row * ic + col));
-    raw[r] = v;
-    const uint32_t words[4] = {v.x, v.y, v.z, v.w};
-    float mn = INFINITY, mx = -INFINITY;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const uint32_t lo = words[k] & 0xFFFFu, hi = words[k] >> 16;
-      bad |= ((lo & 0x7C00u) == 0x7C00u) | ((hi & 0x7C00u) == 0x7C00u);
-      const float a = h2f_bits(lo), b = h2f_bits(hi);
-      mn = fminf(mn, fminf(a, b));
-      mx = fmaxf(mx, fmaxf(a, b));
-    }
+    if (col_in && r0 + r < oc) v = __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * ic));
+    // an all-ones exponent carries into bit 15 of its half
+    bad |= ((v.x & 0x7C007C00u) + 0x04000400u) | ((v.y & 0x7C007C00u) + 0x04000400u) |
+           ((v.z & 0x7C007C00u) + 0x04000400u) | ((v.w & 0x7C007C00u) + 0x04000400u);
+    __half2 mn2 = __hmin2(__hmin2(as_h2(v.x), as_h2(v.y)), __hmin2(as_h2(v.z), as_h2(v.w)));
+    __half2 mx2 = __hmax2(__hmax2(as_h2(v.x), as_h2(v.y)), __hmax2(as_h2(v.z), as_h2(v.w)));
 #pragma unroll
     for (int off = 8; off >= 1; off >>= 1) {
-      mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
-      mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+      mn2 = __hmin2(mn2, as_h2(__shfl_xor_sync(0xFFFFFFFFu, as_u32(mn2), off)));
+      mx2 = __hmax2(mx2, as_h2(__shfl_xor_sync(0xFFFFFFFFu, as_u32(mx2), off)));
     }
-    if ((lane & 15) == r) { my_mn = mn; my_mx = mx; }
+    if ((lane & 15) == r) {
+      my_mn = fminf(__low2float(mn2), __high2float(mn2));
+      my_mx = fmaxf(__low2float(mx2), __high2float(mx2));
+    }
   }
-  if (bad) atomicOr(flags, kFlagNonFinite);
+  if (bad & 0x80008000u) atomicOr(flags, kFlagNonFinite);
   // (s, z) of (row lane & 15, group half), Eq. 2; a constant group c is coded exactly:
   // c == 0 -> (1, 0, q 0), c > 0 -> (c, 0, q 1), c < 0 -> (|c|, 1, q 0).
   float my_s, my_z;
-  int my_deg;     // 0: regular, 1: constant with q = 0, 2: constant with q = 1
   {
     const double mn = (double)my_mn, mx = (double)my_mx;
     const __half s16 = __double2half((mx - mn) / 7.0);
     const double s = (double)__half2float(s16);
+    uint32_t* thr = thr_all[warp][half][lane & 15];
+    const uint32_t kNever = 0x7C007C00u, kAlways = 0xFC00FC00u;     // +inf, -inf
     if (mx == mn || s == 0.0) {
       my_s = mn == 0.0 ? 1.f : fabsf(my_mn);
       my_z = mn < 0.0 ? 1.f : 0.f;
-      my_deg = mn > 0.0 ? 2 : 1;
+      thr[0] = mn > 0.0 ? kAlways : kNever;
+#pragma unroll
+      for (int k = 1; k < 7; ++k) thr[k] = kNever;
     } else {
       my_s = (float)s;
       my_z = (float)fmin(7.0, fmax(0.0, rint(-mn / s)));
-      my_deg = 0;
-    }
-  }
 #pragma unroll
-  for (int r = 0; r < 16; ++r) {
-    const int src = r + 16 * half;
-    const float s = __shfl_sync(0xFFFFFFFFu, my_s, src);
-    const float z = __shfl_sync(0xFFFFFFFFu, my_z, src);
-    const int deg = __shfl_sync(0xFFFFFFFFu, my_deg, src);
-    const uint32_t words[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
-    uint32_t out[2] = {0u, 0u};
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const uint32_t hbits = (words[k >> 1] >> (16 * (k & 1))) & 0xFFFFu;
-      uint32_t q;
-      if (deg) {
-        q = deg == 2 ? 1u : 0u;
-      } else {
-        const float v = rintf(__fdiv_rn(h2f_bits(hbits), s)) + z;
-        q = (uint32_t)fminf(7.f, fmaxf(0.f, v));
+      for (int k = 1; k <= 7; ++k) {
+        const float m = (float)k - my_z;
+        const float theta = (m - 0.5f) * my_s;                  // exact
+        __half t16 = __float2half_ru(theta);                   // smallest fp16 >= theta (+inf / -65504 beyond the range)
+        if (((int)m & 1) && __half2float(t16) == theta) {       // m odd: the tie rounds down, so w must exceed theta
+          const unsigned short hb = __half_as_ushort(t16);
+          t16 = __ushort_as_half((hb & 0x7FFFu) == 0 ? (unsigned short)1 : (hb & 0x8000u) ? (unsigned short)(hb - 1) : (unsigned short)(hb + 1));
+        }
+        const uint32_t tb = __half_as_ushort(t16);
+        thr[k - 1] = tb | (tb << 16);
       }
-      out[k >> 2] |= q << (8 * (k & 3));
     }
-    const bool inside = col_in && (r0 + r) < oc;
-    *reinterpret_cast<uint2*>(codes + r * kSqRowStride + 8 * lane) = inside ? make_uint2(out[0], out[1]) : make_uint2(0u, 0u);
+    thr[7] = 0u;
   }
   __syncwarp();
-  // Bit packing of format.h: lane (g, t) owns rows g and g + 8; triple i covers columns 64 i ..
+#pragma unroll 4
+  for (int r = 0; r < 16; ++r) {
+    const bool inside = col_in && (r0 + r) < oc;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (inside) v = __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * ic));
+    const uint4 ta = *reinterpret_cast<const uint4*>(thr_all[warp][half][r]);
+    const uint4 tb = *reinterpret_cast<const uint4*>(thr_all[warp][half][r] + 4);
+    const uint32_t words[4] = {v.x, v.y, v.z, v.w};
+    uint32_t qw[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const __half2 x = as_h2(words[k]);
+      __half2 acc = as_h2(0x64006400u);       // 1024: the count appears in the low mantissa bits
+      acc = __hadd2(acc, __hge2(x, as_h2(ta.x)));
+      acc = __hadd2(acc, __hge2(x, as_h2(ta.y)));
+      acc = __hadd2(acc, __hge2(x, as_h2(ta.z)));
+      acc = __hadd2(acc, __hge2(x, as_h2(ta.w)));
+      acc = __hadd2(acc, __hge2(x, as_h2(tb.x)));
+      acc = __hadd2(acc, __hge2(x, as_h2(tb.y)));
+      acc = __hadd2(acc, __hge2(x, as_h2(tb.z)));
+      qw[k] = as_u32(acc) & 0x00070007u;
+    }
+    const uint2 out = make_uint2(__byte_perm(qw[0], qw[1], 0x6420u), __byte_perm(qw[2], qw[3], 0x6420u));
+    *reinterpret_cast<uint2*>(codes + r * kSqRowStride + 8 * lane) = inside ? out : make_uint2(0u, 0u);
+  }
+  __syncwarp();
+  // Bit packing of format.h: lane (g, t) owns rows g and g + 8 and, in every tensor-core step,
+  // the four columns 4t .. 4t+3 (one 32-bit read of the staging area = registers R and R + 2).
   const int g = lane >> 2, t = lane & 3;
   uint8_t* rec = payload + ((size_t)blockIdx.x * 8 + warp) * RWKVQ_SQ_RECORD_BYTES;
   uint32_t wd[12];
@@ -116,17 +138,21 @@ __global__ void __launch_bounds__(256) sq_quantize_kernel(const uint16_t* __rest
   for (int i = 0; i < 4; ++i) {
     uint32_t w3[3] = {0u, 0u, 0u};
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-      const int m = e >> 2, R = e & 3;
-      const int row = g + 8 * (R & 1);
-      const int cc = 64 * i + 16 * m + 4 * t + 2 * (R >> 1);
-      const uint32_t two = *reinterpret_cast<const unsigned short*>(codes + row * kSqRowStride + cc);
-      const uint32_t pair = (two & 0xFFu) | ((two >> 8) << 16);
-      if (e < 15) {
-        w3[e / 5] |= pair << (3 * (e % 5));
-      } else {
+    for (int m = 0; m < 4; ++m) {
 #pragma unroll
-        for (int b = 0; b < 3; ++b) w3[b] |= ((pair >> b) & 0x00010001u) << 15;
+      for (int hrow = 0; hrow < 2; ++hrow) {
+        const uint32_t four = *reinterpret_cast<const uint32_t*>(codes + (g + 8 * hrow) * kSqRowStride + 64 * i + 16 * m + 4 * t);
+#pragma unroll
+        for (int cp = 0; cp < 2; ++cp) {
+          const int e = 4 * m + 2 * cp + hrow;             // register R = 2 * cp + hrow of step m
+          const uint32_t pair = __byte_perm(four, 0u, cp ? 0x4342u : 0x4140u);   // (even column) | (odd column) << 16
+          if (e < 15) {
+            w3[e / 5] |= pair << (3 * (e % 5));
+          } else {
+#pragma unroll
+            for (int b = 0; b < 3; ++b) w3[b] |= ((pair >> b) & 0x00010001u) << 15;
+          }
+        }
       }
     }
     wd[3 * i] = w3[0]; wd[3 * i + 1] = w3[1]; wd[3 * i + 2] = w3[2];

@@ -2,7 +2,8 @@
 the device, plus the activation buffers of one decode step.
 
 Only marshalling lives here: the selection runs in rwkvq_proxy_select, quantization and packing in
-rwkvq_pack, the products in rwkvq_gemv / rwkvq_step_run.
+rwkvq_pack (or, with quantizer="device", in rwkvq_quantize_dev), the products in rwkvq_gemv /
+rwkvq_step_run.
 """
 from __future__ import annotations
 
@@ -34,6 +35,27 @@ class MatrixEntry:
                  "desc", "image", "mu_desc", "mu_image", "x", "xprev", "y", "act_off")
 
 
+class _DeviceBlob:
+    """A matrix quantized and packed by rwkvq_quantize_dev: same surface as binding.Blob."""
+
+    def __init__(self, desc, image):
+        self.desc, self._image = desc, image
+
+    def to_device(self, device="cuda"):
+        return self._image.clone()
+
+    def export_codes(self):
+        return B.rwkvq_image_unpack(self._image.cpu().numpy())[1]
+
+
+def _device_blob(w_dev, oc, ic, method, bits, kmeans_iters, seed):
+    d = B.rwkvq_desc_for(oc, ic, method, bits)
+    image = torch.empty(int(d.image_bytes), dtype=torch.uint8, device=w_dev.device)
+    ws = torch.empty(B.rwkvq_quantize_workspace_bytes(), dtype=torch.uint8, device=w_dev.device)
+    d = B.rwkvq_quantize_dev(w_dev, oc, ic, method, bits, image, ws, kmeans_iters=kmeans_iters, seed=seed)
+    return _DeviceBlob(d, image)
+
+
 class Stack:
     """All projection matrices of `layers` RWKV-6 blocks of width d and channel-mix width h.
 
@@ -49,7 +71,9 @@ class Stack:
     def __init__(self, d: int, h: int, layers: int, entries: int, batch: int, n_outliers: int = 8,
                  heavy_fraction: float = 0.1, tag: str = "stack", device: str = "cuda",
                  distinct_layers: int = 0, force_method: int | None = None, kmeans_iters: int = 10,
-                 verbose: bool = False):
+                 verbose: bool = False, quantizer: str = "host"):
+        assert quantizer in ("host", "device")
+        self.quantizer = quantizer
         self.d, self.h, self.layers, self.entries, self.batch = d, h, layers, entries, batch
         self.tag, self.device = tag, device
         self.vq_bits = 6 if entries == 64 else 8
@@ -85,22 +109,29 @@ class Stack:
             mats = [torch.from_numpy(host_w[(l, name)][0]).to(device) for (name, *_r) in shapes]
             ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(mats)), dtype=torch.uint8, device=device)
             _, _, phi = B.rwkvq_proxy_select(mats, 4, self.tau_c, self.tau_f, ws)
-            del mats, ws
-            for (name, oc, ic, has_mu, stage), p in zip(shapes, phi):
+            del ws
+            for (name, oc, ic, has_mu, stage), p, w_dev in zip(shapes, phi, mats):
                 w, kind, seed, pc_v, pf_v = host_w[(l, name)]
                 method = int(p) if force_method is None else force_method
-                if method == B.RWKVQ_SQ:
+                if quantizer == "device":
+                    bits = 3 if method == B.RWKVQ_SQ else self.vq_bits
+                    blob = _device_blob(w_dev, oc, ic, method, bits, kmeans_iters, seed)
+                elif method == B.RWKVQ_SQ:
                     blob = B.rwkvq_pack(w, oc, ic, B.RWKVQ_SQ, 3)
                 else:
                     blob = B.rwkvq_pack(w, oc, ic, B.RWKVQ_VQ, self.vq_bits, kmeans_iters=kmeans_iters, seed=seed)
                 mu_blob = None
-                if has_mu:
+                if has_mu and quantizer == "device":
+                    mu = torch.from_numpy(inputs.gen_mu(seed ^ 0xABCD, ic)).to(device)
+                    mu_blob = _device_blob(mu, 1, ic, B.RWKVQ_VQ, self.vq_bits, kmeans_iters, seed + 1)
+                elif has_mu:
                     mu = inputs.gen_mu(seed ^ 0xABCD, ic)
                     mu_blob = B.rwkvq_pack(mu.reshape(1, -1), 1, ic, B.RWKVQ_VQ, self.vq_bits,
                                            kmeans_iters=kmeans_iters, seed=seed + 1)
                 packed[(l, name)] = (blob, mu_blob, kind, seed, method, pc_v, pf_v)
                 if verbose:
                     print(f"layer {l} {name}: {kind} pc={pc_v:.3f} -> {'SQ' if method else 'VQ'}", flush=True)
+            del mats
             for (name, *_r) in shapes:
                 host_w.pop((l, name))
         self.setup_seconds["select+pack"] = time.time() - t0

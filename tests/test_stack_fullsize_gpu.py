@@ -25,9 +25,12 @@ def _oracle_product(st, op):
     return orc.gemv(w_hat, x), orc.tolerance(w_hat, x)
 
 
-@pytest.mark.parametrize("name,batch", [("c2_1p6b", 1), ("c3_7b", 8), ("c4_14b", 16)])
-def test_whole_step_at_benchmark_size_matches_oracle_on_sampled_products(name, batch):
-    st = stack_mod.from_name(name, batch=batch, distinct_layers=1, kmeans_iters=2)
+@pytest.mark.parametrize("name,batch,quantizer", [("c2_1p6b", 1, "host"), ("c3_7b", 8, "host"), ("c4_14b", 16, "host"),
+                                                  ("c2_1p6b", 1, "device")])
+def test_whole_step_at_benchmark_size_matches_oracle_on_sampled_products(name, batch, quantizer):
+    # quantizer = "device": the images come from rwkvq_quantize_dev, the oracle decodes the codes
+    # unpacked from those images
+    st = stack_mod.from_name(name, batch=batch, distinct_layers=1, kmeans_iters=2, quantizer=quantizer)
     st.plan_step()
     for _ in range(2):                      # a second run must reproduce the first (outputs are cleared in the kernel)
         st.run_step()
