@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
 # profiles/step_kernel_c2_1p6b_b1.md.  Valid only for that workload and for the kernel as it was
 # when the counters were taken: set an entry to None when step.cu changes.
-NCU_TRAFFIC_BYTES = {("c2_1p6b", 1, "step", None, 4): 541_582_592}
+NCU_TRAFFIC_BYTES = {("c2_1p6b", 1, "step", None, 4): None}
 
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
@@ -56,6 +56,10 @@ def parse_args(argv=None):
                     help="step = one persistent launch per step; ops = one rwkvq_gemv launch per product")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill leg (one 7B-class layer, M = 2048)")
+    ap.add_argument("--stage-group", type=int, default=0,
+                    help="diagnostic: put this many consecutive products into one stage instead of the layer's own "
+                         "four dependent stages (0 = the real dependencies); a large value removes every grid barrier "
+                         "and shows the streaming rate of the kernel alone")
     ap.add_argument("--quantizer", default="host", choices=["host", "device"],
                     help="where the stack's weights are quantized and packed: rwkvq_pack or rwkvq_quantize_dev")
     ap.add_argument("--no-quantize", action="store_true", help="skip the device-quantizer leg (one 7B-class layer)")
@@ -400,6 +404,10 @@ def run_ours(args):
     st = stack_mod.Stack(sp["d"], sp["h"], sp["layers"], sp["entries"], batch, n_outliers=sp["outliers"],
                          tag=args.workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force,
                          quantizer=args.quantizer)
+    if args.stage_group > 0:
+        for i, o in enumerate(st.ops):
+            o.stage = i // args.stage_group
+        st.n_stages = len({o.stage for o in st.ops})
     if args.mode == "step":
         st.plan_step()
     setup_s = time.time() - t_setup
@@ -481,7 +489,8 @@ def run_ours(args):
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
     achieved = alg_bytes / launches_per_step / (avg_launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, batch, args.mode, args.force_method, args.distinct_layers)),
+                "traffic": (NCU_TRAFFIC_BYTES.get((args.workload, batch, args.mode, args.force_method, args.distinct_layers))
+                            if args.stage_group == 0 and args.quantizer == "host" else None),
                 "peak_kind": f"of {peak_kind}", "kernel": "step_kernel" if args.mode == "step" else "gemv_kernel",
                 "algorithmic_bytes_per_launch": alg_bytes / launches_per_step,
                 "launch_ms_avg": avg_launch_ms, "launch_ms_median": statistics.median(per_launch_ms),
@@ -514,7 +523,7 @@ def run_ours(args):
         "config": {"workload": workload_name(args.workload, batch), "batch": batch, "mode": args.mode,
                    "matrices": len(st.ops), "sq_matrices": st.n_sq, "stages": st.n_stages,
                    "weights": st.n_weights, "packed_bytes_per_step": st.stream_bytes,
-                   "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src, "quantizer": st.quantizer,
+                   "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src, "quantizer": st.quantizer, "stage_group": args.stage_group,
                    "l2": "inputs larger than L2: every step streams the whole packed stack once",
                    "replicas": "independent replica per GPU, no exchange step" if world > 1 else "single GPU",
                    "not_included": "WKV recurrence, norms, gates, embedding and head are not part of the workload",

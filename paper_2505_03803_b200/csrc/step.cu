@@ -20,7 +20,7 @@
 //     the end of a run along K.
 //
 // The host plans the step once: every stage's units are dealt to the CTAs in contiguous,
-// byte-balanced ranges cut at one eighth of a unit (one warp's records), and written as a per-CTA
+// cost-balanced ranges cut at one eighth of a unit (one warp's records), and written as a per-CTA
 // list of 128-byte unit descriptors plus a list of 64-byte input events (segments and barrier
 // arrivals).
 #include <cuda_runtime.h>
@@ -688,9 +688,12 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
     }
   };
   uint8_t* rep = replicas + (size_t)grp * a.replica_bytes;
-  for (uint32_t i = (uint32_t)grp; i < n_units; i += kGroups) {
-    const int slot = (int)(i % (uint32_t)a.n_slots);
-    const uint32_t round = i / (uint32_t)a.n_slots;
+  // slot and round of unit i (i % n_slots, i / n_slots), advanced without dividing
+  const uint32_t n_slots_u = (uint32_t)a.n_slots;
+  uint32_t slot_u = (uint32_t)grp % n_slots_u, round = (uint32_t)grp / n_slots_u;
+  for (uint32_t i = (uint32_t)grp; i < n_units; i += kGroups, slot_u += kGroups) {
+    while (slot_u >= n_slots_u) { slot_u -= n_slots_u; ++round; }
+    const int slot = (int)slot_u;
     const uint8_t* sl = smem + kCtrlBytes + (size_t)slot * a.slot_bytes;
     const StepUnit* u = reinterpret_cast<const StepUnit*>(sl);
     if (!dead && !mbar_wait_warp(&ctrl->full[slot], round & 1u, abortp, a.status)) dead = true;
@@ -991,16 +994,25 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
           units.push_back(h);
         }
     }
-    // contiguous, byte-balanced ranges cut at one eighth of a unit (the records of one warp)
+    // contiguous, cost-balanced ranges cut at one eighth of a unit (the records of one warp).  The
+    // cost of a unit is its record count weighted by what a record of its format costs the consumer
+    // warps (measured with every product in one stage: a VQ record with 64 entries takes about 1.45
+    // times, one with 256 entries about 1.25 times as long as an SQ record), so that the CTAs that
+    // get a stage's VQ matrix do not finish last.
+    auto cost_of = [&](const HostUnit& h) -> uint64_t {
+      const uint64_t recs = (h.u.bytes0 + h.u.bytes1) / h.u.rec_bytes;
+      const uint64_t wgt = !(h.u.flags & UF_VQ) ? 20u : (h.u.flags & UF_BITS8) ? 25u : 29u;
+      return recs * wgt * 64u;
+    };
     uint64_t total = 0;
-    for (const HostUnit& h : units) total += h.u.bytes0 + h.u.bytes1;
+    for (const HostUnit& h : units) total += cost_of(h);
     uint64_t run = 0;
     auto cta_of = [&](uint64_t mid) {
       int c = (int)((mid * (uint64_t)P) / (total ? total : 1));
       return c >= P ? P - 1 : c;
     };
     for (const HostUnit& h : units) {
-      const uint64_t e8 = (h.u.bytes0 + h.u.bytes1) / 8;
+      const uint64_t e8 = cost_of(h) / 8;
       int w = 0;
       while (w < 8) {
         const int c = cta_of(run + (uint64_t)w * e8 + e8 / 2);
@@ -1017,7 +1029,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         cta_units[c].push_back(part);
         w = w1;
       }
-      run += h.u.bytes0 + h.u.bytes1;
+      run += cost_of(h);
     }
     for (int c = 0; c < P; ++c) make_arrival(c, s + 1, s + 1);
   }
