@@ -17,6 +17,8 @@ Passages followed (RWKVQuant, arXiv 2505.03803):
   * coarse proxy P_c                     -- Section 4.1, Eqs. 5-9
   * fine proxy P_f                       -- Section 4.1, Eqs. 10-17
   * selection rule phi                   -- Section 4.1, Eq. 18
+  * other statistics of G' (ablation)    -- Section 5.3 (Variance, CV, Range, MAD, IE); thresholds for a
+                                            target SQ share -- Section 5.1
   * token shift mix and projections      -- Appendix A.1, Eqs. 20-22, 24-26
   * weighted loss for element-wise mu    -- Section 4.2, Eq. 19 (weighted k-means; representative X by
                                             percentile clipping before the mean)
@@ -288,6 +290,45 @@ def proxy_taylor_signed(w: np.ndarray, K: int) -> float:
         mk = float((delta ** k).sum()) / n
         tot += (-1.0) ** k * float(n) ** k / (k * (k - 1)) * mk
     return tot
+
+
+def proxy_family(w: np.ndarray) -> dict:
+    """The simpler statistics of the normalised gaps G' that the ablation of Section 5.3 puts in
+    the proxy's place (Variance, Coefficient of Variation, Range, Mean Absolute Deviation, and the
+    information entropy alone), each in its textbook form on the n values G'_i (mean 1/n):
+
+        variance = sum (G' - 1/n)^2 / n        cv = sqrt(variance) / (1/n)
+        range    = max G' - min G'             mad = sum |G' - 1/n| / n
+        ie       = -sum G' ln G'   (0 ln 0 := 0; P_c = ln n - ie)
+
+    A constant matrix returns inf for all five."""
+    flat = np.sort(np.asarray(w, dtype=np.float64).reshape(-1))
+    g = flat[1:] - flat[:-1]
+    n = g.size
+    tot = g.sum()
+    if not tot > 0.0:
+        return {k: math.inf for k in ("variance", "cv", "range", "mad", "ie")}
+    gp = g / tot
+    mean = 1.0 / n
+    var = float(((gp - mean) ** 2).sum()) / n
+    nz = gp[gp > 0.0]
+    return {"variance": var, "cv": math.sqrt(var) / mean, "range": float(gp.max() - gp.min()),
+            "mad": float(np.abs(gp - mean).sum()) / n, "ie": -float((nz * np.log(nz)).sum())}
+
+
+def tau_for_fraction(values, sq_fraction: float) -> float:
+    """Threshold that sends the given fraction of the matrices to scalar quantization under
+    "SQ iff value < tau" (Section 5.1 sets the thresholds so that nine tenths of the layers use SQ):
+    with the M values sorted and k = round(sq_fraction * M), tau lies halfway between the k-th and
+    the (k+1)-th smallest; k = 0 gives -inf and k = M gives +inf."""
+    v = np.sort(np.asarray(values, dtype=np.float64))
+    m = v.size
+    k = int(np.rint(sq_fraction * m))
+    if k <= 0:
+        return -math.inf
+    if k >= m:
+        return math.inf
+    return 0.5 * (float(v[k - 1]) + float(v[k]))
 
 
 def select(pc: float, pf: float, tau_c: float, tau_f: float) -> int:

@@ -9,10 +9,11 @@
 
 namespace rwkvq {
 
-// (a & mask) | orv in one LOP3.
-__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t orv) {
+// (a & MASK) | orv in one LOP3; the mask is an immediate of the instruction.
+template <uint32_t MASK>
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t orv) {
   uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "n"(MASK), "r"(orv));
   return r;
 }
 
@@ -25,24 +26,24 @@ __host__ __device__ constexpr uint32_t sq_exp2(int pos) {
 // holding q + (1024 >> rwkvq_sq_pos(e)) exactly.  21 integer instructions for 32 codes.
 __device__ __forceinline__ void sq_unpack_triple(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t (&r)[16]) {
   const uint32_t ua = wa >> 9, ub = wb >> 8, uc = wc >> 7;
-  r[0] = and_or(wa, 0x00070007u, sq_exp2(0));
-  r[1] = and_or(wa, 0x00380038u, sq_exp2(3));
-  r[2] = and_or(wa, 0x01C001C0u, sq_exp2(6));
-  r[3] = and_or(ua, 0x00070007u, sq_exp2(0));
-  r[4] = and_or(ua, 0x00380038u, sq_exp2(3));
-  r[5] = and_or(wb, 0x00070007u, sq_exp2(0));
-  r[6] = and_or(wb, 0x00380038u, sq_exp2(3));
-  r[7] = and_or(wb, 0x01C001C0u, sq_exp2(6));
-  r[8] = and_or(ub, 0x000E000Eu, sq_exp2(1));
-  r[9] = and_or(ub, 0x00700070u, sq_exp2(4));
-  r[10] = and_or(wc, 0x00070007u, sq_exp2(0));
-  r[11] = and_or(wc, 0x00380038u, sq_exp2(3));
-  r[12] = and_or(wc, 0x01C001C0u, sq_exp2(6));
-  r[13] = and_or(uc, 0x001C001Cu, sq_exp2(2));
-  r[14] = and_or(uc, 0x00E000E0u, sq_exp2(5));
-  uint32_t s = and_or(ua, 0x00400040u, sq_exp2(6));
-  s = and_or(ub, 0x00800080u, s);
-  r[15] = and_or(uc, 0x01000100u, s);
+  r[0] = and_or<0x00070007u>(wa, sq_exp2(0));
+  r[1] = and_or<0x00380038u>(wa, sq_exp2(3));
+  r[2] = and_or<0x01C001C0u>(wa, sq_exp2(6));
+  r[3] = and_or<0x00070007u>(ua, sq_exp2(0));
+  r[4] = and_or<0x00380038u>(ua, sq_exp2(3));
+  r[5] = and_or<0x00070007u>(wb, sq_exp2(0));
+  r[6] = and_or<0x00380038u>(wb, sq_exp2(3));
+  r[7] = and_or<0x01C001C0u>(wb, sq_exp2(6));
+  r[8] = and_or<0x000E000Eu>(ub, sq_exp2(1));
+  r[9] = and_or<0x00700070u>(ub, sq_exp2(4));
+  r[10] = and_or<0x00070007u>(wc, sq_exp2(0));
+  r[11] = and_or<0x00380038u>(wc, sq_exp2(3));
+  r[12] = and_or<0x01C001C0u>(wc, sq_exp2(6));
+  r[13] = and_or<0x001C001Cu>(uc, sq_exp2(2));
+  r[14] = and_or<0x00E000E0u>(uc, sq_exp2(5));
+  uint32_t s = and_or<0x00400040u>(ua, sq_exp2(6));
+  s = and_or<0x00800080u>(ub, s);
+  r[15] = and_or<0x01000100u>(uc, s);
 }
 
 // Index n (0..63) of a lane's VQ stream of NW words; compile-time n folds the funnel shift.

@@ -250,6 +250,44 @@ def test_proxy_hand_worked_three_elements():
     assert abs(pc - pc_g) < 1e-13 and abs(pf2 - pf2_g) < 1e-13 and abs(pf4 - pf4_g) < 1e-13
 
 
+def test_proxy_family_hand_worked_and_closed_forms():
+    # Three weights 3, 0, 1: sorted 0, 1, 3, gaps 1, 2, G' = 1/3, 2/3, n = 2, mean 1/2.  By hand:
+    # variance = ((1/6)^2 + (1/6)^2) / 2 = 1/36, cv = (1/6) / (1/2) = 1/3, range = 1/3, mad = 1/6,
+    # ie = -(1/3 ln 1/3 + 2/3 ln 2/3) = ln 3 - (2/3) ln 2.
+    f = orc.proxy_family(np.array([[3.0, 0.0, 1.0]]))
+    assert abs(f["variance"] - 1.0 / 36.0) < 1e-15 and abs(f["cv"] - 1.0 / 3.0) < 1e-15
+    assert abs(f["range"] - 1.0 / 3.0) < 1e-15 and abs(f["mad"] - 1.0 / 6.0) < 1e-15
+    assert abs(f["ie"] - (np.log(3.0) - 2.0 / 3.0 * np.log(2.0))) < 1e-15
+    # equispaced weights: every gap equal, so every dispersion statistic is 0 and ie = ln n
+    w = np.random.default_rng(0).permutation(np.arange(4096) * 0.125 - 7.0).reshape(64, 64)
+    f = orc.proxy_family(w)
+    assert max(f["variance"], f["cv"], f["range"], f["mad"]) < 1e-12 and abs(f["ie"] - np.log(4095.0)) < 1e-9
+    # m + 1 levels each repeated r times: m gaps of 1/m, n - m ties, n = (m + 1) r - 1
+    m, r = 7, 5
+    w = np.repeat(np.arange(m + 1.0), r)
+    n = (m + 1) * r - 1
+    f = orc.proxy_family(w.reshape(1, -1))
+    var = (m * (1.0 / m - 1.0 / n) ** 2 + (n - m) * (1.0 / n) ** 2) / n
+    assert abs(f["variance"] - var) < 1e-15 and abs(f["cv"] - np.sqrt(var) * n) < 1e-12
+    assert abs(f["range"] - 1.0 / m) < 1e-15 and abs(f["ie"] - np.log(m)) < 1e-14
+    assert abs(f["mad"] - (m * (1.0 / m - 1.0 / n) + (n - m) / n) / n) < 1e-15
+    # ties to the coarse proxy and to the second moment of the fine proxy
+    w = (np.random.default_rng(3).standard_normal((32, 48)) * 0.02).astype(np.float16)
+    f = orc.proxy_family(w)
+    pc, pf2 = orc.proxy(w, K=2)
+    nn = w.size - 1
+    assert abs((np.log(nn) - f["ie"]) - pc) < 1e-12 and abs(f["variance"] * nn ** 2 / 2.0 - pf2) < 1e-9 * pf2
+    assert all(np.isinf(v) for v in orc.proxy_family(np.full((4, 4), 0.5)).values())
+
+
+def test_tau_for_fraction_sends_the_stated_share_to_sq():
+    vals = np.random.default_rng(5).permutation(np.arange(20) * 1.5 + 0.25)
+    for frac, k in ((0.9, 18), (0.5, 10), (0.0, 0), (1.0, 20), (0.33, 7)):
+        tau = orc.tau_for_fraction(vals, frac)
+        assert int((vals < tau).sum()) == k
+    assert orc.tau_for_fraction([1.0, 2.0, 4.0, 8.0], 0.5) == 3.0
+
+
 def test_proxy_equispaced_is_zero():
     w = (np.arange(4096, dtype=np.float64) * 0.125 - 7.0).reshape(64, 64)
     rng = np.random.default_rng(0)
