@@ -125,6 +125,25 @@ rwkvq_status rwkvq_proxy_select(const void* const* w_fp16_dev, const int* oc, co
                                 size_t workspace_bytes, void* stream);
 
 /*
+ * The statistics of the normalised gaps G' (Eq. 6) that the ablation of Section 5.3 tries in the
+ * proxy's place, from the same histogram pass: for each matrix stats_host[5*m + {0,1,2,3,4}] =
+ * variance, coefficient of variation, range, mean absolute deviation of G' and its information
+ * entropy -sum G' ln G' (P_c = ln n - entropy).  A constant matrix yields +inf for all five.
+ * Arguments and errors as rwkvq_proxy_select (same workspace size).
+ */
+rwkvq_status rwkvq_proxy_family(const void* const* w_fp16_dev, const int* oc, const int* ic, int n_mats,
+                                double* stats_host, void* workspace_dev, size_t workspace_bytes,
+                                void* stream);
+/*
+ * Threshold that sends the share sq_fraction of n matrices to scalar quantization under the rule
+ * "SQ iff value < tau" (Section 5.1 sets the thresholds so that nine tenths of the layers use SQ):
+ * with the values sorted and k = round(sq_fraction * n), tau is halfway between the k-th and the
+ * (k+1)-th smallest; k = 0 gives -inf, k = n gives +inf.  Host only.  Errors: EINVAL (NULL,
+ * n <= 0, fraction outside [0, 1], NaN among the values).
+ */
+rwkvq_status rwkvq_tau_for_fraction(const double* values_host, int n, double sq_fraction, double* tau_out);
+
+/*
  * Decode product y[b][i] = sum_j w_hat[i][j] * x_mix[b][j], 1 <= B <= 16 (Appendix A.1, the
  * W.(...) products), with the token-shift mix x_mix = x + (x_prev - x) (.) mu_hat fused into the
  * input stage when mu_image_dev != NULL (Eq. 20 with mu_paper = 1 - mu_hat).

@@ -61,6 +61,7 @@ EXPORTS = [
     "rwkvq_step_run_host",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
+    "rwkvq_proxy_family", "rwkvq_tau_for_fraction",
     "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
 ]
 
@@ -104,6 +105,9 @@ def lib() -> C.CDLL:
         L.rwkvq_proxy_workspace_bytes.restype = sz
         L.rwkvq_proxy_select.argtypes = [C.POINTER(vp), C.POINTER(i32), C.POINTER(i32), i32, i32, dbl, dbl,
                                          C.POINTER(dbl), C.POINTER(dbl), C.POINTER(i32), vp, sz, vp]
+    if hasattr(L, "rwkvq_proxy_family"):
+        L.rwkvq_proxy_family.argtypes = [C.POINTER(vp), C.POINTER(i32), C.POINTER(i32), i32, C.POINTER(dbl), vp, sz, vp]
+        L.rwkvq_tau_for_fraction.argtypes = [C.POINTER(dbl), i32, dbl, C.POINTER(dbl)]
     if hasattr(L, "rwkvq_step_plan"):
         L.rwkvq_step_plan_bytes.argtypes = [C.POINTER(GemvOp), i32, i32]
         L.rwkvq_step_plan_bytes.restype = sz
@@ -306,6 +310,28 @@ def rwkvq_proxy_select(mats, K: int, tau_c: float, tau_f: float, workspace, stre
                                     _dev_ptr(workspace), workspace.numel() * workspace.element_size(),
                                     _stream_ptr(stream)), "rwkvq_proxy_select")
     return pc, pf, phi
+
+
+def rwkvq_proxy_family(mats, workspace, stream=None):
+    """rwkvq_proxy_family on a list of torch float16 [oc, ic] device tensors.  Returns a dict of numpy
+    arrays: variance, cv, range, mad, ie."""
+    n = len(mats)
+    ptrs = (C.c_void_p * n)(*[m.data_ptr() for m in mats])
+    ocs = (C.c_int * n)(*[m.shape[0] for m in mats])
+    ics = (C.c_int * n)(*[m.shape[1] for m in mats])
+    stats = np.empty((n, 5), np.float64)
+    _check(lib().rwkvq_proxy_family(ptrs, ocs, ics, n, stats.ctypes.data_as(C.POINTER(C.c_double)),
+                                    _dev_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                    _stream_ptr(stream)), "rwkvq_proxy_family")
+    return {k: stats[:, i].copy() for i, k in enumerate(("variance", "cv", "range", "mad", "ie"))}
+
+
+def rwkvq_tau_for_fraction(values, sq_fraction: float) -> float:
+    v = np.ascontiguousarray(values, dtype=np.float64)
+    tau = C.c_double()
+    _check(lib().rwkvq_tau_for_fraction(v.ctypes.data_as(C.POINTER(C.c_double)), v.size, float(sq_fraction),
+                                        C.byref(tau)), "rwkvq_tau_for_fraction")
+    return float(tau.value)
 
 
 def make_ops(entries):

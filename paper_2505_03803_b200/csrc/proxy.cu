@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 #include <math.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "../../include/rwkvq.h"
@@ -31,6 +32,8 @@ struct ProxyResult {
   unsigned long long count;
   int distinct, nonfinite;
   int pad[2];
+  double variance, cv, range, mad, ie;   // the ablation's statistics of G' (Section 5.3)
+  double pad2;
 };
 
 // Order-preserving key of an fp16 bit pattern: key = 0x8000 - |bits| for negative values,
@@ -115,7 +118,10 @@ __global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* h
   const int mn = s_first[0], mx = s_first[1], D = s_dist[0];
   const unsigned long long N = s_cnt[0];
   if (D < 2 || N < 2) {
-    if (t == 0) { res->pc = INFINITY; res->pf = INFINITY; res->count = N; res->distinct = D; }
+    if (t == 0) {
+      res->pc = INFINITY; res->pf = INFINITY; res->count = N; res->distinct = D;
+      res->variance = res->cv = res->range = res->mad = res->ie = INFINITY;
+    }
     return;
   }
   const double R = value_of_key((unsigned)mx) - value_of_key((unsigned)mn);
@@ -123,6 +129,7 @@ __global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* h
   double acc[8];  // [0] = sum g' ln g', [k-1] = sum t^k for k = 2..8
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0;
+  double abs_t = 0.0, gmax = 0.0, gmin = INFINITY;   // sum |t_j|, largest and smallest positive gap
   int prev = s_last[t];
   for (int k = k0; k < k0 + 64; ++k) {
     if (hist[k] == 0u) continue;
@@ -132,6 +139,9 @@ __global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* h
       const double tt = n * gp - 1.0;
       double pw = tt;
       for (int kk = 2; kk <= K; ++kk) { pw *= tt; acc[kk - 1] += pw; }
+      abs_t += fabs(tt);
+      gmax = fmax(gmax, gp);
+      gmin = fmin(gmin, gp);
     }
     prev = k;
   }
@@ -146,8 +156,26 @@ __global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* h
     }
     tot[i] = s_red[0];
   }
+  // three more reductions of the same shape: sum |t|, max and min positive gap
+  double extra[3];
+  for (int i = 0; i < 3; ++i) {
+    __syncthreads();
+    s_red[t] = i == 0 ? abs_t : i == 1 ? gmax : gmin;
+    __syncthreads();
+    for (int s = 512; s > 0; s >>= 1) {
+      if (t < s) s_red[t] = i == 0 ? s_red[t] + s_red[t + s] : i == 1 ? fmax(s_red[t], s_red[t + s]) : fmin(s_red[t], s_red[t + s]);
+      __syncthreads();
+    }
+    extra[i] = s_red[0];
+  }
   if (t == 0) {
     const double ties = n - (double)(D - 1);
+    // with t = n G' - 1 (ties: t = -1):  variance = sum t^2 / n^3,  mad = sum |t| / n^2
+    res->variance = (tot[1] + ties) / (n * n * n);
+    res->cv = sqrt(res->variance) * n;
+    res->range = extra[1] - (ties > 0.0 ? 0.0 : extra[2]);
+    res->mad = (extra[0] + ties) / (n * n);
+    res->ie = -tot[0];
     double pf = 0.0;
     for (int kk = 2; kk <= K; ++kk) {
       const double sign = (kk & 1) ? -1.0 : 1.0;
@@ -173,10 +201,9 @@ size_t rwkvq_proxy_workspace_bytes(int n_mats) {
   return (size_t)n_mats * per_matrix_bytes() + round_up_sz((size_t)n_mats * sizeof(ProxyResult), 256);
 }
 
-rwkvq_status rwkvq_proxy_select(const void* const* w, const int* oc, const int* ic, int n_mats, int K,
-                                double tau_c, double tau_f, double* Pc, double* Pf, int* phi, void* ws,
-                                size_t ws_bytes, void* stream) {
-  if (!w || !oc || !ic || !Pc || !Pf || !phi || n_mats <= 0) return RWKVQ_EINVAL;
+static rwkvq_status run_proxy(const void* const* w, const int* oc, const int* ic, int n_mats, int K, void* ws,
+                              size_t ws_bytes, void* stream, std::vector<ProxyResult>* out) {
+  if (!w || !oc || !ic || n_mats <= 0) return RWKVQ_EINVAL;
   if (K < 2 || K > 8) return RWKVQ_EINVAL;
   if (!ws || ws_bytes < rwkvq_proxy_workspace_bytes(n_mats)) return RWKVQ_ENOMEM;
   if (!aligned16(ws)) return RWKVQ_EALIGN;
@@ -204,17 +231,52 @@ rwkvq_status rwkvq_proxy_select(const void* const* w, const int* oc, const int* 
   proxy_reduce_kernel<<<n_mats, 1024, 0, s>>>(hist, res, K);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_status(e);
-  std::vector<ProxyResult> host(n_mats);
-  e = cudaMemcpyAsync(host.data(), res, (size_t)n_mats * sizeof(ProxyResult), cudaMemcpyDeviceToHost, s);
+  out->resize(n_mats);
+  e = cudaMemcpyAsync(out->data(), res, (size_t)n_mats * sizeof(ProxyResult), cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return cuda_status(e);
-  bool bad = false;
+  for (int m = 0; m < n_mats; ++m)
+    if ((*out)[m].nonfinite) return RWKVQ_ENONFINITE;
+  return RWKVQ_OK;
+}
+
+rwkvq_status rwkvq_proxy_select(const void* const* w, const int* oc, const int* ic, int n_mats, int K,
+                                double tau_c, double tau_f, double* Pc, double* Pf, int* phi, void* ws,
+                                size_t ws_bytes, void* stream) {
+  if (!Pc || !Pf || !phi) return RWKVQ_EINVAL;
+  std::vector<ProxyResult> host;
+  const rwkvq_status st = run_proxy(w, oc, ic, n_mats, K, ws, ws_bytes, stream, &host);
+  if (st != RWKVQ_OK && st != RWKVQ_ENONFINITE) return st;
   for (int m = 0; m < n_mats; ++m) {
     Pc[m] = host[m].pc; Pf[m] = host[m].pf;
     phi[m] = (host[m].pc < tau_c && host[m].pf < tau_f) ? RWKVQ_SQ : RWKVQ_VQ;   // Eq. 18, strict <
-    if (host[m].nonfinite) bad = true;
   }
-  return bad ? RWKVQ_ENONFINITE : RWKVQ_OK;
+  return st;
+}
+
+rwkvq_status rwkvq_proxy_family(const void* const* w, const int* oc, const int* ic, int n_mats, double* stats,
+                                void* ws, size_t ws_bytes, void* stream) {
+  if (!stats) return RWKVQ_EINVAL;
+  std::vector<ProxyResult> host;
+  const rwkvq_status st = run_proxy(w, oc, ic, n_mats, 2, ws, ws_bytes, stream, &host);
+  if (st != RWKVQ_OK && st != RWKVQ_ENONFINITE) return st;
+  for (int m = 0; m < n_mats; ++m) {
+    double* o = stats + (size_t)m * 5;
+    o[0] = host[m].variance; o[1] = host[m].cv; o[2] = host[m].range; o[3] = host[m].mad; o[4] = host[m].ie;
+  }
+  return st;
+}
+
+rwkvq_status rwkvq_tau_for_fraction(const double* values, int n, double sq_fraction, double* tau_out) {
+  if (!values || !tau_out || n <= 0 || !(sq_fraction >= 0.0) || !(sq_fraction <= 1.0)) return RWKVQ_EINVAL;
+  std::vector<double> v(values, values + n);
+  for (double x : v) if (x != x) return RWKVQ_EINVAL;
+  std::sort(v.begin(), v.end());
+  const long k = lrint(sq_fraction * (double)n);
+  if (k <= 0) *tau_out = -INFINITY;
+  else if (k >= n) *tau_out = INFINITY;
+  else *tau_out = 0.5 * (v[k - 1] + v[k]);
+  return RWKVQ_OK;
 }
 
 }  // extern "C"

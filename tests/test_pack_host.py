@@ -253,3 +253,17 @@ def test_desc_for_matches_the_packer():
             assert getattr(d, f) == getattr(e, f), f
     with pytest.raises(B.RwkvqError):
         B.rwkvq_desc_for(100, 384, B.RWKVQ_SQ, 3)
+
+
+def test_tau_for_fraction_matches_oracle():
+    from oracle import rwkvq_oracle as orc
+    rng = np.random.default_rng(8)
+    for m in (1, 2, 7, 40):
+        vals = rng.standard_normal(m) * 3.0
+        for frac in (0.0, 0.1, 0.5, 0.9, 1.0):
+            a, b = B.rwkvq_tau_for_fraction(vals, frac), orc.tau_for_fraction(vals, frac)
+            assert a == b or (np.isinf(a) and np.isinf(b) and a * b > 0)
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_tau_for_fraction([1.0, float("nan")], 0.5)
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_tau_for_fraction([1.0], 1.5)

@@ -63,3 +63,37 @@ def test_proxy_degenerate_and_nonfinite():
     assert e.value.status == 4
     with pytest.raises(B.RwkvqError):
         _run([const], K=9)
+
+
+def test_proxy_family_matches_oracle():
+    # Section 5.3's other statistics of G', from the same histogram pass
+    mats = [inputs.gen_weight(0, 512, 512, "gauss"), inputs.gen_weight(1, 256, 768, "student"),
+            inputs.gen_weight(2, 128, 384, "uniform"), inputs.gen_weight(3, 3, 37, "gauss"),
+            (np.arange(4096).reshape(64, 64) % 17 - 8).astype(np.float16),
+            (np.arange(2048).reshape(32, 64) * 0.25 - 100.0).astype(np.float16),      # no ties: minimum gap > 0
+            np.full((16, 16), 0.25, np.float16)]
+    dev = [torch.from_numpy(np.ascontiguousarray(m)).cuda() for m in mats]
+    ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(dev)), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xCD)
+    got = B.rwkvq_proxy_family(dev, ws)
+    for i, m in enumerate(mats):
+        ref = orc.proxy_family(m.astype(np.float64))
+        for k, v in ref.items():
+            if math.isinf(v):
+                assert math.isinf(got[k][i]), (i, k)
+            else:
+                assert abs(got[k][i] - v) <= 1e-9 * abs(v) + 1e-13, (i, k, got[k][i], v)   # equal gaps: exact 0 vs rounding
+    # the entropy is the coarse proxy in other words
+    pc, _, _ = _run(mats[:6], K=2)
+    for i in range(6):
+        assert _close(math.log(mats[i].size - 1) - got["ie"][i], pc[i])
+
+
+def test_thresholds_for_a_target_sq_share():
+    # Section 5.1: thresholds set so that a stated share of the matrices uses SQ
+    mats = [inputs.gen_weight(20 + i, 128, 256, "student" if i % 5 == 0 else "gauss") for i in range(10)]
+    pc, _, _ = _run(mats, tau_c=math.inf, tau_f=math.inf)
+    tau = B.rwkvq_tau_for_fraction(pc, 0.8)
+    assert tau == orc.tau_for_fraction(pc, 0.8)
+    _, _, phi = _run(mats, tau_c=tau, tau_f=math.inf)
+    assert int(phi.sum()) == 8 and phi[0] == B.RWKVQ_VQ and phi[5] == B.RWKVQ_VQ
