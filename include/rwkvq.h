@@ -283,6 +283,19 @@ rwkvq_status rwkvq_quantize_dev(const void* w_fp16_dev, int oc, int ic, const rw
 rwkvq_status rwkvq_calib_representative(const float* samples_dev, int n_samples, int n, double pct,
                                         float* rep_dev, float* rep_sq_dev, void* stream);
 
+/*
+ * Quantization error of a packed matrix against the fp16 matrix it was made from:
+ * *sse_host = sum over all weights of (w - w_hat)^2, accumulated in fp64 with the decode routines
+ * of rwkvq_dequant (per-record sums combined in a fixed order, so the value is reproducible).
+ * Comparing it between an SQ and a VQ image of the same matrix is the "MSE" selector of the
+ * ablation in Section 5.3.  Matrices only.  workspace_dev: rwkvq_quant_error_workspace_bytes()
+ * bytes, 16-byte aligned.  Synchronizes `stream`.  Errors: EINVAL, ESHAPE, EALIGN, ENOMEM, ECUDA.
+ */
+size_t rwkvq_quant_error_workspace_bytes(const rwkvq_desc* W_desc);
+rwkvq_status rwkvq_quant_error(const void* w_fp16_dev, const rwkvq_desc* W_desc, const void* W_image_dev,
+                               double* sse_host, void* workspace_dev, size_t workspace_bytes,
+                               void* stream);
+
 /* Device status word of the last launches on this device: RWKVQ_OK, or ETIMEOUT if a bounded
  * wait inside a kernel gave up.  Synchronizes `stream`; clears the word. */
 rwkvq_status rwkvq_device_status(void* stream);

@@ -316,6 +316,13 @@ def proxy_family(w: np.ndarray) -> dict:
             "mad": float(np.abs(gp - mean).sum()) / n, "ie": -float((nz * np.log(nz)).sum())}
 
 
+def quant_sse(w: np.ndarray, w_hat: np.ndarray) -> float:
+    """Sum of squared quantization errors sum (w - w_hat)^2 in float64: the quantity the "MSE"
+    selector of Section 5.3 compares between the SQ and the VQ coding of a matrix."""
+    d = np.asarray(w, dtype=np.float64) - np.asarray(w_hat, dtype=np.float64)
+    return float((d * d).sum())
+
+
 def tau_for_fraction(values, sq_fraction: float) -> float:
     """Threshold that sends the given fraction of the matrices to scalar quantization under
     "SQ iff value < tau" (Section 5.1 sets the thresholds so that nine tenths of the layers use SQ):

@@ -61,7 +61,7 @@ EXPORTS = [
     "rwkvq_step_run_host",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
-    "rwkvq_proxy_family", "rwkvq_tau_for_fraction",
+    "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
     "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
 ]
 
@@ -108,6 +108,10 @@ def lib() -> C.CDLL:
     if hasattr(L, "rwkvq_proxy_family"):
         L.rwkvq_proxy_family.argtypes = [C.POINTER(vp), C.POINTER(i32), C.POINTER(i32), i32, C.POINTER(dbl), vp, sz, vp]
         L.rwkvq_tau_for_fraction.argtypes = [C.POINTER(dbl), i32, dbl, C.POINTER(dbl)]
+    if hasattr(L, "rwkvq_quant_error"):
+        L.rwkvq_quant_error_workspace_bytes.argtypes = [C.POINTER(Desc)]
+        L.rwkvq_quant_error_workspace_bytes.restype = sz
+        L.rwkvq_quant_error.argtypes = [vp, C.POINTER(Desc), vp, C.POINTER(dbl), vp, sz, vp]
     if hasattr(L, "rwkvq_step_plan"):
         L.rwkvq_step_plan_bytes.argtypes = [C.POINTER(GemvOp), i32, i32]
         L.rwkvq_step_plan_bytes.restype = sz
@@ -332,6 +336,16 @@ def rwkvq_tau_for_fraction(values, sq_fraction: float) -> float:
     _check(lib().rwkvq_tau_for_fraction(v.ctypes.data_as(C.POINTER(C.c_double)), v.size, float(sq_fraction),
                                         C.byref(tau)), "rwkvq_tau_for_fraction")
     return float(tau.value)
+
+
+def rwkvq_quant_error(w, desc: Desc, W_image, stream=None) -> float:
+    """rwkvq_quant_error: sum of squared differences between the fp16 CUDA tensor `w` and the decoded image."""
+    import torch
+    ws = torch.empty(int(lib().rwkvq_quant_error_workspace_bytes(C.byref(desc))), dtype=torch.uint8, device=w.device)
+    sse = C.c_double()
+    _check(lib().rwkvq_quant_error(_dev_ptr(w), C.byref(desc), _dev_ptr(W_image), C.byref(sse), _dev_ptr(ws),
+                                   ws.numel(), _stream_ptr(stream)), "rwkvq_quant_error")
+    return float(sse.value)
 
 
 def make_ops(entries):

@@ -116,9 +116,12 @@ __global__ void __launch_bounds__(256, 2) gemv_kernel(const GemvArgs a) {
 // ---------------------------------------------------------------------------------------------
 // Dequantisation probe: one warp per record, same unpack routines as the products.
 // ---------------------------------------------------------------------------------------------
+// With `ref` (the fp16 matrix the image was made from) nothing is stored: each warp instead adds up
+// (w - w_hat)^2 over its record in fp64 and writes the sum to sse_partial[record].
 template <int FMT>
 __global__ void dequant_kernel(const uint8_t* payload, const uint8_t* aux, int oc, int ic, int KT,
-                               int entries, void* out, int dtype, int n_records) {
+                               int entries, void* out, int dtype, int n_records, const __half* ref = nullptr,
+                               double* sse_partial = nullptr) {
   const int lane = threadIdx.x & 31;
   const int recid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (recid >= n_records) return;
@@ -126,6 +129,7 @@ __global__ void dequant_kernel(const uint8_t* payload, const uint8_t* aux, int o
   const int mb = chunk / KT, kt = chunk % KT;
   const int g = lane >> 2, t = lane & 3;
   const int r0 = mb * 128 + rt * 16, c0 = kt * 256;
+  double sse = 0.0;
   if constexpr (FMT == FMT_SQ3) {
     SqRecord rec;
     rec.load(payload + (size_t)recid * RWKVQ_SQ_RECORD_BYTES, lane);
@@ -150,8 +154,14 @@ __global__ void dequant_kernel(const uint8_t* payload, const uint8_t* aux, int o
         const float v0 = __fmul_rn(s, __fsub_rn(q0, z));
         const float v1 = __fmul_rn(s, __fsub_rn(q1, z));
         if (row < oc && col < ic) {
-          store_w(out, dtype, (size_t)row * ic + col, v0);
-          store_w(out, dtype, (size_t)row * ic + col + 1, v1);
+          if (ref) {
+            const float2 wv = __half22float2(*reinterpret_cast<const __half2*>(ref + (size_t)row * ic + col));
+            const double d0 = (double)wv.x - (double)v0, d1 = (double)wv.y - (double)v1;
+            sse += d0 * d0 + d1 * d1;
+          } else {
+            store_w(out, dtype, (size_t)row * ic + col, v0);
+            store_w(out, dtype, (size_t)row * ic + col + 1, v1);
+          }
         }
       }
     }
@@ -167,10 +177,35 @@ __global__ void dequant_kernel(const uint8_t* payload, const uint8_t* aux, int o
       const int col = c0 + 16 * j + 4 * t + 2 * (R >> 1);
       const uint32_t v = cb[vq_index<BITS, VqRecord<BITS>::NW>(rec.w, n)];
       const __half2 h = *reinterpret_cast<const __half2*>(&v);
-      store_w(out, dtype, (size_t)row * ic + col, __half2float(__low2half(h)));
-      store_w(out, dtype, (size_t)row * ic + col + 1, __half2float(__high2half(h)));
+      if (ref) {
+        const float2 wv = __half22float2(*reinterpret_cast<const __half2*>(ref + (size_t)row * ic + col));
+        const double d0 = (double)wv.x - (double)__half2float(__low2half(h)), d1 = (double)wv.y - (double)__half2float(__high2half(h));
+        sse += d0 * d0 + d1 * d1;
+      } else {
+        store_w(out, dtype, (size_t)row * ic + col, __half2float(__low2half(h)));
+        store_w(out, dtype, (size_t)row * ic + col + 1, __half2float(__high2half(h)));
+      }
     }
   }
+  if (ref) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) sse += __shfl_xor_sync(0xFFFFFFFFu, sse, off);
+    if (lane == 0) sse_partial[recid] = sse;
+  }
+}
+
+// Sum of n doubles in a fixed order (one block): the result does not depend on scheduling.
+__global__ void __launch_bounds__(1024) sum_fixed_kernel(const double* v, int n, double* out) {
+  __shared__ double s_red[1024];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n; i += 1024) acc += v[i];
+  s_red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int s = 512; s > 0; s >>= 1) {
+    if ((int)threadIdx.x < s) s_red[threadIdx.x] += s_red[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = s_red[0];
 }
 
 __global__ void dequant_vector_kernel(const uint8_t* payload, const uint8_t* aux, int ic, int bits,
@@ -337,6 +372,39 @@ rwkvq_status rwkvq_dequant(const rwkvq_desc* d, const void* W, void* out, int dt
   else if (fmt == FMT_VQ6) dequant_kernel<FMT_VQ6><<<grid, 128, 0, s>>>(payload, aux, d->oc, d->ic, KT, d->entries, out, dtype, nrec);
   else dequant_kernel<FMT_VQ8><<<grid, 128, 0, s>>>(payload, aux, d->oc, d->ic, KT, d->entries, out, dtype, nrec);
   return cuda_status(cudaGetLastError());
+}
+
+size_t rwkvq_quant_error_workspace_bytes(const rwkvq_desc* d) {
+  if (!d || d->oc == 1 || check_matrix_desc(d) != RWKVQ_OK) return 0;
+  return (size_t)(d->oc_pad / 128) * (d->ic_pad / 256) * 8 * sizeof(double) + 256;
+}
+
+rwkvq_status rwkvq_quant_error(const void* w, const rwkvq_desc* d, const void* W, double* sse_host, void* ws,
+                               size_t ws_bytes, void* stream) {
+  if (!w || !d || !W || !sse_host || !ws) return RWKVQ_EINVAL;
+  if (d->oc == 1) return RWKVQ_ESHAPE;
+  rwkvq_status st = check_matrix_desc(d);
+  if (st != RWKVQ_OK) return st;
+  if (!aligned16(w) || !aligned16(W) || !aligned16(ws)) return RWKVQ_EALIGN;
+  if (ws_bytes < rwkvq_quant_error_workspace_bytes(d)) return RWKVQ_ENOMEM;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const uint8_t* img = static_cast<const uint8_t*>(W);
+  const int KT = d->ic_pad / 256, nrec = (d->oc_pad / 128) * KT * 8;
+  const uint8_t* payload = img + RWKVQ_HEADER_BYTES;
+  const uint8_t* aux = img + matrix_aux_offset(d);
+  double* total = static_cast<double*>(ws);
+  double* partial = reinterpret_cast<double*>(static_cast<uint8_t*>(ws) + 256);
+  const __half* ref = static_cast<const __half*>(w);
+  const int fmt = fmt_of(d);
+  dim3 grid((nrec + 3) / 4);
+  if (fmt == FMT_SQ3) dequant_kernel<FMT_SQ3><<<grid, 128, 0, s>>>(payload, aux, d->oc, d->ic, KT, d->entries, nullptr, 0, nrec, ref, partial);
+  else if (fmt == FMT_VQ6) dequant_kernel<FMT_VQ6><<<grid, 128, 0, s>>>(payload, aux, d->oc, d->ic, KT, d->entries, nullptr, 0, nrec, ref, partial);
+  else dequant_kernel<FMT_VQ8><<<grid, 128, 0, s>>>(payload, aux, d->oc, d->ic, KT, d->entries, nullptr, 0, nrec, ref, partial);
+  sum_fixed_kernel<<<1, 1024, 0, s>>>(partial, nrec, total);
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaMemcpyAsync(sse_host, total, sizeof(double), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return cuda_status(e);
 }
 
 }  // extern "C"

@@ -280,6 +280,16 @@ def test_proxy_family_hand_worked_and_closed_forms():
     assert all(np.isinf(v) for v in orc.proxy_family(np.full((4, 4), 0.5)).values())
 
 
+def test_quant_sse_closed_forms():
+    assert orc.quant_sse(np.array([[0.0, 1.0], [2.0, 3.0]]), np.array([[0.0, 1.0], [2.0, 5.0]])) == 4.0
+    # uniform quantization of a dense ramp with step s: errors are k*s/m - round, sum known
+    w16 = (np.arange(128) % 8 * 0.125).astype(np.float16).reshape(1, 128)      # exactly representable levels
+    q, s_, z = orc.sq_encode(w16)
+    assert orc.quant_sse(w16, orc.sq_decode(q, s_, z)) == 0.0
+    # two values around one level: errors +-d each
+    assert abs(orc.quant_sse(np.array([0.25, 0.75]), np.array([0.5, 0.5])) - 0.125) < 1e-16
+
+
 def test_tau_for_fraction_sends_the_stated_share_to_sq():
     vals = np.random.default_rng(5).permutation(np.arange(20) * 1.5 + 0.25)
     for frac, k in ((0.9, 18), (0.5, 10), (0.0, 0), (1.0, 20), (0.33, 7)):

@@ -245,3 +245,36 @@ def test_quantize_dev_error_paths():
     with pytest.raises(B.RwkvqError) as e:
         B.rwkvq_calib_representative(torch.zeros((1, 8), device="cuda"), 1.0, torch.zeros(8, device="cuda"))
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("method,bits,oc,ic", [(B.RWKVQ_SQ, 3, 272, 384), (B.RWKVQ_SQ, 3, 512, 512), (B.RWKVQ_VQ, 6, 256, 512),
+                                               (B.RWKVQ_VQ, 8, 256, 256)])
+def test_quant_error_matches_oracle(method, bits, oc, ic):
+    rng = np.random.default_rng(oc + ic + bits)
+    w16 = (rng.standard_t(3, (oc, ic)) * 0.01).astype(np.float16)
+    d, img = quantize_dev(w16, method, bits, seed=2, iters=3)
+    _, codes = B.rwkvq_image_unpack(img.cpu().numpy())
+    if method == B.RWKVQ_SQ:
+        w_hat = orc.sq_decode(np.asarray(codes["q"]).reshape(oc, ic), np.asarray(codes["scale"]), np.asarray(codes["zero"]))
+    else:
+        w_hat = orc.vq_decode(np.asarray(codes["codebook"]).reshape(oc // 256, ic // 256, 1 << bits, 2),
+                              np.asarray(codes["q"]).reshape(oc, ic // 2))
+    wd = torch.from_numpy(w16).cuda()
+    sse = B.rwkvq_quant_error(wd, d, img)
+    ref = orc.quant_sse(w16, w_hat)
+    assert abs(sse - ref) <= 1e-12 * ref
+    assert sse == B.rwkvq_quant_error(wd, d, img)          # reproducible
+
+
+def test_mse_selector_picks_the_smaller_error():
+    # Section 5.3's "MSE" selector: code the matrix both ways, keep the coding with the smaller error
+    rng = np.random.default_rng(77)
+    for kind in ("gauss", "student"):
+        w16 = ((rng.standard_normal((256, 512)) * 0.02) if kind == "gauss" else rng.standard_t(3, (256, 512)) * 0.01).astype(np.float16)
+        wd = torch.from_numpy(w16).cuda()
+        dq, iq = quantize_dev(w16, B.RWKVQ_SQ, 3)
+        dv, iv = quantize_dev(w16, B.RWKVQ_VQ, 6, seed=1)
+        e_sq, e_vq = B.rwkvq_quant_error(wd, dq, iq), B.rwkvq_quant_error(wd, dv, iv)
+        q, s, z = orc.sq_encode(w16)
+        assert abs(e_sq - orc.quant_sse(w16, orc.sq_decode(q, s, z))) <= 1e-12 * e_sq
+        assert e_sq > 0.0 and e_vq > 0.0 and (e_sq < e_vq) == (orc.quant_sse(w16, orc.sq_decode(q, s, z)) < e_vq)
