@@ -55,7 +55,7 @@ def _check(ops, Bn):
     return worst
 
 
-@pytest.mark.parametrize("Bn,bits", [(1, 6), (8, 6), (16, 8), (3, 8)])
+@pytest.mark.parametrize("Bn,bits", [(1, 6), (8, 6), (16, 8), (3, 8), (2, 6), (4, 6), (7, 8), (9, 6), (12, 8)])
 def test_step_matches_oracle_small_stack(Bn, bits):
     ops = _build_ops(512, 1280, 2, Bn, bits, seed=10 * Bn + bits)   # h = 5 column tiles: odd tile count
     plan = _plan(ops, Bn)
@@ -74,6 +74,19 @@ def test_step_matches_oracle_1p6b_layer(method):
     torch.cuda.synchronize()
     assert B.rwkvq_device_status() == 0
     _check(ops, 1)
+
+
+@pytest.mark.parametrize("Bn", [1, 5, 16])
+def test_step_ragged_sq_shapes(Bn):
+    # d = 384, h = 896: row counts that end in a half unit (one 128-row chunk) and input lengths
+    # whose last 256-column tile is half empty
+    ops = _build_ops(384, 896, 2, Bn, 6, seed=300 + Bn, all_method=B.RWKVQ_SQ)
+    plan = _plan(ops, Bn)
+    for rep in range(2):
+        B.rwkvq_step_run(plan)
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        _check(ops, Bn)
 
 
 def test_step_agrees_with_single_product_calls():
