@@ -273,6 +273,20 @@ rwkvq_status rwkvq_quantize_dev(const void* w_fp16_dev, int oc, int ic, const rw
                                 void* stream);
 
 /*
+ * rwkvq_quantize_dev in two halves, for quantizing many matrices without a host round trip per
+ * matrix.  rwkvq_quantize_dev_async only enqueues the kernels (same arguments and argument errors);
+ * a NaN/Inf weight sets a flag in the first word of workspace_dev, which must be zero before the
+ * first call and is shared by every call that uses the same workspace.  rwkvq_quantize_check
+ * synchronizes `stream`, returns RWKVQ_ENONFINITE if the flag was set by any call since the last
+ * check (RWKVQ_OK otherwise) and clears it.
+ */
+rwkvq_status rwkvq_quantize_dev_async(const void* w_fp16_dev, int oc, int ic, const rwkvq_quant_cfg* cfg,
+                                      const float* elem_weight_dev, void* image_dev, size_t image_bytes,
+                                      rwkvq_desc* desc_out, void* workspace_dev, size_t workspace_bytes,
+                                      void* stream);
+rwkvq_status rwkvq_quantize_check(void* workspace_dev, void* stream);
+
+/*
  * Representative X of a batch of calibration activations (Section 4.2): for each of the n
  * positions, the n_samples values samples_dev[s][j] (fp32, row-major [n_samples][n],
  * 2 <= n_samples <= 1024) are limited to the range between their pct-th and (100 - pct)-th

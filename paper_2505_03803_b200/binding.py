@@ -63,6 +63,7 @@ EXPORTS = [
     "rwkvq_status_str", "rwkvq_last_cuda_error",
     "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
     "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
+    "rwkvq_quantize_dev_async", "rwkvq_quantize_check",
 ]
 
 _lib = None
@@ -128,6 +129,8 @@ def lib() -> C.CDLL:
         L.rwkvq_quantize_workspace_bytes.restype = sz
         L.rwkvq_quantize_dev.argtypes = [vp, i32, i32, C.POINTER(QuantCfg), vp, vp, sz, C.POINTER(Desc), vp, sz, vp]
         L.rwkvq_calib_representative.argtypes = [vp, i32, i32, dbl, vp, vp, vp]
+        L.rwkvq_quantize_dev_async.argtypes = L.rwkvq_quantize_dev.argtypes
+        L.rwkvq_quantize_check.argtypes = [vp, vp]
     _lib = L
     return L
 
@@ -433,6 +436,25 @@ def rwkvq_quantize_dev(w, oc: int, ic: int, method: int, bits: int, image, works
                                     workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
            "rwkvq_quantize_dev")
     return d
+
+
+def rwkvq_quantize_dev_async(w, oc: int, ic: int, method: int, bits: int, image, workspace, *, elem_weight=None,
+                             group: int = 128, vec_dim: int = 2, tile: int = 256, kmeans_iters: int = 10,
+                             seed: int = 0, stream=None) -> Desc:
+    """rwkvq_quantize_dev_async: enqueue only; `workspace` must have been zero-filled once."""
+    cfg = QuantCfg(method=method, bits=bits, group=group, vec_dim=vec_dim, tile=tile, kmeans_iters=kmeans_iters,
+                   seed=seed, codes_in=None)
+    d = Desc()
+    _check(lib().rwkvq_quantize_dev_async(_dev_ptr(w), oc, ic, C.byref(cfg), _dev_ptr(elem_weight), _dev_ptr(image),
+                                          image.numel() * image.element_size(), C.byref(d), _dev_ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+           "rwkvq_quantize_dev_async")
+    return d
+
+
+def rwkvq_quantize_check(workspace, stream=None) -> int:
+    """rwkvq_quantize_check: status code (0 = OK, 4 = a NaN/Inf weight was seen); synchronizes."""
+    return int(lib().rwkvq_quantize_check(_dev_ptr(workspace), _stream_ptr(stream)))
 
 
 def rwkvq_calib_representative(samples, pct: float, rep=None, rep_sq=None, stream=None):

@@ -554,9 +554,9 @@ extern "C" {
 
 size_t rwkvq_quantize_workspace_bytes(void) { return 256; }
 
-rwkvq_status rwkvq_quantize_dev(const void* w_dev, int oc, int ic, const rwkvq_quant_cfg* cfg, const float* elem_weight_dev,
-                                void* image_dev, size_t image_bytes, rwkvq_desc* desc_out, void* workspace_dev,
-                                size_t workspace_bytes, void* stream) {
+static rwkvq_status quantize_enqueue(const void* w_dev, int oc, int ic, const rwkvq_quant_cfg* cfg, const float* elem_weight_dev,
+                                     void* image_dev, size_t image_bytes, rwkvq_desc* desc_out, void* workspace_dev,
+                                     size_t workspace_bytes, void* stream, bool clear_flag) {
   using namespace rwkvq;
   if (!w_dev || !cfg || !image_dev || !workspace_dev || cfg->codes_in) return RWKVQ_EINVAL;
   rwkvq_desc d;
@@ -577,8 +577,11 @@ rwkvq_status rwkvq_quantize_dev(const void* w_dev, int oc, int ic, const rwkvq_q
   rwkvq_fill_header(&h, d.method, d.bits, d.oc, d.ic, d.oc_pad, d.ic_pad, d.group, d.vec_dim, d.tile, d.entries, is_vector,
                     d.image_bytes, d.stream_bytes);
   h.reserved1 = RWKVQ_IMAGE_FLAG_NO_CRC;
-  cudaError_t e = cudaMemsetAsync(flags, 0, sizeof(int), s);
-  if (e != cudaSuccess) return cuda_status(e);
+  cudaError_t e = cudaSuccess;
+  if (clear_flag) {
+    e = cudaMemsetAsync(flags, 0, sizeof(int), s);
+    if (e != cudaSuccess) return cuda_status(e);
+  }
   write_header_kernel<<<1, 64, 0, s>>>(h, img);
   if (d.method == RWKVQ_SQ) {
     const int MB = d.oc_pad / 128, KT = d.ic_pad / 256;
@@ -609,13 +612,36 @@ rwkvq_status rwkvq_quantize_dev(const void* w_dev, int oc, int ic, const rwkvq_q
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_status(e);
-  int host_flags = 0;
-  e = cudaMemcpyAsync(&host_flags, flags, sizeof(int), cudaMemcpyDeviceToHost, s);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-  if (e != cudaSuccess) return cuda_status(e);
-  if (host_flags & kFlagNonFinite) return RWKVQ_ENONFINITE;
   if (desc_out) *desc_out = d;
   return RWKVQ_OK;
+}
+
+rwkvq_status rwkvq_quantize_check(void* workspace_dev, void* stream) {
+  using namespace rwkvq;
+  if (!workspace_dev) return RWKVQ_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int host_flags = 0;
+  cudaError_t e = cudaMemcpyAsync(&host_flags, workspace_dev, sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(workspace_dev, 0, sizeof(int), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_status(e);
+  return (host_flags & kFlagNonFinite) ? RWKVQ_ENONFINITE : RWKVQ_OK;
+}
+
+rwkvq_status rwkvq_quantize_dev_async(const void* w_dev, int oc, int ic, const rwkvq_quant_cfg* cfg, const float* elem_weight_dev,
+                                      void* image_dev, size_t image_bytes, rwkvq_desc* desc_out, void* workspace_dev,
+                                      size_t workspace_bytes, void* stream) {
+  return quantize_enqueue(w_dev, oc, ic, cfg, elem_weight_dev, image_dev, image_bytes, desc_out, workspace_dev,
+                          workspace_bytes, stream, false);
+}
+
+rwkvq_status rwkvq_quantize_dev(const void* w_dev, int oc, int ic, const rwkvq_quant_cfg* cfg, const float* elem_weight_dev,
+                                void* image_dev, size_t image_bytes, rwkvq_desc* desc_out, void* workspace_dev,
+                                size_t workspace_bytes, void* stream) {
+  rwkvq_status st = quantize_enqueue(w_dev, oc, ic, cfg, elem_weight_dev, image_dev, image_bytes, desc_out, workspace_dev,
+                                     workspace_bytes, stream, true);
+  if (st != RWKVQ_OK) return st;
+  return rwkvq_quantize_check(workspace_dev, stream);
 }
 
 rwkvq_status rwkvq_calib_representative(const float* samples_dev, int n_samples, int n, double pct, float* rep_dev,

@@ -278,3 +278,25 @@ def test_mse_selector_picks_the_smaller_error():
         q, s, z = orc.sq_encode(w16)
         assert abs(e_sq - orc.quant_sse(w16, orc.sq_decode(q, s, z))) <= 1e-12 * e_sq
         assert e_sq > 0.0 and e_vq > 0.0 and (e_sq < e_vq) == (orc.quant_sse(w16, orc.sq_decode(q, s, z)) < e_vq)
+
+
+def test_async_quantizer_and_check():
+    rng = np.random.default_rng(9)
+    ws = torch.zeros(B.rwkvq_quantize_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    mats = [(rng.standard_normal((256, 384)) * 0.02).astype(np.float16) for _ in range(3)]
+    imgs = []
+    for w16 in mats:
+        d0 = B.rwkvq_desc_for(256, 384, B.RWKVQ_SQ, 3)
+        img = torch.empty(int(d0.image_bytes), dtype=torch.uint8, device="cuda")
+        B.rwkvq_quantize_dev_async(torch.from_numpy(w16).cuda(), 256, 384, B.RWKVQ_SQ, 3, img, ws)
+        imgs.append(img)
+    assert B.rwkvq_quantize_check(ws) == 0
+    for w16, img in zip(mats, imgs):
+        ref = B.rwkvq_pack(w16, 256, 384, B.RWKVQ_SQ, 3).image()
+        assert np.array_equal(img.cpu().numpy()[256:], ref[256:])
+    bad = mats[1].copy()
+    bad[7, 300] = np.float16(np.inf)
+    for w16 in (mats[0], bad, mats[2]):           # the flag of the middle call survives the later one
+        B.rwkvq_quantize_dev_async(torch.from_numpy(w16).cuda(), 256, 384, B.RWKVQ_SQ, 3, imgs[0], ws)
+    assert B.rwkvq_quantize_check(ws) == 4
+    assert B.rwkvq_quantize_check(ws) == 0        # cleared by the check
