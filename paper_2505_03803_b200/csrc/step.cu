@@ -213,8 +213,7 @@ __device__ __forceinline__ uint32_t smem_ld_acquire(const uint32_t* p) {
 __device__ __forceinline__ bool wait_count(const uint32_t* p, uint32_t target, volatile int* abort_flag, int* status) {
   for (uint32_t it = 0; it < (kPollLimit << 4); ++it) {
     if (smem_ld_acquire(p) >= target) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;
-    __nanosleep(32);
+    if ((it & 255u) == 255u && *abort_flag) return false;     // no back-off: this wait ends a stage
   }
   *abort_flag = 1;
   atomicExch(status, (int)RWKVQ_ETIMEOUT);
