@@ -642,11 +642,13 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
   int held = -1;              // input segment this warp currently holds
   uint32_t seg_next = 0;      // number of segment events passed so far
   uint32_t cur_ev = 0;        // last event processed (event 0 is the clearing arrival: nothing to do)
-  // Report the current stage as finished.  Every lane first makes its own reductions into y
-  // visible GPU-wide (all lanes and warps wait in parallel), so that the stager's single arrival
-  // at the grid barrier has nothing left to wait for.
+  // Report the current stage as finished.  The lanes' reductions into y are ordered before lane
+  // 0's CTA-scope release of the completion count (warp barrier, then release); the stager thread
+  // that acquires the count posts the CTA's arrival with a GPU-scope release, which by the
+  // cumulativity of release / acquire chains covers every warp's reductions -- the same pattern as a
+  // grid barrier made of a block barrier followed by one thread's fence and arrival.  A GPU-scope
+  // fence in each consumer lane would only add its latency to the end of every stage.
   auto arrive_stage = [&]() {
-    __threadfence();
     __syncwarp();
     if (lane == 0 && !dead) smem_add_release(&ctrl->cdone, 1u);
   };
