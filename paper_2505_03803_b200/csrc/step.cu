@@ -201,34 +201,55 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
 __device__ __forceinline__ void red_release_gpu(unsigned* p, unsigned v) {
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void smem_add_release(uint32_t* p, uint32_t v) {
-  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t smem_ld_acquire(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
-  return v;
-}
-// Bounded wait until a shared-memory counter reaches `target`.
-__device__ __forceinline__ bool wait_count(const uint32_t* p, uint32_t target, volatile int* abort_flag, int* status) {
-  for (uint32_t it = 0; it < (kPollLimit << 4); ++it) {
-    if (smem_ld_acquire(p) >= target) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;     // no back-off: this wait ends a stage
-  }
-  *abort_flag = 1;
-  atomicExch(status, (int)RWKVQ_ETIMEOUT);
-  return false;
+__device__ __forceinline__ uint32_t smem_add_acq_rel(uint32_t* p, uint32_t v) {
+  uint32_t old;
+  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
+  return old;
 }
 
 struct Ctrl {
   uint64_t full[kMaxSlots], empty[kMaxSlots];
   uint64_t xfull[4], xempty[4];
-  uint32_t cdone;            // stage completions reported by consumer warps: 16 per finished stage.  A
-                             // plain counter, not an mbarrier: consumers of a CTA without work in the
-                             // coming stages may run any number of stages ahead of the stagers.
+  uint32_t stage_cnt[64];    // one 8-bit count per grid barrier (four per word): how many of the seventeen
+                             // parties of this CTA (sixteen consumer warps, the stagers) have reported the
+                             // stage that the barrier closes.  Per barrier, not one running total: consumer
+                             // warps of a CTA without work in the coming stages may run any number of
+                             // stages ahead of the stagers.
+  uint32_t cdone;            // running total of stage reports of the consumer warps (two-batch-block launches)
   int abort_flag;
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
+constexpr uint32_t kMaxBarriers = 256;   // barriers that close a stage (8-bit counts in Ctrl::stage_cnt)
+
+// One of the seventeen parties of grid barrier `b` reports that its part of the stage the barrier
+// closes is done; whoever reports last posts the CTA's arrival.  The count is an acquire-release
+// read-modify-write at CTA scope and the arrival a GPU-scope release, so the arrival is ordered
+// after everything every party did before reporting (the consumers' reductions into y, the
+// stagers' clearing of the next outputs): block-level synchronisation followed by one thread's
+// release, the pattern of a cooperative grid barrier.
+__device__ __forceinline__ void stage_report(Ctrl* ctrl, const StepArgs& a, uint32_t b) {
+  const uint32_t sh = 8u * (b & 3u);
+  const uint32_t old = smem_add_acq_rel(&ctrl->stage_cnt[b >> 2], 1u << sh);
+  if (((old >> sh) & 0xFFu) == (uint32_t)kConsumerWarps) red_release_gpu(a.counter + b, 1u);
+}
+// Where the consumer warps are the busy role (two batch blocks per record) they only add to one
+// running total, and a stager thread, which has nothing else to do at that point, waits (bounded)
+// for the sixteen reports of the stage and arrives: the release, which waits for the CTA's
+// outstanding reductions, and the bookkeeping of a barrier number stay off the consumer warps.
+__device__ __forceinline__ void stage_report_total(Ctrl* ctrl) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(&ctrl->cdone)), "r"(1u) : "memory");
+}
+__device__ __forceinline__ bool stage_wait_total_and_arrive(Ctrl* ctrl, const StepArgs& a, uint32_t b, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < (kPollLimit << 4); ++it) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&ctrl->cdone)) : "memory");
+    if (v >= (uint32_t)kConsumerWarps * b) { red_release_gpu(a.counter + b, 1u); return true; }
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicExch(a.status, (int)RWKVQ_ETIMEOUT);
+  return false;
+}
 
 // ---- roles -------------------------------------------------------------------------------------
 
@@ -371,9 +392,10 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
 }
 
 // Stagers walk the CTA's event list.
-//  EV_ARRIVE: clear this CTA's slice of the next stage's outputs, then (deferred until the next
-//    segment's barrier-independent preparation is done) wait for the consumer warps to finish
-//    the stage, publish with one cumulative fence and add this CTA's arrival to the grid barrier.
+//  EV_ARRIVE: clear this CTA's slice of the next stage's outputs, then report the stage as done on
+//    the stagers' side (stage_report: the last of the consumer warps and the stagers to report
+//    adds this CTA's arrival to the grid barrier, so the arrival never waits for a role that is
+//    busy with something else).
 //  EV_SEGMENT: x_mix and, for SQ, the per-group sums of the segment, into buffer (segment number
 //    & 1).  The decoded token-shift vector mu_hat and the previous token's activations go to
 //    shared memory BEFORE the stage barrier, so that only one round of vector loads of x, the
@@ -386,26 +408,11 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
   const int lane = stid & 31;
   volatile int* abortp = &ctrl->abort_flag;
   uint32_t nseg = 0;          // segments staged so far
-  uint32_t narrive = 0;       // arrivals posted so far
-  int pending = -1;           // barrier index of an arrival not yet posted
   uint32_t passed2 = 0xFFFFFFFFu;   // second-stage barrier this CTA has already passed
   bool ok = true;
-  // posts the pending arrival (thread 0 acts; the others only keep count)
-  auto post_arrival = [&]() {
-    if (pending < 0) return;
-    if (stid == 0 && ok) {
-      // barrier 0 (the clearing pass) has no consumer work before it; barrier j closes stage j - 1,
-      // which all sixteen consumer warps must have reported, like every stage before it
-      if (pending > 0) ok = wait_count(&ctrl->cdone, (uint32_t)kConsumerWarps * narrive, abortp, a.status);
-      if (ok) red_release_gpu(a.counter + pending, 1u);
-    }
-    ++narrive;
-    pending = -1;
-  };
   for (uint32_t ei = e0; ei < e1; ++ei) {
     const StepEvent ev = *reinterpret_cast<const StepEvent*>(reinterpret_cast<const uint8_t*>(a.events) + (size_t)ei * 64);
     if (ev.kind == EV_ARRIVE) {
-      post_arrival();                         // an earlier arrival with no segment in between
 #pragma unroll
       for (int k = 0; k < 3; ++k) {
         float* z = reinterpret_cast<float*>(ev.arr.zptr[k]);
@@ -413,12 +420,17 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       }
       // the clearing stores of every stager thread must precede thread 0's fence
       ok = named_bar_and(4, kStagerThreads, ok);
-      pending = (int)ev.barrier;
       if (!ok) break;
+      // The stagers' part of the stage is done.  Barrier 0 (the clearing pass) has no consumer work
+      // before it: arrive directly.  Otherwise report; the last of the seventeen parties arrives.
+      if (stid == 0) {
+        if (ev.barrier == 0u) red_release_gpu(a.counter, 1u);
+        else if constexpr (NB == 2) ok = stage_wait_total_and_arrive(ctrl, a, ev.barrier, abortp);
+        else stage_report(ctrl, a, ev.barrier);
+      }
       if constexpr (MIX) {
-        // no preparation to overlap: arrive now, then, once the barrier opens, do this CTA's share
-        // of the new stage's pre-pass and publish it through the stage's second barrier
-        post_arrival();
+        // once the barrier opens, do this CTA's share of the new stage's pre-pass and publish it
+        // through the stage's second barrier
         if (ev.barrier < (uint32_t)a.n_stages) {
           if (ok && stid == 0) {
             uint32_t it = 0;
@@ -511,7 +523,6 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
         *reinterpret_cast<uint4*>(xb + (size_t)b * xstride + (size_t)c8 * 16) = r;
       }
     }
-    post_arrival();
     if (ok && ev.barrier && stid == 0) {
       // grid-wide stage barrier: every CTA has finished (and published) the previous stage.  Each
       // barrier has its own arrival counter, so a CTA without work may run ahead and arrive at
@@ -579,7 +590,6 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
     ++nseg;
     if (!ok) break;
   }
-  if (ok) post_arrival();
 }
 
 // Six words of one 128-column group of the record of lane `lane` (planes of 512 bytes, 16 bytes
@@ -642,15 +652,18 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
   int held = -1;              // input segment this warp currently holds
   uint32_t seg_next = 0;      // number of segment events passed so far
   uint32_t cur_ev = 0;        // last event processed (event 0 is the clearing arrival: nothing to do)
-  // Report the current stage as finished.  The lanes' reductions into y are ordered before lane
-  // 0's CTA-scope release of the completion count (warp barrier, then release); the stager thread
-  // that acquires the count posts the CTA's arrival with a GPU-scope release, which by the
-  // cumulativity of release / acquire chains covers every warp's reductions -- the same pattern as a
-  // grid barrier made of a block barrier followed by one thread's fence and arrival.  A GPU-scope
-  // fence in each consumer lane would only add its latency to the end of every stage.
+  // Report the current stage as finished (stage_report).  The lanes' reductions into y are ordered
+  // before lane 0's report by the warp barrier; no lane fences at GPU scope itself: that would only
+  // add its latency to the end of every stage.
+  uint32_t next_bar = 1u;     // every CTA arrives at barriers 1, 2, ... in this order, once per stage
   auto arrive_stage = [&]() {
     __syncwarp();
-    if (lane == 0 && !dead) smem_add_release(&ctrl->cdone, 1u);
+    if constexpr (NB == 2) {
+      if (lane == 0 && !dead) stage_report_total(ctrl);
+    } else {
+      if (lane == 0 && !dead) stage_report(ctrl, a, next_bar);
+      ++next_bar;
+    }
   };
   auto release_held = [&]() {
     __syncwarp();
@@ -818,6 +831,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.n_slots; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], kGroupWarps); }
     for (int b = 0; b < 4; ++b) { mbar_init(&ctrl->xfull[b], kStagerWarps); mbar_init(&ctrl->xempty[b], kConsumerWarps); }
+    for (int k = 0; k < 64; ++k) ctrl->stage_cnt[k] = 0u;
     ctrl->cdone = 0u;
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -924,6 +938,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     i = j;
   }
   const int n_stages = (int)stage_ranges.size();
+  if ((uint32_t)n_stages + 1u > kMaxBarriers) return RWKVQ_EUNSUPPORTED;   // per-barrier counts in the control block
   info->n_stages = n_stages;
   info->n_barriers = ((uint32_t)n_stages + 1) * (mix ? 2u : 1u);   // the pre-pass has a barrier of its own per stage
 
