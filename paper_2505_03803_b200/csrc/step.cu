@@ -1020,6 +1020,37 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       const uint64_t wgt = !(h.u.flags & UF_VQ) ? 20u : (h.u.flags & UF_BITS8) ? 25u : 29u;
       return recs * wgt * 64u;
     };
+    // Small stages (at most two units per CTA) are bound by latency, not by bytes: a CTA's time is
+    // one unit per consumer group plus about 1.7 us for every further input segment it has to
+    // stage, however few of a unit's records it holds.  Such a stage is dealt in WHOLE units, two
+    // neighbouring column tiles of one row of tiles per CTA (one unit per group, one segment), and
+    // the CTAs left over idle through it; measured on the 1.6B-class stack, the cost-balanced cut
+    // gave a fifth of the CTAs a second segment or a third piece and the stage waited for them.
+    bool dealt = false;
+    if (units.size() <= (size_t)2 * (size_t)P) {
+      std::vector<std::pair<size_t, size_t>> pairs;      // [first, last) unit of a CTA
+      for (size_t i = 0; i < units.size();) {
+        size_t j = i + 1;
+        if (j < units.size() && units[j].op == units[i].op && units[j].tr == units[i].tr) ++j;
+        pairs.emplace_back(i, j);
+        i = j;
+      }
+      if (pairs.size() <= (size_t)P) {
+        // start at a CTA that moves with the stage, so that the idle CTAs are not always the same SMs
+        const size_t first = ((size_t)s * 37u) % (size_t)P;
+        for (size_t k = 0; k < pairs.size(); ++k) {
+          const int c = (int)((first + k) % (size_t)P);
+          for (size_t i = pairs[k].first; i < pairs[k].second; ++i) {
+            HostUnit part = units[i];
+            part.w0 = 0; part.w1 = 8;
+            part.u.off0 = 0;
+            part.u.flags |= (0u << 8) | (8u << 12);
+            cta_units[c].push_back(part);
+          }
+        }
+        dealt = true;
+      }
+    }
     uint64_t total = 0;
     for (const HostUnit& h : units) total += cost_of(h);
     uint64_t run = 0;
@@ -1028,6 +1059,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       return c >= P ? P - 1 : c;
     };
     for (const HostUnit& h : units) {
+      if (dealt) break;
       const uint64_t e8 = cost_of(h) / 8;
       int w = 0;
       while (w < 8) {
