@@ -1020,35 +1020,59 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       const uint64_t wgt = !(h.u.flags & UF_VQ) ? 20u : (h.u.flags & UF_BITS8) ? 25u : 29u;
       return recs * wgt * 64u;
     };
-    // Small stages (at most two units per CTA) are bound by latency, not by bytes: a CTA's time is
-    // one unit per consumer group plus about 1.7 us for every further input segment it has to
-    // stage, however few of a unit's records it holds.  Such a stage is dealt in WHOLE units, two
-    // neighbouring column tiles of one row of tiles per CTA (one unit per group, one segment), and
-    // the CTAs left over idle through it; measured on the 1.6B-class stack, the cost-balanced cut
-    // gave a fifth of the CTAs a second segment or a third piece and the stage waited for them.
+    // A consumer group spends about the same time on a piece of a unit as on a whole unit (the
+    // warps without a record idle), and every further input segment of a CTA costs about 1.7 us of
+    // serial staging; traces of all CTAs' barrier arrivals showed the stages waiting for the CTAs
+    // with the most pieces and segments, not for the most bytes.  So units are dealt WHOLE, and
+    // where it balances, row by row: each row of tiles (one product, one 256-row block: one input
+    // segment) gets a number of CTAs, greedily the row with the largest cost per CTA first, and
+    // its units are split into that many runs of neighbouring column tiles.  This is taken when no
+    // CTA ends up more than one unit above the even share; small stages leave some CTAs idle.
     bool dealt = false;
-    if (units.size() <= (size_t)2 * (size_t)P) {
-      std::vector<std::pair<size_t, size_t>> pairs;      // [first, last) unit of a CTA
+    auto push_whole = [&](int c, const HostUnit& h) {
+      HostUnit part = h;
+      part.w0 = 0; part.w1 = 8;
+      part.u.off0 = 0;
+      part.u.flags |= (0u << 8) | (8u << 12);
+      cta_units[c].push_back(part);
+    };
+    {
+      struct Row { size_t first, count; uint64_t cost; int k; };
+      std::vector<Row> rows;
       for (size_t i = 0; i < units.size();) {
-        size_t j = i + 1;
-        if (j < units.size() && units[j].op == units[i].op && units[j].tr == units[i].tr) ++j;
-        pairs.emplace_back(i, j);
+        size_t j = i;
+        uint64_t cst = 0;
+        while (j < units.size() && units[j].op == units[i].op && units[j].tr == units[i].tr) { cst += cost_of(units[j]); ++j; }
+        rows.push_back(Row{i, j - i, cst, 1});
         i = j;
       }
-      if (pairs.size() <= (size_t)P) {
-        // start at a CTA that moves with the stage, so that the idle CTAs are not always the same SMs
-        const size_t first = ((size_t)s * 37u) % (size_t)P;
-        for (size_t k = 0; k < pairs.size(); ++k) {
-          const int c = (int)((first + k) % (size_t)P);
-          for (size_t i = pairs[k].first; i < pairs[k].second; ++i) {
-            HostUnit part = units[i];
-            part.w0 = 0; part.w1 = 8;
-            part.u.off0 = 0;
-            part.u.flags |= (0u << 8) | (8u << 12);
-            cta_units[c].push_back(part);
+      if (!rows.empty() && rows.size() <= (size_t)P) {
+        int spare = P - (int)rows.size();
+        while (spare > 0) {
+          size_t best = rows.size();
+          uint64_t best_cost = 0;
+          for (size_t r = 0; r < rows.size(); ++r) {
+            if ((size_t)rows[r].k >= rows[r].count) continue;          // one unit per CTA at most
+            const uint64_t per = rows[r].cost / (uint64_t)rows[r].k;
+            if (per > best_cost) { best_cost = per; best = r; }
           }
+          if (best == rows.size()) break;
+          ++rows[best].k; --spare;
         }
-        dealt = true;
+        size_t max_units = 0;
+        for (const Row& r : rows) max_units = std::max(max_units, (r.count + (size_t)r.k - 1) / (size_t)r.k);
+        const size_t even = (units.size() + (size_t)P - 1) / (size_t)P;
+        if (max_units <= even + 1) {
+          // start at a CTA that moves with the stage, so that idle CTAs are not always the same SMs
+          size_t c = ((size_t)s * 37u) % (size_t)P;
+          for (const Row& r : rows)
+            for (int q = 0; q < r.k; ++q) {
+              const size_t lo = r.count * (size_t)q / (size_t)r.k, hi = r.count * (size_t)(q + 1) / (size_t)r.k;
+              for (size_t i = lo; i < hi; ++i) push_whole((int)c, units[r.first + i]);
+              c = (c + 1) % (size_t)P;
+            }
+          dealt = true;
+        }
       }
     }
     uint64_t total = 0;
@@ -1058,8 +1082,14 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       int c = (int)((mid * (uint64_t)P) / (total ? total : 1));
       return c >= P ? P - 1 : c;
     };
+    const bool whole_units = units.size() >= (size_t)4 * (size_t)P;   // many units per CTA: a whole unit at its cost midpoint
     for (const HostUnit& h : units) {
       if (dealt) break;
+      if (whole_units) {
+        push_whole(cta_of(run + cost_of(h) / 2), h);
+        run += cost_of(h);
+        continue;
+      }
       const uint64_t e8 = cost_of(h) / 8;
       int w = 0;
       while (w < 8) {
