@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
 # profiles/step_kernel_c2_1p6b_b1.md.  Valid only for that workload and for the kernel as it was
 # when the counters were taken: set an entry to None when step.cu changes.
-NCU_TRAFFIC_BYTES = {("c2_1p6b", 1, "step", None, 4): None}
+NCU_TRAFFIC_BYTES = {("c2_1p6b", 1, "step", None, 4): 540_035_328}
 
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
