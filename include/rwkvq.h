@@ -197,7 +197,8 @@ typedef struct {
 /*
  * A whole decode step (all projections of all layers, Appendix A.1) as ONE persistent launch:
  * packed weights are streamed through shared memory continuously across products and stages
- * while a grid-wide barrier enforces the stage order.  rwkvq_step_plan builds the schedule on
+ * while a grid-wide barrier enforces the stage order.  Every output row is summed in a fixed
+ * order and written with plain stores: two runs of a plan on the same inputs give the same bits.  rwkvq_step_plan builds the schedule on
  * the host and copies it into plan_dev (rwkvq_step_plan_bytes() bytes, caller-owned); the plan
  * embeds the pointers of `ops`, so the buffers must stay where they are.  rwkvq_step_run launches
  * it.  ops must be sorted by stage (non-decreasing).  Errors as rwkvq_gemv plus ETIMEOUT through
@@ -207,6 +208,46 @@ size_t rwkvq_step_plan_bytes(const rwkvq_gemv_op* ops, int n_ops, int B);
 rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* plan_dev,
                              size_t plan_bytes, void* stream);
 rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream);
+/* Forget the host-side record of the plan written to plan_dev (call it before the buffer is freed
+ * or reused for something else: the record is keyed by the buffer's address).  EINVAL if there is
+ * no such plan.  Host only. */
+rwkvq_status rwkvq_step_plan_release(const void* plan_dev);
+/*
+ * Waits inside the step kernel are bounded: a warp that has polled a barrier poll_limit times
+ * (default 2^22, several seconds) gives up, the kernel returns and rwkvq_device_status reports
+ * ETIMEOUT.  After an ETIMEOUT the caller must call rwkvq_device_status before the plan's next
+ * rwkvq_step_run, which then clears the plan's barrier words and starts over; outputs of the run
+ * that gave up are undefined.  This call sets the limit for later runs of one plan (0 = default).
+ * wait_skew is added to every barrier target; any value but 0 makes every stage barrier
+ * unreachable and exists so that a test can watch the waits run out.  Host only.
+ */
+rwkvq_status rwkvq_step_set_wait(const void* plan_dev, uint32_t poll_limit, uint32_t wait_skew);
+/*
+ * Cycle accounting of the step kernel, for diagnosis.  After rwkvq_step_trace(plan, trace_dev, n)
+ * every rwkvq_step_run of the plan launches an instrumented copy of the kernel that overwrites
+ * trace_dev (device memory, 8-byte aligned, at least rwkvq_step_trace_bytes(plan) bytes) with 16
+ * 64-bit counters per warp, laid out [CTA][warp][16]: consumer warps first (SM clock cycles spent
+ * waiting for weights, waiting for the stage barrier, fetching before and mixing inputs after it,
+ * inside the record loop, in the flush / publish tail of the record loop; records consumed; total
+ * cycles; cycles waiting for plan records and for input windows), then the producer warp (loop
+ * passes, records issued by its lane 0, total cycles, idle passes, cycles of passes that did
+ * work), then the auxiliary warp (cycles waiting for stage barriers, barriers waited for, cycles
+ * copying plan records, total cycles).  trace_dev == NULL switches back to the ordinary kernel.
+ * The instrumented kernel is slower; its outputs are the same.  Host only.
+ */
+size_t rwkvq_step_trace_bytes(const void* plan_dev);
+rwkvq_status rwkvq_step_trace(const void* plan_dev, void* trace_dev, size_t trace_bytes);
+/*
+ * Host-only check of the schedule rwkvq_step_plan would build for n_ctas CTAs (no device is
+ * touched; device pointers are only stored): counts_host[n_counts] receives, product after product,
+ * for every 16-row slice and every 256-column tile [oc/16][ic_pad/256] how many times the schedule
+ * hands that record to a consumer warp (the caller zero-fills it; a correct schedule writes 1
+ * everywhere), and cta_items_host[n_ctas] (may be NULL) the records each CTA consumes.  The
+ * products must have distinct y_dev.  Errors as rwkvq_step_plan_bytes, plus EINVAL for a
+ * schedule that is inconsistent with itself and ENOMEM for a short counts array.
+ */
+rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, int n_ctas,
+                                   uint32_t* counts_host, size_t n_counts, uint32_t* cta_items_host);
 /*
  * The same step for callers whose activations live in host memory: copies act_bytes from act_host
  * to act_dev (the device buffer the plan's x / x_prev pointers lie in), runs the step, and copies

@@ -1,7 +1,9 @@
-"""Host side of the whole-step launch: rwkvq_step_plan_bytes builds the complete plan on the host (no GPU
-needed: device pointers are only stored), so shapes, ordering and argument checks are tested here."""
+"""Host side of the whole-step launch: rwkvq_step_plan_bytes / rwkvq_step_plan_cover build the complete
+schedule on the host (no GPU needed: device pointers are only stored), so shapes, ordering, argument
+checks and the schedule's coverage are tested here."""
 import ctypes as C
 
+import numpy as np
 import pytest
 
 from paper_2505_03803_b200 import binding as B
@@ -27,17 +29,18 @@ def _mu_desc(ic, bits=6):
                   image_bytes=0, stream_bytes=0)
 
 
-def _ops(d, h, layers, vq_every=3, bits=6, y_dtype=B.RWKVQ_F32):
+def _ops(d, h, layers, vq_every=3, bits=6, y_dtype=B.RWKVQ_F32, one_stage=False):
     rows = []
     addr = 1 << 30
     for l in range(layers):
         for (name, oc, ic, has_mu, stage) in inputs.layer_shapes(d, h):
-            rows.append((oc, ic, has_mu, 4 * l + stage))
+            rows.append((oc, ic, has_mu, 0 if one_stage else 4 * l + stage))
     rows.sort(key=lambda r: r[3])
     arr = (B.GemvOp * len(rows))()
     for k, (oc, ic, has_mu, stage) in enumerate(rows):
         o = arr[k]
-        o.W_desc = _desc(B.RWKVQ_VQ if k % vq_every == 0 else B.RWKVQ_SQ, oc, ic, bits)
+        vq = vq_every > 0 and k % vq_every == 0 and oc % 256 == 0 and ic % 256 == 0
+        o.W_desc = _desc(B.RWKVQ_VQ if vq else B.RWKVQ_SQ, oc, ic, bits)
         for field in ("W_image_dev", "x_fp16_dev", "y_dev"):
             setattr(o, field, addr)
             addr += 1 << 26
@@ -55,15 +58,45 @@ def test_plan_is_built_for_benchmark_shapes(d, h, layers, Bn, bits):
     ops = _ops(d, h, layers, bits=bits)
     n = B.rwkvq_step_plan_bytes(ops, Bn)
     assert n > 0 and n % 256 == 0
-    # the plan grows with the number of units: twice the layers, roughly twice the descriptors
+    # the plan grows with the number of stages: twice the layers, roughly twice the descriptors
     n2 = B.rwkvq_step_plan_bytes(_ops(d, h, 2 * layers, bits=bits), Bn)
-    assert 1.5 * n < n2 < 2.5 * n
+    assert 1.3 * n < n2 < 2.5 * n
+
+
+# Every record (product, 16-row slice, 256-column tile) must reach exactly one consumer warp exactly
+# once: shapes with few slices per CTA, many slices per CTA, fewer items than warps, ragged tiles
+# (ic not a multiple of 256), every batch regime (inputs mixed per CTA; one window of the stage
+# pre-pass; several windows with two accumulator sets per warp), few and many CTAs.
+@pytest.mark.parametrize("d,h,layers,Bn,bits,n_ctas,one_stage", [
+    (512, 1280, 2, 1, 6, 148, False),
+    (384, 896, 2, 5, 6, 148, False),
+    (2048, 7168, 2, 1, 6, 148, False),
+    (4096, 14336, 1, 1, 6, 148, False),
+    (4096, 14336, 1, 2, 6, 148, False),
+    (4096, 14336, 1, 8, 6, 148, False),
+    (4096, 14336, 1, 16, 8, 148, False),
+    (4096, 14336, 1, 16, 8, 7, False),        # many slices per CTA: phases are cut to the warp count
+    (2048, 7168, 3, 1, 6, 148, True),         # every product in one stage
+    (2048, 7168, 1, 8, 6, 33, True),
+    (512, 1280, 1, 12, 8, 1, False),
+])
+def test_schedule_covers_every_record_once(d, h, layers, Bn, bits, n_ctas, one_stage):
+    ops = _ops(d, h, layers, bits=bits, one_stage=one_stage)
+    counts, per_cta = B.rwkvq_step_plan_cover(ops, Bn, n_ctas)
+    assert counts.size == sum((o.W_desc.oc // 16) * (o.W_desc.ic_pad // 256) for o in ops)
+    assert (counts == 1).all(), f"{int((counts != 1).sum())} records not dealt exactly once"
+    assert int(per_cta.sum()) == counts.size
+    if n_ctas == 148 and not one_stage:
+        # whole slices are dealt by cost: no CTA carries more than its even share plus one slice per stage
+        n_stages = len({o.stage for o in ops})
+        kt_max = max(o.W_desc.ic_pad // 256 for o in ops)
+        assert per_cta.max() <= counts.size / n_ctas + n_stages * kt_max * 1.9
 
 
 def test_plan_rejects_bad_arguments():
     ops = _ops(512, 1280, 1)
     assert B.rwkvq_step_plan_bytes(ops, 0) == 0 and B.rwkvq_step_plan_bytes(ops, 17) == 0
-    assert B.rwkvq_step_plan_bytes(_ops(512, 1280, 1, y_dtype=B.RWKVQ_F16), 1) == 0      # atomics need fp32 outputs
+    assert B.rwkvq_step_plan_bytes(_ops(512, 1280, 1, y_dtype=B.RWKVQ_F16), 1) == 0      # the step writes fp32 outputs
     bad = _ops(512, 1280, 1)
     bad[2].stage = -1                                                                  # stages must not decrease
     assert B.rwkvq_step_plan_bytes(bad, 1) == 0
@@ -76,3 +109,7 @@ def test_plan_rejects_bad_arguments():
     lib = B.lib()
     assert lib.rwkvq_step_run(None, 0, None) == 1
     assert lib.rwkvq_step_run(C.c_void_p(4096), 1 << 20, None) == 1                     # not a buffer a plan was written to
+    assert lib.rwkvq_step_plan_release(C.c_void_p(4096)) == 1
+    assert lib.rwkvq_step_set_wait(C.c_void_p(4096), 0, 0) == 1
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_step_plan_cover(_ops(512, 1280, 1), 0, 148)
