@@ -232,7 +232,11 @@ rwkvq_status rwkvq_step_set_wait(const void* plan_dev, uint32_t poll_limit, uint
  * cycles; cycles waiting for plan records and for input windows), then the producer warp (loop
  * passes, records issued by its lane 0, total cycles, idle passes, cycles of passes that did
  * work), then the auxiliary warp (cycles waiting for stage barriers, barriers waited for, cycles
- * copying plan records, total cycles).  trace_dev == NULL switches back to the ordinary kernel.
+ * copying plan records, total cycles).  Behind the counters follows a timeline [CTA][64][4] of
+ * the first 64 stages: SM clock when the CTA's last warp published the stage, when its auxiliary
+ * warp saw the barrier before the stage open, when its first consumer warp woke up and when the
+ * stage's inputs were staged (comparable within a CTA only).  trace_dev == NULL switches back to
+ * the ordinary kernel.
  * The instrumented kernel is slower; its outputs are the same.  Host only.
  */
 size_t rwkvq_step_trace_bytes(const void* plan_dev);
