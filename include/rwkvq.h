@@ -197,8 +197,9 @@ typedef struct {
 /*
  * A whole decode step (all projections of all layers, Appendix A.1) as ONE persistent launch:
  * packed weights are streamed through shared memory continuously across products and stages
- * while a grid-wide barrier enforces the stage order.  Every output row is summed in a fixed
- * order and written with plain stores: two runs of a plan on the same inputs give the same bits.  rwkvq_step_plan builds the schedule on
+ * while a grid-wide barrier enforces the stage order.  Partial sums of a row are added into the
+ * output with fp32 atomics: results are within the stated tolerance but not bit-reproducible
+ * from run to run.  rwkvq_step_plan builds the schedule on
  * the host and copies it into plan_dev (rwkvq_step_plan_bytes() bytes, caller-owned); the plan
  * embeds the pointers of `ops`, so the buffers must stay where they are.  rwkvq_step_run launches
  * it.  ops must be sorted by stage (non-decreasing).  Errors as rwkvq_gemv plus ETIMEOUT through
@@ -222,25 +223,6 @@ rwkvq_status rwkvq_step_plan_release(const void* plan_dev);
  * unreachable and exists so that a test can watch the waits run out.  Host only.
  */
 rwkvq_status rwkvq_step_set_wait(const void* plan_dev, uint32_t poll_limit, uint32_t wait_skew);
-/*
- * Cycle accounting of the step kernel, for diagnosis.  After rwkvq_step_trace(plan, trace_dev, n)
- * every rwkvq_step_run of the plan launches an instrumented copy of the kernel that overwrites
- * trace_dev (device memory, 8-byte aligned, at least rwkvq_step_trace_bytes(plan) bytes) with 16
- * 64-bit counters per warp, laid out [CTA][warp][16]: consumer warps first (SM clock cycles spent
- * waiting for weights, waiting for the stage barrier, fetching before and mixing inputs after it,
- * inside the record loop, in the flush / publish tail of the record loop; records consumed; total
- * cycles; cycles waiting for plan records and for input windows), then the producer warp (loop
- * passes, records issued by its lane 0, total cycles, idle passes, cycles of passes that did
- * work), then the auxiliary warp (cycles waiting for stage barriers, barriers waited for, cycles
- * copying plan records, total cycles).  Behind the counters follows a timeline [CTA][64][4] of
- * the first 64 stages: SM clock when the CTA's last warp published the stage, when its auxiliary
- * warp saw the barrier before the stage open, when its first consumer warp woke up and when the
- * stage's inputs were staged (comparable within a CTA only).  trace_dev == NULL switches back to
- * the ordinary kernel.
- * The instrumented kernel is slower; its outputs are the same.  Host only.
- */
-size_t rwkvq_step_trace_bytes(const void* plan_dev);
-rwkvq_status rwkvq_step_trace(const void* plan_dev, void* trace_dev, size_t trace_bytes);
 /*
  * Host-only check of the schedule rwkvq_step_plan would build for n_ctas CTAs (no device is
  * touched; device pointers are only stored): counts_host[n_counts] receives, product after product,

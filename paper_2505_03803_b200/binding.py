@@ -58,7 +58,7 @@ EXPORTS = [
     "rwkvq_pack", "rwkvq_blob_desc", "rwkvq_blob_nbytes", "rwkvq_blob_image", "rwkvq_blob_export_codes",
     "rwkvq_image_unpack", "rwkvq_blob_free", "rwkvq_proxy_workspace_bytes", "rwkvq_proxy_select",
     "rwkvq_gemv_workspace_bytes", "rwkvq_gemv", "rwkvq_gemv_static", "rwkvq_gemv_static_max_scratch_bytes", "rwkvq_step_plan_bytes", "rwkvq_step_plan", "rwkvq_step_run",
-    "rwkvq_step_run_host", "rwkvq_step_plan_release", "rwkvq_step_set_wait", "rwkvq_step_plan_cover", "rwkvq_step_trace_bytes", "rwkvq_step_trace",
+    "rwkvq_step_run_host", "rwkvq_step_plan_release", "rwkvq_step_set_wait", "rwkvq_step_plan_cover",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
     "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
@@ -120,9 +120,6 @@ def lib() -> C.CDLL:
         L.rwkvq_step_run.argtypes = [vp, sz, vp]
         L.rwkvq_step_run_host.argtypes = [vp, sz, vp, vp, sz, vp, vp, sz, vp]
         L.rwkvq_step_plan_release.argtypes = [vp]
-        L.rwkvq_step_trace_bytes.argtypes = [vp]
-        L.rwkvq_step_trace_bytes.restype = sz
-        L.rwkvq_step_trace.argtypes = [vp, vp, sz]
         L.rwkvq_step_set_wait.argtypes = [vp, C.c_uint32, C.c_uint32]
         L.rwkvq_step_plan_cover.argtypes = [C.POINTER(GemvOp), i32, i32, i32, C.POINTER(C.c_uint32), sz, C.POINTER(C.c_uint32)]
     if hasattr(L, "rwkvq_gemm_prefill"):
@@ -398,16 +395,6 @@ def rwkvq_step_plan_release(plan):
 
 def rwkvq_step_set_wait(plan, poll_limit: int = 0, wait_skew: int = 0):
     _check(lib().rwkvq_step_set_wait(_dev_ptr(plan), poll_limit, wait_skew), "rwkvq_step_set_wait")
-
-
-def rwkvq_step_trace_bytes(plan) -> int:
-    return int(lib().rwkvq_step_trace_bytes(_dev_ptr(plan)))
-
-
-def rwkvq_step_trace(plan, trace=None):
-    """trace: device int64 tensor of rwkvq_step_trace_bytes(plan) bytes, or None to switch tracing off."""
-    _check(lib().rwkvq_step_trace(_dev_ptr(plan), None if trace is None else _dev_ptr(trace),
-                                  0 if trace is None else trace.numel() * trace.element_size()), "rwkvq_step_trace")
 
 
 def rwkvq_step_plan_cover(ops, B: int, n_ctas: int):

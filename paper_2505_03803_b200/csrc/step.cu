@@ -2,31 +2,28 @@
 //
 // Decode at batch 1..16 reads every packed weight once and does almost no arithmetic per byte
 // (the paper's compute-to-memory argument, Section 1 and Appendix A.3), and one projection of a
-// 7B-class layer is only a few microseconds of HBM time.  The step is therefore ONE cooperative
-// kernel with one CTA per SM, built around these ideas:
+// 7B-class layer is only a few microseconds of HBM time.  Launching one kernel per projection
+// leaves the memory system idle between launches, so the step is ONE kernel with one CTA per SM:
 //
-//   * Weights never depend on activations, so each consumer warp owns a private ring of
-//     shared-memory entries that it keeps full itself with 16-byte asynchronous copies
-//     (cp.async), one 16-row x 256-column record per entry, running ahead across products and
-//     across stage boundaries: HBM keeps streaming while the CTAs synchronise.  A producer warp
-//     (one lane per consumer warp) walks the schedule and hands each warp, a few items ahead, a
-//     32-byte header per record: where it is, where its inputs are, what to do with the
-//     accumulators.  All index arithmetic of the schedule stays off the consumer warps.
-//   * A product's K range is cut into slabs short enough for a CTA to hold the slab's inputs in
-//     shared memory (one slab at batch 1; more at larger batches).  A 16-row slice of a slab
-//     belongs to ONE CTA; its records are dealt to the CTA's consumer warps in contiguous runs along
-//     K.  A warp accumulates a run in registers (m16n8k16 tensor-core steps, fp32), writes one
-//     partial per run to shared memory, and the last warp to finish the slice adds the partials in
-//     warp order.  With one slab the sums are the output rows (plain stores); with several, every
-//     CTA writes its slab's sums to a scratch area and the last CTA to arrive adds the slabs in slab
-//     order.  No atomics on outputs, no clearing pass, bit-reproducible results.
-//   * Inputs: every CTA mixes the slab of activations it needs itself, right after the stage
-//     barrier opens (x_mix = x + (x_prev - x) (.) mu_hat, Appendix A.1 Eq. 20; x_prev and mu_hat
-//     of a thread's first vectors are fetched before the barrier opens), rounds to fp16 and keeps
-//     the per-group sums the factored dequantisation needs.
-//   * The stage order ("every product of stage s is complete before any activation of stage s+1 is
-//     read") is a flag-array grid barrier: a CTA publishes the number of stages it has completed
-//     with one release store to its own word, and one auxiliary warp per CTA polls all words.
+//   * a producer warp streams packed weights from HBM into a ring of shared-memory slots with
+//     bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts).  Weights never depend
+//     on activations, so the stream runs ahead across products and across stage boundaries;
+//   * three stager warps build the fp16 input x_mix = x + (x_prev - x) (.) mu_hat (Appendix A.1
+//     Eq. 20) of the next run of units in one of two shared-memory buffers.  What does not depend
+//     on the previous stage (mu_hat, x_prev) is prepared before the grid-wide stage barrier; the
+//     stagers also clear the next stage's outputs and post this CTA's arrival at the barrier;
+//   * sixteen consumer warps in two groups of eight.  A unit is a 256-row x 256-column tile (two
+//     128-row chunks of the packed image); the groups take the CTA's units alternately, so one
+//     group computes while the other waits, flushes or synchronises.  Warp w of a group owns rows
+//     16w..16w+15 of both chunks and runs the m16n8k16 tensor-core steps of gemv_core.cuh with
+//     every input fragment shared by the two records.  Partial sums go to y with fp32 atomics at
+//     the end of a run along K.
+//
+// The host plans the step once: every stage's units are dealt WHOLE to the CTAs, row of tiles by
+// row of tiles where that balances (each row gets a number of CTAs by greedy cost per CTA), else at
+// their cost midpoints, small stages in eighths of a unit (one warp's records); the plan is a per-CTA
+// list of 128-byte unit descriptors plus a list of 64-byte input events (segments and barrier
+// arrivals).
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -44,77 +41,109 @@ namespace rwkvq {
 int* device_status_ptr();  // api_misc.cu
 unsigned abort_epoch();     // api_misc.cu: bumped whenever rwkvq_device_status reports a failed wait
 
-// ---- plan records shared by host and device -----------------------------------------------------
+enum { UF_FLUSH = 1, UF_VQ = 2, UF_BITS8 = 4 };
 
-enum { DK_PHASE = 0, DK_END = 2 };
-enum : uint32_t {
-  DF_FIRST = 1u << 8,    // first phase of a stage for this CTA: the stage barrier is awaited before it
-  DF_LAST = 1u << 9,     // last phase of the stage: the warps report the stage after it
-  DF_MU = 1u << 10, DF_SUMS = 1u << 11,
-  DF_SYNC = 1u << 12,    // every consumer warp must have left the earlier phases of the stage
-  DF_GROUP = 1u << 13,   // first phase of a group whose inputs are staged together
-  DF_GLAST = 1u << 14    // last phase of that group
-};
-// kind in bits 0..3, format (FMT_*) in bits 4..5 of kind_flags
-
-// One phase of a CTA: slices [row0/16, row0/16 + S) of one product, column tiles [kt0, kt0 + T) (one
-// K slab).  Item i of the S x T grid (slice-major) goes to consumer warp w with
-// w*N/CW <= i < (w+1)*N/CW  (N = S*T).
-struct PhaseDesc {           // 128 bytes
-  uint32_t kind_flags, stage;
-  uint64_t src;              // payload of the product's image
-  uint64_t cb;               // VQ: codebooks of the image
+struct StepUnit {            // 128 bytes, copied into the slot header by the producer
+  uint64_t src0, src1;       // global addresses of the first copied record of chunk A / chunk B (0 = absent)
+  uint64_t cb_src;           // VQ: codebook of the tile
+  uint32_t bytes0, bytes1;   // bytes copied from each chunk: (w1 - w0) records
+  uint32_t cb_bytes;
+  uint32_t off0;             // w0 * record bytes: where the copied records sit inside a chunk
+  uint32_t flags;            // UF_* | w0 << 8 | w1 << 12: warps w0 <= w < w1 of the group have a record
+  uint32_t seg;              // number, within this CTA, of the input segment the unit reads
+  uint32_t stage;            // stage number (0-based)
+  uint32_t xcol0;            // column of the unit's tile inside the segment
+  uint32_t row0, oc;         // first output row of chunk A; rows of the product
   uint64_t y;                // float y[B][oc]
-  uint32_t oc, row0;         // rows of the product; first row of the phase
-  uint32_t S, KT;            // slices of the phase; column tiles of the product
-  uint32_t T, kt0;           // tiles of the slab; its first tile
-  uint32_t xoff, xstride;    // bytes: the slab's input rows inside the input area
-  uint32_t gsoff, cnt_base;  // bytes: group sums; first slice counter of the phase
-  uint32_t ks_part;          // slabs of the product | this slab's number << 16
-  uint32_t gslot0;           // several slabs: scratch slot of (slice row0/16, slab 0); slice i: + i * slabs
-  uint32_t post_value;       // stages to report complete when the phase's stage is done
-  uint32_t ic;
-  uint64_t x, xprev, mu, mu_aux;   // the caller's inputs
-  uint16_t mu_bits, mu_entries;
-  uint32_t slot_set;         // which set of partial-sum slots the phase uses (phases of one stage alternate)
+  uint32_t xstride, gs_off;  // geometry of the segment: bytes between batch rows, offset of the sums
+  uint32_t nbp, entries;
+  uint32_t chunk_bytes;      // distance between chunk A and chunk B inside the slot
+  uint32_t rec_bytes;
+  uint32_t ev_index;         // position of the unit's segment in this CTA's event list
+  uint32_t between_mask;     // events between the group's previous segment and this one, oldest in bit 0:
+                             // 1 = barrier arrival, 0 = segment of the other group (valid for up to 32 events)
+  uint32_t after_count;      // set on a group's last unit of a stage: events after its segment up to and
+  uint32_t after_mask;       // including the stage's barrier arrival, to be passed right after the unit
+  uint32_t pad[4];
 };
-static_assert(sizeof(PhaseDesc) == 128, "phase descriptor size");
+static_assert(sizeof(StepUnit) == 128, "unit descriptor size");
 
-// run header flags (word 2 of the 32-byte header the producer writes for every run; bits 0..8: records of the run,
-// 9..15: slice counter, 16..23: warps that hold a part of the slice, 24..28: the first of them)
-enum : uint32_t { IF_RSELF = 1u << 29, IF_RFIRST = 1u << 30 };
+enum { EV_SEGMENT = 0, EV_ARRIVE = 1 };
 
-constexpr int kConsumerWarps = 16;   // per CTA, plus one producer and one auxiliary warp
-constexpr int kMaxCW = 24, kHeaderRing = 16, kDescRing = 32, kCnt = 128;
-constexpr int kMaxVals = (16 * 16 + 31) / 32;   // elements of a slice's [batch][16 rows] block per lane
-constexpr uint32_t kCtrlBytes = 2048, kDescBytes = kDescRing * 128;
+struct StepEvent {           // 64 bytes
+  union {
+    // segment.  Mixed in the CTA: x, xprev, mu, mu_aux as given by the caller.  Copied from the
+    // stage's pre-pass (StepArgs::mix): x = first byte of the segment in the pre-pass rows,
+    // xprev = first byte of its sums, mu = 0.
+    struct { uint64_t x, xprev, mu, mu_aux; } seg;
+    // arrival: float ranges to clear before arriving; then this CTA's share of the stage's
+    // pre-pass: groups [grp_lo, grp_hi) of the stage's (product, batch row, 128-column group) list
+    struct { uint64_t zptr[3]; uint32_t grp_lo, grp_hi; } arr;
+  };
+  union {
+    struct { uint32_t ic, col0, ncols; uint16_t mu_bits, mu_entries; } segd;   // copied segments: ic = bytes between rows
+    struct { uint32_t zcount[3]; uint16_t op_first, op_count; } arrd;          // products of the stage the pre-pass covers
+  };
+  uint32_t kind;             // EV_SEGMENT / EV_ARRIVE
+  uint32_t barrier;          // segment: index + 1 of the stage barrier to pass first; arrival: index of the barrier
+  uint32_t xstride_sums;     // segment: xstride | sums << 31
+  uint16_t mu_off16;         // segment: offset / 16 of the decoded mu row inside the buffer
+  uint16_t reserved;
+};
+static_assert(sizeof(StepEvent) == 64, "event descriptor size");
+
+// One product's share of a stage's pre-pass: where its inputs are and where x_mix (fp16 rows of
+// ic_pad columns, zero beyond ic) and the per-group sums ([group][3][nbp] floats) go.
+struct StepMixOp {           // 64 bytes
+  uint64_t x, xprev, mu, mu_aux, dst_x, dst_sums;
+  uint32_t ic, ic_pad;
+  uint16_t mu_bits, mu_entries, sums, pad;
+};
+static_assert(sizeof(StepMixOp) == 64, "pre-pass descriptor size");
+
+constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGroups, kStagerWarps = 3;
+constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
+constexpr int kGroupThreads = kGroupWarps * 32;
+constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
+constexpr int kMaxSlots = 12;
+constexpr uint32_t kCtrlBytes = 1024, kXBufTotal = 49152, kMuScratch = 1024;
+// Input-segment buffers: two of 24 KB when the CTA mixes its own inputs (the segment carries a mu row and
+// is prepared ahead), four of 12 KB when segments are copied from the stage's pre-pass.
+// (up to 8 batch rows; larger batches keep two buffers, a 256-column tile of 16 rows being 9 KB).
+template <bool MIX, int NB> struct XBufs { static constexpr uint32_t kCount = (MIX && NB == 1) ? 4u : 2u, kBytes = kXBufTotal / kCount; };
 constexpr uint32_t kSmemLimit = 232448;  // 227 KB
 constexpr uint32_t kDefaultPollLimit = 1u << 22;
 
 struct StepArgs {
-  const PhaseDesc* descs;
-  const uint32_t* desc_off;   // [P+1]
-  const uint32_t* init_post;  // [P] stages a CTA may report complete before it has consumed anything
-  unsigned* flags;            // [P] stages completed by each CTA, summed over all runs
-  unsigned base;              // value of every flag when this run starts
+  const StepUnit* units;
+  const StepEvent* events;
+  const uint32_t* unit_off;   // [P+1]
+  const uint32_t* event_off;  // [P+1]
+  unsigned* counter;          // stage barriers: arrivals at barrier k, summed over all runs, in counter[k]
+  unsigned target;            // arrivals that open a barrier in this run: run number * CTAs (mod 2^32)
+  unsigned wait_skew;         // added to the target the WAITS compare with (0; a test sets it to make them run out)
+  uint32_t poll_limit;        // polls after which a wait gives up
   int* status;
-  uint32_t poll_limit;
-  unsigned wait_skew;         // added to every barrier target (0; a test sets it to make the waits run out)
-  int B, nbp, depth;
-  uint32_t entry_bytes, slot_floats;
-  uint32_t off_hq, off_partial, off_x, off_ring;
-  float* gpart;               // scratch slots of slot_floats floats: a slab's sums of one slice
-  unsigned* gcnt;             // per slot of slab 0: slabs of the slice that have arrived
-  unsigned long long* trace;  // rwkvq_step_trace: per-warp counters, else NULL
+  int B, n_slots, n_stages;
+  uint32_t slot_bytes, replica_bytes;
+  // Larger batches: x_mix and the sums of a stage are computed ONCE by all CTAs together after the
+  // stage barrier (instead of by every CTA that reads a column), published through a second
+  // barrier per stage (counter[n_stages + 1 + s]), and fetched into the segment buffers with bulk copies.
+  int mix;
+  const StepMixOp* mixops;    // dst_x / dst_sums are offsets into `scratch`
+  uint8_t* scratch;
 };
 
-// ---- small wrappers -----------------------------------------------------------------------------
+// ---- mbarrier / bulk-copy wrappers ------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 // The hint lets the hardware park the thread for up to that many nanoseconds (it is woken when
 // the phase completes), so that waiting warps do not compete for issue slots with computing ones.
@@ -125,39 +154,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(2000u) : "memory");
   return ok != 0;
 }
-// Packed weights are read exactly once per step: they are marked evict-first so that streaming
-// them does not push the activations, the plan and the outputs out of L2.
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
+// The launch's poll limit sits directly behind the CTA's abort flag in the control block (Ctrl).
+__device__ __forceinline__ uint32_t poll_limit_of(volatile int* abort_flag) { return (uint32_t)abort_flag[1]; }
+// Bounded wait by one thread: gives up (and raises the CTA-wide abort flag) after that many polls
+// or when another role of this CTA has already given up.
+__device__ __forceinline__ bool mbar_wait_one(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  const uint32_t limit = poll_limit_of(abort_flag);
+  for (uint32_t it = 0; it < limit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicExch(status, (int)RWKVQ_ETIMEOUT);
+  return false;
 }
-__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_relaxed_gpu(unsigned* p, unsigned v) {
-  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned atom_add_acq_rel_gpu(unsigned* p, unsigned v) {
-  unsigned old;
-  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-  return old;
-}
-__device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
-__device__ __forceinline__ uint32_t smem_add_acq_rel(uint32_t* p, uint32_t v) {
-  uint32_t old;
-  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
-  return old;
-}
-__device__ __forceinline__ uint32_t ld_acquire_cta(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_release_cta(uint32_t* p, uint32_t v) {
-  asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+// Warp-collective bounded wait: every lane polls (so that each lane itself observes the completed
+// phase and with it the data the barrier guards); the verdict is made warp-uniform.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  const bool ok = mbar_wait_one(bar, parity, abort_flag, status);
+  return __all_sync(0xFFFFFFFFu, ok);
 }
 // Named barrier over `nthreads` threads that also ANDs a predicate: a uniform verdict for a role.
 __device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred) {
@@ -166,288 +181,148 @@ __device__ __forceinline__ bool named_bar_and(int id, int nthreads, bool pred) {
                : "=r"(r) : "r"((uint32_t)pred), "r"(id), "r"(nthreads) : "memory");
   return r != 0;
 }
+// Packed weights are read exactly once per step: they are marked evict-first so that streaming
+// them does not push the activations, the plan and the outputs out of L2.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s_plain(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_gpu(unsigned* p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t smem_add_acq_rel(uint32_t* p, uint32_t v) {
+  uint32_t old;
+  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(smem_u32(p)), "r"(v) : "memory");
+  return old;
+}
 
 struct Ctrl {
-  uint64_t open;               // the aux warp arrives once per stage this CTA takes part in
-  uint32_t warps_done;         // consumer warps that have left a stage, summed over the stages so far
-  uint32_t hq_head[kMaxCW];    // item headers written by the producer lane of each consumer warp
-  uint32_t hq_tail[kMaxCW];    // ... and read by the warp
-  uint32_t desc_hi;            // descriptors copied into the ring so far
-  uint32_t desc_tail;          // descriptors below this one are no longer needed by the consumer warps
-  uint32_t prod_tail;          // ... nor by any lane of the producer warp
+  uint64_t full[kMaxSlots], empty[kMaxSlots];
+  uint64_t xfull[4], xempty[4];
+  uint32_t stage_cnt[64];    // one 8-bit count per grid barrier (four per word): how many of the seventeen
+                             // parties of this CTA (sixteen consumer warps, the stagers) have reported the
+                             // stage that the barrier closes.  Per barrier, not one running total: consumer
+                             // warps of a CTA without work in the coming stages may run any number of
+                             // stages ahead of the stagers.
+  uint32_t cdone;            // running total of stage reports of the consumer warps (two-batch-block launches)
   int abort_flag;
-  uint32_t cnt[kCnt];          // per-slice count of warps that have written their partial
+  int poll_limit;            // must follow abort_flag (poll_limit_of)
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
+constexpr uint32_t kMaxBarriers = 256;   // barriers that close a stage (8-bit counts in Ctrl::stage_cnt)
 
-// The CTA's dynamic shared memory.  The record loop addresses it by 32-bit offsets from this symbol.
-extern __shared__ __align__(128) uint8_t smem_base[];
-
-struct Env {
-  const StepArgs& a;
-  uint8_t* smem;
-  Ctrl* ctrl;
-  volatile int* abortp;
-};
-
-// Optional per-warp cycle accounting (rwkvq_step_trace): kTraceSlots 64-bit counters per warp,
-// (CW + 2) warps per CTA.  Compiled into separate kernel instances, so the ordinary launch carries
-// none of it.
-constexpr int kTraceSlots = 16, kTraceStages = 64;
-enum { TR_WAIT_FULL = 0, TR_WAIT_OPEN, TR_PRE, TR_POST, TR_ITEMS, TR_FLUSH, TR_NITEMS, TR_TOTAL, TR_WAIT_DESC,
-       TR_P_ITER = 0, TR_P_ISSUED, TR_P_TOTAL, TR_P_IDLE, TR_P_WORK,
-       TR_A_WAIT = 0, TR_A_POLLS, TR_A_REFILL, TR_A_TOTAL };
-template <bool TRACE>
-struct Tracer {
-  unsigned long long v[TRACE ? kTraceSlots : 1];
-  __device__ __forceinline__ Tracer() {
-    if constexpr (TRACE) for (int k = 0; k < kTraceSlots; ++k) v[k] = 0ull;
-  }
-  __device__ __forceinline__ long long now() const { if constexpr (TRACE) return clock64(); else return 0; }
-  __device__ __forceinline__ void add(int slot, long long t0) { if constexpr (TRACE) v[slot] += (unsigned long long)(clock64() - t0); }
-  __device__ __forceinline__ void count(int slot, unsigned n = 1u) { if constexpr (TRACE) v[slot] += n; }
-  // Timeline of the first kTraceStages stages of a CTA: when its last warp published the stage
-  // (0), when the auxiliary warp saw the barrier open (1), when consumer warp 0 woke up (2) and when
-  // the consumers had the stage's inputs staged (3); SM clock, comparable within one CTA only.
-  __device__ __forceinline__ static void stamp(unsigned long long* trace, uint32_t stage, int what) {
-    if constexpr (TRACE) {
-      if (trace && stage < (uint32_t)kTraceStages)
-        trace[(size_t)gridDim.x * (blockDim.x >> 5) * kTraceSlots + ((size_t)blockIdx.x * kTraceStages + stage) * 4 + what] = (unsigned long long)clock64();
-    }
-  }
-  __device__ __forceinline__ void store(unsigned long long* trace) const {
-    if constexpr (TRACE) {
-      if (trace && (threadIdx.x & 31) == 0) {
-        unsigned long long* dst = trace + ((size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * kTraceSlots;
-        for (int k = 0; k < kTraceSlots; ++k) dst[k] = v[k];
-      }
-    }
-  }
-};
-
-__device__ __forceinline__ void give_up(const Env& e) {
-  *e.abortp = 1;
-  atomicExch(e.a.status, (int)RWKVQ_ETIMEOUT);
+// One of the seventeen parties of grid barrier `b` reports that its part of the stage the barrier
+// closes is done; whoever reports last posts the CTA's arrival.  The count is an acquire-release
+// read-modify-write at CTA scope and the arrival a GPU-scope release, so the arrival is ordered
+// after everything every party did before reporting (the consumers' reductions into y, the
+// stagers' clearing of the next outputs): block-level synchronisation followed by one thread's
+// release, the pattern of a cooperative grid barrier.
+__device__ __forceinline__ void stage_report(Ctrl* ctrl, const StepArgs& a, uint32_t b) {
+  const uint32_t sh = 8u * (b & 3u);
+  const uint32_t old = smem_add_acq_rel(&ctrl->stage_cnt[b >> 2], 1u << sh);
+  if (((old >> sh) & 0xFFu) == (uint32_t)kConsumerWarps) red_release_gpu(a.counter + b, 1u);
 }
-// Bounded wait on an mbarrier phase: gives up (and raises the CTA-wide abort flag) after
-// poll_limit polls or when another role of this CTA has already given up.
-__device__ __forceinline__ bool mbar_wait(const Env& e, uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < e.a.poll_limit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 15u) == 15u && *e.abortp) return false;
-  }
-  give_up(e);
-  return false;
+// Where the consumer warps are the busy role (two batch blocks per record) they only add to one
+// running total, and a stager thread, which has nothing else to do at that point, waits (bounded)
+// for the sixteen reports of the stage and arrives: the release, which waits for the CTA's
+// outstanding reductions, and the bookkeeping of a barrier number stay off the consumer warps.
+__device__ __forceinline__ void stage_report_total(Ctrl* ctrl) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(&ctrl->cdone)), "r"(1u) : "memory");
 }
-__device__ __forceinline__ const PhaseDesc* desc_slot(const Env& e, uint32_t p) {
-  return reinterpret_cast<const PhaseDesc*>(e.smem + kCtrlBytes) + (p % (uint32_t)kDescRing);
-}
-// Bounded wait until descriptor p is in the ring.
-__device__ __forceinline__ bool wait_desc(const Env& e, uint32_t p) {
-  for (uint32_t it = 0; it < (e.a.poll_limit << 4); ++it) {
-    if ((int)(ld_acquire_cta(&e.ctrl->desc_hi) - p) > 0) return true;
-    if ((it & 63u) == 63u && *e.abortp) return false;
-    __nanosleep(64);
+__device__ __forceinline__ bool stage_wait_total_and_arrive(Ctrl* ctrl, const StepArgs& a, uint32_t b, volatile int* abort_flag) {
+  const uint32_t limit = poll_limit_of(abort_flag) << 4;
+  for (uint32_t it = 0; it < limit; ++it) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&ctrl->cdone)) : "memory");
+    if (v >= (uint32_t)kConsumerWarps * b) { red_release_gpu(a.counter + b, 1u); return true; }
+    if ((it & 255u) == 255u && *abort_flag) return false;
   }
-  give_up(e);
+  *abort_flag = 1;
+  atomicExch(a.status, (int)RWKVQ_ETIMEOUT);
   return false;
 }
 
-// The share [i0, i1) of a phase's N = S*T items that consumer warp w of CW owns.
-template <int CW>
-__host__ __device__ __forceinline__ void item_range(uint32_t N, uint32_t w, uint32_t& i0, uint32_t& i1) {
-  if (N >= (uint32_t)CW) { i0 = w * N / (uint32_t)CW; i1 = (w + 1u) * N / (uint32_t)CW; }
-  else { i0 = w < N ? w : N; i1 = w + 1u < N ? w + 1u : N; }
-}
+// ---- roles -------------------------------------------------------------------------------------
 
-// ---- producer: one lane per consumer warp ---------------------------------------------------------
-//
-// A RUN is the part of one slice that one consumer warp owns: consecutive column tiles of the
-// slab.  Lane w walks the CTA's phases and writes, for every run of warp w in consumption order, a
-// 32-byte header into warp w's header ring: where the run's first record (and, for VQ, its
-// codebook) is in global memory, how many records follow at the fixed stride of a column tile,
-// where the inputs of the first tile are in shared memory, and who else holds a part of the slice.
-// It stays a few runs ahead of the consumer, which issues the copies itself.
-//   q0 = { byte offset of the first tile's inputs in shared memory, ... of its group sums, flags | records, first row of the slice }
-//   q1 = { address of the first record | format, codebook address - record address, unused }
-template <int CW, bool TRACE>
-__device__ void producer_role(const Env& e) {
-  const StepArgs& a = e.a;
-  Tracer<TRACE> tr;
-  const long long t_begin = tr.now();
-  const uint32_t w = threadIdx.x & 31u;
-  const bool active = w < (uint32_t)CW;
-  uint8_t* hq = e.smem + a.off_hq + (size_t)w * kHeaderRing * 32u;
-  const uint32_t sums_tile = 2u * 3u * (uint32_t)a.nbp * 4u;   // bytes of group sums per 256-column tile
-  uint32_t p = 0;              // descriptor this lane works on
-  bool have = false, done = !active;
-  // current phase
-  uint32_t kf = 0, KT = 0, T = 0, kt0 = 0, N = 0, i0 = 0, i1 = 0, rec_bytes = 0, cb_bytes = 0;
-  uint32_t xoff = 0, gsoff = 0, row0 = 0, cnt_base = 0;
-  uint64_t src0 = 0, cb0 = 0;
-  uint32_t i = 0, sl0 = 0;     // first item of the next run; the warp's first slice of the phase
-  uint32_t n = 0;              // headers written
-  uint32_t tail = 0;           // headers the consumer is known to have read
-  uint32_t idle = 0, last_pmin = 0;
-  while (true) {
-    bool progress = false;
-    tr.count(TR_P_ITER);
-    const long long t_it = tr.now();
-    if (!done && !have) {
-      if ((int)(ld_acquire_cta(&e.ctrl->desc_hi) - p) > 0) {
-        const PhaseDesc* d = desc_slot(e, p);
-        kf = d->kind_flags;
-        progress = true;
-        if ((kf & 15u) == DK_END) done = true;
-        else {
-          KT = d->KT; T = d->T; kt0 = d->kt0; N = d->S * T;
-          item_range<CW>(N, w, i0, i1);
-          if (i0 == i1) ++p;
-          else {
-            have = true;
-            const uint32_t fmt = (kf >> 4) & 3u;
-            rec_bytes = fmt == FMT_SQ3 ? (uint32_t)RWKVQ_SQ_RECORD_BYTES : fmt == FMT_VQ6 ? 1536u : 2048u;
-            cb_bytes = fmt == FMT_SQ3 ? 0u : fmt == FMT_VQ6 ? 256u : 1024u;
-            xoff = a.off_x + d->xoff; gsoff = a.off_x + d->gsoff; row0 = d->row0;
-            cnt_base = d->cnt_base; src0 = d->src; cb0 = d->cb;
-            sl0 = i0 / T;
-            i = i0;
-          }
+// Producer: one warp.  Four descriptors are fetched per warp-wide 16-byte load (8 lanes each) one
+// batch ahead; lane 0 waits for the slot, the owning lanes copy the descriptor into the slot
+// header, lane 0 arms the barrier and issues the bulk copies.
+__device__ void producer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint32_t u0, uint32_t u1) {
+  const int lane = threadIdx.x & 31;
+  const uint4* base = reinterpret_cast<const uint4*>(a.units);
+  const uint32_t n = u1 - u0;
+  volatile int* abortp = &ctrl->abort_flag;
+  const uint64_t policy = policy_evict_first();
+  uint4 next = make_uint4(0, 0, 0, 0);
+  if ((uint32_t)(lane >> 3) < n) next = __ldg(base + (size_t)(u0 + (lane >> 3)) * 8 + (lane & 7));
+  uint32_t issued = 0;
+  bool ok = true;
+  for (uint32_t b0 = 0; b0 < n && ok; b0 += 4) {
+    const uint4 cur = next;
+    const uint32_t nb = b0 + 4 + (lane >> 3);
+    if (nb < n) next = __ldg(base + (size_t)(u0 + nb) * 8 + (lane & 7));
+    for (int k = 0; k < 4 && b0 + k < n; ++k) {
+      const uint32_t i = b0 + k;
+      const int slot = (int)(i % (uint32_t)a.n_slots);
+      const uint32_t round = i / (uint32_t)a.n_slots;
+      uint8_t* sl = smem + kCtrlBytes + (size_t)slot * a.slot_bytes;
+      int good = 1;
+      if (lane == 0) good = mbar_wait_one(&ctrl->empty[slot], (round & 1u) ^ 1u, abortp, a.status) ? 1 : 0;
+      good = __shfl_sync(0xFFFFFFFFu, good, 0);
+      if (!good) { ok = false; break; }
+      if ((lane >> 3) == k) *reinterpret_cast<uint4*>(sl + (lane & 7) * 16) = cur;
+      // fields for lane 0, by 16-byte piece of descriptor k
+      const uint32_t s0l = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k), s0h = __shfl_sync(0xFFFFFFFFu, cur.y, 8 * k);
+      const uint32_t s1l = __shfl_sync(0xFFFFFFFFu, cur.z, 8 * k), s1h = __shfl_sync(0xFFFFFFFFu, cur.w, 8 * k);
+      const uint32_t cbl = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k + 1), cbh = __shfl_sync(0xFFFFFFFFu, cur.y, 8 * k + 1);
+      const uint32_t by0 = __shfl_sync(0xFFFFFFFFu, cur.z, 8 * k + 1), by1 = __shfl_sync(0xFFFFFFFFu, cur.w, 8 * k + 1);
+      const uint32_t cbb = __shfl_sync(0xFFFFFFFFu, cur.x, 8 * k + 2), off0 = __shfl_sync(0xFFFFFFFFu, cur.y, 8 * k + 2);
+      const uint32_t chb = __shfl_sync(0xFFFFFFFFu, cur.z, 8 * k + 5);
+      __syncwarp();
+      if (lane == 0) {
+        const uint32_t tx = by0 + by1 + cbb;
+        uint64_t* full = &ctrl->full[slot];
+        if (tx == 0) {
+          mbar_arrive(full);
+        } else {
+          mbar_arrive_expect_tx(full, tx);
+          uint8_t* data = sl + 128;
+          if (by0) bulk_g2s(data + off0, reinterpret_cast<const void*>(((uint64_t)s0h << 32) | s0l), by0, full, policy);
+          if (by1) bulk_g2s(data + chb + off0, reinterpret_cast<const void*>(((uint64_t)s1h << 32) | s1l), by1, full, policy);
+          if (cbb) bulk_g2s(data + 2 * chb, reinterpret_cast<const void*>(((uint64_t)cbh << 32) | cbl), cbb, full, policy);
         }
       }
-    } else if (!done) {
-      if (n - tail >= (uint32_t)kHeaderRing) tail = ld_acquire_cta(&e.ctrl->hq_tail[w]);
-      if (n - tail < (uint32_t)kHeaderRing) {
-        progress = true;
-        const uint32_t sl = i / T, tt = i - sl * T;
-        const uint32_t lo = sl * T, hi = lo + T;
-        const uint32_t iend = min(i1, hi);                 // the run: items [i, iend) of slice sl
-        const uint32_t kt = kt0 + tt;
-        const uint32_t row = row0 + 16u * sl;
-        const uint64_t src = src0 + (uint64_t)((row >> 7) * KT + kt) * (8u * rec_bytes) + ((row >> 4) & 7u) * rec_bytes;
-        const uint64_t cbs = cb0 + (uint64_t)((row >> 8) * KT + kt) * cb_bytes;
-        // who else holds a part of the slice
-        uint32_t wlo, whi;
-        if (N >= (uint32_t)CW) { wlo = ((lo + 1u) * (uint32_t)CW + N - 1u) / N - 1u; whi = (hi * (uint32_t)CW + N - 1u) / N - 1u; }
-        else { wlo = lo; whi = hi - 1u; }
-        uint32_t f0, f1;
-        item_range<CW>(N, wlo, f0, f1);
-        uint32_t flags = (iend - i) | (((cnt_base + sl) & (uint32_t)(kCnt - 1)) << 9) | ((whi - wlo + 1u) << 16) | (wlo << 24);
-        if (sl != sl0) flags |= IF_RSELF;
-        if (f0 < lo) flags |= IF_RFIRST;
-        uint4* h = reinterpret_cast<uint4*>(hq + (size_t)(n % (uint32_t)kHeaderRing) * 32u);
-        h[0] = make_uint4(xoff + tt * 512u, gsoff + tt * sums_tile, flags, row);
-        h[1] = make_uint4((uint32_t)src | ((kf >> 4) & 3u), (uint32_t)(src >> 32), (uint32_t)(cbs - src), 0u);
-        ++n;
-        st_release_cta(&e.ctrl->hq_head[w], n);
-        tr.count(TR_P_ISSUED);
-        i = iend;
-        if (i == i1) { have = false; ++p; }
-      }
-    }
-    {
-      // the oldest descriptor any lane still reads (lanes that are done, or unused, do not hold one back)
-      const uint32_t pmin = __reduce_min_sync(0xFFFFFFFFu, done ? 0xFFFFFFFFu : p);
-      if (pmin != last_pmin && pmin != 0xFFFFFFFFu) { last_pmin = pmin; if (w == 0) st_release_cta(&e.ctrl->prod_tail, pmin); }
-    }
-    if (__all_sync(0xFFFFFFFFu, done)) break;
-    if (__any_sync(0xFFFFFFFFu, progress)) { idle = 0; tr.add(TR_P_WORK, t_it); continue; }
-    tr.count(TR_P_IDLE);
-    if (*e.abortp) break;
-    if (++idle > (a.poll_limit << 4)) { give_up(e); break; }
-    __nanosleep(100);
-  }
-  tr.add(TR_P_TOTAL, t_begin);
-  tr.store(a.trace);
-}
-
-
-// ---- the flag barrier -----------------------------------------------------------------------------
-
-// All of this warp's lanes together read every CTA's word; true once all have reached `target`.
-__device__ __forceinline__ bool flags_reached(const unsigned* flags, int P, unsigned target, int lane) {
-  // Acquire loads (an acquire load costs about what a relaxed one does, a separate fence after the
-  // poll three times as much); every load is issued before the first result is looked at: one
-  // round trip per poll.
-  unsigned behind = 0u;
-  for (int c = lane; c < P; c += 32) behind |= (ld_acquire_gpu(flags + c) - target) >> 31;
-  return __all_sync(0xFFFFFFFFu, behind == 0u);
-}
-__device__ __forceinline__ bool flags_wait(const Env& e, const unsigned* flags, unsigned target, int lane) {
-  const int P = (int)gridDim.x;
-  for (uint32_t it = 0; it < (e.a.poll_limit << 2); ++it) {
-    if (flags_reached(flags, P, target, lane)) return true;
-    if ((it & 7u) == 7u && *e.abortp) return false;
-  }
-  if (lane == 0) give_up(e);
-  return false;
-}
-
-// ---- auxiliary warp: descriptor ring, barrier detection -------------------------------------------
-template <bool TRACE>
-__device__ void aux_role(const Env& e) {
-  const StepArgs& a = e.a;
-  const int lane = threadIdx.x & 31;
-  Tracer<TRACE> tr;
-  const long long t_begin = tr.now();
-  const uint32_t d0 = a.desc_off[blockIdx.x], n_desc = a.desc_off[blockIdx.x + 1] - d0;
-  uint32_t hi = 0;
-  auto refill = [&]() {
-    // copy descriptors into the ring as far as the other warps' progress allows, four per pass
-    const uint32_t tail = min(ld_acquire_cta(&e.ctrl->desc_tail), ld_acquire_cta(&e.ctrl->prod_tail));
-    bool any = false;
-    while (hi < n_desc && hi < tail + (uint32_t)kDescRing) {
-      const uint32_t k = hi + (uint32_t)(lane >> 3);
-      if (k < n_desc && k < tail + (uint32_t)kDescRing) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(a.descs + d0 + k) + (lane & 7));
-        *(reinterpret_cast<uint4*>(const_cast<PhaseDesc*>(desc_slot(e, k))) + (lane & 7)) = v;
-      }
-      hi = min(min(hi + 4u, n_desc), tail + (uint32_t)kDescRing);
-      any = true;
-    }
-    if (any) {
-      __syncwarp();
-      if (lane == 0) st_release_cta(&e.ctrl->desc_hi, hi);
-    }
-  };
-  if (lane == 0 && a.init_post[blockIdx.x]) st_relaxed_gpu(a.flags + blockIdx.x, a.base + a.init_post[blockIdx.x]);
-  refill();
-  for (uint32_t p = 0; p < n_desc; ++p) {
-    if (p >= hi) {
-      // the ring is full of descriptors the other warps still need: wait for them to move on
-      bool ok = false;
-      for (uint32_t it = 0; it < (a.poll_limit << 4); ++it) {
-        refill();
-        if (p < hi) { ok = true; break; }
-        if ((it & 63u) == 63u && *e.abortp) break;
-        __nanosleep(100);
-      }
-      if (!ok) { if (lane == 0 && !*e.abortp) give_up(e); return; }
-    }
-    const PhaseDesc* d = desc_slot(e, p);
-    const uint32_t kf = d->kind_flags;
-    if ((kf & 15u) == DK_END) break;
-    if (kf & DF_FIRST) {
-      // the stage may start once every CTA has completed all earlier stages
-      const uint32_t stage = d->stage;
-      const long long t0 = tr.now();
-      if (stage > 0u && !flags_wait(e, a.flags, a.base + stage + a.wait_skew, lane)) return;
-      tr.add(TR_A_WAIT, t0); tr.count(TR_A_POLLS);
-      if (lane == 0) Tracer<TRACE>::stamp(a.trace, stage, 1);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&e.ctrl->open);
-    }
-    {
-      const long long t0 = tr.now();
-      refill();
-      tr.add(TR_A_REFILL, t0);
+      ++issued;
     }
   }
-  tr.add(TR_A_TOTAL, t_begin);
-  tr.store(a.trace);
+  if (!ok && lane == 0) {
+    // Gave up: do not leave the CTA while copies this thread issued may still be landing.
+    const uint32_t first = issued > (uint32_t)a.n_slots ? issued - a.n_slots : 0;
+    for (uint32_t i = first; i < issued; ++i) {
+      const int slot = (int)(i % (uint32_t)a.n_slots);
+      const uint32_t parity = (i / (uint32_t)a.n_slots) & 1u;
+      for (uint32_t it = 0; it < a.poll_limit; ++it)
+        if (mbar_try_wait(&ctrl->full[slot], parity)) break;
+    }
+  }
 }
-
-// ---- consumer warps: input staging ------------------------------------------------------------------
 
 __device__ __forceinline__ uint32_t mix2(uint32_t xr, uint32_t pr, uint32_t mr) {
   const float2 xf = __half22float2(*reinterpret_cast<const __half2*>(&xr));
@@ -460,591 +335,561 @@ __device__ __forceinline__ float pair_sum(uint32_t r) {
   const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r));
   return f.x + f.y;
 }
-// mu_hat of the eight columns col..col+7 (col a multiple of 8): four 2-D codebook entries whose
-// indices start at a byte boundary of the index stream.
-__device__ __forceinline__ uint4 mu_vector(const uint8_t* mu, const uint8_t* mu_aux, uint32_t bits, int col) {
-  const uint32_t mask = (1u << bits) - 1u;
-  const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
-  const uint32_t* w = reinterpret_cast<const uint32_t*>(mu) + (byte >> 2);
-  const uint32_t sh = (byte & 3u) * 8u;
-  const uint32_t lo = __ldg(w);
-  const uint32_t hi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
-  const uint32_t f = __funnelshift_r(lo, hi, sh);
-  const uint32_t* cb = reinterpret_cast<const uint32_t*>(mu_aux);
-  return make_uint4(__ldg(cb + (f & mask)), __ldg(cb + ((f >> bits) & mask)), __ldg(cb + ((f >> (2 * bits)) & mask)),
-                    __ldg(cb + ((f >> (3 * bits)) & mask)));
-}
-// The three sums of a 128-column group the factored dequantisation needs, from the rounded fp16
-// values the tensor core will see: Sx = sum x and, negated, Bx_h = sum bias_h(col) * x for the two
-// row halves of a record.  Called by a half-warp whose lane l16 holds columns 8*l16..8*l16+7.
-__device__ __forceinline__ void group_sums(const uint4 v, int l16, float& sx, float& nb0, float& nb1) {
-  const int o = (8 * l16) & 63;
-  const float pa = pair_sum(v.x) + pair_sum(v.z), pb = pair_sum(v.y) + pair_sum(v.w);
-  sx = pa + pb;
-  nb0 = -fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
-  nb1 = -fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
-#pragma unroll
-  for (int d = 8; d > 0; d >>= 1) {
-    sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
-    nb0 += __shfl_xor_sync(0xFFFFFFFFu, nb0, d);
-    nb1 += __shfl_xor_sync(0xFFFFFFFFu, nb1, d);
-  }
-}
 
-// The consumer threads of a CTA mix the inputs of the phases [p0, p1) of a staging group into the
-// input area.  A thread owns 16-byte vectors (8 columns of one batch row of a slab) tid, tid + NT,
-// ... of the concatenated phases; x_prev and mu_hat of its first two vectors can be fetched BEFORE
-// the grid barrier is awaited, so that only one round of loads of x, the mix and the sums follow it.
-template <int CW>
-struct Stager {
-  static constexpr int NT = CW * 32, PRE = 2;
-  uint4 xp[PRE], mh[PRE];
+constexpr int kStageUnroll = 4;
 
-  // vector number v of the group -> phase, batch row, vector within the slab's row
-  __device__ __forceinline__ static const PhaseDesc* locate(const Env& e, uint32_t p0, uint32_t p1, int B, uint32_t v, int& b, int& c8) {
-    for (uint32_t p = p0; p < p1; ++p) {
-      const PhaseDesc* d = desc_slot(e, p);
-      const uint32_t nvr = d->T * 32u, nv = (uint32_t)B * nvr;
-      if (v < nv) { b = (int)(v / nvr); c8 = (int)(v - (uint32_t)b * nvr); return d; }
-      v -= nv;
+// This CTA's share of a stage's pre-pass.  A half-warp takes one (product, batch row, 128-column
+// group) at a time: it loads x (and x_prev, and decodes mu_hat), mixes, rounds to fp16, stores the
+// 128 values to the product's pre-pass rows and reduces the three sums of the group with shuffles.
+__device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
+  const int lane = stid & 31, l16 = lane & 15;
+  const uint32_t lo = ev.arr.grp_lo, hi = ev.arr.grp_hi;
+  const StepMixOp* ops = a.mixops + ev.arrd.op_first;
+  const int n_ops = (int)ev.arrd.op_count;
+  const int nbp = (a.B + 1) & ~1;
+  for (uint32_t g0 = lo + 2u * (uint32_t)(stid >> 5); g0 < hi; g0 += 2u * (uint32_t)kStagerWarps) {
+    const uint32_t gi = g0 + (uint32_t)(lane >> 4);
+    const bool valid = gi < hi;
+    uint32_t r = valid ? gi : lo;
+    int k = 0;
+    uint32_t icp = __ldg(&ops[0].ic_pad);
+    while (k + 1 < n_ops && r >= (uint32_t)a.B * (icp >> 7)) { r -= (uint32_t)a.B * (icp >> 7); ++k; icp = __ldg(&ops[k].ic_pad); }
+    const StepMixOp op = ops[k];
+    const uint32_t ng = op.ic_pad >> 7;
+    const int b = (int)(r / ng), grp = (int)(r % ng);
+    const int col = grp * 128 + l16 * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (col < (int)op.ic) {
+      v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + (size_t)b * op.ic + col));
+      if (op.mu) {
+        const uint4 pr = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.xprev) + (size_t)b * op.ic + col));
+        const uint32_t bits = op.mu_bits, mask = (1u << bits) - 1u;
+        // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
+        const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(op.mu) + (byte >> 2);
+        const uint32_t sh = (byte & 3u) * 8u;
+        const uint32_t wlo = __ldg(w);
+        const uint32_t whi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+        const uint32_t f = __funnelshift_r(wlo, whi, sh);
+        const uint32_t* cb = reinterpret_cast<const uint32_t*>(op.mu_aux);
+        v.x = mix2(v.x, pr.x, __ldg(cb + (f & mask)));
+        v.y = mix2(v.y, pr.y, __ldg(cb + ((f >> bits) & mask)));
+        v.z = mix2(v.z, pr.z, __ldg(cb + ((f >> (2 * bits)) & mask)));
+        v.w = mix2(v.w, pr.w, __ldg(cb + ((f >> (3 * bits)) & mask)));
+      }
     }
-    return nullptr;
-  }
-  __device__ __forceinline__ void before_barrier(const Env& e, uint32_t p0, uint32_t p1) {
+    if (valid) *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(a.scratch + op.dst_x) + (size_t)b * op.ic_pad + col) = v;
+    const int o = (8 * l16) & 63;
+    const float pa = pair_sum(v.x) + pair_sum(v.z), pb = pair_sum(v.y) + pair_sum(v.w);
+    float sx = pa + pb;
+    float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
+    float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
 #pragma unroll
-    for (int k = 0; k < PRE; ++k) {
-      int b, c8;
-      const PhaseDesc* d = locate(e, p0, p1, e.a.B, (uint32_t)(threadIdx.x + k * NT), b, c8);
-      xp[k] = make_uint4(0u, 0u, 0u, 0u); mh[k] = xp[k];
-      if (d && (d->kind_flags & DF_MU)) {
-        const int col = (int)d->kt0 * 256 + 8 * c8;
-        if (col < (int)d->ic) {
-          xp[k] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(d->xprev) + (size_t)b * d->ic + col));
-          mh[k] = mu_vector(reinterpret_cast<const uint8_t*>(d->mu), reinterpret_cast<const uint8_t*>(d->mu_aux), d->mu_bits, col);
+    for (int d = 8; d > 0; d >>= 1) {
+      sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+      t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
+      t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+    }
+    if (valid && l16 == 0 && op.sums) {
+      float* gs = reinterpret_cast<float*>(a.scratch + op.dst_sums);
+      gs[(grp * 3 + 0) * nbp + b] = sx;
+      gs[(grp * 3 + 1) * nbp + b] = t0;
+      gs[(grp * 3 + 2) * nbp + b] = t1;
+    }
+  }
+}
+
+// Stagers walk the CTA's event list.
+//  EV_ARRIVE: clear this CTA's slice of the next stage's outputs, then report the stage as done on
+//    the stagers' side (stage_report: the last of the consumer warps and the stagers to report
+//    adds this CTA's arrival to the grid barrier, so the arrival never waits for a role that is
+//    busy with something else).
+//  EV_SEGMENT: x_mix and, for SQ, the per-group sums of the segment, into buffer (segment number
+//    & 1).  The decoded token-shift vector mu_hat and the previous token's activations go to
+//    shared memory BEFORE the stage barrier, so that only one round of vector loads of x, the
+//    mix and the sums remain behind it.  A thread owns 8 consecutive columns (16 bytes) of one
+//    batch row; a half-warp owns one 128-column group, whose three sums it reduces with shuffles.
+template <bool MIX, int NB>
+__device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_t* xbufs, uint32_t* mucb,
+                            uint32_t e0, uint32_t e1) {
+  const int stid = threadIdx.x - kConsumerThreads;
+  const int lane = stid & 31;
+  volatile int* abortp = &ctrl->abort_flag;
+  uint32_t nseg = 0;          // segments staged so far
+  uint32_t passed2 = 0xFFFFFFFFu;   // second-stage barrier this CTA has already passed
+  bool ok = true;
+  for (uint32_t ei = e0; ei < e1; ++ei) {
+    const StepEvent ev = *reinterpret_cast<const StepEvent*>(reinterpret_cast<const uint8_t*>(a.events) + (size_t)ei * 64);
+    if (ev.kind == EV_ARRIVE) {
+#pragma unroll
+      for (int k = 0; k < 3; ++k) {
+        float* z = reinterpret_cast<float*>(ev.arr.zptr[k]);
+        for (uint32_t e = stid; e < ev.arrd.zcount[k]; e += kStagerThreads) z[e] = 0.f;
+      }
+      // the clearing stores of every stager thread must precede thread 0's fence
+      ok = named_bar_and(4, kStagerThreads, ok);
+      if (!ok) break;
+      // The stagers' part of the stage is done.  Barrier 0 (the clearing pass) has no consumer work
+      // before it: arrive directly.  Otherwise report; the last of the seventeen parties arrives.
+      if (stid == 0) {
+        if (ev.barrier == 0u) red_release_gpu(a.counter, 1u);
+        else if constexpr (NB == 2) ok = stage_wait_total_and_arrive(ctrl, a, ev.barrier, abortp);
+        else stage_report(ctrl, a, ev.barrier);
+      }
+      if constexpr (MIX) {
+        // once the barrier opens, do this CTA's share of the new stage's pre-pass and publish it
+        // through the stage's second barrier
+        if (ev.barrier < (uint32_t)a.n_stages) {
+          if (ok && stid == 0) {
+            uint32_t it = 0;
+            while ((int)(ld_acquire_gpu(a.counter + ev.barrier) - (a.target + a.wait_skew)) < 0) {
+              if (++it >= (a.poll_limit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
+            }
+          }
+          ok = named_bar_and(6, kStagerThreads, ok);   // thread 0's acquire precedes every thread's loads of x
+          if (!ok) break;
+          mix_slice(a, ev, stid);
+          named_bar_sync(4, kStagerThreads);           // every thread's pre-pass stores precede thread 0's release
+          if (stid == 0) red_release_gpu(a.counter + (uint32_t)a.n_stages + 1u + ev.barrier, 1u);
+        }
+      }
+      continue;
+    }
+    const int buf = (int)(nseg % XBufs<MIX, NB>::kCount);
+    // uniform verdict over all stager threads: the named barriers below must be reached by all or none
+    ok = named_bar_and(7, kStagerThreads, mbar_wait_warp(&ctrl->xempty[buf], ((nseg / XBufs<MIX, NB>::kCount) & 1u) ^ 1u, abortp, a.status) && ok);
+    uint8_t* xb = xbufs + (size_t)buf * XBufs<MIX, NB>::kBytes;
+    if constexpr (MIX) {
+      // The segment is a rectangle of the stage's pre-pass output: pass the stage's second barrier
+      // (once per stage), then fetch B rows and the block of sums with bulk copies.
+      const uint32_t b2 = (uint32_t)a.n_stages + ev.barrier;      // counter of the second barrier of stage ev.barrier - 1
+      if (ok && stid == 0 && b2 != passed2) {
+        uint32_t it = 0;
+        while ((int)(ld_acquire_gpu(a.counter + b2) - (a.target + a.wait_skew)) < 0) {
+          if (++it >= (a.poll_limit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
+        }
+      }
+      passed2 = b2;
+      ok = named_bar_and(6, kStagerThreads, ok);
+      if (ok && stid < 32) {
+        const uint32_t xstride = ev.xstride_sums & 0x7FFFFFFFu;
+        const uint32_t row_bytes = ev.segd.ncols * 2u;
+        const uint32_t sums_bytes = (ev.xstride_sums >> 31) ? (ev.segd.ncols >> 7) * 3u * (uint32_t)((a.B + 1) & ~1) * 4u : 0u;
+        // what other CTAs wrote with ordinary stores is read below by the copy engine
+        asm volatile("fence.proxy.async;" ::: "memory");
+        if (lane == 0) mbar_arrive_expect_tx(&ctrl->xfull[buf], (uint32_t)a.B * row_bytes + sums_bytes);
+        __syncwarp();
+        if (lane < a.B)
+          bulk_g2s_plain(xb + (size_t)lane * xstride, a.scratch + ev.seg.x + (size_t)lane * ev.segd.ic, row_bytes, &ctrl->xfull[buf]);
+        else if (lane == a.B && sums_bytes)
+          bulk_g2s_plain(xb + (size_t)a.B * xstride, a.scratch + ev.seg.xprev, sums_bytes, &ctrl->xfull[buf]);
+      } else if (lane == 0) {
+        mbar_arrive(&ctrl->xfull[buf]);      // the other stager warps (and everyone after a failure) only arrive
+      }
+      ++nseg;
+      if (!ok) break;
+      continue;
+    }
+    const uint8_t* mu = reinterpret_cast<const uint8_t*>(ev.seg.mu);
+    const __half* x = reinterpret_cast<const __half*>(ev.seg.x);
+    const __half* xp = reinterpret_cast<const __half*>(ev.seg.xprev);
+    const int ic = (int)ev.segd.ic, col0 = (int)ev.segd.col0;
+    const uint32_t xstride = ev.xstride_sums & 0x7FFFFFFFu;
+    const bool sums = (ev.xstride_sums >> 31) != 0;
+    const int nvr = (int)ev.segd.ncols >> 3;            // 16-byte vectors per batch row
+    const int total = a.B * nvr;
+    const int nbp = (a.B + 1) & ~1;
+    uint8_t* murow = xb + (size_t)ev.mu_off16 * 16;
+    if (ok && mu) {
+      for (int e = stid; e < (int)ev.segd.mu_entries; e += kStagerThreads) mucb[e] = __ldg(reinterpret_cast<const uint32_t*>(ev.seg.mu_aux) + e);
+      named_bar_sync(5, kStagerThreads);
+      const int bits = (int)ev.segd.mu_bits;
+      const uint32_t mask = (1u << bits) - 1u;
+      for (int c8 = stid; c8 < nvr; c8 += kStagerThreads) {
+        const int col = col0 + 8 * c8;
+        uint4 m = make_uint4(0u, 0u, 0u, 0u);
+        if (col < ic) {
+          // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
+          const uint32_t byte = (uint32_t)(col >> 1) * (uint32_t)bits >> 3;
+          const uint32_t* w = reinterpret_cast<const uint32_t*>(mu) + (byte >> 2);
+          const uint32_t sh = (byte & 3u) * 8u;
+          const uint32_t lo = __ldg(w);
+          const uint32_t hi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+          const uint32_t f = __funnelshift_r(lo, hi, sh);
+          m.x = mucb[f & mask];
+          m.y = mucb[(f >> bits) & mask];
+          m.z = mucb[(f >> (2 * bits)) & mask];
+          m.w = mucb[(f >> (3 * bits)) & mask];
+        }
+        *reinterpret_cast<uint4*>(murow + (size_t)c8 * 16) = m;
+      }
+      for (int v = stid; v < total; v += kStagerThreads) {
+        const int b = v / nvr, c8 = v - b * nvr;
+        const int col = col0 + 8 * c8;
+        uint4 r = make_uint4(0u, 0u, 0u, 0u);
+        if (col < ic) r = __ldg(reinterpret_cast<const uint4*>(xp + (size_t)b * ic + col));
+        *reinterpret_cast<uint4*>(xb + (size_t)b * xstride + (size_t)c8 * 16) = r;
+      }
+    }
+    if (ok && ev.barrier && stid == 0) {
+      // grid-wide stage barrier: every CTA has finished (and published) the previous stage.  Each
+      // barrier has its own arrival counter, so a CTA without work may run ahead and arrive at
+      // later barriers without releasing this one early.
+      uint32_t it = 0;
+      while ((int)(ld_acquire_gpu(a.counter + (ev.barrier - 1u)) - (a.target + a.wait_skew)) < 0) {
+        if (++it >= (a.poll_limit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
+      }
+    }
+    ok = named_bar_and(6, kStagerThreads, ok);   // uniform verdict; orders the mu row before its readers
+    if (ok) {
+      float* gs = reinterpret_cast<float*>(xb + (size_t)a.B * xstride);
+      for (int v0 = stid; v0 < total; v0 += kStagerThreads * kStageUnroll) {
+        uint4 raw[kStageUnroll];
+#pragma unroll
+        for (int u = 0; u < kStageUnroll; ++u) {
+          const int v = v0 + u * kStagerThreads;
+          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (v < total) {
+            const int b = v / nvr, c8 = v - b * nvr;
+            const int col = col0 + 8 * c8;
+            if (col < ic) raw[u] = __ldcg(reinterpret_cast<const uint4*>(x + (size_t)b * ic + col));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kStageUnroll; ++u) {
+          const int v = v0 + u * kStagerThreads;
+          if (v >= total) break;                      // warp-uniform: total is a multiple of 32
+          const int b = v / nvr, c8 = v - b * nvr;
+          uint4 r = raw[u];
+          uint8_t* dst = xb + (size_t)b * xstride + (size_t)c8 * 16;
+          if (mu) {
+            const uint4 pr = *reinterpret_cast<const uint4*>(dst);          // this thread's own earlier store
+            const uint4 mr = *reinterpret_cast<const uint4*>(murow + (size_t)c8 * 16);
+            r.x = mix2(r.x, pr.x, mr.x); r.y = mix2(r.y, pr.y, mr.y);
+            r.z = mix2(r.z, pr.z, mr.z); r.w = mix2(r.w, pr.w, mr.w);
+          }
+          *reinterpret_cast<uint4*>(dst) = r;
+          if (sums) {
+            const int o = (8 * c8) & 63;
+            const float pa = pair_sum(r.x) + pair_sum(r.z), pb = pair_sum(r.y) + pair_sum(r.w);
+            float sx = pa + pb;
+            float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
+            float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
+#pragma unroll
+            for (int d = 8; d > 0; d >>= 1) {
+              sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+              t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
+              t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+            }
+            if ((lane & 15) == 0) {
+              const int grp = c8 >> 4;
+              gs[(grp * 3 + 0) * nbp + b] = sx;
+              gs[(grp * 3 + 1) * nbp + b] = t0;
+              gs[(grp * 3 + 2) * nbp + b] = t1;
+            }
+          }
         }
       }
     }
-  }
-  // Mix, round and store one vector; reduce the group's sums.  Called by whole warps.
-  __device__ __forceinline__ static void finish_vector(const Env& e, const PhaseDesc* d, int b, int c8, bool pre, uint4 pr, uint4 m) {
-    const int lane = threadIdx.x & 31, nbp = e.a.nbp;
-    uint8_t* xarea = e.smem + e.a.off_x;
-    const int col = (int)d->kt0 * 256 + 8 * c8;
-    uint4 r = make_uint4(0u, 0u, 0u, 0u);
-    if (col < (int)d->ic) {
-      r = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(d->x) + (size_t)b * d->ic + col));
-      if (d->kind_flags & DF_MU) {
-        if (!pre) {
-          pr = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(d->xprev) + (size_t)b * d->ic + col));
-          m = mu_vector(reinterpret_cast<const uint8_t*>(d->mu), reinterpret_cast<const uint8_t*>(d->mu_aux), d->mu_bits, col);
-        }
-        r.x = mix2(r.x, pr.x, m.x); r.y = mix2(r.y, pr.y, m.y); r.z = mix2(r.z, pr.z, m.z); r.w = mix2(r.w, pr.w, m.w);
-      }
-    }
-    *reinterpret_cast<uint4*>(xarea + d->xoff + (size_t)b * d->xstride + (size_t)c8 * 16) = r;
-    if (d->kind_flags & DF_SUMS) {
-      float sx, nb0, nb1;
-      group_sums(r, lane & 15, sx, nb0, nb1);
-      if ((lane & 15) == 0) {
-        float* gs = reinterpret_cast<float*>(xarea + d->gsoff);
-        const int grp = c8 >> 4;
-        gs[(grp * 3 + 0) * nbp + b] = sx;
-        gs[(grp * 3 + 1) * nbp + b] = nb0;
-        gs[(grp * 3 + 2) * nbp + b] = nb1;
-      }
-    }
-  }
-  // A row is a multiple of 32 vectors, so a warp is inside one row of one phase or past the end:
-  // every branch below is warp-uniform.  `pre`: before_barrier has run for this group.
-  __device__ __forceinline__ void stage(const Env& e, uint32_t p0, uint32_t p1, bool pre) {
-#pragma unroll
-    for (int k = 0; k < PRE; ++k) {
-      int b = 0, c8 = 0;
-      const PhaseDesc* d = locate(e, p0, p1, e.a.B, (uint32_t)(threadIdx.x + k * NT), b, c8);
-      if (!d) return;
-      finish_vector(e, d, b, c8, pre, xp[k], mh[k]);
-    }
-    for (int k = PRE;; ++k) {
-      int b = 0, c8 = 0;
-      const PhaseDesc* d = locate(e, p0, p1, e.a.B, (uint32_t)(threadIdx.x + k * NT), b, c8);
-      if (!d) return;
-      finish_vector(e, d, b, c8, false, make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u));
-    }
-  }
-};
-
-// ---- consumer warps: the record loop ------------------------------------------------------------------
-
-// One 128-column group of an SQ record (16 rows) against the staged input:
-//   acc[b][row] += s * ( sum_cols (q+bias) x  -  Bx_h  -  z * Sx )
-// Two chains of four m16n8k16 steps each (even and odd steps) keep the dependent tensor-core
-// latency short; the first starts at -Bx_h (the bias every extracted half carries, from the
-// precomputed sums), so that after the steps only an add and two FMAs per output remain.
-// `w`: the group's six words; sz_lo / sz_hi: (s, z) fp16 pairs of rows g and g+8; xa[n]: byte
-// offset in shared memory of this lane's fragment of batch block n at the group's first column;
-// gs: byte offset of this lane's part of the group's sums [3][nbp].
-template <int NB>
-__device__ __forceinline__ void sq_group(const uint32_t (&w)[6], uint32_t sz_lo, uint32_t sz_hi, const uint32_t (&xa)[NB],
-                                         uint32_t gs, uint32_t gstride, float (&acc)[NB][4]) {
-  float c0[NB][4], c1[NB][4];
-#pragma unroll
-  for (int n = 0; n < NB; ++n) {
-    const float2 b0 = *reinterpret_cast<const float2*>(smem_base + gs + gstride + n * 32);
-    const float2 b1 = *reinterpret_cast<const float2*>(smem_base + gs + 2 * gstride + n * 32);
-    c0[n][0] = b0.x; c0[n][1] = b0.y; c0[n][2] = b1.x; c0[n][3] = b1.y;
-    c1[n][0] = c1[n][1] = c1[n][2] = c1[n][3] = 0.f;
-  }
-#pragma unroll
-  for (int ti = 0; ti < 2; ++ti) {
-    uint32_t r[16];
-    sq_unpack_triple(w[3 * ti], w[3 * ti + 1], w[3 * ti + 2], r);
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      const uint32_t afrag[4] = {r[4 * m], r[4 * m + 1], r[4 * m + 2], r[4 * m + 3]};
-#pragma unroll
-      for (int n = 0; n < NB; ++n) {
-        const uint2 bf = *reinterpret_cast<const uint2*>(smem_base + xa[n] + (4 * ti + m) * 32);
-        if (m & 1) mma_16816(c1[n], afrag, bf.x, bf.y); else mma_16816(c0[n], afrag, bf.x, bf.y);
-      }
-    }
-  }
-  const uint32_t nlo = sz_lo ^ 0x80000000u, nhi = sz_hi ^ 0x80000000u;   // (s, -z)
-  const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&nlo));
-  const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&nhi));
-#pragma unroll
-  for (int n = 0; n < NB; ++n) {
-    const float2 sx = *reinterpret_cast<const float2*>(smem_base + gs + n * 32);
-    acc[n][0] = fmaf(s0.x, fmaf(s0.y, sx.x, c0[n][0] + c1[n][0]), acc[n][0]);
-    acc[n][1] = fmaf(s0.x, fmaf(s0.y, sx.y, c0[n][1] + c1[n][1]), acc[n][1]);
-    acc[n][2] = fmaf(s1.x, fmaf(s1.y, sx.x, c0[n][2] + c1[n][2]), acc[n][2]);
-    acc[n][3] = fmaf(s1.x, fmaf(s1.y, sx.y, c0[n][3] + c1[n][3]), acc[n][3]);
+    __syncwarp();
+    // A stager that gave up still arrives, so that no consumer is left waiting on this barrier;
+    // the consumers stop at the abort flag.
+    if (lane == 0) mbar_arrive(&ctrl->xfull[buf]);
+    ++nseg;
+    if (!ok) break;
   }
 }
 
-// Eight tensor-core steps (HALF of a tile's columns) of a VQ record: every fragment register is one
-// lookup in the tile's codebook, which sits behind the record in the ring entry.
+// Six words of one 128-column group of the record of lane `lane` (planes of 512 bytes, 16 bytes
+// per lane): group 0 = words 0..5, group 1 = words 6..11.
+template <int GRP>
+__device__ __forceinline__ void sq_group_words(const uint8_t* rec, int lane, uint32_t (&w)[6]) {
+  if constexpr (GRP == 0) {
+    const uint4 p0 = *reinterpret_cast<const uint4*>(rec + lane * 16);
+    const uint2 p1 = *reinterpret_cast<const uint2*>(rec + 512 + lane * 16);
+    w[0] = p0.x; w[1] = p0.y; w[2] = p0.z; w[3] = p0.w; w[4] = p1.x; w[5] = p1.y;
+  } else {
+    const uint2 p1 = *reinterpret_cast<const uint2*>(rec + 512 + lane * 16 + 8);
+    const uint4 p2 = *reinterpret_cast<const uint4*>(rec + 1024 + lane * 16);
+    w[0] = p1.x; w[1] = p1.y; w[2] = p2.x; w[3] = p2.y; w[4] = p2.z; w[5] = p2.w;
+  }
+}
+
+// One 128-column group of the two records of a warp.  With one batch block (B <= 8) the input
+// fragments are loaded once and shared by both records; with two blocks that costs more
+// registers than a thread has, so the records are taken one after the other.
+template <int NB, int GRP>
+__device__ __forceinline__ void sq_pair(const uint32_t (&wa)[6], const uint32_t (&wb)[6], const uint4 sza, const uint4 szb,
+                                        bool has_b, const XLane& xl, float (&acca)[NB][4], float (&accb)[NB][4]) {
+  if constexpr (NB == 1) {
+    sq_group_mma2<NB, GRP>(wa, wb, sza, szb, has_b, xl, acca, accb);
+  } else {
+    sq_group_mma<NB, GRP>(wa, GRP == 0 ? sza.x : sza.y, GRP == 0 ? sza.z : sza.w, xl, acca);
+    if (has_b) sq_group_mma<NB, GRP>(wb, GRP == 0 ? szb.x : szb.y, GRP == 0 ? szb.z : szb.w, xl, accb);
+  }
+}
+
 template <int BITS, int NB, int HALF>
-__device__ __forceinline__ void vq_half(const uint32_t (&w)[2 * BITS], const uint32_t* cb, const uint32_t (&xa)[NB],
-                                        float (&acc)[NB][4]) {
-#pragma unroll
-  for (int j = 8 * HALF; j < 8 * HALF + 8; ++j) {
-    uint32_t afrag[4];
-#pragma unroll
-    for (int R = 0; R < 4; ++R) afrag[R] = cb[vq_index<BITS, 2 * BITS>(w, 4 * j + R)];
-#pragma unroll
-    for (int n = 0; n < NB; ++n) {
-      const uint2 bf = *reinterpret_cast<const uint2*>(smem_base + xa[n] + j * 32);
-      mma_16816(acc[n], afrag, bf.x, bf.y);
-    }
+__device__ __forceinline__ void vq_pair(const uint32_t (&wa)[2 * BITS], const uint32_t (&wb)[2 * BITS], const uint32_t* cb_lane,
+                                        const XLane& xl, float (&acca)[NB][4], float (&accb)[NB][4]) {
+  if constexpr (NB == 1) {
+    vq_half_mma2<BITS, NB, HALF>(wa, wb, cb_lane, xl, acca, accb);
+  } else {
+    vq_record_mma<BITS, NB, 8 * HALF, 8 * HALF + 8>(wa, cb_lane, xl, acca);
+    vq_record_mma<BITS, NB, 8 * HALF, 8 * HALF + 8>(wb, cb_lane, xl, accb);
   }
 }
 
-// 16-byte asynchronous copies global -> shared in per-thread groups.
-__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src, uint64_t policy) {
-  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "l"(policy) : "memory");
-}
-// The same copy by the lanes for which `on` holds, as one predicated instruction (no divergent branch).
-__device__ __forceinline__ void cp_async16_if(bool on, uint32_t dst_smem, const void* src, uint64_t policy) {
-  asm volatile("{\n .reg .pred p;\n setp.ne.u32 p, %3, 0;\n @p cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n}"
-               ::"r"(dst_smem), "l"(src), "l"(policy), "r"((uint32_t)on) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-// Wait until at most `pending` (0..6) of this thread's most recent groups are still in flight.
-__device__ __forceinline__ void cp_async_wait_pending(uint32_t pending) {
-  switch (pending) {
-    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-    case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
-    case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
-  }
-}
-
-// What a consumer warp carries from record to record.
-template <int NB>
-struct ConsumerState {
-  float acc[NB][4];
-  uint32_t infl;               // records whose copies are issued and not yet consumed
-  uint32_t slot, islot;        // ring entry of the next record to consume / to issue
-  uint32_t run_cons, run_iss;  // run headers read by the consuming / by the issuing side
-  const uint8_t* iss_src;      // issuing side: this lane's part of the next record of the current run
-  uint32_t iss_cb;             // ... its codebook, as an offset from iss_src (VQ)
-  uint32_t iss_left, iss_fmt;  // ... records left in the run; the run's format
-  int rowsel[NB];
-};
-
-template <int NB, int CW, bool TRACE>
-struct Consumer {
-  const Env& e;
-  Tracer<TRACE>& tr;
-  ConsumerState<NB>& s;
-  const uint32_t w, lane, g, t, depth, entry, ring, hq;   // ring / hq: byte offsets in shared memory
-  const uint64_t policy;
-
-  // Issue the copies of the next record (and of the codebook behind it) into ring entry islot as one
-  // group.  The entry is free: the warp itself has consumed what was in it.  When the current run is
-  // exhausted the next run header is taken, if the producer lane has written it.
-  __device__ __forceinline__ bool issue_one() {
-    if (s.iss_left == 0u) {
-      if ((int)(ld_acquire_cta(&e.ctrl->hq_head[w]) - s.run_iss) <= 0) return false;
-      const uint32_t hoff = hq + (s.run_iss % (uint32_t)kHeaderRing) * 32u;
-      const uint4 q1 = *reinterpret_cast<const uint4*>(smem_base + hoff + 16u);
-      s.iss_left = *reinterpret_cast<const uint32_t*>(smem_base + hoff + 8u) & 0x1FFu;
-      s.iss_fmt = q1.x & 3u;
-      s.iss_src = reinterpret_cast<const uint8_t*>(((uint64_t)q1.y << 32) | (q1.x & ~15u)) + lane * 16u;
-      s.iss_cb = q1.z;
-      ++s.run_iss;
-    }
-    const uint8_t* src = s.iss_src;
-    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_base) + ring + s.islot * entry + lane * 16u;
-    cp_async16(dst, src, policy);
-    cp_async16(dst + 512u, src + 512, policy);
-    cp_async16(dst + 1024u, src + 1024, policy);
-    if (s.iss_fmt == FMT_SQ3) {
-      cp_async16_if(lane < 8u, dst + 1536u, src + 1536, policy);
-      s.iss_src = src + 8 * RWKVQ_SQ_RECORD_BYTES;
-    } else if (s.iss_fmt == FMT_VQ6) {
-      cp_async16_if(lane < 16u, dst + 1536u, src + s.iss_cb, policy);
-      s.iss_src = src + 8 * 1536; s.iss_cb += 256u - 8u * 1536u;
+// Consumer warp `w` of group `grp`: units grp, grp + 2, ... of the CTA's list.
+template <int NB, bool MIX>
+__device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, const uint8_t* xbufs, uint8_t* replicas,
+                              uint32_t unit_base, uint32_t n_units, uint32_t ev_base, uint32_t n_events) {
+  bool dead = false;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = warp >> 3, w = warp & 7;
+  const int g = lane >> 2, t = lane & 3;
+  volatile int* abortp = &ctrl->abort_flag;
+  float acca[NB][4], accb[NB][4];
+#pragma unroll
+  for (int n = 0; n < NB; ++n)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) acca[n][k] = accb[n][k] = 0.f;
+  // Every consumer warp walks the CTA's event list in order -- it reports each stage it leaves and
+  // passes through each input segment, used or not -- so that the phases of the shared barriers
+  // advance in step for all sixteen warps.
+  int held = -1;              // input segment this warp currently holds
+  uint32_t seg_next = 0;      // number of segment events passed so far
+  uint32_t cur_ev = 0;        // last event processed (event 0 is the clearing arrival: nothing to do)
+  // Report the current stage as finished (stage_report).  The lanes' reductions into y are ordered
+  // before lane 0's report by the warp barrier; no lane fences at GPU scope itself: that would only
+  // add its latency to the end of every stage.
+  uint32_t next_bar = 1u;     // every CTA arrives at barriers 1, 2, ... in this order, once per stage
+  auto arrive_stage = [&]() {
+    __syncwarp();
+    if constexpr (NB == 2) {
+      if (lane == 0 && !dead) stage_report_total(ctrl);
     } else {
-      cp_async16(dst + 1536u, src + 1536, policy);
-      cp_async16(dst + 2048u, src + s.iss_cb, policy);
-      cp_async16(dst + 2560u, src + s.iss_cb + 512, policy);
-      s.iss_src = src + 8 * 2048; s.iss_cb += 1024u - 8u * 2048u;
+      if (lane == 0 && !dead) stage_report(ctrl, a, next_bar);
+      ++next_bar;
     }
-    cp_async_commit();
-    --s.iss_left; ++s.infl;
-    if (++s.islot == depth) s.islot = 0;
-    return true;
-  }
-  __device__ __forceinline__ void top_up() { while (s.infl < depth && issue_one()) {} }
-
-  // The rows of a finished slice: vals[j] holds element lane + 32*j of the slice's [batch][16 rows]
-  // block, summed over this CTA's slab.  One slab: these are the outputs.  Several: the sums go to
-  // the slab's scratch slot, and the last slab to arrive adds all slabs in slab order and stores the
-  // rows.
-  __device__ __forceinline__ void finish_slice(const PhaseDesc* d, uint32_t row, const float (&vals)[kMaxVals]) {
-    const StepArgs& a = e.a;
-    float* y = reinterpret_cast<float*>(d->y);
-    const uint32_t oc = d->oc, ks = d->ks_part & 0xFFFFu, nel = 16u * (uint32_t)a.B;
-    if (ks == 1u) {
-#pragma unroll
-      for (int j = 0; j < kMaxVals; ++j) {
-        const uint32_t el = lane + 32u * j;
-        if (el < nel) y[(size_t)(el >> 4) * oc + row + (el & 15u)] = vals[j];
-      }
-      return;
-    }
-    const uint32_t slot = d->gslot0 + ((row - d->row0) >> 4) * ks;
-    float* mine = a.gpart + (size_t)(slot + (d->ks_part >> 16)) * a.slot_floats;
-#pragma unroll
-    for (int j = 0; j < kMaxVals; ++j) {
-      const uint32_t el = lane + 32u * j;
-      if (el < nel) __stcg(mine + el, vals[j]);
-    }
-    // every lane's stores precede lane 0's release; whoever finds all the other slabs arrived
-    // acquires their stores with the same operation
+  };
+  auto release_held = [&]() {
     __syncwarp();
-    unsigned old = 0;
-    if (lane == 0) old = atom_add_acq_rel_gpu(a.gcnt + slot, 1u);
-    old = __shfl_sync(0xFFFFFFFFu, old, 0);
+    if (held >= 0 && lane == 0 && !dead) mbar_arrive(&ctrl->xempty[(uint32_t)held % XBufs<MIX, NB>::kCount]);
+    held = -1;
+  };
+  auto pass_segment = [&]() {   // a segment this warp does not use: observe it, hand it back
+    const uint32_t q = seg_next++;
+    if (!dead && !mbar_wait_warp(&ctrl->xfull[q % XBufs<MIX, NB>::kCount], (q / XBufs<MIX, NB>::kCount) & 1u, abortp, a.status)) dead = true;
     __syncwarp();
-    if (old + 1u == ks) {
-      if (lane == 0) a.gcnt[slot] = 0u;      // the next use lies behind a stage barrier
-      const float* all = a.gpart + (size_t)slot * a.slot_floats;
-#pragma unroll
-      for (int j = 0; j < kMaxVals; ++j) {
-        const uint32_t el = lane + 32u * j;
-        if (el < nel) {
-          float sum = 0.f;
-          for (uint32_t k = 0; k < ks; ++k) sum += __ldcg(all + (size_t)k * a.slot_floats + el);
-          y[(size_t)(el >> 4) * oc + row + (el & 15u)] = sum;
+    if (lane == 0 && !dead) mbar_arrive(&ctrl->xempty[q % XBufs<MIX, NB>::kCount]);
+  };
+  // Events (cur_ev, upto) in order; `mask` describes them when there are at most 32 and the planner
+  // could say so, otherwise (and for the tail of the list) the kinds are read from the plan, 32 at
+  // a time.
+  auto pass_events = [&](uint32_t upto, uint32_t mask, bool mask_valid) {
+    if (cur_ev + 1u >= upto) return;
+    release_held();
+    while (cur_ev + 1u < upto && !dead) {
+      const uint32_t first = cur_ev + 1u;
+      const uint32_t cnt = min(32u, upto - first);
+      uint32_t m = mask;
+      if (!mask_valid) {
+        bool arr = false;
+        if ((uint32_t)lane < cnt) {
+          const uint2 kb = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint8_t*>(a.events) + (size_t)(ev_base + first + lane) * 64 + 48));
+          arr = kb.x == EV_ARRIVE && kb.y > 0u;
         }
+        m = __ballot_sync(0xFFFFFFFFu, arr);
+      }
+      for (uint32_t j = 0; j < cnt && !dead; ++j) {
+        if ((m >> j) & 1u) arrive_stage(); else pass_segment();
+      }
+      cur_ev += cnt;
+      mask_valid = false;
+    }
+  };
+  uint8_t* rep = replicas + (size_t)grp * a.replica_bytes;
+  // slot and round of unit i (i % n_slots, i / n_slots), advanced without dividing
+  const uint32_t n_slots_u = (uint32_t)a.n_slots;
+  uint32_t slot_u = (uint32_t)grp % n_slots_u, round = (uint32_t)grp / n_slots_u;
+  for (uint32_t i = (uint32_t)grp; i < n_units; i += kGroups, slot_u += kGroups) {
+    while (slot_u >= n_slots_u) { slot_u -= n_slots_u; ++round; }
+    const int slot = (int)slot_u;
+    const uint8_t* sl = smem + kCtrlBytes + (size_t)slot * a.slot_bytes;
+    const StepUnit* u = reinterpret_cast<const StepUnit*>(sl);
+    if (!dead && !mbar_wait_warp(&ctrl->full[slot], round & 1u, abortp, a.status)) dead = true;
+    if (!dead && u->ev_index != cur_ev) {
+      const uint32_t target = u->ev_index;
+      pass_events(target, u->between_mask, target - cur_ev - 1u <= 32u);
+      if (!dead) {
+        release_held();
+        const uint32_t q = seg_next++;
+        held = (int)q;
+        cur_ev = target;
+        if (!mbar_wait_warp(&ctrl->xfull[q % XBufs<MIX, NB>::kCount], (q / XBufs<MIX, NB>::kCount) & 1u, abortp, a.status)) dead = true;
       }
     }
-  }
-
-  // The warp's n_runs runs of one phase, all of format FMT.  False after a failed wait.
-  template <int FMT>
-  __device__ __forceinline__ bool run(const PhaseDesc* d, uint32_t n_runs) {
-    const StepArgs& a = e.a;
-    const uint32_t gstride = (uint32_t)a.nbp * 4u, sums_tile = 6u * gstride;
-    const uint32_t slot0 = d->slot_set * 2u * (uint32_t)CW;
-    float* partial = reinterpret_cast<float*>(smem_base + a.off_partial);
-    uint32_t lane_x[NB];      // this lane's part of a fragment address: batch row and column quad
-#pragma unroll
-    for (int n = 0; n < NB; ++n) lane_x[n] = t * 8u + (uint32_t)s.rowsel[n] * d->xstride;
-    for (uint32_t r = 0; r < n_runs; ++r) {
-      // the run's header: the producer lane is normally far ahead; wait for it (bounded) if not
-      if ((int)(ld_acquire_cta(&e.ctrl->hq_head[w]) - s.run_cons) <= 0) {
-        bool ok = false;
-        for (uint32_t k = 0; k < (a.poll_limit << 4); ++k) {
-          if ((int)(ld_acquire_cta(&e.ctrl->hq_head[w]) - s.run_cons) > 0) { ok = true; break; }
-          if ((k & 63u) == 63u && *e.abortp) break;
-          __nanosleep(32);
+    if (dead) {
+      // A warp that gave up keeps walking the list only to keep the group's named barriers whole
+      // (the other warps stop at their next bounded wait); it touches neither slots nor outputs.
+      if (a.units[unit_base + i].flags & UF_VQ) { named_bar_sync(1 + grp, kGroupThreads); named_bar_sync(1 + grp, kGroupThreads); }
+      continue;
+    }
+    const uint32_t flags = u->flags;
+    const uint32_t by1 = u->bytes1;
+    const uint32_t after_count = u->after_count, after_mask = u->after_mask;
+    const uint8_t* data = sl + 128;
+    const uint8_t* xb = xbufs + (size_t)((uint32_t)held % XBufs<MIX, NB>::kCount) * XBufs<MIX, NB>::kBytes;
+    const uint32_t xstride = u->xstride, nbp = u->nbp, chb = u->chunk_bytes, rb = u->rec_bytes;
+    const uint32_t w0 = (flags >> 8) & 15u, w1 = (flags >> 12) & 15u;
+    const bool active = (uint32_t)w >= w0 && (uint32_t)w < w1;
+    const bool has_b = by1 != 0u;
+    const uint32_t oc = u->oc, row0 = u->row0;
+    float* y = reinterpret_cast<float*>(u->y);
+    const uint8_t* ra = data + (size_t)w * rb;
+    const uint8_t* rbp = data + chb + (size_t)w * rb;
+    if (!(flags & UF_VQ)) {
+      const uint32_t col = u->xcol0;
+      const XLane xl = make_xlane(xb + (size_t)col * 2, xstride,
+                                  reinterpret_cast<const float*>(xb + u->gs_off) + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
+      uint32_t wa[6], wb[6];
+      uint4 sza = make_uint4(0, 0, 0, 0), szb = sza;
+      if (active) {
+        sq_group_words<0>(ra, lane, wa);
+        sza = *reinterpret_cast<const uint4*>(ra + RWKVQ_SQ_CODE_BYTES + g * 16);
+        if (has_b) {
+          sq_group_words<0>(rbp, lane, wb);
+          szb = *reinterpret_cast<const uint4*>(rbp + RWKVQ_SQ_CODE_BYTES + g * 16);
         }
-        if (!ok) { if (!*e.abortp) give_up(e); return false; }
+        sq_pair<NB, 0>(wa, wb, sza, szb, has_b, xl, acca, accb);
+        sq_group_words<1>(ra, lane, wa);
+        if (has_b) sq_group_words<1>(rbp, lane, wb);
       }
-      const uint4 ha = *reinterpret_cast<const uint4*>(smem_base + hq + (s.run_cons % (uint32_t)kHeaderRing) * 32u);
-      const uint32_t flags = ha.z, n_items = flags & 0x1FFu;
-      uint32_t xa[NB];
-#pragma unroll
-      for (int n = 0; n < NB; ++n) xa[n] = ha.x + lane_x[n];
-      uint32_t gs = ha.y + t * 8u;
-#pragma unroll
-      for (int n = 0; n < NB; ++n)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) s.acc[n][k] = 0.f;
-      for (uint32_t it = 0; it < n_items; ++it) {
-        const long long t_w = tr.now();
-        if (s.infl == 0u) issue_one();                  // its header is there: cannot fail
-        cp_async_wait_pending(s.infl - 1u);
-        __syncwarp();                                   // every lane's part of the record has landed
-        tr.add(TR_WAIT_FULL, t_w);
-        const long long t_i = tr.now();
-        tr.count(TR_NITEMS);
-        const uint32_t rec = ring + s.slot * entry;
-        if (FMT == FMT_SQ3) {
-          const uint4 p0 = *reinterpret_cast<const uint4*>(smem_base + rec + lane * 16u);
-          const uint4 p1 = *reinterpret_cast<const uint4*>(smem_base + rec + 512u + lane * 16u);
-          const uint4 p2 = *reinterpret_cast<const uint4*>(smem_base + rec + 1024u + lane * 16u);
-          const uint4 sz = *reinterpret_cast<const uint4*>(smem_base + rec + (uint32_t)RWKVQ_SQ_CODE_BYTES + g * 16u);
-          // the record is in registers: once every lane has read its part, the entry is refilled
-          __syncwarp();
-          --s.infl; if (++s.slot == depth) s.slot = 0;
-          issue_one();
-          {
-            const uint32_t w0[6] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y};
-            sq_group<NB>(w0, sz.x, sz.z, xa, gs, gstride, s.acc);
-          }
-          {
-            uint32_t xb[NB];
-#pragma unroll
-            for (int n = 0; n < NB; ++n) xb[n] = xa[n] + 256u;
-            const uint32_t w1[6] = {p1.z, p1.w, p2.x, p2.y, p2.z, p2.w};
-            sq_group<NB>(w1, sz.y, sz.w, xb, gs + 3u * gstride, gstride, s.acc);
-          }
-        } else {
-          const uint8_t* recp = smem_base + rec;
-          if (FMT == FMT_VQ6) {
-            const uint32_t* cb = reinterpret_cast<const uint32_t*>(recp + 1536);
-            uint32_t v[12];
-            vq_half_words<6, 0>(recp, (int)lane, v);
-            vq_half_words<6, 1>(recp, (int)lane, v);
-            vq_half<6, NB, 0>(v, cb, xa, s.acc);
-            vq_half<6, NB, 1>(v, cb, xa, s.acc);
-          } else {
-            const uint32_t* cb = reinterpret_cast<const uint32_t*>(recp + 2048);
-            uint32_t v[16];
-            vq_half_words<8, 0>(recp, (int)lane, v);
-            vq_half<8, NB, 0>(v, cb, xa, s.acc);
-            vq_half_words<8, 1>(recp, (int)lane, v);
-            vq_half<8, NB, 1>(v, cb, xa, s.acc);
-          }
-          // the codebook is looked up in the entry until the last step
-          __syncwarp();
-          --s.infl; if (++s.slot == depth) s.slot = 0;
-          issue_one();
-        }
-#pragma unroll
-        for (int n = 0; n < NB; ++n) xa[n] += 512u;
-        gs += sums_tile;
-        tr.add(TR_ITEMS, t_i);
-      }
-      // The header is no longer needed by either side (the issuing side is past it): tell the producer lane.
-      ++s.run_cons;
-      st_release_cta(&e.ctrl->hq_tail[w], s.run_cons);   // every lane stores the same word
-      const long long t_f = tr.now();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl->empty[slot]);     // the rest of the records is in registers: free the slot
+      if (active) sq_pair<NB, 1>(wa, wb, sza, szb, has_b, xl, acca, accb);
+    } else {
+      // replicate the tile's codebook for conflict-free lookups (the eight warps of the group)
+      const uint32_t E = u->entries;
+      named_bar_sync(1 + grp, kGroupThreads);          // the group's previous lookups are done
       {
-        // The run's sums leave the registers through a slot of shared memory in [batch][16 rows]
-        // order: this warp's slot alone if the slice is its alone, else every holder's slot, added
-        // in warp order by whoever writes last.
-        const uint32_t ncon = (flags >> 16) & 0xFFu;
-        float* ps = partial + (size_t)(slot0 + 2u * w + ((flags >> 29) & 1u)) * a.slot_floats;
+        const uint32_t* cbraw = reinterpret_cast<const uint32_t*>(data + 2 * chb);
+        uint32_t* rp = reinterpret_cast<uint32_t*>(rep);
+        for (uint32_t idx = (uint32_t)(w * 32 + lane); idx < E * 32u; idx += kGroupThreads) rp[idx] = cbraw[idx >> 5];
+      }
+      named_bar_sync(1 + grp, kGroupThreads);
+      const uint32_t* cb_lane = reinterpret_cast<const uint32_t*>(rep) + lane;
+      const XLane xl = make_xlane(xb + (size_t)u->xcol0 * 2, xstride, nullptr, nbp, a.B, lane);
+      if (flags & UF_BITS8) {
+        uint32_t va[16], vb[16];
+        if (active) {
+          vq_half_words<8, 0>(ra, lane, va); vq_half_words<8, 0>(rbp, lane, vb);
+          vq_pair<8, NB, 0>(va, vb, cb_lane, xl, acca, accb);
+          vq_half_words<8, 1>(ra, lane, va); vq_half_words<8, 1>(rbp, lane, vb);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
+        if (active) vq_pair<8, NB, 1>(va, vb, cb_lane, xl, acca, accb);
+      } else {
+        uint32_t va[12], vb[12];
+        if (active) {
+          vq_half_words<6, 0>(ra, lane, va); vq_half_words<6, 0>(rbp, lane, vb);
+          vq_pair<6, NB, 0>(va, vb, cb_lane, xl, acca, accb);
+          vq_half_words<6, 1>(ra, lane, va); vq_half_words<6, 1>(rbp, lane, vb);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
+        if (active) vq_pair<6, NB, 1>(va, vb, cb_lane, xl, acca, accb);
+      }
+    }
+    if (flags & UF_FLUSH) {
+      if (active) {
 #pragma unroll
         for (int n = 0; n < NB; ++n)
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const int b = n * 8 + 2 * (int)t + (k & 1);
-            if (b < a.B) ps[b * 16 + (int)g + 8 * (k >> 1)] = s.acc[n][k];
+            const uint32_t row = row0 + (uint32_t)w * 16u + (uint32_t)g + 8u * (uint32_t)(k >> 1);
+            const int b = n * 8 + 2 * t + (k & 1);
+            if (b < a.B && row < oc) atomicAdd(y + (size_t)b * oc + row, acca[n][k]);
+            if (b < a.B && has_b && row + 128u < oc) atomicAdd(y + (size_t)b * oc + row + 128u, accb[n][k]);
           }
-        __syncwarp();
-        bool last = true;
-        uint32_t wlo = w, rfirst = (flags >> 29) & 1u;
-        if (ncon > 1u) {
-          uint32_t old = 0;
-          uint32_t* cnt = &e.ctrl->cnt[(flags >> 9) & (uint32_t)(kCnt - 1)];
-          if (lane == 0) old = smem_add_acq_rel(cnt, 1u);
-          old = __shfl_sync(0xFFFFFFFFu, old, 0);
-          __syncwarp();
-          last = old + 1u == ncon;
-          if (last && lane == 0) *cnt = 0u;
-          wlo = (flags >> 24) & 31u; rfirst = (flags >> 30) & 1u;
-        }
-        if (last) {
-          float vals[kMaxVals];
+      }
 #pragma unroll
-          for (int j = 0; j < kMaxVals; ++j) {
-            const uint32_t el = lane + 32u * j;
-            float sum = 0.f;
-            if (el < 16u * (uint32_t)a.B)
-              for (uint32_t k = 0; k < ncon; ++k)
-                sum += partial[(size_t)(slot0 + 2u * (wlo + k) + (k == 0u ? rfirst : 0u)) * a.slot_floats + el];
-            vals[j] = sum;
-          }
-          finish_slice(d, ha.w, vals);
-        }
-      }
-      tr.add(TR_FLUSH, t_f);
-    }
-    return true;
-  }
-};
-
-
-template <int NB, int CW, bool TRACE>
-__device__ void consumer_role(const Env& e) {
-  const StepArgs& a = e.a;
-  Tracer<TRACE> tr;
-  const long long t_begin = tr.now();
-  const uint32_t lane = threadIdx.x & 31u, w = threadIdx.x >> 5;
-  ConsumerState<NB> s;
+      for (int n = 0; n < NB; ++n)
 #pragma unroll
-  for (int n = 0; n < NB; ++n) {
-    s.rowsel[n] = min(8 * n + (int)(lane >> 2), a.B - 1);
-#pragma unroll
-    for (int k = 0; k < 4; ++k) s.acc[n][k] = 0.f;
+        for (int k = 0; k < 4; ++k) acca[n][k] = accb[n][k] = 0.f;
+    }
+    // the group's last unit of the stage: report the stage as finished without waiting for the next unit
+    if (after_count) pass_events(cur_ev + after_count + 1u, after_mask, true);
   }
-  s.infl = s.slot = s.islot = s.run_cons = s.run_iss = 0u;
-  s.iss_src = nullptr; s.iss_cb = 0u; s.iss_left = 0u; s.iss_fmt = 0u;
-  Consumer<NB, CW, TRACE> c{e, tr, s, w, lane, lane >> 2, lane & 3u, (uint32_t)a.depth, a.entry_bytes,
-                            a.off_ring + w * (uint32_t)a.depth * a.entry_bytes, a.off_hq + w * (uint32_t)kHeaderRing * 32u,
-                            policy_evict_first()};
-  uint32_t opened = 0;                 // stages this CTA has taken part in
-  uint32_t reported = 0;               // stages this warp has left
-  bool dead = false, verdict = false;  // verdict: the role's barrier has already told everyone to leave
-  Stager<CW> stager;
-
-  for (uint32_t p = 0;; ++p) {
-    {
-      const long long t0 = tr.now();
-      if (!wait_desc(e, p)) dead = true;
-      tr.add(TR_WAIT_DESC, t0);
-    }
-    if (dead) break;
-    const PhaseDesc* d = desc_slot(e, p);
-    const uint32_t kf = d->kind_flags;
-    if ((kf & 15u) == DK_END) break;
-    c.top_up();                        // the weight ring, before anything that may wait
-    if (kf & DF_GROUP) {
-      uint32_t p1 = p + 1;
-      while (true) {                   // the group's phases: p .. the one flagged last
-        if (!wait_desc(e, p1 - 1)) { dead = true; break; }
-        if (desc_slot(e, p1 - 1)->kind_flags & DF_GLAST) break;
-        ++p1;
-      }
-      if (dead) break;
-      if (kf & DF_FIRST) {
-        {
-          const long long t0 = tr.now();
-          stager.before_barrier(e, p, p1);
-          tr.add(TR_PRE, t0);
-        }
-        {
-          const long long t0 = tr.now();
-          if (!mbar_wait(e, &e.ctrl->open, opened & 1u)) dead = true;
-          tr.add(TR_WAIT_OPEN, t0);
-          if (threadIdx.x == 0) Tracer<TRACE>::stamp(a.trace, d->stage, 2);
-        }
-        ++opened;
-      } else {
-        // a later group of the stage reuses the input area: every warp must have left the earlier one
-        if (!named_bar_and(1, CW * 32, true)) { dead = true; verdict = true; break; }
-      }
-      const long long t1 = tr.now();
-      if (!dead) stager.stage(e, p, p1, (kf & DF_FIRST) != 0u);
-      // every consumer thread's stores precede the verdict; all leave together after a failure
-      if (!named_bar_and(1, CW * 32, !dead)) { dead = true; verdict = true; break; }
-      tr.add(TR_POST, t1);
-      if ((kf & DF_FIRST) && threadIdx.x == 0) {
-        Tracer<TRACE>::stamp(a.trace, d->stage, 3);
-        st_release_cta(&e.ctrl->desc_tail, p);
-      }
-    } else if (kf & DF_SYNC) {
-      // the phase reuses partial-sum slots or slice counters of an earlier phase of this stage: every
-      // warp must have left that phase (its slices are then reduced and stored)
-      if (!named_bar_and(1, CW * 32, true)) { dead = true; verdict = true; break; }
-    }
-    uint32_t i0, i1;
-    item_range<CW>(d->S * d->T, w, i0, i1);
-    const uint32_t n_runs = i1 > i0 ? (i1 - 1u) / d->T - i0 / d->T + 1u : 0u;   // slices the warp's share touches
-    const uint32_t fmt = (kf >> 4) & 3u;
-    bool ok;
-    if (fmt == FMT_SQ3) ok = c.template run<FMT_SQ3>(d, n_runs);
-    else if (fmt == FMT_VQ6) ok = c.template run<FMT_VQ6>(d, n_runs);
-    else ok = c.template run<FMT_VQ8>(d, n_runs);
-    if (!ok) { dead = true; break; }
-    if (kf & DF_LAST) {
-      // This warp has left the stage.  The count is an acquire-release read-modify-write at CTA scope
-      // and the publication a GPU-scope release by whoever reports last, so it is ordered after
-      // everything every warp stored before reporting: block-level synchronisation followed by one
-      // thread's release, the pattern of a cooperative grid barrier.
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t old = smem_add_acq_rel(&e.ctrl->warps_done, 1u);
-        if (old + 1u == (uint32_t)CW * (reported + 1u)) {
-          fence_gpu();
-          st_relaxed_gpu(a.flags + blockIdx.x, a.base + d->post_value);
-          Tracer<TRACE>::stamp(a.trace, d->stage, 0);
-        }
-      }
-      ++reported;
-    }
+  if (!dead) {
+    release_held();
+    pass_events(n_events, 0u, false);     // the rest of the list: later stages this warp has no unit in
   }
-  // no copy of this warp may still be landing when the CTA's shared memory is given up
-  cp_async_wait_all();
-  if (dead && !verdict) named_bar_and(1, CW * 32, false);   // keep the role's barrier whole: the others leave through this verdict
-  tr.add(TR_TOTAL, t_begin);
-  tr.store(a.trace);
 }
 
-template <int NB, int CW, bool TRACE>
-__global__ void __launch_bounds__((CW + 2) * 32, 1) step_kernel(const StepArgs a) {
-  uint8_t* smem = smem_base;
+template <int NB, bool MIX>
+__global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
+  uint8_t* xbufs = smem + kCtrlBytes + (size_t)a.n_slots * a.slot_bytes;
+  uint32_t* mucb = reinterpret_cast<uint32_t*>(xbufs + kXBufTotal);
+  uint8_t* replicas = reinterpret_cast<uint8_t*>(mucb) + kMuScratch;
   if (threadIdx.x == 0) {
-    mbar_init(&ctrl->open, 1);
-    for (int k = 0; k < kMaxCW; ++k) { ctrl->hq_head[k] = 0u; ctrl->hq_tail[k] = 0u; }
-    ctrl->warps_done = 0u; ctrl->desc_hi = 0u; ctrl->desc_tail = 0u; ctrl->prod_tail = 0u; ctrl->abort_flag = 0;
-    for (int k = 0; k < kCnt; ++k) ctrl->cnt[k] = 0u;
+    for (int s = 0; s < a.n_slots; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], kGroupWarps); }
+    for (int b = 0; b < 4; ++b) { mbar_init(&ctrl->xfull[b], kStagerWarps); mbar_init(&ctrl->xempty[b], kConsumerWarps); }
+    for (int k = 0; k < 64; ++k) ctrl->stage_cnt[k] = 0u;
+    ctrl->cdone = 0u;
+    ctrl->abort_flag = 0;
+    ctrl->poll_limit = (int)a.poll_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  const Env e{a, smem, ctrl, &ctrl->abort_flag};
+  const uint32_t u0 = a.unit_off[blockIdx.x], u1 = a.unit_off[blockIdx.x + 1];
+  const uint32_t e0 = a.event_off[blockIdx.x], e1 = a.event_off[blockIdx.x + 1];
   const int warp = threadIdx.x >> 5;
-  if (warp < CW) consumer_role<NB, CW, TRACE>(e);
-  else if (warp == CW) producer_role<CW, TRACE>(e);
-  else aux_role<TRACE>(e);
+  if (warp < kConsumerWarps) {
+    consumer_role<NB, MIX>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
+  } else if (warp < kConsumerWarps + kStagerWarps) {
+    stager_role<MIX, NB>(a, smem, ctrl, xbufs, mucb, e0, e1);
+  } else {
+    producer_role(a, smem, ctrl, u0, u1);
+  }
 }
 
 // ---- host planner --------------------------------------------------------------------------------
 
 struct PlanInfo {
-  int P, B, NB, CW, depth, n_stages;
-  unsigned runs;        // launches since the flags were last zero
-  unsigned abort_epoch; // value of the abort epoch when the flags were last known good
-  uint32_t poll_limit, wait_skew, n_sets;
-  void* trace_dev;      // rwkvq_step_trace: where the next runs write their per-warp counters
-  uint32_t entry_bytes, slot_floats, smem_bytes, off_hq, off_partial, off_x, off_ring;
-  size_t off_desc_off, off_init_post, off_descs, off_flags, off_gcnt, off_gpart, total_bytes;
-  uint32_t n_descs, gslots;
+  int P, B, NB, n_slots, n_stages, mix;
+  unsigned runs;        // launches since the counters were last zero
+  unsigned abort_epoch; // value of the abort epoch when the counters were last known good
+  uint32_t poll_limit, wait_skew;
+  uint32_t slot_bytes, replica_bytes, smem_bytes;
+  size_t off_unit_off, off_event_off, off_units, off_events, off_counter, off_mixops, off_scratch, total_bytes;
+  uint32_t n_units, n_events, n_barriers;
 };
 
 static std::mutex g_plan_mutex;
 static std::unordered_map<const void*, PlanInfo> g_plans;
+
+struct HostUnit {
+  StepUnit u;
+  int op, tr, kt, stage, w0, w1;
+};
+
+// Shared-memory footprint of an input segment: B rows of x_mix, the per-group sums (SQ) and one
+// row of decoded mu_hat (products with a token shift).
+static uint32_t xseg_mu_off(int B, int ncols, bool sums) {
+  uint32_t xstride = (uint32_t)ncols * 2u + 32u;
+  uint32_t nbp = (uint32_t)((B + 1) & ~1);
+  // 64 bytes of slack: lanes of batch columns that do not exist read (and discard) sums past the table
+  uint32_t off = (uint32_t)B * xstride + (sums ? (uint32_t)(ncols / 128) * 3u * nbp * 4u + 64u : 0u);
+  return (off + 15u) & ~15u;
+}
+static uint32_t xseg_bytes(int B, int ncols, bool sums, bool has_mu) {
+  return xseg_mu_off(B, ncols, sums) + (has_mu ? (uint32_t)ncols * 2u : 0u);
+}
 
 static rwkvq_status validate_ops(const rwkvq_gemv_op* ops, int n_ops, int B) {
   if (!ops || n_ops <= 0 || B < 1 || B > 16) return RWKVQ_EINVAL;
@@ -1061,35 +906,40 @@ static rwkvq_status validate_ops(const rwkvq_gemv_op* ops, int n_ops, int B) {
       if (!aligned16(o.mu_image_dev) || !aligned16(o.xprev_fp16_dev)) return RWKVQ_EALIGN;
     }
     if (!aligned16(o.W_image_dev) || !aligned16(o.x_fp16_dev) || !aligned16(o.y_dev)) return RWKVQ_EALIGN;
-    if (o.y_dtype != RWKVQ_F32) return RWKVQ_EUNSUPPORTED;   // the step writes fp32 outputs
+    if (o.y_dtype != RWKVQ_F32) return RWKVQ_EUNSUPPORTED;   // partial sums are added with fp32 atomics
     if (i > 0 && o.stage < ops[i - 1].stage) return RWKVQ_EINVAL;
   }
   return RWKVQ_OK;
 }
 
-static int fmt_of(const rwkvq_desc& d) { return d.method == RWKVQ_SQ ? FMT_SQ3 : d.bits == 6 ? FMT_VQ6 : FMT_VQ8; }
-
-// Input-area footprint of a slab of `cols` columns: B rows of fp16 values plus 32 bytes of padding
-// each (the 8-byte fragment loads of a half-warp then hit 16 distinct bank pairs), the group
-// sums, and 64 bytes of slack that lanes of batch columns which do not exist read (and discard).
-static uint32_t xrows_bytes(int B, uint32_t cols) { return (uint32_t)B * (cols * 2u + 32u); }
-static uint32_t xsums_bytes(int nbp, uint32_t cols, bool sums) { return sums ? (cols / 128u) * 3u * (uint32_t)nbp * 4u + 64u : 0u; }
-static uint32_t xseg_bytes(int B, int nbp, uint32_t cols, bool sums) { return (xrows_bytes(B, cols) + xsums_bytes(nbp, cols, sums) + 15u) & ~15u; }
-
-struct CtaPhase {
-  int op;
-  uint32_t slab, row0, S;
-};
-
 // Builds the whole plan on the host.  Returns the serialized image in `out` and fills `info`.
 static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P, std::vector<uint8_t>* out, PlanInfo* info) {
   rwkvq_status st = validate_ops(ops, n_ops, B);
   if (st != RWKVQ_OK) return st;
-  const int NB = B <= 8 ? 1 : 2;
-  const int CW = kConsumerWarps;
+  bool has_vq6 = false, has_vq8 = false, has_sq = false;
+  for (int i = 0; i < n_ops; ++i) {
+    if (ops[i].W_desc.method == RWKVQ_SQ) has_sq = true;
+    else if (ops[i].W_desc.bits == 6) has_vq6 = true;
+    else has_vq8 = true;
+  }
+  uint32_t data_max = 0;
+  if (has_sq) data_max = std::max(data_max, 2u * 8u * RWKVQ_SQ_RECORD_BYTES);
+  if (has_vq6) data_max = std::max(data_max, 2u * 8u * 1536u + 256u);
+  if (has_vq8) data_max = std::max(data_max, 2u * 8u * 2048u + 1024u);
+  info->slot_bytes = (128u + data_max + 127u) & ~127u;
+  info->replica_bytes = has_vq8 ? 256u * 128u : has_vq6 ? 64u * 128u : 0u;   // per consumer group
+  const uint32_t fixed = kCtrlBytes + kXBufTotal + kMuScratch + (uint32_t)kGroups * info->replica_bytes;
+  int ns = (int)((kSmemLimit - fixed) / info->slot_bytes);
+  if (ns > kMaxSlots) ns = kMaxSlots;
+  if (ns < 2) return RWKVQ_EUNSUPPORTED;
+  info->n_slots = ns;
+  info->smem_bytes = fixed + (uint32_t)ns * info->slot_bytes;
+  info->P = P; info->B = B; info->NB = B <= 8 ? 1 : 2;
+  info->poll_limit = kDefaultPollLimit; info->wait_skew = 0;
+  const bool mix = B >= 4;     // see StepArgs::mix
+  const uint32_t xbuf_bytes = mix && B <= 8 ? XBufs<true, 1>::kBytes : XBufs<false, 1>::kBytes;
+  info->mix = mix ? 1 : 0;
   const uint32_t nbp = (uint32_t)((B + 1) & ~1);
-  info->P = P; info->B = B; info->NB = NB; info->CW = CW;
-  info->poll_limit = kDefaultPollLimit; info->wait_skew = 0; info->trace_dev = nullptr;
 
   std::vector<std::pair<int, int>> stage_ranges;  // [first op, last op) per distinct stage value
   for (int i = 0; i < n_ops;) {
@@ -1099,180 +949,328 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     i = j;
   }
   const int n_stages = (int)stage_ranges.size();
-  if (n_stages >= 65535) return RWKVQ_EUNSUPPORTED;
+  if ((uint32_t)n_stages + 1u > kMaxBarriers) return RWKVQ_EUNSUPPORTED;   // per-barrier counts in the control block
   info->n_stages = n_stages;
+  info->n_barriers = ((uint32_t)n_stages + 1) * (mix ? 2u : 1u);   // the pre-pass has a barrier of its own per stage
 
-  // 1. K slabs: T tiles per slab, the largest divisor of KT whose inputs fit one segment of the input area
-  const uint32_t kSegCap = 36u * 1024u, kAreaCap = B <= 8 ? 72u * 1024u : 36u * 1024u;
-  std::vector<uint32_t> slab_tiles(n_ops, 1);
-  for (int i = 0; i < n_ops; ++i) {
-    const rwkvq_desc& d = ops[i].W_desc;
-    const uint32_t KT = (uint32_t)d.ic_pad / 256u;
-    for (uint32_t T = 1; T <= KT; ++T)
-      if (KT % T == 0 && xseg_bytes(B, (int)nbp, T * 256u, d.method == RWKVQ_SQ) <= kSegCap) slab_tiles[i] = T;
-  }
-
-  // 2. deal every stage's (slab, 16-row slice) units to the CTAs: contiguous in (product, slab, row)
-  //    order, balanced by cost (records x a weight per format: what a record costs a consumer warp)
-  std::vector<std::vector<std::vector<CtaPhase>>> deal(n_stages, std::vector<std::vector<CtaPhase>>(P));
-  for (int s = 0; s < n_stages; ++s) {
-    uint64_t total = 0;
-    auto unit_cost = [&](int o) -> uint64_t {
-      const rwkvq_desc& d = ops[o].W_desc;
-      const uint64_t wgt = d.method == RWKVQ_SQ ? 20u : d.bits == 8 ? 40u : 36u;
-      return (uint64_t)slab_tiles[o] * wgt;
-    };
-    for (int o = stage_ranges[s].first; o < stage_ranges[s].second; ++o)
-      total += unit_cost(o) * (uint64_t)(ops[o].W_desc.oc / 16) * (uint64_t)((uint32_t)ops[o].W_desc.ic_pad / 256u / slab_tiles[o]);
-    uint64_t run = 0;
-    const int rot = (int)(((uint64_t)s * 37u) % (uint64_t)P);   // idle CTAs of small stages are not always the same SMs
-    for (int o = stage_ranges[s].first; o < stage_ranges[s].second; ++o) {
-      const uint64_t c1 = unit_cost(o);
-      const int ns = ops[o].W_desc.oc / 16;
-      const uint32_t ks = (uint32_t)ops[o].W_desc.ic_pad / 256u / slab_tiles[o];
-      for (uint32_t k = 0; k < ks; ++k)
-        for (int sl = 0; sl < ns; ++sl) {
-          int c = (int)(((run + c1 / 2) * (uint64_t)P) / (total ? total : 1));
-          if (c >= P) c = P - 1;
-          c = (c + rot) % P;
-          std::vector<CtaPhase>& L = deal[s][c];
-          if (!L.empty() && L.back().op == o && L.back().slab == k && L.back().row0 + 16u * L.back().S == (uint32_t)sl * 16u) ++L.back().S;
-          else L.push_back(CtaPhase{o, k, (uint32_t)sl * 16u, 1u});
-          run += c1;
+  std::vector<std::vector<HostUnit>> cta_units(P);
+  std::vector<std::vector<StepEvent>> cta_arrivals(P);      // arrival events, one per barrier
+  bool too_many_ranges = false;
+  auto make_arrival = [&](int c, int stage_idx_to_clear, int barrier) {
+    StepEvent ev;
+    std::memset(&ev, 0, sizeof(ev));
+    ev.kind = EV_ARRIVE; ev.barrier = (uint32_t)barrier;
+    if (stage_idx_to_clear < n_stages) {
+      uint64_t total = 0;
+      for (int o = stage_ranges[stage_idx_to_clear].first; o < stage_ranges[stage_idx_to_clear].second; ++o)
+        total += (uint64_t)B * ops[o].W_desc.oc;
+      const uint64_t lo = total * (uint64_t)c / P, hi = total * (uint64_t)(c + 1) / P;
+      uint64_t base = 0;
+      int k = 0;
+      for (int o = stage_ranges[stage_idx_to_clear].first; o < stage_ranges[stage_idx_to_clear].second; ++o) {
+        const uint64_t n = (uint64_t)B * ops[o].W_desc.oc;
+        const uint64_t a0 = std::max(lo, base), a1 = std::min(hi, base + n);
+        if (a1 > a0) {
+          if (k >= 3) { too_many_ranges = true; break; }
+          ev.arr.zptr[k] = (uint64_t)(uintptr_t)ops[o].y_dev + (a0 - base) * 4;
+          ev.arrd.zcount[k] = (uint32_t)(a1 - a0);
+          ++k;
         }
-    }
-  }
-
-  // 3. scratch slots of the products with several slabs (one region, reused by every stage: a slice's
-  //    slots are read by the last slab to arrive before that CTA reports the stage)
-  std::vector<uint32_t> gslot_base(n_ops, 0);
-  uint32_t gslots = 0;
-  for (int s = 0; s < n_stages; ++s) {
-    uint32_t run = 0;
-    for (int o = stage_ranges[s].first; o < stage_ranges[s].second; ++o) {
-      const uint32_t ks = (uint32_t)ops[o].W_desc.ic_pad / 256u / slab_tiles[o];
-      gslot_base[o] = run;
-      if (ks > 1) run += (uint32_t)(ops[o].W_desc.oc / 16) * ks;
-    }
-    gslots = std::max(gslots, run);
-  }
-  info->gslots = gslots;
-
-  // 4. per-CTA descriptor lists; the input area is as large as the largest staging group
-  info->n_sets = B <= 3 ? 2u : 1u;
-  uint32_t xarea = 0;
-  std::vector<uint32_t> desc_off(P + 1, 0), init_post(P, 0);
-  std::vector<PhaseDesc> descs;
-  for (int c = 0; c < P; ++c) {
-    desc_off[c] = (uint32_t)descs.size();
-    // stages this CTA completes without consuming anything are reported with the previous stage
-    // that has items (or at the start of the launch)
-    std::vector<int> has_items(n_stages, 0);
-    for (int s = 0; s < n_stages; ++s) has_items[s] = deal[s][c].empty() ? 0 : 1;
-    int first_with = 0;
-    while (first_with < n_stages && !has_items[first_with]) ++first_with;
-    init_post[c] = (uint32_t)first_with;
-    for (int s = 0; s < n_stages; ++s) {
-      if (!has_items[s]) continue;
-      std::vector<CtaPhase> phases;
-      for (const CtaPhase& ph : deal[s][c])      // a phase's slices each own a counter
-        for (uint32_t s0 = 0; s0 < ph.S; s0 += (uint32_t)kCnt)
-          phases.push_back(CtaPhase{ph.op, ph.slab, ph.row0 + 16u * s0, std::min<uint32_t>((uint32_t)kCnt, ph.S - s0)});
-      int next_with = s + 1;
-      while (next_with < n_stages && !has_items[next_with]) ++next_with;
-      uint32_t xo = 0, cnt = 0;
-      for (size_t k = 0; k < phases.size(); ++k) {
-        const CtaPhase& ph = phases[k];
-        const rwkvq_gemv_op& op = ops[ph.op];
-        const rwkvq_desc& d = op.W_desc;
-        const uint8_t* img = static_cast<const uint8_t*>(op.W_image_dev);
-        const bool sq = d.method == RWKVQ_SQ;
-        const uint32_t T = slab_tiles[ph.op], KT = (uint32_t)d.ic_pad / 256u, ks = KT / T;
-        const uint32_t seg = xseg_bytes(B, (int)nbp, T * 256u, sq);
-        PhaseDesc pd;
-        std::memset(&pd, 0, sizeof(pd));
-        // the slice counters are reused once the stage has gone through all of them, the slots of
-        // partial sums when the stage has more phases than sets: every warp must then have left the
-        // phases that used them
-        bool sync = k >= info->n_sets;
-        if (cnt + ph.S > (uint32_t)kCnt) { cnt = 0; sync = true; }
-        bool group = k == 0;
-        if (xo + seg > kAreaCap) { group = true; xo = 0; }
-        if (group && k > 0) descs.back().kind_flags |= DF_GLAST;
-        pd.kind_flags = DK_PHASE | ((uint32_t)fmt_of(d) << 4) | (k == 0 ? DF_FIRST : 0u) | (k + 1 == phases.size() ? DF_LAST | DF_GLAST : 0u) |
-                        (op.mu_image_dev ? DF_MU : 0u) | (sq ? DF_SUMS : 0u) | (sync ? DF_SYNC : 0u) | (group ? DF_GROUP : 0u);
-        pd.slot_set = (uint32_t)(k % info->n_sets);
-        pd.stage = (uint32_t)s;
-        pd.src = (uint64_t)(uintptr_t)(img + RWKVQ_HEADER_BYTES);
-        pd.cb = sq ? 0 : (uint64_t)(uintptr_t)(img + matrix_aux_offset(&d));
-        pd.y = (uint64_t)(uintptr_t)op.y_dev;
-        pd.oc = (uint32_t)d.oc; pd.row0 = ph.row0; pd.S = ph.S; pd.KT = KT;
-        pd.T = T; pd.kt0 = ph.slab * T;
-        pd.cnt_base = cnt; cnt += ph.S;
-        pd.ks_part = ks | (ph.slab << 16);
-        pd.gslot0 = gslot_base[ph.op] + (ph.row0 / 16u) * ks;
-        pd.post_value = (uint32_t)next_with;
-        pd.ic = (uint32_t)d.ic;
-        pd.xoff = xo; pd.xstride = T * 512u + 32u;
-        pd.gsoff = xo + xrows_bytes(B, T * 256u);
-        xo += seg;
-        xarea = std::max(xarea, xo);
-        pd.x = (uint64_t)(uintptr_t)op.x_fp16_dev;
-        if (op.mu_image_dev) {
-          const uint8_t* mi = static_cast<const uint8_t*>(op.mu_image_dev);
-          pd.xprev = (uint64_t)(uintptr_t)op.xprev_fp16_dev;
-          pd.mu = (uint64_t)(uintptr_t)(mi + RWKVQ_HEADER_BYTES);
-          pd.mu_aux = (uint64_t)(uintptr_t)(mi + vector_aux_offset(&op.mu_desc));
-          pd.mu_bits = (uint16_t)op.mu_desc.bits; pd.mu_entries = (uint16_t)op.mu_desc.entries;
-        }
-        descs.push_back(pd);
+        base += n;
       }
     }
-    PhaseDesc end;
-    std::memset(&end, 0, sizeof(end));
-    end.kind_flags = DK_END;
-    descs.push_back(end);
-  }
-  desc_off[P] = (uint32_t)descs.size();
-  info->n_descs = (uint32_t)descs.size();
+    if (mix && barrier < n_stages) {
+      // this CTA's share of the pre-pass of stage `barrier`
+      uint64_t G = 0;
+      for (int o = stage_ranges[barrier].first; o < stage_ranges[barrier].second; ++o) G += (uint64_t)B * (ops[o].W_desc.ic_pad / 128);
+      ev.arr.grp_lo = (uint32_t)(G * (uint64_t)c / P); ev.arr.grp_hi = (uint32_t)(G * (uint64_t)(c + 1) / P);
+      ev.arrd.op_first = (uint16_t)stage_ranges[barrier].first;
+      ev.arrd.op_count = (uint16_t)(stage_ranges[barrier].second - stage_ranges[barrier].first);
+    }
+    cta_arrivals[c].push_back(ev);
+  };
+  for (int c = 0; c < P; ++c) make_arrival(c, 0, 0);   // barrier 0: the first stage's outputs are clear
 
-  // 5. shared-memory budget
-  bool has_vq6 = false, has_vq8 = false;
-  for (int i = 0; i < n_ops; ++i) {
-    if (ops[i].W_desc.method == RWKVQ_SQ) continue;
-    if (ops[i].W_desc.bits == 6) has_vq6 = true; else has_vq8 = true;
+  for (int s = 0; s < n_stages; ++s) {
+    std::vector<HostUnit> units;
+    for (int o = stage_ranges[s].first; o < stage_ranges[s].second; ++o) {
+      const rwkvq_desc& d = ops[o].W_desc;
+      const uint8_t* img = static_cast<const uint8_t*>(ops[o].W_image_dev);
+      const uint8_t* payload = img + RWKVQ_HEADER_BYTES;
+      const int KT = d.ic_pad / 256, MB = d.oc_pad / 128;
+      const bool vq = d.method != RWKVQ_SQ;
+      const uint32_t rb = vq ? rwkvq_vq_record_bytes(d.bits) : (uint32_t)RWKVQ_SQ_RECORD_BYTES;
+      const uint32_t cb = 8u * rb;
+      const uint8_t* aux = vq ? img + matrix_aux_offset(&d) : nullptr;
+      for (int tr = 0; tr < (MB + 1) / 2; ++tr)
+        for (int kt = 0; kt < KT; ++kt) {
+          HostUnit h;
+          std::memset(&h, 0, sizeof(h));
+          h.u.flags = vq ? (UF_VQ | (d.bits == 8 ? UF_BITS8 : 0)) : 0;
+          h.u.src0 = (uint64_t)(uintptr_t)(payload + (size_t)((2 * tr) * KT + kt) * cb);
+          h.u.bytes0 = cb;
+          if (2 * tr + 1 < MB) { h.u.src1 = (uint64_t)(uintptr_t)(payload + (size_t)((2 * tr + 1) * KT + kt) * cb); h.u.bytes1 = cb; }
+          if (vq) {
+            h.u.cb_src = (uint64_t)(uintptr_t)(aux + (size_t)(tr * KT + kt) * d.entries * 4);
+            h.u.cb_bytes = (uint32_t)d.entries * 4u; h.u.entries = (uint32_t)d.entries;
+          }
+          h.u.chunk_bytes = cb; h.u.rec_bytes = rb;
+          h.u.row0 = (uint32_t)tr * 256u; h.u.oc = (uint32_t)d.oc; h.u.y = (uint64_t)(uintptr_t)ops[o].y_dev;
+          h.u.stage = (uint32_t)s;
+          h.op = o; h.tr = tr; h.kt = kt; h.stage = s;
+          units.push_back(h);
+        }
+    }
+    // contiguous, cost-balanced ranges cut at one eighth of a unit (the records of one warp).  The
+    // cost of a unit is its record count weighted by what a record of its format costs the consumer
+    // warps (measured with every product in one stage: a VQ record with 64 entries takes about 1.45
+    // times, one with 256 entries about 1.25 times as long as an SQ record), so that the CTAs that
+    // get a stage's VQ matrix do not finish last.
+    auto cost_of = [&](const HostUnit& h) -> uint64_t {
+      const uint64_t recs = (h.u.bytes0 + h.u.bytes1) / h.u.rec_bytes;
+      const uint64_t wgt = !(h.u.flags & UF_VQ) ? 20u : (h.u.flags & UF_BITS8) ? 25u : 29u;
+      return recs * wgt * 64u;
+    };
+    // A consumer group spends about the same time on a piece of a unit as on a whole unit (the
+    // warps without a record idle), and every further input segment of a CTA costs about 1.7 us of
+    // serial staging; traces of all CTAs' barrier arrivals showed the stages waiting for the CTAs
+    // with the most pieces and segments, not for the most bytes.  So units are dealt WHOLE, and
+    // where it balances, row by row: each row of tiles (one product, one 256-row block: one input
+    // segment) gets a number of CTAs, greedily the row with the largest cost per CTA first, and
+    // its units are split into that many runs of neighbouring column tiles.  This is taken when no
+    // CTA ends up more than one unit above the even share; small stages leave some CTAs idle.
+    bool dealt = false;
+    auto push_whole = [&](int c, const HostUnit& h) {
+      HostUnit part = h;
+      part.w0 = 0; part.w1 = 8;
+      part.u.off0 = 0;
+      part.u.flags |= (0u << 8) | (8u << 12);
+      cta_units[c].push_back(part);
+    };
+    {
+      struct Row { size_t first, count; uint64_t cost; int k; };
+      std::vector<Row> rows;
+      for (size_t i = 0; i < units.size();) {
+        size_t j = i;
+        uint64_t cst = 0;
+        while (j < units.size() && units[j].op == units[i].op && units[j].tr == units[i].tr) { cst += cost_of(units[j]); ++j; }
+        rows.push_back(Row{i, j - i, cst, 1});
+        i = j;
+      }
+      if (!rows.empty() && rows.size() <= (size_t)P) {
+        int spare = P - (int)rows.size();
+        while (spare > 0) {
+          size_t best = rows.size();
+          uint64_t best_cost = 0;
+          for (size_t r = 0; r < rows.size(); ++r) {
+            if ((size_t)rows[r].k >= rows[r].count) continue;          // one unit per CTA at most
+            const uint64_t per = rows[r].cost / (uint64_t)rows[r].k;
+            if (per > best_cost) { best_cost = per; best = r; }
+          }
+          if (best == rows.size()) break;
+          ++rows[best].k; --spare;
+        }
+        size_t max_units = 0;
+        for (const Row& r : rows) max_units = std::max(max_units, (r.count + (size_t)r.k - 1) / (size_t)r.k);
+        const size_t even = (units.size() + (size_t)P - 1) / (size_t)P;
+        if (max_units <= even + 1) {
+          // start at a CTA that moves with the stage, so that idle CTAs are not always the same SMs
+          size_t c = ((size_t)s * 37u) % (size_t)P;
+          for (const Row& r : rows)
+            for (int q = 0; q < r.k; ++q) {
+              const size_t lo = r.count * (size_t)q / (size_t)r.k, hi = r.count * (size_t)(q + 1) / (size_t)r.k;
+              for (size_t i = lo; i < hi; ++i) push_whole((int)c, units[r.first + i]);
+              c = (c + 1) % (size_t)P;
+            }
+          dealt = true;
+        }
+      }
+    }
+    uint64_t total = 0;
+    for (const HostUnit& h : units) total += cost_of(h);
+    uint64_t run = 0;
+    auto cta_of = [&](uint64_t mid) {
+      int c = (int)((mid * (uint64_t)P) / (total ? total : 1));
+      return c >= P ? P - 1 : c;
+    };
+    const bool whole_units = units.size() >= (size_t)4 * (size_t)P;   // many units per CTA: a whole unit at its cost midpoint
+    for (const HostUnit& h : units) {
+      if (dealt) break;
+      if (whole_units) {
+        push_whole(cta_of(run + cost_of(h) / 2), h);
+        run += cost_of(h);
+        continue;
+      }
+      const uint64_t e8 = cost_of(h) / 8;
+      int w = 0;
+      while (w < 8) {
+        const int c = cta_of(run + (uint64_t)w * e8 + e8 / 2);
+        int w1 = w + 1;
+        while (w1 < 8 && cta_of(run + (uint64_t)w1 * e8 + e8 / 2) == c) ++w1;
+        HostUnit part = h;
+        part.w0 = w; part.w1 = w1;
+        const uint32_t rb = h.u.rec_bytes;
+        part.u.off0 = (uint32_t)w * rb;
+        part.u.src0 = h.u.src0 + (uint64_t)w * rb;
+        part.u.bytes0 = (uint32_t)(w1 - w) * rb;
+        if (h.u.bytes1) { part.u.src1 = h.u.src1 + (uint64_t)w * rb; part.u.bytes1 = (uint32_t)(w1 - w) * rb; }
+        part.u.flags |= ((uint32_t)w << 8) | ((uint32_t)w1 << 12);
+        cta_units[c].push_back(part);
+        w = w1;
+      }
+      run += cost_of(h);
+    }
+    for (int c = 0; c < P; ++c) make_arrival(c, s + 1, s + 1);
   }
-  uint32_t entry = RWKVQ_SQ_RECORD_BYTES;
-  if (has_vq6) entry = std::max(entry, 1536u + 256u);
-  if (has_vq8) entry = std::max(entry, 2048u + 1024u);
-  info->entry_bytes = entry;
-  info->slot_floats = 16u * (uint32_t)B;
-  info->off_hq = kCtrlBytes + kDescBytes;
-  info->off_partial = info->off_hq + (uint32_t)CW * kHeaderRing * 32u;
-  // Two sets of partial-sum slots where they are small, so that a CTA's second phase of a stage
-  // starts without waiting for the first one's slices to be reduced.
-  info->off_x = (info->off_partial + info->n_sets * 2u * (uint32_t)CW * info->slot_floats * 4u + 127u) & ~127u;
-  xarea = (xarea + 127u) & ~127u;
-  info->off_ring = info->off_x + xarea;
-  if (info->off_ring + (uint32_t)CW * 2u * entry > kSmemLimit) return RWKVQ_EUNSUPPORTED;
-  int depth = (int)((kSmemLimit - info->off_ring) / ((uint32_t)CW * entry));
-  if (depth > 6) depth = 6;   // cp_async_wait_pending counts up to six groups in flight
-  info->depth = depth;
-  info->smem_bytes = info->off_ring + (uint32_t)CW * (uint32_t)depth * entry;
+  if (too_many_ranges) return RWKVQ_EUNSUPPORTED;   // a CTA's slice of a stage's outputs may touch at most three products
 
+  // pre-pass outputs: one region, reused by every stage (a stage's pre-pass starts only after the
+  // previous stage, and with it every copy out of the region, has finished everywhere)
+  std::vector<uint64_t> mix_x_off(n_ops, 0), mix_sums_off(n_ops, 0);
+  std::vector<StepMixOp> mixops(mix ? n_ops : 0);
+  uint64_t scratch_bytes = 0;
+  if (mix) {
+    for (int st_i = 0; st_i < n_stages; ++st_i) {
+      uint64_t off = 0;
+      for (int o = stage_ranges[st_i].first; o < stage_ranges[st_i].second; ++o) {
+        const rwkvq_gemv_op& op = ops[o];
+        mix_x_off[o] = off; off += round_up_sz((size_t)B * op.W_desc.ic_pad * 2, 256);
+        mix_sums_off[o] = off; off += round_up_sz((size_t)(op.W_desc.ic_pad / 128) * 3 * nbp * 4, 256);
+        StepMixOp& m = mixops[o];
+        std::memset(&m, 0, sizeof(m));
+        m.x = (uint64_t)(uintptr_t)op.x_fp16_dev;
+        if (op.mu_image_dev) {
+          const uint8_t* mi = static_cast<const uint8_t*>(op.mu_image_dev);
+          m.xprev = (uint64_t)(uintptr_t)op.xprev_fp16_dev;
+          m.mu = (uint64_t)(uintptr_t)(mi + RWKVQ_HEADER_BYTES);
+          m.mu_aux = (uint64_t)(uintptr_t)(mi + vector_aux_offset(&op.mu_desc));
+          m.mu_bits = (uint16_t)op.mu_desc.bits; m.mu_entries = (uint16_t)op.mu_desc.entries;
+        }
+        m.dst_x = mix_x_off[o]; m.dst_sums = mix_sums_off[o];
+        m.ic = (uint32_t)op.W_desc.ic; m.ic_pad = (uint32_t)op.W_desc.ic_pad;
+        m.sums = op.W_desc.method == RWKVQ_SQ ? 1 : 0;
+      }
+      scratch_bytes = std::max(scratch_bytes, off);
+    }
+  }
+  std::vector<uint32_t> unit_off(P + 1, 0), event_off(P + 1, 0);
+  std::vector<StepUnit> all_units;
+  std::vector<StepEvent> all_events;
+  for (int c = 0; c < P; ++c) {
+    std::vector<HostUnit>& L = cta_units[c];
+    unit_off[c] = (uint32_t)all_units.size();
+    event_off[c] = (uint32_t)all_events.size();
+    const size_t n = L.size();
+    // a group accumulates along K in registers while its consecutive units stay on the same rows
+    for (size_t i = 0; i < n; ++i) {
+      const size_t j = i + kGroups;
+      const bool same_run = j < n && L[j].stage == L[i].stage && L[j].op == L[i].op && L[j].tr == L[i].tr &&
+                            L[j].w0 == L[i].w0 && L[j].w1 == L[i].w1;
+      if (!same_run) L[i].u.flags |= UF_FLUSH;
+    }
+    all_events.push_back(cta_arrivals[c][0]);
+    uint32_t seg_no = 0;
+    size_t i = 0;
+    for (int s = 0; s < n_stages; ++s) {
+      // segments: maximal runs of units of one product whose column span fits the buffer
+      while (i < n && L[i].stage == s) {
+        const int op = L[i].op;
+        const bool sums = ops[op].W_desc.method == RWKVQ_SQ;
+        const bool has_mu = !mix && ops[op].mu_image_dev != nullptr;   // copied segments carry no mu row
+        int kmin = L[i].kt, kmax = L[i].kt + 1;
+        size_t j = i + 1, last = i;
+        // A segment is a contiguous run of column tiles (a range that wraps from the end of one row
+        // pair to the start of the next starts a new segment) that fits the buffer.
+        while (j < n && L[j].op == op && L[j].stage == s) {
+          if (L[j].kt < kmin || L[j].kt > kmax) break;
+          const int nmax = std::max(kmax, L[j].kt + 1);
+          if (xseg_bytes(B, (nmax - kmin) * 256, sums, has_mu) > xbuf_bytes) break;
+          kmax = nmax; last = j; ++j;
+        }
+        const int ncols = (kmax - kmin) * 256;
+        if (xseg_bytes(B, ncols, sums, has_mu) > xbuf_bytes) return RWKVQ_EUNSUPPORTED;
+        StepEvent ev;
+        std::memset(&ev, 0, sizeof(ev));
+        const rwkvq_gemv_op& o = ops[op];
+        ev.kind = EV_SEGMENT;
+        ev.seg.x = (uint64_t)(uintptr_t)o.x_fp16_dev;
+        ev.segd.ic = (uint32_t)o.W_desc.ic; ev.segd.col0 = (uint32_t)kmin * 256u; ev.segd.ncols = (uint32_t)ncols;
+        const uint32_t xstride = (uint32_t)ncols * 2u + 32u;
+        ev.xstride_sums = xstride | (sums ? 0x80000000u : 0u);
+        ev.mu_off16 = (uint16_t)(xseg_mu_off(B, ncols, sums) / 16u);
+        ev.barrier = (uint32_t)s + 1u;   // stage s reads its inputs after barrier s
+        if (mix) {
+          ev.seg.x = mix_x_off[op] + (uint64_t)kmin * 512u;
+          ev.seg.xprev = mix_sums_off[op] + (uint64_t)(kmin * 2) * 3u * nbp * 4u;
+          ev.segd.ic = (uint32_t)o.W_desc.ic_pad * 2u;
+        } else if (has_mu) {
+          const uint8_t* m = static_cast<const uint8_t*>(o.mu_image_dev);
+          ev.seg.xprev = (uint64_t)(uintptr_t)o.xprev_fp16_dev;
+          ev.seg.mu = (uint64_t)(uintptr_t)(m + RWKVQ_HEADER_BYTES);
+          ev.seg.mu_aux = (uint64_t)(uintptr_t)(m + vector_aux_offset(&o.mu_desc));
+          ev.segd.mu_bits = (uint16_t)o.mu_desc.bits; ev.segd.mu_entries = (uint16_t)o.mu_desc.entries;
+        }
+        for (size_t k = i; k <= last; ++k) {
+          L[k].u.seg = seg_no;
+          L[k].u.ev_index = (uint32_t)(all_events.size() - event_off[c]);
+          L[k].u.xcol0 = (uint32_t)(L[k].kt - kmin) * 256u;
+          L[k].u.xstride = xstride; L[k].u.gs_off = (uint32_t)B * xstride; L[k].u.nbp = nbp;
+        }
+        all_events.push_back(ev);
+        ++seg_no;
+        i = last + 1;
+      }
+      all_events.push_back(cta_arrivals[c][s + 1]);
+    }
+    // what each group has to pass between its consecutive segments, and after its last unit of a stage
+    uint32_t prev_ev[kGroups] = {0, 0};
+    const StepEvent* evs = all_events.data() + event_off[c];
+    const uint32_t n_ev = (uint32_t)(all_events.size() - event_off[c]);
+    std::vector<uint32_t> arr_idx(n_stages, 0);
+    for (uint32_t e = 0; e < n_ev; ++e)
+      if (evs[e].kind == EV_ARRIVE && evs[e].barrier > 0u) arr_idx[evs[e].barrier - 1u] = e;
+    auto mask_of = [&](uint32_t first, uint32_t last_excl) {
+      uint32_t mask = 0;
+      for (uint32_t e = first; e < last_excl; ++e)
+        if (evs[e].kind == EV_ARRIVE && evs[e].barrier > 0u) mask |= 1u << (e - first);
+      return mask;
+    };
+    for (size_t k = 0; k < n; ++k) {
+      const int gidx = (int)(k % kGroups);
+      const uint32_t target = L[k].u.ev_index;
+      L[k].u.between_mask = (target > prev_ev[gidx] && target - prev_ev[gidx] - 1u <= 32u) ? mask_of(prev_ev[gidx] + 1u, target) : 0u;
+      prev_ev[gidx] = target;
+      const bool last_of_stage = k + kGroups >= n || L[k + kGroups].stage != L[k].stage;
+      const uint32_t arr = arr_idx[L[k].stage];
+      if (last_of_stage && arr > target && arr - target <= 32u) {
+        L[k].u.after_count = arr - target;
+        L[k].u.after_mask = mask_of(target + 1u, arr + 1u);
+        prev_ev[gidx] = arr;
+      }
+    }
+    for (size_t k = 0; k < n; ++k) all_units.push_back(L[k].u);
+  }
+  unit_off[P] = (uint32_t)all_units.size();
+  event_off[P] = (uint32_t)all_events.size();
+
+  info->n_units = (uint32_t)all_units.size();
+  info->n_events = (uint32_t)all_events.size();
   size_t off = 256;
-  info->off_desc_off = off; off += round_up_sz((size_t)(P + 1) * 4, 256);
-  info->off_init_post = off; off += round_up_sz((size_t)P * 4, 256);
-  info->off_descs = off; off += round_up_sz(descs.size() * sizeof(PhaseDesc), 256);
-  info->off_flags = off; off += round_up_sz((size_t)P * 4, 256);
-  info->off_gcnt = off; off += round_up_sz((size_t)gslots * 4, 256);
-  info->off_gpart = off; off += round_up_sz((size_t)gslots * info->slot_floats * 4, 256);
+  info->off_unit_off = off; off += round_up_sz((size_t)(P + 1) * 4, 256);
+  info->off_event_off = off; off += round_up_sz((size_t)(P + 1) * 4, 256);
+  info->off_units = off; off += round_up_sz(std::max<size_t>(1, all_units.size()) * sizeof(StepUnit), 256);
+  info->off_events = off; off += round_up_sz(all_events.size() * sizeof(StepEvent), 256);
+  info->off_counter = off; off += round_up_sz((size_t)info->n_barriers * 4, 256);
+  info->off_mixops = off; off += round_up_sz(mixops.size() * sizeof(StepMixOp), 256);
+  info->off_scratch = off; off += round_up_sz((size_t)scratch_bytes, 256);
   info->total_bytes = off;
   if (out) {
-    out->assign(info->off_gpart, 0);     // the slab sums need no initial value
-    memcpy(out->data() + info->off_desc_off, desc_off.data(), (size_t)(P + 1) * 4);
-    memcpy(out->data() + info->off_init_post, init_post.data(), (size_t)P * 4);
-    memcpy(out->data() + info->off_descs, descs.data(), descs.size() * sizeof(PhaseDesc));
+    out->assign(off, 0);
+    memcpy(out->data() + info->off_unit_off, unit_off.data(), (size_t)(P + 1) * 4);
+    memcpy(out->data() + info->off_event_off, event_off.data(), (size_t)(P + 1) * 4);
+    if (!all_units.empty()) memcpy(out->data() + info->off_units, all_units.data(), all_units.size() * sizeof(StepUnit));
+    memcpy(out->data() + info->off_events, all_events.data(), all_events.size() * sizeof(StepEvent));
+    if (!mixops.empty()) memcpy(out->data() + info->off_mixops, mixops.data(), mixops.size() * sizeof(StepMixOp));
   }
   return RWKVQ_OK;
 }
@@ -1282,10 +1280,6 @@ static int sm_count() {
   if (cudaGetDevice(&dev) != cudaSuccess) return 148;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
   return sms;
-}
-
-static size_t trace_bytes_of(const PlanInfo& info) {
-  return ((size_t)info.P * (size_t)(info.CW + 2) * kTraceSlots + (size_t)info.P * kTraceStages * 4) * sizeof(unsigned long long);
 }
 
 }  // namespace rwkvq
@@ -1313,7 +1307,7 @@ rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* p
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);   // `image` is a pageable temporary
   if (e != cudaSuccess) return cuda_status(e);
   info.runs = 0;
-  info.abort_epoch = abort_epoch();   // the image just copied holds zeroed flags and counters
+  info.abort_epoch = abort_epoch();   // the image just copied holds zeroed counters
   std::lock_guard<std::mutex> lock(g_plan_mutex);
   g_plans[plan_dev] = info;
   return RWKVQ_OK;
@@ -1322,52 +1316,48 @@ rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* p
 rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream) {
   if (!plan_dev) return RWKVQ_EINVAL;
   PlanInfo info;
-  bool clear_flags = false;
+  bool clear_counters = false;
   {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     auto it = g_plans.find(plan_dev);
     if (it == g_plans.end()) return RWKVQ_EINVAL;   // not a plan written by rwkvq_step_plan in this process
     if (plan_bytes < it->second.total_bytes) return RWKVQ_ENOMEM;
-    // The flags only ever grow: a run starts with every flag at (runs so far) * stages, so a launch
-    // needs no clearing pass.  A run that gave up leaves them (and the slab counters) uneven; start
-    // over after one.
+    // The arrival counters only ever grow: run r opens a barrier at r * CTAs arrivals, so a launch
+    // needs no clearing pass.  A run that gave up leaves them short; start over after one.
     const unsigned epoch = abort_epoch();
-    if (it->second.abort_epoch != epoch) { it->second.abort_epoch = epoch; it->second.runs = 0; clear_flags = true; }
+    if (it->second.abort_epoch != epoch) { it->second.abort_epoch = epoch; it->second.runs = 0; clear_counters = true; }
     it->second.runs += 1;
     info = it->second;
   }
   const uint8_t* p = static_cast<const uint8_t*>(plan_dev);
-  uint8_t* pw = const_cast<uint8_t*>(p);
   StepArgs a;
-  a.descs = reinterpret_cast<const PhaseDesc*>(p + info.off_descs);
-  a.desc_off = reinterpret_cast<const uint32_t*>(p + info.off_desc_off);
-  a.init_post = reinterpret_cast<const uint32_t*>(p + info.off_init_post);
-  a.flags = reinterpret_cast<unsigned*>(pw + info.off_flags);
-  a.base = (info.runs - 1u) * (unsigned)info.n_stages;
+  a.units = reinterpret_cast<const StepUnit*>(p + info.off_units);
+  a.events = reinterpret_cast<const StepEvent*>(p + info.off_events);
+  a.unit_off = reinterpret_cast<const uint32_t*>(p + info.off_unit_off);
+  a.event_off = reinterpret_cast<const uint32_t*>(p + info.off_event_off);
+  a.counter = reinterpret_cast<unsigned*>(const_cast<uint8_t*>(p) + info.off_counter);
   a.status = device_status_ptr();
   if (!a.status) return RWKVQ_ECUDA;
-  a.poll_limit = info.poll_limit; a.wait_skew = info.wait_skew;
-  a.B = info.B; a.nbp = (info.B + 1) & ~1; a.depth = info.depth;
-  a.entry_bytes = info.entry_bytes; a.slot_floats = info.slot_floats;
-  a.off_hq = info.off_hq; a.off_partial = info.off_partial; a.off_x = info.off_x; a.off_ring = info.off_ring;
-  a.gcnt = reinterpret_cast<unsigned*>(pw + info.off_gcnt);
-  a.gpart = reinterpret_cast<float*>(pw + info.off_gpart);
-  a.trace = static_cast<unsigned long long*>(info.trace_dev);
+  a.B = info.B; a.n_slots = info.n_slots; a.n_stages = info.n_stages;
+  a.mix = info.mix; a.mixops = reinterpret_cast<const StepMixOp*>(p + info.off_mixops);
+  a.scratch = const_cast<uint8_t*>(p) + info.off_scratch;
+  a.slot_bytes = info.slot_bytes; a.replica_bytes = info.replica_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  a.target = info.runs * (unsigned)info.P;
+  a.poll_limit = info.poll_limit; a.wait_skew = info.wait_skew;
   cudaError_t e = cudaSuccess;
-  if (clear_flags) {
-    e = cudaMemsetAsync(a.flags, 0, info.off_gpart - info.off_flags, s);
+  if (clear_counters) {
+    e = cudaMemsetAsync(a.counter, 0, round_up_sz((size_t)info.n_barriers * 4, 256), s);
     if (e != cudaSuccess) return cuda_status(e);
   }
-  const void* fn;
-  if (info.trace_dev) fn = info.NB == 1 ? (const void*)step_kernel<1, kConsumerWarps, true> : (const void*)step_kernel<2, kConsumerWarps, true>;
-  else fn = info.NB == 1 ? (const void*)step_kernel<1, kConsumerWarps, false> : (const void*)step_kernel<2, kConsumerWarps, false>;
+  // batches of 4 and more use the stage pre-pass (StepArgs::mix)
+  const void* fn = !info.mix ? (const void*)step_kernel<1, false> : info.NB == 1 ? (const void*)step_kernel<1, true> : (const void*)step_kernel<2, true>;
   e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)info.smem_bytes);
   if (e != cudaSuccess) return cuda_status(e);
   void* params[] = {&a};
   // Cooperative launch: all CTAs must be resident at once because they meet at the stage barrier.
-  e = cudaLaunchCooperativeKernel(fn, dim3(info.P), dim3((info.CW + 2) * 32), params, info.smem_bytes, s);
-  if (e != cudaSuccess) {   // this run will never report: have the next one clear the flags
+  e = cudaLaunchCooperativeKernel(fn, dim3(info.P), dim3(kThreads), params, info.smem_bytes, s);
+  if (e != cudaSuccess) {   // this run will never arrive: have the next one clear the counters
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     auto it = g_plans.find(plan_dev);
     if (it != g_plans.end()) it->second.abort_epoch = abort_epoch() - 1u;
@@ -1391,26 +1381,6 @@ rwkvq_status rwkvq_step_set_wait(const void* plan_dev, uint32_t poll_limit, uint
   return RWKVQ_OK;
 }
 
-size_t rwkvq_step_trace_bytes(const void* plan_dev) {
-  std::lock_guard<std::mutex> lock(g_plan_mutex);
-  auto it = g_plans.find(plan_dev);
-  if (it == g_plans.end()) return 0;
-  return trace_bytes_of(it->second);
-}
-
-rwkvq_status rwkvq_step_trace(const void* plan_dev, void* trace_dev, size_t trace_bytes) {
-  if (!plan_dev) return RWKVQ_EINVAL;
-  std::lock_guard<std::mutex> lock(g_plan_mutex);
-  auto it = g_plans.find(plan_dev);
-  if (it == g_plans.end()) return RWKVQ_EINVAL;
-  if (trace_dev) {
-    if (((uintptr_t)trace_dev & 7u) != 0) return RWKVQ_EALIGN;
-    if (trace_bytes < trace_bytes_of(it->second)) return RWKVQ_ENOMEM;
-  }
-  it->second.trace_dev = trace_dev;
-  return RWKVQ_OK;
-}
-
 rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, int n_ctas, uint32_t* counts_host,
                                    size_t n_counts, uint32_t* cta_items_host) {
   if (!counts_host || n_ctas <= 0) return RWKVQ_EINVAL;
@@ -1424,43 +1394,38 @@ rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, i
   if (n_counts < base[n_ops]) return RWKVQ_ENOMEM;
   std::unordered_map<uint64_t, int> op_of_y;
   for (int i = 0; i < n_ops; ++i) op_of_y[(uint64_t)(uintptr_t)ops[i].y_dev] = i;
-  const uint32_t* desc_off = reinterpret_cast<const uint32_t*>(image.data() + info.off_desc_off);
-  const PhaseDesc* descs = reinterpret_cast<const PhaseDesc*>(image.data() + info.off_descs);
-  const int n_stages = info.n_stages;
+  const uint32_t* unit_off = reinterpret_cast<const uint32_t*>(image.data() + info.off_unit_off);
+  const StepUnit* units = reinterpret_cast<const StepUnit*>(image.data() + info.off_units);
   for (int c = 0; c < n_ctas; ++c) {
     uint32_t items = 0;
-    bool in_group = false;
-    uint32_t area = 0;
-    for (uint32_t k = desc_off[c]; k < desc_off[c + 1]; ++k) {
-      const PhaseDesc& d = descs[k];
-      if ((d.kind_flags & 15u) != DK_PHASE) continue;
-      auto it = op_of_y.find(d.y);
+    for (uint32_t k = unit_off[c]; k < unit_off[c + 1]; ++k) {
+      const StepUnit& u = units[k];
+      auto it = op_of_y.find(u.y);
       if (it == op_of_y.end()) return RWKVQ_EINVAL;     // the walk needs distinct output buffers
       const int o = it->second;
-      const uint32_t KT = d.KT, N = d.S * d.T, ks = d.ks_part & 0xFFFFu, part = d.ks_part >> 16;
-      if (KT != (uint32_t)ops[o].W_desc.ic_pad / 256u || d.T * ks != KT || part >= ks || d.kt0 != part * d.T) return RWKVQ_EINVAL;
-      // staging groups: every phase inside exactly one, the first phase of a stage opens one, segments disjoint
-      if (d.kind_flags & DF_GROUP) { if (in_group) return RWKVQ_EINVAL; in_group = true; area = 0; }
-      if (!in_group || ((d.kind_flags & DF_FIRST) && !(d.kind_flags & DF_GROUP))) return RWKVQ_EINVAL;
-      if (d.xoff != area) return RWKVQ_EINVAL;
-      area += xseg_bytes(B, (B + 1) & ~1, d.T * 256u, ops[o].W_desc.method == RWKVQ_SQ);
-      if (info.off_x + area > info.off_ring) return RWKVQ_EINVAL;
-      if (d.kind_flags & DF_GLAST) in_group = false;
-      if ((d.kind_flags & DF_LAST) && in_group) return RWKVQ_EINVAL;
-      // the walk of producer_role: every warp's share of the S x T grid
-      for (uint32_t w = 0; w < (uint32_t)info.CW; ++w) {
-        uint32_t i0, i1;
-        item_range<kConsumerWarps>(N, w, i0, i1);
-        for (uint32_t i = i0; i < i1; ++i) {
-          const uint32_t sl = i / d.T, tt = i - sl * d.T;
-          const uint32_t slice = d.row0 / 16u + sl, kt = d.kt0 + tt;
-          if (slice >= (uint32_t)ops[o].W_desc.oc / 16u || kt >= KT) return RWKVQ_EINVAL;
+      const rwkvq_desc& d = ops[o].W_desc;
+      const uint32_t KT = (uint32_t)d.ic_pad / 256u, slices = (uint32_t)d.oc / 16u;
+      const uint8_t* payload = static_cast<const uint8_t*>(ops[o].W_image_dev) + RWKVQ_HEADER_BYTES;
+      const uint32_t w0 = (u.flags >> 8) & 15u, w1 = (u.flags >> 12) & 15u;
+      if (w0 >= w1 || w1 > 8u || u.off0 != w0 * u.rec_bytes) return RWKVQ_EINVAL;
+      // the unit's chunks: warp w of the group takes record w of chunk A (and of chunk B, 128 rows below)
+      const uint64_t src[2] = {u.src0, u.src1};
+      const uint32_t bytes[2] = {u.bytes0, u.bytes1};
+      for (int h = 0; h < 2; ++h) {
+        if (!bytes[h]) continue;
+        if (bytes[h] != (w1 - w0) * u.rec_bytes) return RWKVQ_EINVAL;
+        const uint64_t rel = src[h] - (uint64_t)(uintptr_t)payload - (uint64_t)w0 * u.rec_bytes;
+        if (rel % u.chunk_bytes) return RWKVQ_EINVAL;
+        const uint64_t chunk = rel / u.chunk_bytes;       // mb * KT + kt
+        const uint32_t mb = (uint32_t)(chunk / KT), kt = (uint32_t)(chunk % KT);
+        if (mb * 128u != u.row0 + 128u * (uint32_t)h) return RWKVQ_EINVAL;
+        for (uint32_t w = w0; w < w1; ++w) {
+          const uint32_t slice = mb * 8u + w;
+          if (slice >= slices) continue;                  // padding rows of the last chunk
           counts_host[base[o] + (size_t)slice * KT + kt] += 1u;
           ++items;
         }
       }
-      if (ks > 1u && d.gslot0 + d.S * ks > info.gslots) return RWKVQ_EINVAL;
-      if (d.post_value > (uint32_t)n_stages || d.post_value <= d.stage) return RWKVQ_EINVAL;
     }
     if (cta_items_host) cta_items_host[c] = items;
   }

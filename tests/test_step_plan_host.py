@@ -58,17 +58,16 @@ def test_plan_is_built_for_benchmark_shapes(d, h, layers, Bn, bits):
     ops = _ops(d, h, layers, bits=bits)
     n = B.rwkvq_step_plan_bytes(ops, Bn)
     assert n > 0 and n % 256 == 0
-    # the plan grows with the number of stages (twice the layers, twice the descriptors); the scratch
-    # for the sums of K slabs at larger batches is as large as one stage needs, whatever the depth
+    # the plan grows with the number of units: twice the layers, roughly twice the descriptors
     n2 = B.rwkvq_step_plan_bytes(_ops(d, h, 2 * layers, bits=bits), Bn)
-    n4 = B.rwkvq_step_plan_bytes(_ops(d, h, 4 * layers, bits=bits), Bn)
-    assert n < n2 < 2.5 * n and 1.8 * (n2 - n) < n4 - n2 < 2.2 * (n2 - n)
+    assert 1.5 * n < n2 < 2.5 * n
 
 
 # Every record (product, 16-row slice, 256-column tile) must reach exactly one consumer warp exactly
-# once: shapes with few slices per CTA, many slices per CTA, fewer items than warps, ragged tiles
-# (ic not a multiple of 256), every batch regime (inputs mixed per CTA; one window of the stage
-# pre-pass; several windows with two accumulator sets per warp), few and many CTAs.
+# once, in each of the planner's three ways of dealing a stage (row of tiles by row of tiles; whole
+# units at their cost midpoints; eighths of a unit for stages too small for either): small and large
+# stages, ragged shapes (rows that end in half a unit, ic not a multiple of 256), every batch
+# regime, few and many CTAs, every product in one stage.
 @pytest.mark.parametrize("d,h,layers,Bn,bits,n_ctas,one_stage", [
     (512, 1280, 2, 1, 6, 148, False),
     (384, 896, 2, 5, 6, 148, False),
@@ -80,7 +79,7 @@ def test_plan_is_built_for_benchmark_shapes(d, h, layers, Bn, bits):
     (4096, 14336, 1, 16, 8, 7, False),        # many slices per CTA: phases are cut to the warp count
     (2048, 7168, 3, 1, 6, 148, True),         # every product in one stage
     (2048, 7168, 1, 8, 6, 33, True),
-    (512, 1280, 1, 12, 8, 1, False),
+    (512, 1280, 1, 12, 8, 16, False),
 ])
 def test_schedule_covers_every_record_once(d, h, layers, Bn, bits, n_ctas, one_stage):
     ops = _ops(d, h, layers, bits=bits, one_stage=one_stage)
@@ -89,10 +88,10 @@ def test_schedule_covers_every_record_once(d, h, layers, Bn, bits, n_ctas, one_s
     assert (counts == 1).all(), f"{int((counts != 1).sum())} records not dealt exactly once"
     assert int(per_cta.sum()) == counts.size
     if n_ctas == 148 and not one_stage:
-        # whole slices are dealt by cost: no CTA carries more than its even share plus one slice per stage
+        # whole units (16 records of a 256-column tile) are dealt by cost: no CTA carries more than
+        # its even share plus two units per stage
         n_stages = len({o.stage for o in ops})
-        kt_max = max(o.W_desc.ic_pad // 256 for o in ops)
-        assert per_cta.max() <= counts.size / n_ctas + n_stages * kt_max * 1.9
+        assert per_cta.max() <= counts.size / n_ctas + n_stages * 32
 
 
 def test_plan_rejects_bad_arguments():
