@@ -4,6 +4,8 @@
 // the per-record routines below.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "../../include/rwkvq.h"
 #include "gemv_core.cuh"
 #include "host_util.h"
@@ -285,9 +287,9 @@ size_t rwkvq_gemv_workspace_bytes(const rwkvq_desc* d, int B) {
   return p.ws_bytes;
 }
 
-rwkvq_status rwkvq_gemv(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu,
-                        const void* x, const void* xprev, int B, void* y, int y_dtype, void* ws,
-                        size_t ws_bytes, void* stream) {
+// Every argument check of the decode product, made on the host before anything is enqueued.
+static rwkvq_status check_gemv_args(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu, const void* x,
+                                    const void* xprev, int B, const void* y, int y_dtype, GemvPlan* p) {
   if (!d || !W || !x || !y) return RWKVQ_EINVAL;
   if ((mu == nullptr) != (xprev == nullptr)) return RWKVQ_EINVAL;
   if (mu && !mud) return RWKVQ_EINVAL;
@@ -296,12 +298,14 @@ rwkvq_status rwkvq_gemv(const rwkvq_desc* d, const void* W, const rwkvq_desc* mu
     rwkvq_status st = check_vector_desc(mud, d->ic);
     if (st != RWKVQ_OK) return st;
   }
-  GemvPlan p;
-  rwkvq_status st = plan_gemv(d, B, mu != nullptr, mu ? mud->entries : 0, &p);
+  rwkvq_status st = plan_gemv(d, B, mu != nullptr, mu ? mud->entries : 0, p);
   if (st != RWKVQ_OK) return st;
-  if (!aligned16(W) || !aligned16(x) || !aligned16(y) || (mu && (!aligned16(mu) || !aligned16(xprev))) || (ws && !aligned16(ws)))
-    return RWKVQ_EALIGN;
-  if (!ws || ws_bytes < p.ws_bytes) return RWKVQ_ENOMEM;
+  if (!aligned16(W) || !aligned16(x) || !aligned16(y) || (mu && (!aligned16(mu) || !aligned16(xprev)))) return RWKVQ_EALIGN;
+  return RWKVQ_OK;
+}
+
+static rwkvq_status run_gemv(const GemvPlan& p, const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu,
+                             const void* x, const void* xprev, int B, void* y, int y_dtype, void* ws, void* stream) {
   GemvArgs a;
   fill_gemv_args(&a, d, W, mud, mu, x, xprev, B, y, y_dtype);
   a.KT = p.KT; a.S = p.S; a.nkt = p.nkt;
@@ -314,6 +318,17 @@ rwkvq_status rwkvq_gemv(const rwkvq_desc* d, const void* W, const rwkvq_desc* mu
   return cuda_status(e);
 }
 
+rwkvq_status rwkvq_gemv(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu,
+                        const void* x, const void* xprev, int B, void* y, int y_dtype, void* ws,
+                        size_t ws_bytes, void* stream) {
+  GemvPlan p;
+  rwkvq_status st = check_gemv_args(d, W, mud, mu, x, xprev, B, y, y_dtype, &p);
+  if (st != RWKVQ_OK) return st;
+  if (ws && !aligned16(ws)) return RWKVQ_EALIGN;
+  if (!ws || ws_bytes < p.ws_bytes) return RWKVQ_ENOMEM;
+  return run_gemv(p, d, W, mud, mu, x, xprev, B, y, y_dtype, ws, stream);
+}
+
 // ---------------------------------------------------------------------------------------------
 // rwkvq_gemv for callers that cannot allocate device memory: the split-K scratch lives in a
 // file-scope device array.  In host code the array's name is only a handle; its device address
@@ -321,31 +336,34 @@ rwkvq_status rwkvq_gemv(const rwkvq_desc* d, const void* W, const rwkvq_desc* mu
 // ---------------------------------------------------------------------------------------------
 #define RWKVQ_STATIC_SCRATCH_BYTES (8u << 20)
 static __device__ __align__(256) unsigned char g_static_scratch[RWKVQ_STATIC_SCRATCH_BYTES];
-static void* g_static_scratch_addr[64] = {nullptr};
+// One entry per device ordinal, written once; atomic because any host thread may make the first
+// call.  The address stays valid for the life of the device's primary context: after
+// cudaDeviceReset the library has to be loaded afresh (as every other device allocation).
+static std::atomic<void*> g_static_scratch_addr[64];
 
 size_t rwkvq_gemv_static_max_scratch_bytes(void) { return RWKVQ_STATIC_SCRATCH_BYTES; }
 
 rwkvq_status rwkvq_gemv_static(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu,
                                const void* x, const void* xprev, int B, void* y, int y_dtype, void* stream) {
-  if (!d) return RWKVQ_EINVAL;
+  // every argument error is reported before anything reaches the stream
   GemvPlan p;
-  rwkvq_status st = plan_gemv(d, B, mu != nullptr, (mu && mud) ? mud->entries : 0, &p);
+  rwkvq_status st = check_gemv_args(d, W, mud, mu, x, xprev, B, y, y_dtype, &p);
   if (st != RWKVQ_OK) return st;
   if (p.ws_bytes > RWKVQ_STATIC_SCRATCH_BYTES) return RWKVQ_ENOMEM;   // this product needs more scratch than the built-in array holds
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_status(e);
   if (dev < 0 || dev >= 64) return RWKVQ_EUNSUPPORTED;
-  void* ws = g_static_scratch_addr[dev];
+  void* ws = g_static_scratch_addr[dev].load(std::memory_order_acquire);
   if (!ws) {
     e = cudaGetSymbolAddress(&ws, g_static_scratch);
     if (e != cudaSuccess) return cuda_status(e);
-    g_static_scratch_addr[dev] = ws;
+    g_static_scratch_addr[dev].store(ws, std::memory_order_release);
   }
   // The array keeps whatever the previous call left: the arrival counters must start at zero.
   e = cudaMemsetAsync(ws, 0, p.counters_bytes, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_status(e);
-  return rwkvq_gemv(d, W, mud, mu, x, xprev, B, y, y_dtype, ws, RWKVQ_STATIC_SCRATCH_BYTES, stream);
+  return run_gemv(p, d, W, mud, mu, x, xprev, B, y, y_dtype, ws, stream);
 }
 
 rwkvq_status rwkvq_dequant(const rwkvq_desc* d, const void* W, void* out, int dtype, void* stream) {

@@ -157,3 +157,34 @@ def test_argument_errors_are_reported_before_launch():
         B.rwkvq_gemv(W.desc, W.dev, mu.desc, mu.dev, x, x, 1, y, ws)
     assert e.value.status == 2
     assert B.rwkvq_device_status() == 0
+
+
+def _extreme_sq_codes(seed, oc, ic):
+    """Valid logical SQ codes whose scales cover the whole fp16 range (subnormals, the smallest
+    subnormal 2^-24, scales of 2^15 and above) and whose zero points include non-integers: Eq. 2's
+    decode s * (q - z) is defined for all of them (two fp32 operations, no FMA contraction)."""
+    rng = np.random.default_rng(seed)
+    codes = H.random_sq_codes(seed, oc, ic)
+    s = codes["scale"].astype(np.float64)
+    pick = [2.0 ** -24, 3 * 2.0 ** -24, 2.0 ** -15, 6.0e-5, 2.0 ** 15, 40000.0, 65504.0, 1.0, 0.013]
+    s[:] = rng.choice(pick, size=s.shape)
+    codes["scale"] = s.astype(np.float16)
+    z = codes["zero"].astype(np.float64)
+    frac = rng.random(z.shape) < 0.3
+    z[frac] = rng.choice([0.5, 2.25, 3.125, 6.75, 0.0009765625], size=int(frac.sum()))
+    codes["zero"] = z.astype(np.float16)
+    return codes
+
+
+@pytest.mark.parametrize("oc,ic,Bn", [(64, 512, 1), (256, 1024, 8), (128, 2048, 16)])
+def test_sq_extreme_scales_and_fractional_zero_points(oc, ic, Bn):
+    W = H.pack_sq(_extreme_sq_codes(oc + ic + Bn, oc, ic))
+    s = W.codes["scale"].astype(np.float64)
+    assert (s < 6.2e-5).any() and (s >= 2.0 ** 15).any()               # subnormal and very large scales are present
+    assert (W.codes["zero"].astype(np.float64) % 1 != 0).any()          # and zero points that are no integers
+    _check_decode_exact(W)
+    # Scales this far apart make rows that differ by ten orders of magnitude: activations with a
+    # few large channels exercise the fp32 accumulation of the per-group terms.
+    x, xp = inputs.gen_activation_pair(Bn + ic, Bn, ic, n_outliers=8)
+    mu = H.pack_mu(H.random_mu_codes(ic, ic)) if Bn != 8 else None
+    _check_gemv(W, mu, x.astype(np.float16), xp.astype(np.float16))

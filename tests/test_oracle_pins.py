@@ -241,6 +241,25 @@ def test_mu_roundtrip_shapes():
     assert mh.shape == (512,) and np.abs(mh - mu.astype(np.float64)).max() < 0.02
 
 
+def test_mu_encode_reproduces_few_distinct_pairs_in_order():
+    # A vector made of no more distinct (even, odd) pairs than codebook entries is coded without
+    # error, and decoding puts every pair back at its own position: a reshape that paired the wrong
+    # elements (stride ic/2 instead of 2, or columns swapped) would either need more than `entries`
+    # centres or return the halves in the wrong order.
+    rng = np.random.default_rng(5)
+    pairs = (rng.random((48, 2)) * 0.9 + 0.05).astype(np.float16)
+    pairs[:, 1] += np.float16(1.0)                       # odd elements in (1, 2), even ones in (0, 1)
+    which = rng.integers(0, 48, size=300)
+    mu = pairs[which].reshape(-1)                        # [x0, y0, x1, y1, ...]
+    cb, ix = orc.mu_encode(mu, entries=64, iters=10, seed=3)
+    mh = orc.mu_decode(cb, ix)
+    assert np.array_equal(mh, mu.astype(np.float64))
+    assert (mh[0::2] < 1.0).all() and (mh[1::2] >= 1.0).all()
+    # the indices name the pair each position holds: equal pairs share an index, different pairs do not
+    for a, b in [(0, 1), (5, 200), (17, 299)]:
+        assert (ix[a] == ix[b]) == bool((pairs[which[a]] == pairs[which[b]]).all())
+
+
 # ---------------------------------------------------------------- proxy (Eqs. 5-18)
 
 def test_proxy_hand_worked_three_elements():

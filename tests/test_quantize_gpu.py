@@ -88,6 +88,30 @@ def test_sq_device_image_feeds_the_products():
     assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - ref) <= tol)
 
 
+def test_sq_device_image_of_special_groups_feeds_the_products():
+    # the matrix of degenerate groups (constants, +-0, the full fp16 range, subnormals): its device
+    # image must decode to the oracle's values bit for bit and multiply within the tolerance
+    w16 = sq_cases()["special_256x1024"]
+    oc, ic = w16.shape
+    d, img = quantize_dev(w16, B.RWKVQ_SQ, 3)
+    q, s, z = orc.sq_encode(w16)
+    w_hat = orc.sq_decode(q, s, z)
+    out = torch.empty((oc, ic), dtype=torch.float32, device="cuda")
+    B.rwkvq_dequant(d, img, out)
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), w_hat)
+    rng = np.random.default_rng(12)
+    for Bn in (1, 5):
+        x = rng.standard_normal((Bn, ic)).astype(np.float16)
+        y = torch.empty((Bn, oc), dtype=torch.float32, device="cuda")
+        ws = torch.zeros(max(256, B.rwkvq_gemv_workspace_bytes(d, Bn)), dtype=torch.uint8, device="cuda")
+        B.rwkvq_gemv(d, img, None, None, torch.from_numpy(x).cuda(), None, Bn, y, ws)
+        torch.cuda.synchronize()
+        ref = orc.gemv(w_hat, x.astype(np.float64))
+        tol = orc.tolerance(w_hat, x.astype(np.float64))
+        got = y.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all() and np.all(np.abs(got - ref) <= tol)
+
+
 def tile_vectors(w16, tr, tc):
     return w16[tr * 256:(tr + 1) * 256, tc * 256:(tc + 1) * 256].astype(np.float64).reshape(-1, 2)
 

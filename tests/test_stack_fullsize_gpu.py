@@ -26,7 +26,7 @@ def _oracle_product(st, op):
 
 
 @pytest.mark.parametrize("name,batch,quantizer", [("c2_1p6b", 1, "host"), ("c3_7b", 8, "host"), ("c4_14b", 16, "host"),
-                                                  ("c2_1p6b", 1, "device")])
+                                                  ("c2_1p6b", 1, "device"), ("c3_7b", 1, "device")])
 def test_whole_step_at_benchmark_size_matches_oracle_on_sampled_products(name, batch, quantizer):
     # quantizer = "device": the images come from rwkvq_quantize_dev, the oracle decodes the codes
     # unpacked from those images

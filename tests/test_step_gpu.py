@@ -108,3 +108,74 @@ def test_step_rejects_bad_plans():
     arr = B.make_ops([dict(desc=e["W"].desc, W=e["W"].dev, mu_desc=None, mu=None, x=e["xd"], xprev=None,
                            y=e["y"].half(), stage=e["stage"]) for e in ops[:1]])
     assert B.rwkvq_step_plan_bytes(arr, 1) == 0   # fp16 outputs are not supported by the step launch
+
+
+def test_step_run_host_matches_oracle():
+    """rwkvq_step_run_host (the call behind the benchmark's end-to-end figure): activations come from
+    pinned host memory, results go back to pinned host memory, compared with the oracle there."""
+    Bn = 4
+    ops = _build_ops(512, 1280, 2, Bn, 6, seed=91)
+    # one arena for the activations and one for the outputs, as the stack runner lays them out
+    def al(n):
+        return (n + 255) // 256 * 256
+    act_off, y_off, slots = 0, 0, []
+    for e in ops:
+        xo = act_off; act_off += al(e["x16"].nbytes)
+        po = None
+        if e["mu"] is not None:
+            po = act_off; act_off += al(e["xp16"].nbytes)
+        slots.append((xo, po, y_off)); y_off += al(Bn * e["W"].oc * 4)
+    act_host = torch.zeros(act_off, dtype=torch.uint8).pin_memory()
+    y_host = torch.zeros(y_off, dtype=torch.uint8).pin_memory()
+    act_dev = torch.zeros(act_off, dtype=torch.uint8, device="cuda")
+    y_dev = torch.full((y_off // 4,), float("nan"), dtype=torch.float32, device="cuda").view(torch.uint8)
+    an = act_host.numpy()
+    for e, (xo, po, yo) in zip(ops, slots):
+        an[xo:xo + e["x16"].nbytes] = e["x16"].reshape(-1).view(np.uint8)
+        e["xd"] = act_dev[xo:xo + e["x16"].nbytes].view(torch.float16).view(Bn, -1)
+        if po is not None:
+            an[po:po + e["xp16"].nbytes] = e["xp16"].reshape(-1).view(np.uint8)
+            e["xpd"] = act_dev[po:po + e["xp16"].nbytes].view(torch.float16).view(Bn, -1)
+        e["y"] = y_dev[yo:yo + Bn * e["W"].oc * 4].view(torch.float32).view(Bn, e["W"].oc)
+    plan = _plan(ops, Bn)
+    for rep in range(2):
+        y_host.zero_()
+        B.rwkvq_step_run_host(plan, act_host, act_dev, y_dev, y_host)
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        assert torch.equal(act_dev.cpu(), act_host)                      # the inputs went through the call
+        yn = y_host.numpy()
+        for e, (xo, po, yo) in zip(ops, slots):
+            y = yn[yo:yo + Bn * e["W"].oc * 4].view(np.float32).reshape(Bn, -1).astype(np.float64)
+            ref, tol = H.reference(e["W"], e["mu"], e["x16"], e["xp16"])
+            assert np.isfinite(y).all() and (np.abs(y - ref) <= tol).all()
+    B.rwkvq_step_plan_release(plan)
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_step_run(plan)                                           # the record of the plan is gone
+
+
+def test_bounded_waits_run_out_and_the_plan_recovers():
+    """No wait inside the step kernel is unbounded.  With a barrier target that can never be met
+    (wait_skew) and a small poll limit every CTA gives up at its first stage barrier, the kernel
+    returns, the status word says ETIMEOUT; after the status has been read the next run clears the
+    barrier counters and matches the oracle again.  Nothing traps, faults or hangs."""
+    for Bn in (1, 8):
+        ops = _build_ops(512, 1280, 2, Bn, 6, seed=40 + Bn)
+        plan = _plan(ops, Bn)
+        B.rwkvq_step_run(plan)
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        _check(ops, Bn)
+        B.rwkvq_step_set_wait(plan, poll_limit=2000, wait_skew=1)
+        B.rwkvq_step_run(plan)
+        torch.cuda.synchronize()                                         # the kernel returns by itself
+        assert B.rwkvq_device_status() == 8                              # RWKVQ_ETIMEOUT, and the word is cleared
+        assert B.rwkvq_device_status() == 0
+        B.rwkvq_step_set_wait(plan, poll_limit=0, wait_skew=0)           # defaults again
+        for rep in range(2):
+            for e in ops:
+                e["y"].fill_(float("nan"))
+            B.rwkvq_step_run(plan)
+            torch.cuda.synchronize()
+            assert B.rwkvq_device_status() == 0
+            _check(ops, Bn)

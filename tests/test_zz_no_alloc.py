@@ -1,6 +1,7 @@
 """rwkvq_gemv_static -- the decode product for callers that may not allocate device memory (the
 scratch is an array inside the library) -- must give what rwkvq_gemv gives with a caller-owned
-workspace.  Collected last on purpose: a failure here stops nothing else."""
+workspace, bit for bit (the partial sums are combined in the same fixed order), and both must match
+the oracle.  Collected last on purpose: a failure here stops nothing else."""
 import numpy as np
 import pytest
 import torch
@@ -35,11 +36,13 @@ def test_static_scratch_variant_matches_workspace_variant(fmt, oc, ic, Bn):
     mu = H.pack_mu(H.random_mu_codes(ic, ic)) if Bn != 3 else None
     x, xp = inputs.gen_activation_pair(Bn + ic, Bn, ic, n_outliers=8)
     x16, xp16 = x.astype(np.float16), xp.astype(np.float16)
-    y_ref, ys = _both(W, mu, x16, xp16)
-    _, tol = H.reference(W, mu, x16, xp16)
+    y_ws, ys = _both(W, mu, x16, xp16)
+    ref, tol = H.reference(W, mu, x16, xp16)          # the oracle's fp64 product and the stated tolerance
+    assert (np.abs(y_ws - ref) <= tol).all()
     for y in ys:
         assert np.isfinite(y).all()
-        assert (np.abs(y - y_ref) <= tol).all()
+        assert (np.abs(y - ref) <= tol).all()
+        assert np.array_equal(y, y_ws)
     assert B.rwkvq_device_status() == 0
 
 
