@@ -103,6 +103,49 @@ def test_prefill_7b_shape_sampled(fmt):
     _check(W, mu, M, seed=34, sample_tokens=toks)
 
 
+# The kernel is persistent: with more output tiles (256 weight rows x 256 tokens) than SMs a CTA works
+# through several tiles, carrying the phases of its barriers and handing the accumulators back and
+# forth between the tensor-core issue thread and the epilogue warps.  Every case below has more than
+# 148 tiles; (oc = 640: five chunks, so the last row pair has no second half).
+@pytest.mark.parametrize("fmt,oc,ic,M", [
+    ("sq", 14336, 512, 2048),      # 56 row pairs x 8 token tiles = 448 tiles, short K
+    ("vq6", 7168, 256, 3000),      # 28 x 12 = 336 tiles, ragged last token tile
+    ("vq8", 2048, 512, 5120),      # 8 x 20 = 160 tiles
+    ("sq", 640, 256, 12800),       # 3 x 50 = 150 tiles, second half of the last row pair absent
+    ("vq6", 1280, 512, 8192),      # 5 x 32 = 160 tiles
+])
+def test_prefill_several_tiles_per_cta(fmt, oc, ic, M):
+    bits = 6 if fmt == "vq6" else 8
+    W = H.pack_sq(H.random_sq_codes(oc + M, oc, ic)) if fmt == "sq" else H.pack_vq(H.random_vq_codes(oc + M, oc, ic, bits), bits)
+    mu = H.pack_mu(H.random_mu_codes(oc + 1, ic))
+    rng = np.random.default_rng(M)
+    toks = sorted(set([0, 1, 255, 256, 257, M // 2, M - 257, M - 256, M - 2, M - 1]) | set(int(t) for t in rng.integers(0, M, 40)))
+    _check(W, mu, M, seed=oc + ic, sample_tokens=toks)
+
+
+def test_prefill_identity_probe_over_several_tiles_per_cta():
+    # X = [I; I; ...] stacked to M tokens: every block of ic tokens returns bf16_rne(w_hat) transposed,
+    # bit for bit, whichever tile of whichever CTA computed it (the zeros added in the tensor core are exact)
+    oc, ic, reps = 5120, 256, 8                      # 20 row pairs x 8 token tiles = 160 tiles
+    W = H.pack_sq(H.random_sq_codes(5, oc, ic))
+    M = ic * reps
+    _, Xd = _bf16(np.tile(np.eye(ic, dtype=np.float32), (reps, 1)))
+    Y = _run(W, None, Xd, None, M).cpu().numpy()
+    expect = orc.bf16_rne(W.w_hat).T
+    for r in range(reps):
+        assert np.array_equal(Y[r * ic:(r + 1) * ic], expect), f"block {r}"
+
+
+@pytest.mark.parametrize("fmt,oc,ic", [("sq", 14336, 4096), ("sq", 4096, 14336), ("vq6", 14336, 4096), ("vq6", 4096, 14336)])
+def test_prefill_channel_mix_shapes_of_the_7b_layer_sampled(fmt, oc, ic):
+    # the two 14336-wide products of the timed prefill layer at M = 2048 (448 and 128 tiles), on sampled tokens
+    M = 2048
+    W = H.pack_sq(H.random_sq_codes(61, oc, ic)) if fmt == "sq" else H.pack_vq(H.random_vq_codes(62, oc, ic, 6), 6)
+    mu = H.pack_mu(H.random_mu_codes(63, ic)) if oc > ic else None     # the channel-mix key takes the token shift
+    toks = [0, 1, 255, 256, 511, 512, 1023, 1024, 1500, 2046, 2047]
+    _check(W, mu, M, seed=64, sample_tokens=toks)
+
+
 def test_prefill_argument_errors():
     W = H.pack_sq(H.random_sq_codes(41, 128, 256))
     X = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
