@@ -5,7 +5,12 @@ One step = one decode pass over every projection of every layer of a seeded synt
 RWKV-6-shaped stack (time-mix R/K/V/G/O, channel-mix K/R/V, the five token-shift mixes fused),
 issued as one persistent launch (rwkvq_step_run).  Prints ONE JSON line.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_1p6b|c3_7b|c4_14b] [--batch B]
+  python bench.py [--gpus N] [--steps K] [--warmup W]
+        headline: the 14B-class stack at decode batch 16, every layer's weights distinct, drawn and
+        quantized on the device; the same line carries a "configs" map with the 1.6B-class stack at
+        batch 1 and the 7B-class stack at batch 1 and 8, a prefill leg (one 7B-class layer, M = 2048),
+        a quantizer leg and a proxy leg
+  python bench.py --workload c2_1p6b|c3_7b|c4_14b [--batch B] ...   # one stack only
   python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
 
 With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
@@ -16,6 +21,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -29,10 +35,15 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
-# profiles/step_kernel_c2_1p6b_b1.md.  Valid only for that workload and for the kernel as it was
-# when the counters were taken: set an entry to None when step.cu changes.
-NCU_TRAFFIC_BYTES = {("c2_1p6b", 1, "step", None, 4): 540_035_328}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one step_kernel launch divided by its
+# algorithmic bytes, from an ncu capture of the 1.6B-class stack (about 0.55 GB per launch; the larger
+# stacks are beyond the size a capture should hold on the device).  The packed weights are read once
+# whatever the stack, so the traffic of a larger stack is this ratio times its algorithmic bytes.
+# None = no capture of the kernel as it stands.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = None
+
+HEADLINE = ("c4_14b", 16)
+CONFIGS = (("c2_1p6b", 1), ("c3_7b", 1), ("c3_7b", 8))
 
 METRIC = "decode_tokens_per_s"
 UNIT = "tokens/s"
@@ -45,9 +56,10 @@ def parse_args(argv=None):
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_1p6b", choices=["c2_1p6b", "c3_7b", "c4_14b"])
+    ap.add_argument("--workload", default=None, choices=["c2_1p6b", "c3_7b", "c4_14b"],
+                    help="time this stack only (default: the 14B-class headline plus the configs map)")
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--distinct-layers", type=int, default=4,
+    ap.add_argument("--distinct-layers", type=int, default=0,
                     help="draw and quantize weights for this many layers and reuse their values, in "
                          "separate device buffers, for the others (0 = every layer distinct)")
     ap.add_argument("--force-method", default=None, choices=[None, "sq", "vq"],
@@ -60,8 +72,13 @@ def parse_args(argv=None):
                     help="diagnostic: put this many consecutive products into one stage instead of the layer's own "
                          "four dependent stages (0 = the real dependencies); a large value removes every grid barrier "
                          "and shows the streaming rate of the kernel alone")
-    ap.add_argument("--quantizer", default="host", choices=["host", "device"],
+    ap.add_argument("--quantizer", default="device", choices=["host", "device"],
                     help="where the stack's weights are quantized and packed: rwkvq_pack or rwkvq_quantize_dev")
+    ap.add_argument("--weights", default=None, choices=["host", "device"],
+                    help="where the synthetic weights are drawn: the numpy generators of the inputs module, or a seeded "
+                         "generator on the device (default: device with --quantizer device, else host)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the configs map (the other stacks)")
+    ap.add_argument("--no-proxy", action="store_true", help="skip the proxy leg")
     ap.add_argument("--no-quantize", action="store_true", help="skip the device-quantizer leg (one 7B-class layer)")
     return ap.parse_args(argv)
 
@@ -234,16 +251,17 @@ def run_reference(args):
     if rank != 0:
         return 0
     from paper_2505_03803_b200 import inputs
-    sp = inputs.STACKS[args.workload]
-    batch = args.batch or sp["batches"][0]
+    wl = args.workload or HEADLINE[0]
+    sp = inputs.STACKS[wl]
+    batch = args.batch or (HEADLINE[1] if args.workload is None else sp["batches"][0])
     K = args.steps if args.steps is not None else 5
     W = args.warmup if args.warmup is not None else 1
     # size the per-step sample from a probe so that the whole run stays near two minutes
-    probe = time_oracle(args.workload, batch, steps=1, rows_fraction=0.125)
+    probe = time_oracle(wl, batch, steps=1, rows_fraction=0.125)
     full_layer_s = probe["per_sample_s"] * 8.0
     frac = min(1.0, max(0.125, 120.0 / max(1e-9, full_layer_s * (K + W))))
     frac = max(0.125, int(frac * 8) / 8.0)
-    r = time_oracle(args.workload, batch, steps=K, warmup=W, rows_fraction=frac)
+    r = time_oracle(wl, batch, steps=K, warmup=W, rows_fraction=frac)
     cores = cpu_threads()
     sample = (f"per step: the oracle's decode + token shift + fp64 product over the first {frac:g} of the rows of "
               f"each of the 8 matrices of one layer ({r['sample_weights']} of {r['total_weights']} weights), "
@@ -252,7 +270,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus, "steps": K,
         "warmup": W, "ms_per_step": r["full_step_s"] * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(args.workload, batch), "batch": batch},
+        "config": {"workload": workload_name(wl, batch), "batch": batch},
         "cpu_baseline": {"value": r["value"], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -273,19 +291,17 @@ def measured_bf16_peak():
         return 1590.0, "fallback"
 
 
-def prefill_leg(reps: int = 10, M: int = 2048):
-    """All eight projections of one 7B-class layer (d = 4096, h = 14336) over M tokens: random valid
-    logical codes (the time does not depend on the code values), SQ for the matrices the seeded coin
-    makes Gaussian and VQ-64 for the heavy-tailed ones, token-shift mix on R, K, V, G and cm_k.
-    Returns TFLOP/s over the layer (2*M*oc*ic per matrix) and the fraction of the measured bf16 peak."""
+def _prefill_layer(formats, M):
+    """Device buffers of the eight projections of one 7B-class layer, matrix i packed as formats[i]
+    ("sq" or "vq"): random valid logical codes (the time does not depend on the code values)."""
     import torch
     from paper_2505_03803_b200 import binding as B
     from paper_2505_03803_b200 import inputs
     sp = inputs.STACKS["c3_7b"]
     mats = []
-    for (name, oc, ic, has_mu, stage) in inputs.layer_shapes(sp["d"], sp["h"]):
+    for fmt, (name, oc, ic, has_mu, stage) in zip(formats, inputs.layer_shapes(sp["d"], sp["h"])):
         seed = inputs.seed_of("c5_prefill", name)
-        if inputs.weight_kind(seed) == "gauss":
+        if fmt == "sq":
             blob = B.rwkvq_pack(None, oc, ic, B.RWKVQ_SQ, 3, codes=inputs.random_sq_codes(seed, oc, ic))
         else:
             blob = B.rwkvq_pack(None, oc, ic, B.RWKVQ_VQ, 6, codes=inputs.random_vq_codes(seed, oc, ic, 6))
@@ -295,6 +311,12 @@ def prefill_leg(reps: int = 10, M: int = 2048):
         Y = torch.empty((M, oc), dtype=torch.float32, device="cuda")
         ws = torch.empty(B.rwkvq_prefill_workspace_bytes(blob.desc, M, has_mu), dtype=torch.uint8, device="cuda")
         mats.append((blob.desc, blob.to_device(), mu.desc if mu else None, mu.to_device() if mu else None, X, Y, ws, oc, ic))
+    return mats
+
+
+def _time_prefill_layer(mats, M, reps):
+    import torch
+    from paper_2505_03803_b200 import binding as B
 
     def layer():
         for (d, W, md, m, X, Y, ws, oc, ic) in mats:
@@ -312,14 +334,95 @@ def prefill_leg(reps: int = 10, M: int = 2048):
         raise SystemExit("bench.py: a device-side wait timed out in the prefill leg")
     ms = e0.elapsed_time(e1) / reps
     flops = sum(2.0 * M * oc * ic for (*_r, oc, ic) in mats)
-    tf = flops / (ms * 1e-3) / 1e12
+    return ms, flops, flops / (ms * 1e-3) / 1e12
+
+
+def prefill_formats():
+    """Formats of the timed hybrid layer: per matrix the seeded coin of the decode stacks (heavy-tailed
+    -> VQ-64, Gaussian -> SQ), under the first salt that gives the layer both formats."""
+    from paper_2505_03803_b200 import inputs
+    sp = inputs.STACKS["c3_7b"]
+    names = [name for (name, *_r) in inputs.layer_shapes(sp["d"], sp["h"])]
+    for salt in range(64):
+        f = ["sq" if inputs.weight_kind(inputs.seed_of("c5_prefill", salt, n)) == "gauss" else "vq" for n in names]
+        if 0 < f.count("sq") < len(f):
+            return f
+    raise SystemExit("bench.py: no seeded hybrid layer found")
+
+
+def prefill_leg(reps: int = 10, M: int = 2048):
+    """All eight projections of one 7B-class layer (d = 4096, h = 14336) over M tokens with the
+    token-shift mix on R, K, V, G and cm_k: the hybrid layer (SQ and VQ-64 matrices by the seeded coin),
+    then the same layer all-SQ and all-VQ-64.  TFLOP/s over the layer (2*M*oc*ic per matrix) and the
+    fraction of the measured bf16 peak."""
+    import torch
+    from paper_2505_03803_b200 import binding as B
     peak, kind = measured_bf16_peak()
+    out = {}
+    hybrid = prefill_formats()
+    for label, formats in (("hybrid", hybrid), ("all_sq", ["sq"] * 8), ("all_vq64", ["vq"] * 8)):
+        mats = _prefill_layer(formats, M)
+        ms, flops, tf = _time_prefill_layer(mats, M, reps)
+        out[label] = (ms, flops, tf, sum(1 for m in mats if m[0].method == B.RWKVQ_SQ), len(mats))
+        del mats
+        torch.cuda.empty_cache()
+    ms, flops, tf, n_sq, n = out["hybrid"]
+    assert 0 < n_sq < n
     return {"workload": f"one 7B-class layer (8 projections, d=4096 h=14336), M={M} tokens, hybrid SQ/VQ-64, bf16 x bf16 -> fp32",
-            "ms_per_layer": ms, "flop_per_layer": flops, "launches_per_layer": 2 * len(mats), "sq_matrices":
-            sum(1 for m in mats if m[0].method == B.RWKVQ_SQ),
+            "ms_per_layer": ms, "flop_per_layer": flops, "launches_per_layer": 2 * n, "sq_matrices": n_sq,
+            "formats": hybrid,
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
                          "traffic": None, "peak_kind": f"of {kind} (burst)", "kernel": "prefill_kernel",
-                         "frac_of_2250_nominal": tf / 2250.0}}
+                         "frac_of_2250_nominal": tf / 2250.0},
+            "all_sq": {"ms_per_layer": out["all_sq"][0], "tflops": out["all_sq"][2], "frac": out["all_sq"][2] / peak},
+            "all_vq64": {"ms_per_layer": out["all_vq64"][0], "tflops": out["all_vq64"][2], "frac": out["all_vq64"][2] / peak}}
+
+
+def proxy_leg(reps: int = 10, with_oracle: bool = True):
+    """The proxy pass (Section 4.1) on fp16 matrices resident on the device: rwkvq_proxy_select over one
+    matrix at a time (histogram of the 65 536 bit patterns = the sort of Eq. 5 as a counting sort, then the
+    walk over the occupied bins, then the copy of the two numbers to the host), timed with events around
+    the call.  A 256 x 256 matrix gives the fixed cost of the call (clear, walk, copy, synchronization);
+    the large matrices minus that are the streaming pass, whose algorithmic traffic is 2 bytes per
+    weight.  The oracle's sort-and-difference on the same values is timed beside it."""
+    import torch
+    from paper_2505_03803_b200 import binding as B
+    from paper_2505_03803_b200 import stack as stack_mod
+    peak, kind = measured_hbm_peak()
+    ws = torch.empty(B.rwkvq_proxy_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+
+    def timed(w):
+        B.rwkvq_proxy_select([w], 4, math.inf, math.inf, ws)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            pc, pf, _ = B.rwkvq_proxy_select([w], 4, math.inf, math.inf, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps, float(pc[0]), float(pf[0])
+    small = stack_mod.gen_weight_device(11, 256, 256, "gauss")
+    fixed_ms, _, _ = timed(small)
+    rows = []
+    for (oc, ic, kind_w) in ((4096, 4096, "gauss"), (14336, 4096, "gauss"), (4096, 4096, "student")):
+        w = stack_mod.gen_weight_device(12 + oc, oc, ic, kind_w)
+        ms, pc, pf = timed(w)
+        stream_ms = max(1e-6, ms - fixed_ms)
+        gbs = 2.0 * oc * ic / (stream_ms * 1e-3) / 1e9
+        rows.append({"matrix": f"{oc}x{ic} {kind_w}", "call_ms": ms, "histogram_ms": stream_ms, "P_c": pc, "P_f": pf,
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                  "traffic": None, "peak_kind": f"of {kind}", "kernel": "proxy_hist_kernel",
+                                  "algorithmic_bytes_per_launch": 2 * oc * ic}})
+        if with_oracle and oc == 4096 and kind_w == "gauss":
+            from oracle import rwkvq_oracle as orc
+            wh = w.cpu().numpy().astype(np.float64)
+            t0 = time.perf_counter()
+            orc.proxy(wh, 4)
+            rows[-1]["oracle_s"] = time.perf_counter() - t0
+        del w
+    return {"workload": "rwkvq_proxy_select on one fp16 matrix resident on the device, K = 4", "fixed_call_ms": fixed_ms,
+            "fixed_call": "256 x 256 matrix: workspace clear, proxy_reduce_kernel, copy of the results, synchronization",
+            "matrices": rows}
 
 
 def quantize_leg(reps: int = 5):
@@ -372,7 +475,7 @@ def quantize_leg(reps: int = 5):
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
                          "peak_kind": f"of {kind}", "kernel": "sq_quantize_kernel", "algorithmic_bytes_per_layer": nbytes,
                          "timed": "eight rwkvq_quantize_dev_async calls and one rwkvq_quantize_check (a stream "
-                                  "synchronization) per layer; the kernel alone is in the ncu launch list under profiles/"},
+                                  "synchronization) per layer"},
             "vq": {"matrix": f"{oc}x{ic}, 64 entries, 10 Lloyd iterations", "ms": vq_ms, "tiles": (oc // 256) * (ic // 256),
                    "weights_per_s": oc * ic / (vq_ms * 1e-3)}}
 
@@ -380,65 +483,45 @@ def quantize_leg(reps: int = 5):
 # ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
+def build_stack(args, workload, batch):
     from paper_2505_03803_b200 import binding as B
-    from paper_2505_03803_b200 import build as build_mod
     from paper_2505_03803_b200 import inputs, stack as stack_mod
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; this benchmark has no CPU path (use --impl reference for the oracle)")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    if rank == 0:
-        build_mod.build()
-    if world > 1:
-        dist.barrier()
-    B.lib()
-
-    sp = inputs.STACKS[args.workload]
-    batch = args.batch or sp["batches"][0]
+    sp = inputs.STACKS[workload]
     force = None if args.force_method is None else (B.RWKVQ_SQ if args.force_method == "sq" else B.RWKVQ_VQ)
-    t_setup = time.time()
+    weights = args.weights or ("device" if args.quantizer == "device" else "host")
+    t0 = time.time()
     st = stack_mod.Stack(sp["d"], sp["h"], sp["layers"], sp["entries"], batch, n_outliers=sp["outliers"],
-                         tag=args.workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force,
-                         quantizer=args.quantizer)
+                         tag=workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force,
+                         quantizer=args.quantizer, weights=weights)
+    st.bench_setup_s = time.time() - t0
+    return st
+
+
+def measure_stack(st, args, workload, K, W, world, dist, gpu_id, with_e2e=True):
+    """W warm-up steps, then K timed steps of one stack at its current batch: device-resident timing
+    with one event per step boundary, then the end-to-end loop through rwkvq_step_run_host; clocks are
+    sampled over both."""
+    import torch
+    from paper_2505_03803_b200 import binding as B
+    batch = st.batch
     if args.stage_group > 0:
         for i, o in enumerate(st.ops):
             o.stage = i // args.stage_group
         st.n_stages = len({o.stage for o in st.ops})
     if args.mode == "step":
         st.plan_step()
-    setup_s = time.time() - t_setup
     run = st.run_step if args.mode == "step" else st.run_ops
     launches_per_step = 1 if args.mode == "step" else len(st.ops)
-
-    est_ms = max(0.05, st.stream_bytes / 4.0e9)    # ms per step at 4 TB/s: only sizes the default step count
-    K = args.steps if args.steps is not None else int(min(2000, max(20, 4000.0 / est_ms)))
-    W = args.warmup if args.warmup is not None else 5
-    W = max(W, 3)
-
     stream = torch.cuda.current_stream()
     for _ in range(W):
         run(stream)
     torch.cuda.synchronize()
     if B.rwkvq_device_status() != 0:
         raise SystemExit("bench.py: a device-side wait timed out during warm-up")
-
-    try:
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
-    except Exception:
-        gpu_id = str(local_rank)
     sampler = ClockSampler(gpu_id)
     sampler.start()
     time.sleep(0.3)
 
-    # ---- device-resident timing: K steps, one event per step boundary
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
     if world > 1:
         dist.barrier()
@@ -451,14 +534,13 @@ def run_ours(args):
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    t1 = time.time()
     total_ms = ev[0].elapsed_time(ev[K])
     per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) / launches_per_step for i in range(K)]
     status = B.rwkvq_device_status()
 
     # ---- end to end: activations from pinned host memory, results back to the host, every step
     e2e_ms = None
-    if args.mode == "step":
+    if with_e2e and args.mode == "step":
         for _ in range(3):
             st.run_step_host(stream)
         torch.cuda.synchronize()
@@ -477,64 +559,126 @@ def run_ours(args):
         e2e_ms = a.elapsed_time(b)
     t2 = time.time()
     clocks = sampler.stop(t0, t2)
-    if status != 0:
+    if status != 0 or B.rwkvq_device_status() != 0:
         raise SystemExit("bench.py: a device-side wait timed out during the timed region")
 
     max_ms, tokens = aggregate_over_ranks(total_ms, float(batch * K), dist if world > 1 else None)
-    value = tokens / (max_ms * 1e-3)
     e2e = None
     if e2e_ms is not None:
         m2, tok2 = aggregate_over_ranks(e2e_ms, float(batch * K), dist if world > 1 else None)
         e2e = {"value": tok2 / (m2 * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(st.act_host.numel()),
                "d2h_bytes_per_step": int(st.y_host.numel())}
-
     peak, peak_kind = measured_hbm_peak()
     alg_bytes = st.stream_bytes + st.act_bytes
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
     achieved = alg_bytes / launches_per_step / (avg_launch_ms * 1e-3) / 1e9
+    traffic = None
+    if (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE is not None and args.mode == "step" and args.stage_group == 0
+            and args.force_method is None):
+        traffic = int(NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": (NCU_TRAFFIC_BYTES.get((args.workload, batch, args.mode, args.force_method, args.distinct_layers))
-                            if args.stage_group == 0 and args.quantizer == "host" else None),
-                "peak_kind": f"of {peak_kind}", "kernel": "step_kernel" if args.mode == "step" else "gemv_kernel",
+                "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                "kernel": "step_kernel" if args.mode == "step" else "gemv_kernel",
                 "algorithmic_bytes_per_launch": alg_bytes / launches_per_step,
                 "launch_ms_avg": avg_launch_ms, "launch_ms_median": statistics.median(per_launch_ms),
                 "launch_ms_min": min(per_launch_ms), "frac_of_8TBs_nominal": achieved / 8000.0}
+    config = {"workload": workload_name(workload, batch), "batch": batch, "mode": args.mode,
+              "matrices": len(st.ops), "sq_matrices": st.n_sq, "stages": st.n_stages,
+              "weights": st.n_weights, "packed_bytes_per_step": st.stream_bytes,
+              "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src, "quantizer": st.quantizer,
+              "weights_drawn_on": st.weights, "stage_group": args.stage_group,
+              "l2": "inputs larger than L2: every step streams the whole packed stack once",
+              "not_included": "WKV recurrence, norms, gates, embedding and head are not part of the workload",
+              "tau_c": st.tau_c, "setup_s": round(st.bench_setup_s, 1)}
+    return {"value": tokens / (max_ms * 1e-3), "ms_per_step": max_ms / K, "steps": K, "warmup": W, "roofline": roofline,
+            "e2e": e2e, "clocks": clocks, "gpu_launches": K * launches_per_step, "config": config}
+
+
+def default_steps(st, args):
+    est_ms = max(0.05, st.stream_bytes / 2.0e9)    # ms per step at 2 TB/s: only sizes the default step count
+    K = args.steps if args.steps is not None else int(min(2000, max(20, 2000.0 / est_ms)))
+    W = max(args.warmup if args.warmup is not None else 5, 3)
+    return K, W
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_03803_b200 import binding as B
+    from paper_2505_03803_b200 import build as build_mod
+    from paper_2505_03803_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; this benchmark has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build_mod.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+
+    whole = args.workload is None
+    workload = args.workload or HEADLINE[0]
+    batch = args.batch or (HEADLINE[1] if whole else inputs.STACKS[workload]["batches"][0])
+    st = build_stack(args, workload, batch)
+    K, W = default_steps(st, args)
+    head = measure_stack(st, args, workload, K, W, world, dist, gpu_id)
+    head["config"]["replicas"] = "independent replica per GPU, no exchange step" if world > 1 else "single GPU"
+    del st
+    torch.cuda.empty_cache()
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return 0
 
-    prefill = None
-    if world == 1 and not args.no_prefill:
-        prefill = prefill_leg()
-    quantize = None
-    if world == 1 and not args.no_quantize:
-        quantize = quantize_leg()
+    configs = None
+    if whole and world == 1 and not args.no_configs:
+        configs, st, cur = {}, None, None
+        for (wl, b) in CONFIGS:
+            if cur != wl:
+                del st
+                torch.cuda.empty_cache()
+                st, cur = build_stack(args, wl, b), wl
+            else:
+                st.set_batch(b)
+            k, w = default_steps(st, args)
+            r = measure_stack(st, args, wl, k, w, 1, None, gpu_id)
+            configs[f"{wl}_b{b}"] = {"tokens_per_s": r["value"], "ms_per_step": r["ms_per_step"], "steps": r["steps"],
+                                     "roofline": r["roofline"], "clocks": r["clocks"], "e2e": r["e2e"],
+                                     "config": r["config"]}
+        del st
+        torch.cuda.empty_cache()
+
+    prefill = prefill_leg() if world == 1 and not args.no_prefill else None
+    quantize = quantize_leg() if world == 1 and not args.no_quantize else None
+    proxy = proxy_leg(with_oracle=not args.no_cpu_baseline) if world == 1 and not args.no_proxy else None
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        r = time_oracle(args.workload, batch, budget_s=12.0)
+        sp = inputs.STACKS[workload]
+        r = time_oracle(workload, batch, budget_s=12.0)
         cpu = {"value": r["value"], "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                "sample": (f"the oracle's decode + token shift + fp64 product over the 8 matrices of one layer "
                           f"({r['sample_weights']} of {r['total_weights']} weights), {r['n']} repetitions, "
                           f"{r['per_sample_s']:.3f} s each, scaled to {sp['layers']} layers")}
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": max_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16", "data": "synthetic",
-        "config": {"workload": workload_name(args.workload, batch), "batch": batch, "mode": args.mode,
-                   "matrices": len(st.ops), "sq_matrices": st.n_sq, "stages": st.n_stages,
-                   "weights": st.n_weights, "packed_bytes_per_step": st.stream_bytes,
-                   "activation_bytes_per_step": st.act_bytes, "distinct_layers": st.n_src, "quantizer": st.quantizer, "stage_group": args.stage_group,
-                   "l2": "inputs larger than L2: every step streams the whole packed stack once",
-                   "replicas": "independent replica per GPU, no exchange step" if world > 1 else "single GPU",
-                   "not_included": "WKV recurrence, norms, gates, embedding and head are not part of the workload",
-                   "tau_c": st.tau_c, "setup_s": round(setup_s, 1)},
-        "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-        "gpu_launches": K * launches_per_step,
-        "hbm_gbs": achieved, "prefill": prefill, "quantize": quantize,
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": head["steps"],
+        "warmup": head["warmup"], "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": head["config"],
+        "roofline": head["roofline"], "cpu_baseline": cpu, "e2e": head["e2e"], "clocks": head["clocks"],
+        "gpu_launches": head["gpu_launches"], "hbm_gbs": head["roofline"]["achieved"],
+        "configs": configs, "prefill": prefill, "quantize": quantize, "proxy": proxy,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

@@ -142,6 +142,14 @@ rwkvq_status rwkvq_proxy_family(const void* const* w_fp16_dev, const int* oc, co
  * n <= 0, fraction outside [0, 1], NaN among the values).
  */
 rwkvq_status rwkvq_tau_for_fraction(const double* values_host, int n, double sq_fraction, double* tau_out);
+/*
+ * Threshold for the same rule when the values fall into two clusters (the synthetic stacks mix
+ * Gaussian and heavy-tailed matrices, whose coarse proxies P_c of Eq. 9 are far apart): the
+ * midpoint of the widest gap between neighbouring finite values in sorted order, the first such
+ * gap when several are equally wide.  Fewer than two finite values, or all of them equal, give
+ * +inf (everything scalar-quantized).  Host only.  Errors: EINVAL (NULL, n <= 0, NaN among the values).
+ */
+rwkvq_status rwkvq_tau_largest_gap(const double* values_host, int n, double* tau_out);
 
 /*
  * Decode product y[b][i] = sum_j w_hat[i][j] * x_mix[b][j], 1 <= B <= 16 (Appendix A.1, the

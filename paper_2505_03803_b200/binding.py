@@ -61,7 +61,7 @@ EXPORTS = [
     "rwkvq_step_run_host", "rwkvq_step_plan_release", "rwkvq_step_set_wait", "rwkvq_step_plan_cover",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
-    "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
+    "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_tau_largest_gap", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
     "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
     "rwkvq_quantize_dev_async", "rwkvq_quantize_check",
 ]
@@ -109,6 +109,7 @@ def lib() -> C.CDLL:
     if hasattr(L, "rwkvq_proxy_family"):
         L.rwkvq_proxy_family.argtypes = [C.POINTER(vp), C.POINTER(i32), C.POINTER(i32), i32, C.POINTER(dbl), vp, sz, vp]
         L.rwkvq_tau_for_fraction.argtypes = [C.POINTER(dbl), i32, dbl, C.POINTER(dbl)]
+        L.rwkvq_tau_largest_gap.argtypes = [C.POINTER(dbl), i32, C.POINTER(dbl)]
     if hasattr(L, "rwkvq_quant_error"):
         L.rwkvq_quant_error_workspace_bytes.argtypes = [C.POINTER(Desc)]
         L.rwkvq_quant_error_workspace_bytes.restype = sz
@@ -341,6 +342,14 @@ def rwkvq_tau_for_fraction(values, sq_fraction: float) -> float:
     tau = C.c_double()
     _check(lib().rwkvq_tau_for_fraction(v.ctypes.data_as(C.POINTER(C.c_double)), v.size, float(sq_fraction),
                                         C.byref(tau)), "rwkvq_tau_for_fraction")
+    return float(tau.value)
+
+
+def rwkvq_tau_largest_gap(values) -> float:
+    v = np.ascontiguousarray(values, dtype=np.float64)
+    tau = C.c_double()
+    _check(lib().rwkvq_tau_largest_gap(v.ctypes.data_as(C.POINTER(C.c_double)), v.size, C.byref(tau)),
+           "rwkvq_tau_largest_gap")
     return float(tau.value)
 
 

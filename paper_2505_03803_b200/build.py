@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(PKG_DIR, "librwkvq.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math" if False else "-DRWKVQ_BUILD",
+    "-DRWKVQ_BUILD",
     "-Xcompiler", "-fPIC,-fopenmp,-O3,-fvisibility=default",
 ]
 

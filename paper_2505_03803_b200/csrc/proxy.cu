@@ -14,6 +14,7 @@
 #include <math.h>
 
 #include <algorithm>
+#include <cmath>
 #include <vector>
 
 #include "../../include/rwkvq.h"
@@ -276,6 +277,27 @@ rwkvq_status rwkvq_tau_for_fraction(const double* values, int n, double sq_fract
   if (k <= 0) *tau_out = -INFINITY;
   else if (k >= n) *tau_out = INFINITY;
   else *tau_out = 0.5 * (v[k - 1] + v[k]);
+  return RWKVQ_OK;
+}
+
+rwkvq_status rwkvq_tau_largest_gap(const double* values, int n, double* tau_out) {
+  if (!values || !tau_out || n <= 0) return RWKVQ_EINVAL;
+  std::vector<double> v;
+  v.reserve((size_t)n);
+  for (int i = 0; i < n; ++i) {
+    if (values[i] != values[i]) return RWKVQ_EINVAL;
+    if (std::isfinite(values[i])) v.push_back(values[i]);
+  }
+  std::sort(v.begin(), v.end());
+  *tau_out = INFINITY;
+  if (v.size() < 2 || v.back() == v.front()) return RWKVQ_OK;
+  size_t best = 0;
+  double widest = -1.0;
+  for (size_t i = 0; i + 1 < v.size(); ++i) {
+    const double gap = v[i + 1] - v[i];
+    if (gap > widest) { widest = gap; best = i; }     // the first of equally wide gaps
+  }
+  *tau_out = 0.5 * (v[best] + v[best + 1]);
   return RWKVQ_OK;
 }
 

@@ -17,19 +17,6 @@ from . import binding as B
 from . import inputs
 
 
-def largest_gap_threshold(pc: np.ndarray) -> float:
-    """Threshold in the middle of the widest gap between sorted finite P_c values: separates the
-    two clusters a stack of Gaussian and heavy-tailed matrices produces.  With fewer than two
-    distinct values everything is kept below the threshold."""
-    v = np.sort(np.asarray(pc, dtype=np.float64))
-    v = v[np.isfinite(v)]
-    if v.size < 2 or v[-1] == v[0]:
-        return math.inf
-    gaps = v[1:] - v[:-1]
-    i = int(np.argmax(gaps))
-    return float(0.5 * (v[i] + v[i + 1]))
-
-
 class MatrixEntry:
     __slots__ = ("layer", "name", "oc", "ic", "kind", "seed", "stage", "has_mu", "method", "pc", "pf",
                  "desc", "image", "mu_desc", "mu_image", "x", "xprev", "y", "act_off")
@@ -56,62 +43,91 @@ def _device_blob(w_dev, oc, ic, method, bits, kmeans_iters, seed):
     return _DeviceBlob(d, image)
 
 
+def gen_weight_device(seed: int, oc: int, ic: int, kind: str, device="cuda"):
+    """fp16 weight matrix [oc, ic] drawn on the device from a seeded generator: N(0, std 0.02), or
+    Student-t(nu=3) * 0.01 as a normal variate over the root of a chi-square(3) variate / 3.  Same
+    distributions as inputs.gen_weight, other values: set-up of the large stacks without the host
+    generator's minutes."""
+    gen = torch.Generator(device=device).manual_seed(int(seed) & 0x7FFFFFFFFFFFFFFF)
+    z = torch.randn((oc, ic), generator=gen, device=device, dtype=torch.float32)
+    if kind == "gauss":
+        return (z * 0.02).to(torch.float16)
+    if kind != "student":
+        raise ValueError(kind)
+    chi = torch.zeros_like(z)
+    for _ in range(3):
+        n = torch.randn((oc, ic), generator=gen, device=device, dtype=torch.float32)
+        chi.addcmul_(n, n)
+    return (z * torch.rsqrt(chi / 3.0) * 0.01).to(torch.float16)
+
+
 class Stack:
     """All projection matrices of `layers` RWKV-6 blocks of width d and channel-mix width h.
 
     Per matrix the weight distribution is N(0, 0.02) or Student-t(3)*0.01 by a seeded coin; the
-    SQ/VQ method comes from rwkvq_proxy_select with tau_c at the widest gap of the measured P_c and
-    tau_f = +inf; SQ is 3-bit group-128, VQ uses 2-D vectors with `entries` codebook entries per
-    256x256 tile.  The four time-mix input projections and the channel-mix key projection get a
-    VQ-coded token-shift vector.  `distinct_layers` > 0 draws weights for that many layers only and
-    reuses their values (in separate device buffers) for the remaining layers, to shorten set-up of
-    the large stacks.
+    SQ/VQ method comes from rwkvq_proxy_select with tau_c at the widest gap of the measured P_c
+    (rwkvq_tau_largest_gap) and tau_f = +inf; SQ is 3-bit group-128, VQ uses 2-D vectors with
+    `entries` codebook entries per 256x256 tile.  The four time-mix input projections and the
+    channel-mix key projection get a VQ-coded token-shift vector.  `distinct_layers` > 0 draws
+    weights for that many layers only and reuses their values (in separate device buffers) for the
+    remaining layers.  weights="device" draws the weights with a seeded generator on the device
+    (quantizer="device" only); weights="host" uses the numpy generators of the inputs module.
     """
 
     def __init__(self, d: int, h: int, layers: int, entries: int, batch: int, n_outliers: int = 8,
                  heavy_fraction: float = 0.1, tag: str = "stack", device: str = "cuda",
                  distinct_layers: int = 0, force_method: int | None = None, kmeans_iters: int = 10,
-                 verbose: bool = False, quantizer: str = "host"):
-        assert quantizer in ("host", "device")
-        self.quantizer = quantizer
-        self.d, self.h, self.layers, self.entries, self.batch = d, h, layers, entries, batch
+                 verbose: bool = False, quantizer: str = "host", weights: str = "host"):
+        assert quantizer in ("host", "device") and weights in ("host", "device")
+        if weights == "device" and quantizer != "device":
+            raise ValueError("weights drawn on the device are quantized on the device")
+        self.quantizer, self.weights = quantizer, weights
+        self.d, self.h, self.layers, self.entries = d, h, layers, entries
+        self.n_outliers = n_outliers
         self.tag, self.device = tag, device
         self.vq_bits = 6 if entries == 64 else 8
         self.ops: list[MatrixEntry] = []
         self.setup_seconds = {}
         t0 = time.time()
         shapes = inputs.layer_shapes(d, h)
+        self.shapes = shapes
         n_src = layers if distinct_layers <= 0 else min(layers, distinct_layers)
         self.n_src = n_src
         # pass 1: weights of the source layers, P_c / P_f on the device
-        host_w = {}
+        src_w = {}
         for l in range(n_src):
             mats = []
             for (name, oc, ic, has_mu, stage) in shapes:
                 seed = inputs.seed_of(tag, l, name)
                 kind = inputs.weight_kind(seed, heavy_fraction)
-                w = inputs.gen_weight(seed, oc, ic, kind)
-                host_w[(l, name)] = (w, kind, seed)
-                mats.append(torch.from_numpy(w).to(device))
+                if weights == "device":
+                    w_dev = gen_weight_device(seed, oc, ic, kind, device)
+                    src_w[(l, name)] = (w_dev, kind, seed)
+                else:
+                    w = inputs.gen_weight(seed, oc, ic, kind)
+                    w_dev = torch.from_numpy(w).to(device)
+                    src_w[(l, name)] = (w, kind, seed)
+                mats.append(w_dev)
             ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(mats)), dtype=torch.uint8, device=device)
             pc, pf, _ = B.rwkvq_proxy_select(mats, 4, math.inf, math.inf, ws)
             for (name, *_), a, b in zip(shapes, pc, pf):
-                host_w[(l, name)] += (float(a), float(b))
+                src_w[(l, name)] += (float(a), float(b))
             del mats, ws
         self.setup_seconds["generate+proxy"] = time.time() - t0
         t0 = time.time()
-        all_pc = np.array([v[3] for v in host_w.values()])
-        self.tau_c = largest_gap_threshold(all_pc)
+        all_pc = np.array([v[3] for v in src_w.values()])
+        self.tau_c = B.rwkvq_tau_largest_gap(all_pc)
         self.tau_f = math.inf
         # pass 2: selection (Eq. 18 inside the library), quantize + pack, upload
         packed = {}
         for l in range(n_src):
-            mats = [torch.from_numpy(host_w[(l, name)][0]).to(device) for (name, *_r) in shapes]
+            mats = [src_w[(l, name)][0] if weights == "device" else torch.from_numpy(src_w[(l, name)][0]).to(device)
+                    for (name, *_r) in shapes]
             ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(mats)), dtype=torch.uint8, device=device)
             _, _, phi = B.rwkvq_proxy_select(mats, 4, self.tau_c, self.tau_f, ws)
             del ws
             for (name, oc, ic, has_mu, stage), p, w_dev in zip(shapes, phi, mats):
-                w, kind, seed, pc_v, pf_v = host_w[(l, name)]
+                w, kind, seed, pc_v, pf_v = src_w[(l, name)]
                 method = int(p) if force_method is None else force_method
                 if quantizer == "device":
                     bits = 3 if method == B.RWKVQ_SQ else self.vq_bits
@@ -133,9 +149,32 @@ class Stack:
                     print(f"layer {l} {name}: {kind} pc={pc_v:.3f} -> {'SQ' if method else 'VQ'}", flush=True)
             del mats
             for (name, *_r) in shapes:
-                host_w.pop((l, name))
+                src_w.pop((l, name))
         self.setup_seconds["select+pack"] = time.time() - t0
         t0 = time.time()
+        self._packed = packed  # keeps the blobs (logical codes on request) for parity checks
+        # one device image per (layer, matrix): layers beyond the source layers get copies of their own
+        self._images = {}
+        for l in range(layers):
+            for (name, oc, ic, has_mu, stage) in shapes:
+                blob, mu_blob, *_r = packed[(l % n_src, name)]
+                if l < n_src and isinstance(blob, _DeviceBlob):      # already on the device: no second copy
+                    self._images[(l, name)] = (blob._image, mu_blob._image if has_mu else None)
+                else:
+                    self._images[(l, name)] = (blob.to_device(device), mu_blob.to_device(device) if has_mu else None)
+        self.setup_seconds["upload"] = time.time() - t0
+        self.set_batch(batch)
+
+    def set_batch(self, batch: int):
+        """(Re)builds the activation and output arenas and the product list for a decode batch; the
+        packed images stay where they are."""
+        t0 = time.time()
+        device, shapes, layers = self.device, self.shapes, self.layers
+        self.batch = batch
+        self.ops = []
+        if getattr(self, "_plan", None) is not None:
+            B.rwkvq_step_plan_release(self._plan)
+        self._plan = None
         # Activations of every product live in one device arena and the outputs in another, so a
         # step's inputs arrive in one host-to-device copy and its results leave in one copy back.
         def _al(n):
@@ -158,24 +197,24 @@ class Stack:
         act_np = self.act_host.numpy()
         k = 0
         for l in range(layers):
-            src = l % n_src
+            src = l % self.n_src
             for (name, oc, ic, has_mu, stage) in shapes:
-                blob, mu_blob, kind, seed, method, pc_v, pf_v = packed[(src, name)]
+                blob, mu_blob, kind, seed, method, pc_v, pf_v = self._packed[(src, name)]
                 xo, po, yo = slots[k]
                 k += 1
                 e = MatrixEntry()
                 e.layer, e.name, e.oc, e.ic, e.kind, e.seed = l, name, oc, ic, kind, seed
                 e.stage, e.has_mu, e.method, e.pc, e.pf = 4 * l + stage, has_mu, method, pc_v, pf_v
-                e.desc, e.image = blob.desc, blob.to_device(device)
-                e.mu_desc, e.mu_image = (mu_blob.desc, mu_blob.to_device(device)) if has_mu else (None, None)
-                act_seed = inputs.seed_of(tag, "act", l, name)
+                e.desc, e.image = blob.desc, self._images[(l, name)][0]
+                e.mu_desc, e.mu_image = (mu_blob.desc, self._images[(l, name)][1]) if has_mu else (None, None)
+                act_seed = inputs.seed_of(self.tag, "act", l, name)
                 nb = batch * ic * 2
                 if has_mu:
-                    x, xp = inputs.gen_activation_pair(act_seed, batch, ic, n_outliers)
+                    x, xp = inputs.gen_activation_pair(act_seed, batch, ic, self.n_outliers)
                     act_np[po:po + nb] = xp.astype(np.float16).reshape(-1).view(np.uint8)
                     e.xprev = self.act_arena[po:po + nb].view(torch.float16).view(batch, ic)
                 else:
-                    x = inputs.gen_activation(act_seed, batch, ic, n_outliers)
+                    x = inputs.gen_activation(act_seed, batch, ic, self.n_outliers)
                     e.xprev = None
                 act_np[xo:xo + nb] = x.astype(np.float16).reshape(-1).view(np.uint8)
                 e.x = self.act_arena[xo:xo + nb].view(torch.float16).view(batch, ic)
@@ -184,8 +223,6 @@ class Stack:
                 self.ops.append(e)
         self.act_arena.copy_(self.act_host)
         self.ops.sort(key=lambda o: o.stage)
-        self.setup_seconds["upload"] = time.time() - t0
-        self._packed = packed  # keeps the host blobs (logical codes) for parity checks
         self.n_weights = sum(o.oc * o.ic for o in self.ops)
         self.stream_bytes = sum(int(o.desc.stream_bytes) + (int(o.mu_desc.stream_bytes) if o.has_mu else 0)
                                 for o in self.ops)
@@ -194,7 +231,7 @@ class Stack:
         self.n_stages = len({o.stage for o in self.ops})
         ws_bytes = max(B.rwkvq_gemv_workspace_bytes(o.desc, batch) for o in self.ops)
         self.workspace = torch.zeros(max(ws_bytes, 256), dtype=torch.uint8, device=device)
-        self._plan = None
+        self.setup_seconds["activations"] = time.time() - t0
 
     def host_codes(self, op: MatrixEntry):
         """Logical codes (numpy) of a matrix and of its mu vector, exported by the packer."""

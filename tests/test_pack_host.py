@@ -267,3 +267,18 @@ def test_tau_for_fraction_matches_oracle():
         B.rwkvq_tau_for_fraction([1.0, float("nan")], 0.5)
     with pytest.raises(B.RwkvqError):
         B.rwkvq_tau_for_fraction([1.0], 1.5)
+
+
+def test_tau_largest_gap_separates_two_clusters():
+    """Worked cases: the threshold is the midpoint of the widest gap of the sorted finite values."""
+    assert B.rwkvq_tau_largest_gap([1.0, 1.2, 5.0, 1.1, 5.5]) == 0.5 * (1.2 + 5.0)
+    assert B.rwkvq_tau_largest_gap([3.0, 1.0, 2.0]) == 1.5              # equal gaps: the first one
+    assert B.rwkvq_tau_largest_gap([0.25, float("inf"), 0.75]) == 0.5    # non-finite values are ignored
+    assert np.isinf(B.rwkvq_tau_largest_gap([2.0, 2.0, 2.0])) and B.rwkvq_tau_largest_gap([2.0, 2.0]) > 0
+    assert np.isinf(B.rwkvq_tau_largest_gap([7.0]))
+    rng = np.random.default_rng(3)
+    lo, hi = rng.uniform(0.0, 1.0, 40), rng.uniform(3.0, 4.0, 6)
+    tau = B.rwkvq_tau_largest_gap(rng.permutation(np.concatenate([lo, hi])))
+    assert tau == 0.5 * (lo.max() + hi.min())
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_tau_largest_gap([1.0, float("nan")])

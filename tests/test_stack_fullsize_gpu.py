@@ -25,12 +25,23 @@ def _oracle_product(st, op):
     return orc.gemv(w_hat, x), orc.tolerance(w_hat, x)
 
 
-@pytest.mark.parametrize("name,batch,quantizer", [("c2_1p6b", 1, "host"), ("c3_7b", 8, "host"), ("c4_14b", 16, "host"),
-                                                  ("c2_1p6b", 1, "device"), ("c3_7b", 1, "device")])
-def test_whole_step_at_benchmark_size_matches_oracle_on_sampled_products(name, batch, quantizer):
+@pytest.mark.parametrize("name,batch,quantizer,weights", [
+    ("c2_1p6b", 1, "host", "host"), ("c3_7b", 8, "host", "host"), ("c4_14b", 16, "host", "host"),
+    ("c2_1p6b", 1, "device", "host"), ("c3_7b", 1, "device", "host"),
+    # the set-up bench.py times by default: weights drawn and quantized on the device
+    ("c4_14b", 16, "device", "device"), ("c3_7b", 8, "device", "device")])
+def test_whole_step_at_benchmark_size_matches_oracle_on_sampled_products(name, batch, quantizer, weights):
     # quantizer = "device": the images come from rwkvq_quantize_dev, the oracle decodes the codes
     # unpacked from those images
-    st = stack_mod.from_name(name, batch=batch, distinct_layers=1, kmeans_iters=2, quantizer=quantizer)
+    st = stack_mod.from_name(name, batch=batch, distinct_layers=2 if weights == "device" else 1, kmeans_iters=2,
+                             quantizer=quantizer, weights=weights)
+    _check_step(st, name)
+    if weights == "device" and name == "c3_7b":      # the same images under another batch size
+        st.set_batch(1)
+        _check_step(st, name)
+
+
+def _check_step(st, name):
     st.plan_step()
     for _ in range(2):                      # a second run must reproduce the first (outputs are cleared in the kernel)
         st.run_step()
