@@ -255,9 +255,18 @@ rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const 
 
 /*
  * Prefill product Y[t][i] = sum_j bf16(w_hat[i][j]) * x_mix[t][j] for M tokens, bf16 x bf16 ->
- * fp32 on the tensor cores.  x_mix[t] = X[t] + (X[t-1] - X[t]) (.) mu_hat, with X[-1] = xprev0
- * (zeros if NULL); mu NULL = no mix.  X_bf16_dev: [M][ic]; Y_dev: [M][oc] F32 or BF16.
- * workspace_dev: rwkvq_prefill_workspace_bytes() bytes (holds x_mix when mu is given).
+ * fp32 on the tensor cores (the dense contraction of the path: Appendix A.1, the projections of
+ * Eqs. 21-24 applied to a whole sequence).  bf16(w_hat) is the decoded weight (the fp32 rounding
+ * of s*(q-z), or the fp16 codebook entry) rounded to nearest even.  x_mix[t] = X[t] +
+ * (X[t-1] - X[t]) (.) mu_hat (Eq. 20), with X[-1] = xprev0 (zeros if NULL); mu NULL = no mix.
+ * X_bf16_dev: [M][ic] row-major; Y_dev: [M][oc] row-major, F32 or BF16; all device pointers,
+ * 16-byte aligned, owned by the caller.  workspace_dev: rwkvq_prefill_workspace_bytes() bytes,
+ * 128-byte aligned; it receives x_mix in the tensor core's operand layout and a scheduling word,
+ * and must not be shared by products in flight at the same time.  The call enqueues on `stream`
+ * and returns; a device-side wait that ran out shows in rwkvq_device_status (ETIMEOUT).
+ * Errors: EINVAL (NULL pointer, M <= 0, mu without mu_desc, xprev0 without mu, unknown y_dtype),
+ * ESHAPE (oc == 1, ic not a multiple of 8), EUNSUPPORTED (format), EALIGN, ENOMEM (workspace
+ * too small), ECUDA.
  */
 size_t rwkvq_prefill_workspace_bytes(const rwkvq_desc* W_desc, int M, int has_mu);
 rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* W_desc, const void* W_image_dev,
@@ -265,6 +274,28 @@ rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* W_desc, const void* W_image_de
                                 const void* X_bf16_dev, const void* xprev0_bf16_dev, int M,
                                 void* Y_dev, int y_dtype, void* workspace_dev,
                                 size_t workspace_bytes, void* stream);
+/*
+ * Up to 16 independent prefill products over the same M tokens as ONE persistent launch (plus one
+ * small mix launch per product): the output tiles of all products are handed to the SMs from one
+ * queue, longest contraction first, so no SM idles at the end of a short product.  The products
+ * of one dependency stage of a layer (R, K, V, G; or the channel-mix key and receptance) are such
+ * a group.  Each entry has the arguments of rwkvq_gemm_prefill; outputs and workspaces must be
+ * pairwise distinct.  Errors as rwkvq_gemm_prefill, checked for every product before anything is
+ * enqueued; EUNSUPPORTED for more than 16 products; EINVAL for a shared output or workspace.
+ */
+typedef struct rwkvq_prefill_op {
+  const rwkvq_desc* W_desc;
+  const void* W_image_dev;
+  const rwkvq_desc* mu_desc;      /* NULL with mu_image_dev == NULL */
+  const void* mu_image_dev;
+  const void* X_bf16_dev;
+  const void* xprev0_bf16_dev;    /* may be NULL */
+  void* Y_dev;
+  void* workspace_dev;
+  size_t workspace_bytes;
+} rwkvq_prefill_op;
+rwkvq_status rwkvq_gemm_prefill_grouped(const rwkvq_prefill_op* ops, int n_ops, int M, int y_dtype,
+                                        void* stream);
 
 /*
  * Decode the packed matrix to out_dev[oc][ic]: F32 = the exact value s*(q-z) (two IEEE fp32

@@ -54,12 +54,18 @@ class GemvOp(C.Structure):
                 ("stage", C.c_int32), ("y_dtype", C.c_int32)]
 
 
+class PrefillOp(C.Structure):
+    _fields_ = [("W_desc", C.POINTER(Desc)), ("W_image_dev", C.c_void_p), ("mu_desc", C.POINTER(Desc)),
+                ("mu_image_dev", C.c_void_p), ("X_bf16_dev", C.c_void_p), ("xprev0_bf16_dev", C.c_void_p),
+                ("Y_dev", C.c_void_p), ("workspace_dev", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
 EXPORTS = [
     "rwkvq_pack", "rwkvq_blob_desc", "rwkvq_blob_nbytes", "rwkvq_blob_image", "rwkvq_blob_export_codes",
     "rwkvq_image_unpack", "rwkvq_blob_free", "rwkvq_proxy_workspace_bytes", "rwkvq_proxy_select",
     "rwkvq_gemv_workspace_bytes", "rwkvq_gemv", "rwkvq_gemv_static", "rwkvq_gemv_static_max_scratch_bytes", "rwkvq_step_plan_bytes", "rwkvq_step_plan", "rwkvq_step_run",
     "rwkvq_step_run_host", "rwkvq_step_plan_release", "rwkvq_step_set_wait", "rwkvq_step_plan_cover",
-    "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_dequant", "rwkvq_device_status",
+    "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_gemm_prefill_grouped", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
     "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_tau_largest_gap", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
     "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
@@ -127,6 +133,7 @@ def lib() -> C.CDLL:
         L.rwkvq_prefill_workspace_bytes.argtypes = [C.POINTER(Desc), i32, i32]
         L.rwkvq_prefill_workspace_bytes.restype = sz
         L.rwkvq_gemm_prefill.argtypes = [C.POINTER(Desc), vp, C.POINTER(Desc), vp, vp, vp, i32, vp, i32, vp, sz, vp]
+        L.rwkvq_gemm_prefill_grouped.argtypes = [C.POINTER(PrefillOp), i32, i32, i32, vp]
     if hasattr(L, "rwkvq_quantize_dev"):
         L.rwkvq_desc_for.argtypes = [C.POINTER(QuantCfg), i32, i32, C.POINTER(Desc)]
         L.rwkvq_quantize_workspace_bytes.argtypes = []
@@ -440,6 +447,35 @@ def rwkvq_gemm_prefill(desc: Desc, W_image, mu_desc, mu_image, X, xprev0, M: int
                                     _dev_ptr(workspace),
                                     0 if workspace is None else workspace.numel() * workspace.element_size(),
                                     _stream_ptr(stream)), "rwkvq_gemm_prefill")
+
+
+def make_prefill_ops(entries):
+    """entries: dicts with desc, W, mu_desc, mu, X, xprev0, Y, workspace (CUDA tensors or None).  Returns
+    (array of PrefillOp, objects to keep alive while the array is in use)."""
+    arr = (PrefillOp * len(entries))()
+    keep = []
+    for o, e in zip(arr, entries):
+        o.W_desc = C.pointer(e["desc"])
+        o.W_image_dev = _dev_ptr(e["W"])
+        md = e.get("mu_desc")
+        if md is not None:
+            o.mu_desc = C.pointer(md)
+        o.mu_image_dev = _dev_ptr(e.get("mu"))
+        o.X_bf16_dev = _dev_ptr(e["X"])
+        o.xprev0_bf16_dev = _dev_ptr(e.get("xprev0"))
+        o.Y_dev = _dev_ptr(e["Y"])
+        ws = e.get("workspace")
+        o.workspace_dev = _dev_ptr(ws)
+        o.workspace_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+        keep.append(e)
+    return arr, keep
+
+
+def rwkvq_gemm_prefill_grouped(ops, M: int, y_dtype: int = RWKVQ_F32, stream=None):
+    """rwkvq_gemm_prefill_grouped on an array from make_prefill_ops (or a list of entry dicts)."""
+    if isinstance(ops, (list, tuple)):
+        ops, _keep = make_prefill_ops(ops)
+    _check(lib().rwkvq_gemm_prefill_grouped(ops, len(ops), M, y_dtype, _stream_ptr(stream)), "rwkvq_gemm_prefill_grouped")
 
 
 def rwkvq_desc_for(oc: int, ic: int, method: int, bits: int, *, group: int = 128, vec_dim: int = 2,

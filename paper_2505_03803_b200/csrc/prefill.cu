@@ -1,28 +1,35 @@
 // Prefill product Y[t][i] = sum_j bf16(w_hat[i][j]) * x_mix[t][j] on the tcgen05 tensor cores.
 //
-// Two launches.  (1) A pre-pass applies the token-shift mix of Appendix A.1 Eq. 20 along the
+// (1) A pre-pass per product applies the token-shift mix of Appendix A.1 Eq. 20 along the
 // sequence (x_mix[t] = X[t] + (X[t-1] - X[t]) (.) mu_hat, X[-1] = xprev0), rounds to bf16 and
 // writes the result tile by tile in the shared-memory operand layout of the tensor core (tiles of
 // 256 tokens x 64 columns, 128-byte rows, 128-byte swizzle), so that the main kernel fetches an
-// operand tile with ONE bulk asynchronous copy.  (2) The main kernel is persistent, one CTA per
-// SM, each looping over output tiles of 256 weight rows (two chunks of the packed image) x 256
-// tokens, so that one activation tile feeds two products:
-//   * a producer warp streams packed chunk pairs (27-34 KB per 256 columns) and activation tiles
-//     (32 KB per 64 columns) into shared memory with cp.async.bulk + mbarrier transactions;
-//   * sixteen dequantisation warps (one group of eight per row half, one warp per 16-row record)
-//     turn packed codes into bf16 with
-//     the shared unpack routines, exactly bf16_rne(s * (q - z)) or bf16_rne(codebook entry), and
-//     store them in the K-major 128-byte-swizzled layout; a proxy fence hands them to the tensor core;
+// operand tile with ONE bulk asynchronous copy.  (2) ONE persistent launch, one CTA per SM, covers
+// every product of the call (rwkvq_gemm_prefill_grouped; the single product is a group of one).
+// Output tiles of 128 weight rows (one chunk row of the packed image) x 256 tokens are handed out
+// by an atomic ticket, longest contraction first, so tiles of different products balance:
+//   * a producer thread draws the ticket, publishes the tile to the other roles through a small
+//     queue, and streams packed chunks (12-17 KB per 256 columns, two slots) and activation tiles
+//     (32 KB per 64 columns, three stages) into shared memory with cp.async.bulk + mbarrier
+//     transactions;
+//   * sixteen dequantisation warps in two groups (group g takes the 64-column blocks of parity g,
+//     one warp per 16-row record) turn packed codes into bf16, exactly bf16_rne of the fp32
+//     rounding of s * (q - z) or of the codebook entry, and store them in the K-major
+//     128-byte-swizzled layout, a ring of four tiles; a proxy fence hands them to the tensor core;
 //   * one thread issues tcgen05.mma (A = weights 128 x 16, B = activations 256 x 16, fp32
-//     accumulators in tensor memory, one of 256 columns per row half) and commits to mbarriers;
-//   * four epilogue warps read the accumulators with tcgen05.ld (lane = weight row, so a warp
-//     writes 32 consecutive outputs of one token) while the next tile's operands stream in.
+//     accumulators in tensor memory: two stages of 256 columns) and commits to mbarriers;
+//   * four epilogue warps read an accumulator stage with tcgen05.ld (lane = weight row, so a warp
+//     writes 32 consecutive outputs of one token) while the tensor core fills the other stage
+//     with the next tile.
 // Every wait is bounded; a wait that gives up raises the device status word and all roles leave
 // through the common exit, where tensor memory is freed.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
 
 #include "../../include/rwkvq.h"
 #include "format.h"
@@ -36,17 +43,20 @@ int* device_status_ptr();  // api_misc.cu
 namespace pf {
 
 constexpr int kTileTokens = 256, kTileRows = 128, kKBlock = 64;
-constexpr int kXStages = 3, kWStages = 2;   // rings: activation tiles (32 KB); dequantised weight tiles (16 KB), one ring per row half
+constexpr int kXStages = 3, kWStages = 4;   // rings: activation tiles (32 KB); dequantised weight tiles (16 KB)
 constexpr uint32_t kXTileBytes = kTileTokens * kKBlock * 2;   // 32 KB: activations of one stage
 constexpr uint32_t kWTileBytes = kTileRows * kKBlock * 2;     // 16 KB: dequantised weights of one stage
-constexpr uint32_t kPackedSlot = 2 * 8 * 2048 + 1024;         // two largest chunks (VQ, 8-bit) + their codebook
-constexpr int kPackedSlots = 1;
+constexpr uint32_t kPackedSlot = 8 * 2048 + 1024;             // the largest chunk (VQ, 8-bit) + its codebook
+constexpr int kPackedSlots = 2;
+constexpr int kTileQueue = 4;                                 // tiles the producer may run ahead of the slowest role
 constexpr uint32_t kCtrlBytes = 1024;
-constexpr uint32_t kSmemBytes = kCtrlBytes + kXStages * kXTileBytes + 2 * kWStages * kWTileBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
+constexpr uint32_t kSmemBytes = kCtrlBytes + kXStages * kXTileBytes + kWStages * kWTileBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
 constexpr int kRecordWarps = 8, kDequantGroups = 2, kDequantWarps = kRecordWarps * kDequantGroups, kEpilogueWarps = 4;
 constexpr int kThreads = 32 * (2 + kDequantWarps + kEpilogueWarps);
 constexpr uint32_t kPollLimit = 1u << 22;
-constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kTmemCols = 512;                           // two accumulator stages of kTileTokens columns
+constexpr int kMaxGroup = 16;                                 // products per launch
+constexpr size_t kTicketBytes = 256;                          // tail of a product's workspace: the tile ticket
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -117,7 +127,8 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // 32 lanes x 32 consecutive columns of an accumulator: register c of lane l = D[lane base + l][col + c].
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// The load is asynchronous: the registers hold the data only after tmem_ld_wait on the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
       "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -126,7 +137,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Waits for every tcgen05.ld of this thread; the array is an in/out operand so that no use of it
+// is scheduled before the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+        "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+        "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
 }
 
 // Byte offset of element (row r, column k) of a K-major tile with 128-byte rows (64 bf16) and the
@@ -177,22 +197,31 @@ __global__ void __launch_bounds__(256) prefill_mix_kernel(const __nv_bfloat16* X
   *reinterpret_cast<uint4*>(tile + sw128_offset((uint32_t)r, (uint32_t)(c % kKBlock))) = out;
 }
 
-struct PrefillArgs {
+struct PrefillArgs {          // one product of the group
   const uint8_t* payload;   // chunks of the packed image
   const uint8_t* aux;       // VQ codebooks
   const uint8_t* xtiles;    // x_mix in operand tile layout: [MT][KB] tiles of 32 KB
   void* Y;
-  int* status;
-  int oc, ic, M, KT, KB, MB, MT, n_tiles, fmt, entries, y_dtype;
+  int oc, ic, KT, KB, MB, fmt;
   uint32_t chunk_bytes, rec_bytes, cb_bytes;
+};
+
+struct GroupArgs {
+  PrefillArgs p[kMaxGroup];          // longest contraction first
+  int tile_start[kMaxGroup + 1];     // tickets of product i: tile_start[i] .. tile_start[i + 1] - 1
+  int n, M, MT, y_dtype;
+  unsigned* ticket;                  // cleared before the launch
+  int* status;
 };
 
 enum { PF_SQ3 = 0, PF_VQ6 = 1, PF_VQ8 = 2 };
 
 struct Ctrl {
-  uint64_t wfull[kPackedSlots], wempty[kPackedSlots];
-  uint64_t xfull[kXStages], xempty[kXStages], wready[2][kWStages], wfree[2][kWStages];
-  uint64_t accfull, accempty;
+  uint64_t cfull[kPackedSlots], cempty[kPackedSlots];
+  uint64_t xfull[kXStages], xempty[kXStages], wready[kWStages], wfree[kWStages];
+  uint64_t accfull[2], accempty[2];
+  uint64_t tqfull[kTileQueue], tqempty[kTileQueue];
+  int tileq[kTileQueue];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -204,18 +233,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 }
 
 // 64 columns (one triple) of an SQ record -> bf16 rows of the weight tile.  `r` are the sixteen
-// extracted half2 registers (each half = q + bias exactly); every value is
-// bf16_rne(fmul_rn(s, fsub_rn(q, z))), the rounding of the exact decode.
+// extracted half2 registers (each half = q + bias exactly).  s * q - s * z with one rounding
+// (s * z is exact in fp32: two 11-bit significands) is the fp32 rounding of the exact decode
+// s * (q - z); the tile holds its bf16 rounding.
 __device__ __forceinline__ void sq_store_triple(const uint32_t (&r)[16], uint32_t sz_lo, uint32_t sz_hi, uint8_t* wtile,
                                                 int row_base, int lane) {
   const int g = lane >> 2, t = lane & 3;
   const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sz_lo));   // (s, z) of row g
   const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sz_hi));   // (s, z) of row g + 8
+  const float nsz0 = -__fmul_rn(s0.x, s0.y), nsz1 = -__fmul_rn(s1.x, s1.y);
+  uint8_t* row0 = wtile + (uint32_t)(row_base + g) * 128u + 8u * (uint32_t)(t & 1);
+  const uint32_t sw = (uint32_t)g, c0 = (uint32_t)(t >> 1);     // (row_base + g) % 8 == g: row_base is a multiple of 16
 #pragma unroll
   for (int m = 0; m < 4; ++m) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const float s = h ? s1.x : s0.x, z = h ? s1.y : s0.y;
+      const float s = h ? s1.x : s0.x, nsz = h ? nsz1 : nsz0;
       uint32_t out[2];
 #pragma unroll
       for (int p = 0; p < 2; ++p) {
@@ -223,12 +256,11 @@ __device__ __forceinline__ void sq_store_triple(const uint32_t (&r)[16], uint32_
         // (q + bias) - bias is exact in fp16: both are integers below 2048
         const __half2 bias2 = __float2half2_rn((float)(1024 >> rwkvq_sq_pos(e)));
         const float2 qf = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&r[e]), bias2));
-        const float v0 = __fmul_rn(s, __fsub_rn(qf.x, z));
-        const float v1 = __fmul_rn(s, __fsub_rn(qf.y, z));
-        out[p] = pack_bf16(v0, v1);
+        out[p] = pack_bf16(__fmaf_rn(s, qf.x, nsz), __fmaf_rn(s, qf.y, nsz));
       }
-      const uint32_t off = sw128_offset((uint32_t)(row_base + g + 8 * h), (uint32_t)(16 * m + 4 * t));
-      *reinterpret_cast<uint2*>(wtile + off) = make_uint2(out[0], out[1]);
+      // element (row, 16 m + 4 t): 16-byte chunk (2 m + t / 2) ^ (row % 8), bytes 8 (t % 2) of it; rows g and g + 8 swizzle alike
+      const uint32_t off = (uint32_t)h * 1024u + ((((uint32_t)(2 * m) + c0) ^ sw) << 4);
+      *reinterpret_cast<uint2*>(row0 + off) = make_uint2(out[0], out[1]);
     }
   }
 }
@@ -262,22 +294,73 @@ __device__ __forceinline__ void vq_store_block(const uint32_t (&w)[2 * BITS], in
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs a) {
+// Ticket -> product index; the tile within the product is ticket - tile_start[product].
+__device__ __forceinline__ int product_of(const GroupArgs& ga, int ticket) {
+  int p = 0;
+  while (p + 1 < ga.n && ticket >= ga.tile_start[p + 1]) ++p;
+  return p;
+}
+
+// The next tile of this CTA as published by the producer (-1: none left, or another role gave up).
+// Called by whole warps (every lane reads the entry, lane 0 frees it) or by one thread alone.
+__device__ __forceinline__ int next_tile(Ctrl* ctrl, uint32_t& tq, bool whole_warp, int lane, volatile int* abortp, int* status) {
+  const int slot = (int)(tq % kTileQueue);
+  bool ok = mbar_wait(&ctrl->tqfull[slot], (tq / kTileQueue) & 1u, abortp, status);
+  if (whole_warp) ok = __all_sync(0xFFFFFFFFu, ok);
+  int g = -1;
+  if (ok) g = *reinterpret_cast<volatile int*>(&ctrl->tileq[slot]);
+  if (whole_warp) __syncwarp();
+  if (ok && (!whole_warp || lane == 0)) mbar_arrive(&ctrl->tqempty[slot]);
+  ++tq;
+  return g;
+}
+
+// The blocks of parity DG of one 256-column chunk: registers -> bf16 tiles of the weight ring.
+template <int DG>
+__device__ __forceinline__ bool dequant_chunk(const uint32_t (&w)[16], const uint4 sz, const uint32_t* cb, int fmt, uint32_t kb0,
+                                              Ctrl* ctrl, uint8_t* wring, int dw, int lane, volatile int* abortp, int* status) {
+#pragma unroll
+  for (int qq = 0; qq < 2; ++qq) {
+    const int q = 2 * qq + DG;
+    const uint32_t kb = kb0 + (uint32_t)q;
+    const int st = (int)(kb % kWStages);
+    if (!__all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfree[st], ((kb / kWStages) & 1u) ^ 1u, abortp, status))) return false;
+    uint8_t* wtile = wring + (size_t)st * kWTileBytes;
+    if (fmt == PF_SQ3) {
+      uint32_t r[16];
+      sq_unpack_triple(w[3 * q], w[3 * q + 1], w[3 * q + 2], r);
+      sq_store_triple(r, q < 2 ? sz.x : sz.y, q < 2 ? sz.z : sz.w, wtile, dw * 16, lane);
+    } else if (fmt == PF_VQ6) {
+      const uint32_t (&w6)[12] = *reinterpret_cast<const uint32_t (*)[12]>(&w[0]);
+      vq_store_block<6>(w6, q, cb, wtile, dw * 16, lane);
+    } else {
+      vq_store_block<8>(w, q, cb, wtile, dw * 16, lane);
+    }
+    // generic-proxy stores -> visible to the tensor core (async proxy)
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&ctrl->wready[st]);
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_constant__ GroupArgs ga) {
   extern __shared__ uint8_t smem_raw[];
   // operand tiles need 1024-byte alignment (8 rows of 128 bytes per swizzle group)
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
   uint8_t* xring = smem + kCtrlBytes;                        // [kXStages] activation tiles
-  uint8_t* wring = xring + kXStages * kXTileBytes;           // [2 row halves][kWStages] dequantised weight tiles
-  uint8_t* packed = wring + 2 * kWStages * kWTileBytes;      // [chunk A | chunk B | codebook]
+  uint8_t* wring = xring + kXStages * kXTileBytes;           // [kWStages] dequantised weight tiles
+  uint8_t* packed = wring + kWStages * kWTileBytes;          // [kPackedSlots] chunk | codebook
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abortp = &ctrl->abort_flag;
+  const int total = ga.tile_start[ga.n];
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kPackedSlots; ++s) { mbar_init(&ctrl->wfull[s], 1); mbar_init(&ctrl->wempty[s], kDequantWarps); }
+    for (int s = 0; s < kPackedSlots; ++s) { mbar_init(&ctrl->cfull[s], 1); mbar_init(&ctrl->cempty[s], kDequantWarps); }
     for (int s = 0; s < kXStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->xempty[s], 1); }
-    for (int h = 0; h < 2; ++h)
-      for (int s = 0; s < kWStages; ++s) { mbar_init(&ctrl->wready[h][s], kRecordWarps); mbar_init(&ctrl->wfree[h][s], 1); }
-    mbar_init(&ctrl->accfull, 1); mbar_init(&ctrl->accempty, kEpilogueWarps);
+    for (int s = 0; s < kWStages; ++s) { mbar_init(&ctrl->wready[s], kRecordWarps); mbar_init(&ctrl->wfree[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->accfull[s], 1); mbar_init(&ctrl->accempty[s], kEpilogueWarps); }
+    for (int s = 0; s < kTileQueue; ++s) { mbar_init(&ctrl->tqfull[s], 1); mbar_init(&ctrl->tqempty[s], 1 + kDequantWarps + kEpilogueWarps); }
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -286,28 +369,36 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctrl->tmem_base;
-  // A tile is 256 weight rows (row pair tr: chunks 2 tr and 2 tr + 1 of the image) x 256 tokens: one
-  // activation tile feeds two products, which halves the activation traffic from L2 per FLOP.
-  // The last row pair of a matrix with an odd number of chunks has only its first half.
 
   if (warp == 0) {
     // ---- producer ------------------------------------------------------------------------------
     if (lane == 0) {
-      uint32_t kt_iter = 0, kb_iter = 0;
+      uint32_t tq = 0, ck = 0, kb_iter = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x) {
-        const int tr = tile / a.MT, mt = tile % a.MT;
-        const bool has_b = 2 * tr + 1 < a.MB;
-        for (int kt = 0; kt < a.KT && ok; ++kt, ++kt_iter) {
-          ok = mbar_wait(&ctrl->wempty[0], (kt_iter & 1u) ^ 1u, abortp, a.status);
+      while (ok) {
+        const int slot = (int)(tq % kTileQueue);
+        ok = mbar_wait(&ctrl->tqempty[slot], ((tq / kTileQueue) & 1u) ^ 1u, abortp, ga.status);
+        if (!ok) break;
+        int g = (int)atomicAdd(ga.ticket, 1u);
+        if (g >= total) g = -1;
+        *reinterpret_cast<volatile int*>(&ctrl->tileq[slot]) = g;
+        mbar_arrive(&ctrl->tqfull[slot]);        // release: the entry is visible to whoever sees the phase complete
+        ++tq;
+        if (g < 0) break;
+        const int pi = product_of(ga, g);
+        const PrefillArgs& a = ga.p[pi];
+        const int local = g - ga.tile_start[pi], cr = local / ga.MT, mt = local % ga.MT;
+        for (int kt = 0; kt < a.KT && ok; ++kt, ++ck) {
+          const int c = (int)(ck % kPackedSlots);
+          ok = mbar_wait(&ctrl->cempty[c], ((ck / kPackedSlots) & 1u) ^ 1u, abortp, ga.status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&ctrl->wfull[0], a.chunk_bytes * (has_b ? 2u : 1u) + a.cb_bytes);
-          bulk_g2s(packed, a.payload + (size_t)((2 * tr) * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->wfull[0]);
-          if (has_b) bulk_g2s(packed + a.chunk_bytes, a.payload + (size_t)((2 * tr + 1) * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->wfull[0]);
-          if (a.cb_bytes) bulk_g2s(packed + 2 * a.chunk_bytes, a.aux + (size_t)(tr * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->wfull[0]);
+          uint8_t* slot_base = packed + (size_t)c * kPackedSlot;
+          mbar_arrive_expect_tx(&ctrl->cfull[c], a.chunk_bytes + a.cb_bytes);
+          bulk_g2s(slot_base, a.payload + (size_t)(cr * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->cfull[c]);
+          if (a.cb_bytes) bulk_g2s(slot_base + a.chunk_bytes, a.aux + (size_t)((cr >> 1) * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->cfull[c]);
           for (int q = 0; q < 4 && ok; ++q, ++kb_iter) {
             const int st = (int)(kb_iter % kXStages);
-            ok = mbar_wait(&ctrl->xempty[st], ((kb_iter / kXStages) & 1u) ^ 1u, abortp, a.status);
+            ok = mbar_wait(&ctrl->xempty[st], ((kb_iter / kXStages) & 1u) ^ 1u, abortp, ga.status);
             if (!ok) break;
             mbar_arrive_expect_tx(&ctrl->xfull[st], kXTileBytes);
             bulk_g2s(xring + (size_t)st * kXTileBytes, a.xtiles + ((size_t)mt * a.KB + (kt * 4 + q)) * kXTileBytes, kXTileBytes, &ctrl->xfull[st]);
@@ -317,139 +408,136 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
       // do not leave while copies issued by this thread may still be landing
       for (uint32_t i = (kb_iter > kXStages ? kb_iter - kXStages : 0); i < kb_iter; ++i)
         for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->xfull[i % kXStages], (i / kXStages) & 1u)) break;
-      if (kt_iter > 0)
-        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->wfull[0], (kt_iter - 1u) & 1u)) break;
+      for (uint32_t i = (ck > kPackedSlots ? ck - kPackedSlots : 0); i < ck; ++i)
+        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->cfull[i % kPackedSlots], (i / kPackedSlots) & 1u)) break;
     }
   } else if (warp == 1) {
     // ---- tensor-core issue -----------------------------------------------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16(kTileRows, kTileTokens);
-      uint32_t kb_iter = 0, kb_b = 0, tile_iter = 0;     // kb_b counts the blocks of tiles that have a second half
+      uint32_t tq = 0, kb_iter = 0, tile_iter = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x, ++tile_iter) {
-        const int tr = tile / a.MT;
-        const bool has_b = 2 * tr + 1 < a.MB;
-        ok = mbar_wait(&ctrl->accempty, (tile_iter & 1u) ^ 1u, abortp, a.status);
+      while (ok) {
+        const int g = next_tile(ctrl, tq, false, 0, abortp, ga.status);
+        if (g < 0) break;
+        const int KB = ga.p[product_of(ga, g)].KB;
+        const uint32_t as = tile_iter & 1u;
+        ok = mbar_wait(&ctrl->accempty[as], ((tile_iter >> 1) & 1u) ^ 1u, abortp, ga.status);
         if (!ok) break;
         tc_fence_after();
-        for (int kb = 0; kb < a.KB && ok; ++kb, ++kb_iter) {
-          const int xst = (int)(kb_iter % kXStages), sa = (int)(kb_iter % kWStages);
-          ok = mbar_wait(&ctrl->xfull[xst], (kb_iter / kXStages) & 1u, abortp, a.status) &&
-               mbar_wait(&ctrl->wready[0][sa], (kb_iter / kWStages) & 1u, abortp, a.status);
+        const uint32_t acc = tmem_base + as * (uint32_t)kTileTokens;
+        for (int kb = 0; kb < KB && ok; ++kb, ++kb_iter) {
+          const int xst = (int)(kb_iter % kXStages), wst = (int)(kb_iter % kWStages);
+          ok = mbar_wait(&ctrl->xfull[xst], (kb_iter / kXStages) & 1u, abortp, ga.status) &&
+               mbar_wait(&ctrl->wready[wst], (kb_iter / kWStages) & 1u, abortp, ga.status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t xs = smem_u32(xring + (size_t)xst * kXTileBytes);
-          const uint32_t wa = smem_u32(wring + (size_t)sa * kWTileBytes);
+          const uint32_t wa = smem_u32(wring + (size_t)wst * kWTileBytes);
 #pragma unroll
           for (int k = 0; k < kKBlock / 16; ++k)
-            umma_bf16(tmem_base, smem_desc_sw128(wa + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(&ctrl->wfree[0][sa]);
-          if (has_b) {
-            const int sb = (int)(kb_b % kWStages);
-            ok = mbar_wait(&ctrl->wready[1][sb], (kb_b / kWStages) & 1u, abortp, a.status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t wb = smem_u32(wring + (size_t)(kWStages + sb) * kWTileBytes);
-#pragma unroll
-            for (int k = 0; k < kKBlock / 16; ++k)
-              umma_bf16(tmem_base + (uint32_t)kTileTokens, smem_desc_sw128(wb + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-            umma_commit(&ctrl->wfree[1][sb]);
-            ++kb_b;
-          }
-          umma_commit(&ctrl->xempty[xst]);    // the activation tile is free once both products have read it
+            umma_bf16(acc, smem_desc_sw128(wa + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(&ctrl->wfree[wst]);
+          umma_commit(&ctrl->xempty[xst]);
         }
-        if (ok) umma_commit(&ctrl->accfull);
+        if (ok) umma_commit(&ctrl->accfull[as]);
+        ++tile_iter;
       }
     }
   } else if (warp < 2 + kDequantWarps) {
-    // ---- dequantisation: group dg takes row half dg of the tile, warp dw its record dw (16 rows) ----
-    const int dw = (warp - 2) & 7, dg = (warp - 2) >> 3, g = lane >> 2;
-    uint32_t kt_iter = 0, kbm = 0;      // kbm: 64-column blocks this group has produced
+    // ---- dequantisation: warp dw takes record dw (16 rows) of the chunk, group dg the blocks of parity dg ----
+    const int dw = (warp - 2) & 7, dg = (warp - 2) >> 3, g8 = lane >> 2;
+    uint32_t tq = 0, ck = 0, kb0 = 0;      // kb0: 64-column blocks before the current chunk
     bool ok = true;
-    for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x) {
-      const int tr = tile / a.MT;
-      const bool mine = dg == 0 || 2 * tr + 1 < a.MB;     // the second half may be absent
-      for (int kt = 0; kt < a.KT && ok; ++kt, ++kt_iter) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfull[0], kt_iter & 1u, abortp, a.status));
+    while (ok) {
+      const int g = next_tile(ctrl, tq, true, lane, abortp, ga.status);
+      if (g < 0) break;
+      const PrefillArgs& a = ga.p[product_of(ga, g)];
+      const int fmt = a.fmt, KT = a.KT;
+      const uint32_t chunk_bytes = a.chunk_bytes, rec_bytes = a.rec_bytes;
+      for (int kt = 0; kt < KT && ok; ++kt, ++ck, kb0 += 4) {
+        const int c = (int)(ck % kPackedSlots);
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->cfull[c], (ck / kPackedSlots) & 1u, abortp, ga.status));
         if (!ok) break;
-        const uint8_t* rec = packed + (size_t)dg * a.chunk_bytes + (size_t)dw * a.rec_bytes;
-        const uint32_t* cb = reinterpret_cast<const uint32_t*>(packed + 2 * a.chunk_bytes);
+        const uint8_t* slot_base = packed + (size_t)c * kPackedSlot;
+        const uint8_t* rec = slot_base + (size_t)dw * rec_bytes;
+        const uint32_t* cb = reinterpret_cast<const uint32_t*>(slot_base + chunk_bytes);
         uint32_t w[16];
         uint4 sz = make_uint4(0, 0, 0, 0);
-        const int nplanes = a.fmt == PF_VQ8 ? 4 : 3;
+        const int nplanes = fmt == PF_VQ8 ? 4 : 3;
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
           uint4 v = make_uint4(0, 0, 0, 0);
-          if (mine && p < nplanes) v = *reinterpret_cast<const uint4*>(rec + p * 512 + lane * 16);
+          if (p < nplanes) v = *reinterpret_cast<const uint4*>(rec + p * 512 + lane * 16);
           w[4 * p] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
         }
-        if (mine && a.fmt == PF_SQ3) sz = *reinterpret_cast<const uint4*>(rec + RWKVQ_SQ_CODE_BYTES + g * 16);
-        // SQ needs nothing more from the packed slot (the codes are in registers): free it now so
-        // that the next 256 columns stream in while these are expanded.  VQ still reads the codebook.
-        const bool early = a.fmt == PF_SQ3;
+        if (fmt == PF_SQ3) sz = *reinterpret_cast<const uint4*>(rec + RWKVQ_SQ_CODE_BYTES + g8 * 16);
+        // SQ needs nothing more from the packed slot (the codes are in registers): free it now.
+        // VQ still reads the codebook while it expands the blocks.
+        const bool early = fmt == PF_SQ3;
         __syncwarp();
-        if (early && lane == 0) mbar_arrive(&ctrl->wempty[0]);
-        if (mine) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q, ++kbm) {
-            const int st = (int)(kbm % kWStages);
-            if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->wfree[dg][st], ((kbm / kWStages) & 1u) ^ 1u, abortp, a.status));
-            if (ok) {
-              uint8_t* wtile = wring + (size_t)(dg * kWStages + st) * kWTileBytes;
-              if (a.fmt == PF_SQ3) {
-                uint32_t r[16];
-                sq_unpack_triple(w[3 * q], w[3 * q + 1], w[3 * q + 2], r);
-                sq_store_triple(r, q < 2 ? sz.x : sz.y, q < 2 ? sz.z : sz.w, wtile, dw * 16, lane);
-              } else if (a.fmt == PF_VQ6) {
-                const uint32_t (&w6)[12] = *reinterpret_cast<const uint32_t (*)[12]>(&w[0]);
-                vq_store_block<6>(w6, q, cb, wtile, dw * 16, lane);
-              } else {
-                vq_store_block<8>(w, q, cb, wtile, dw * 16, lane);
-              }
-              // generic-proxy stores -> visible to the tensor core (async proxy)
-              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&ctrl->wready[dg][st]);
-            }
-          }
-        }
+        if (early && lane == 0) mbar_arrive(&ctrl->cempty[c]);
+        ok = dg == 0 ? dequant_chunk<0>(w, sz, cb, fmt, kb0, ctrl, wring, dw, lane, abortp, ga.status)
+                     : dequant_chunk<1>(w, sz, cb, fmt, kb0, ctrl, wring, dw, lane, abortp, ga.status);
         __syncwarp();
-        if (!early && ok && lane == 0) mbar_arrive(&ctrl->wempty[0]);
+        if (!early && ok && lane == 0) mbar_arrive(&ctrl->cempty[c]);
       }
     }
   } else {
-    // ---- epilogue: warp quarter qd reads lanes 32 qd .. 32 qd + 31 (weight rows) of both accumulators ----
+    // ---- epilogue: warp quarter qd reads lanes 32 qd .. 32 qd + 31 (weight rows) of an accumulator stage ----
     const int qd = warp & 3;
-    uint32_t tile_iter = 0;
+    uint32_t tq = 0, tile_iter = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < a.n_tiles && ok; tile += gridDim.x, ++tile_iter) {
-      const int tr = tile / a.MT, mt = tile % a.MT;
-      const int halves = 2 * tr + 1 < a.MB ? 2 : 1;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->accfull, tile_iter & 1u, abortp, a.status));
+    while (ok) {
+      const int g = next_tile(ctrl, tq, true, lane, abortp, ga.status);
+      if (g < 0) break;
+      const int pi = product_of(ga, g);
+      const PrefillArgs& a = ga.p[pi];
+      const int local = g - ga.tile_start[pi], cr = local / ga.MT, mt = local % ga.MT;
+      const uint32_t as = tile_iter & 1u;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->accfull[as], (tile_iter >> 1) & 1u, abortp, ga.status));
       if (!ok) break;
       tc_fence_after();
-      const int t0 = mt * kTileTokens;
-      for (int h = 0; h < halves; ++h) {
-        const int row = (2 * tr + h) * kTileRows + qd * 32 + lane;
+      const int t0 = mt * kTileTokens, row = cr * kTileRows + qd * 32 + lane, oc = a.oc;
+      const uint32_t acc = tmem_base + as * (uint32_t)kTileTokens + ((uint32_t)(qd * 32) << 16);
+      const bool row_ok = row < oc;
+      float* yf = static_cast<float*>(a.Y) + row;
+      __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(a.Y) + row;
+      const bool f32 = ga.y_dtype == RWKVQ_F32;
+      // two register buffers: the load of the next 32 columns is in flight while these are stored
+      uint32_t ra[32], rb[32];
+      tmem_ld32_issue(acc, ra);
 #pragma unroll 1
-        for (int cc = 0; cc < kTileTokens / 32; ++cc) {
-          uint32_t r[32];
-          tmem_ld32(tmem_base + (uint32_t)(h * kTileTokens + cc * 32) + ((uint32_t)(qd * 32) << 16), r);
-          if (row < a.oc) {
+      for (int cc = 0; cc < kTileTokens / 32; cc += 2) {
+        tmem_ld_wait(ra);
+        tmem_ld32_issue(acc + (uint32_t)((cc + 1) * 32), rb);
+        if (row_ok) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int t = t0 + cc * 32 + c;
-              if (t < a.M) {
-                if (a.y_dtype == RWKVQ_F32) static_cast<float*>(a.Y)[(size_t)t * a.oc + row] = __uint_as_float(r[c]);
-                else static_cast<__nv_bfloat16*>(a.Y)[(size_t)t * a.oc + row] = __float2bfloat16_rn(__uint_as_float(r[c]));
-              }
+          for (int c = 0; c < 32; ++c) {
+            const int t = t0 + cc * 32 + c;
+            if (t < ga.M) {
+              if (f32) yf[(size_t)t * oc] = __uint_as_float(ra[c]);
+              else yb[(size_t)t * oc] = __float2bfloat16_rn(__uint_as_float(ra[c]));
+            }
+          }
+        }
+        tmem_ld_wait(rb);
+        if (cc + 2 < kTileTokens / 32) tmem_ld32_issue(acc + (uint32_t)((cc + 2) * 32), ra);
+        if (row_ok) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const int t = t0 + (cc + 1) * 32 + c;
+            if (t < ga.M) {
+              if (f32) yf[(size_t)t * oc] = __uint_as_float(rb[c]);
+              else yb[(size_t)t * oc] = __float2bfloat16_rn(__uint_as_float(rb[c]));
             }
           }
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&ctrl->accempty);
+      if (lane == 0) mbar_arrive(&ctrl->accempty[as]);
+      ++tile_iter;
     }
   }
   // common exit: every role's loops are bounded, so all threads arrive here
@@ -463,71 +551,128 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillArgs 
 
 using namespace rwkvq;
 
+namespace {
+
+struct HostProduct {
+  pf::PrefillArgs a;
+  const void* X; const void* xprev0;
+  const uint8_t* mup; const uint8_t* mua; int mu_bits;
+  uint8_t* ws;
+};
+
+rwkvq_status check_product(const rwkvq_prefill_op& o, int M, HostProduct* out) {
+  const rwkvq_desc* d = o.W_desc;
+  if (!d || !o.W_image_dev || !o.X_bf16_dev || !o.Y_dev) return RWKVQ_EINVAL;
+  if (o.mu_image_dev && !o.mu_desc) return RWKVQ_EINVAL;
+  if (!o.mu_image_dev && o.xprev0_bf16_dev) return RWKVQ_EINVAL;
+  if (d->oc == 1) return RWKVQ_ESHAPE;
+  rwkvq_status st = check_matrix_desc(d);
+  if (st != RWKVQ_OK) return st;
+  if (o.mu_image_dev) {
+    st = check_vector_desc(o.mu_desc, d->ic);
+    if (st != RWKVQ_OK) return st;
+  }
+  if (d->ic % 8) return RWKVQ_ESHAPE;
+  if (!aligned16(o.W_image_dev) || !aligned16(o.X_bf16_dev) || !aligned16(o.Y_dev) || (o.mu_image_dev && !aligned16(o.mu_image_dev)) ||
+      (o.xprev0_bf16_dev && !aligned16(o.xprev0_bf16_dev)))
+    return RWKVQ_EALIGN;
+  const size_t need = rwkvq_prefill_workspace_bytes(d, M, o.mu_image_dev != nullptr);
+  if (!o.workspace_dev || o.workspace_bytes < need) return RWKVQ_ENOMEM;
+  if ((reinterpret_cast<uintptr_t>(o.workspace_dev) & 127u) != 0) return RWKVQ_EALIGN;
+  const uint8_t* img = static_cast<const uint8_t*>(o.W_image_dev);
+  pf::PrefillArgs& a = out->a;
+  a.payload = img + RWKVQ_HEADER_BYTES;
+  a.aux = img + matrix_aux_offset(d);
+  a.xtiles = static_cast<const uint8_t*>(o.workspace_dev);
+  a.Y = o.Y_dev;
+  a.oc = d->oc; a.ic = d->ic;
+  a.KT = d->ic_pad / 256; a.KB = a.KT * 4; a.MB = d->oc_pad / 128;
+  a.fmt = d->method == RWKVQ_SQ ? pf::PF_SQ3 : (d->bits == 6 ? pf::PF_VQ6 : pf::PF_VQ8);
+  a.rec_bytes = d->method == RWKVQ_SQ ? (uint32_t)RWKVQ_SQ_RECORD_BYTES : rwkvq_vq_record_bytes(d->bits);
+  a.chunk_bytes = 8u * a.rec_bytes;
+  a.cb_bytes = d->method == RWKVQ_SQ ? 0u : (uint32_t)d->entries * 4u;
+  out->X = o.X_bf16_dev; out->xprev0 = o.xprev0_bf16_dev;
+  out->mup = nullptr; out->mua = nullptr; out->mu_bits = 0;
+  if (o.mu_image_dev) {
+    const uint8_t* m = static_cast<const uint8_t*>(o.mu_image_dev);
+    out->mup = m + RWKVQ_HEADER_BYTES; out->mua = m + vector_aux_offset(o.mu_desc); out->mu_bits = o.mu_desc->bits;
+  }
+  out->ws = static_cast<uint8_t*>(o.workspace_dev);
+  return RWKVQ_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 size_t rwkvq_prefill_workspace_bytes(const rwkvq_desc* d, int M, int has_mu) {
   (void)has_mu;   // the operand tiles are written whether or not a token shift is applied
   if (!d || M <= 0 || check_matrix_desc(d) != RWKVQ_OK) return 0;
   const size_t MT = ((size_t)M + pf::kTileTokens - 1) / pf::kTileTokens, KB = (size_t)d->ic_pad / pf::kKBlock;
-  return MT * KB * pf::kXTileBytes;
+  return MT * KB * pf::kXTileBytes + pf::kTicketBytes;
 }
 
-rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu, const void* X,
-                                const void* xprev0, int M, void* Y, int y_dtype, void* ws, size_t ws_bytes, void* stream) {
-  if (!d || !W || !X || !Y || M <= 0) return RWKVQ_EINVAL;
+rwkvq_status rwkvq_gemm_prefill_grouped(const rwkvq_prefill_op* ops, int n_ops, int M, int y_dtype, void* stream) {
+  if (!ops || n_ops <= 0 || M <= 0) return RWKVQ_EINVAL;
+  if (n_ops > pf::kMaxGroup) return RWKVQ_EUNSUPPORTED;
   if (y_dtype != RWKVQ_F32 && y_dtype != RWKVQ_BF16) return RWKVQ_EINVAL;
-  if (mu && !mud) return RWKVQ_EINVAL;
-  if (!mu && xprev0) return RWKVQ_EINVAL;
-  if (d->oc == 1) return RWKVQ_ESHAPE;
-  rwkvq_status st = check_matrix_desc(d);
-  if (st != RWKVQ_OK) return st;
-  if (mu) {
-    st = check_vector_desc(mud, d->ic);
+  HostProduct hp[pf::kMaxGroup];
+  for (int i = 0; i < n_ops; ++i) {
+    const rwkvq_status st = check_product(ops[i], M, &hp[i]);
     if (st != RWKVQ_OK) return st;
+    for (int j = 0; j < i; ++j)
+      if (ops[j].Y_dev == ops[i].Y_dev || ops[j].workspace_dev == ops[i].workspace_dev) return RWKVQ_EINVAL;
   }
-  if (d->ic % 8) return RWKVQ_ESHAPE;
-  if (!aligned16(W) || !aligned16(X) || !aligned16(Y) || (mu && !aligned16(mu)) || (xprev0 && !aligned16(xprev0)) || (ws && !aligned16(ws)))
-    return RWKVQ_EALIGN;
-  const size_t need = rwkvq_prefill_workspace_bytes(d, M, mu != nullptr);
-  if (!ws || ws_bytes < need) return RWKVQ_ENOMEM;
-  if ((reinterpret_cast<uintptr_t>(ws) & 127u) != 0) return RWKVQ_EALIGN;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const uint8_t* img = static_cast<const uint8_t*>(W);
-  pf::PrefillArgs a;
-  a.payload = img + RWKVQ_HEADER_BYTES;
-  a.aux = img + matrix_aux_offset(d);
-  a.xtiles = static_cast<const uint8_t*>(ws);
-  a.Y = Y;
-  a.status = device_status_ptr();
-  if (!a.status) return RWKVQ_ECUDA;
-  a.oc = d->oc; a.ic = d->ic; a.M = M;
-  a.KT = d->ic_pad / 256; a.KB = a.KT * 4; a.MB = d->oc_pad / 128;
-  a.MT = (M + pf::kTileTokens - 1) / pf::kTileTokens;
-  a.n_tiles = ((a.MB + 1) / 2) * a.MT;
-  a.fmt = d->method == RWKVQ_SQ ? pf::PF_SQ3 : (d->bits == 6 ? pf::PF_VQ6 : pf::PF_VQ8);
-  a.entries = d->entries; a.y_dtype = y_dtype;
-  a.rec_bytes = d->method == RWKVQ_SQ ? (uint32_t)RWKVQ_SQ_RECORD_BYTES : rwkvq_vq_record_bytes(d->bits);
-  a.chunk_bytes = 8u * a.rec_bytes;
-  a.cb_bytes = d->method == RWKVQ_SQ ? 0u : (uint32_t)d->entries * 4u;
-  // pre-pass
-  const uint8_t* mup = nullptr; const uint8_t* mua = nullptr; int mu_bits = 0;
-  if (mu) {
-    const uint8_t* m = static_cast<const uint8_t*>(mu);
-    mup = m + RWKVQ_HEADER_BYTES; mua = m + vector_aux_offset(mud); mu_bits = mud->bits;
+  const int MT = (M + pf::kTileTokens - 1) / pf::kTileTokens;
+  // longest contraction first: the long tiles are dealt before the short ones fill the gaps
+  int order[pf::kMaxGroup];
+  for (int i = 0; i < n_ops; ++i) order[i] = i;
+  std::stable_sort(order, order + n_ops, [&](int x, int y) { return hp[x].a.KB > hp[y].a.KB; });
+  pf::GroupArgs ga;
+  memset(&ga, 0, sizeof(ga));
+  ga.n = n_ops; ga.M = M; ga.MT = MT; ga.y_dtype = y_dtype;
+  ga.status = device_status_ptr();
+  if (!ga.status) return RWKVQ_ECUDA;
+  long long total = 0;
+  for (int i = 0; i < n_ops; ++i) {
+    ga.p[i] = hp[order[i]].a;
+    ga.tile_start[i] = (int)total;
+    total += (long long)ga.p[i].MB * MT;
+    if (total > 0x3FFFFFFF) return RWKVQ_EUNSUPPORTED;
   }
-  const long long nvec = (long long)a.MT * pf::kTileTokens * a.KB * 8;
-  pf::prefill_mix_kernel<<<(unsigned)((nvec + 255) / 256), 256, 0, s>>>(
-      static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(xprev0), mup, mua, mu_bits, M, d->ic, a.KB, a.MT,
-      static_cast<uint8_t*>(ws));
-  cudaError_t e = cudaGetLastError();
+  ga.tile_start[n_ops] = (int)total;
+  const HostProduct& first = hp[order[0]];
+  ga.ticket = reinterpret_cast<unsigned*>(first.ws + (size_t)MT * first.a.KB * pf::kXTileBytes);
+  cudaError_t e = cudaMemsetAsync(ga.ticket, 0, sizeof(unsigned), s);
+  if (e != cudaSuccess) return cuda_status(e);
+  // pre-pass per product
+  for (int i = 0; i < n_ops; ++i) {
+    const HostProduct& h = hp[i];
+    const long long nvec = (long long)MT * pf::kTileTokens * h.a.KB * 8;
+    pf::prefill_mix_kernel<<<(unsigned)((nvec + 255) / 256), 256, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(h.X), static_cast<const __nv_bfloat16*>(h.xprev0), h.mup, h.mua, h.mu_bits, M, h.a.ic,
+        h.a.KB, MT, h.ws);
+  }
+  e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_status(e);
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   e = cudaFuncSetAttribute(pf::prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pf::kSmemBytes);
   if (e != cudaSuccess) return cuda_status(e);
-  const int grid = a.n_tiles < sms ? a.n_tiles : sms;
-  pf::prefill_kernel<<<grid, pf::kThreads, pf::kSmemBytes, s>>>(a);
+  const int grid = total < sms ? (int)total : sms;
+  pf::prefill_kernel<<<grid, pf::kThreads, pf::kSmemBytes, s>>>(ga);
   return cuda_status(cudaGetLastError());
+}
+
+rwkvq_status rwkvq_gemm_prefill(const rwkvq_desc* d, const void* W, const rwkvq_desc* mud, const void* mu, const void* X,
+                                const void* xprev0, int M, void* Y, int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+  if (!d || !W || !X || !Y || M <= 0) return RWKVQ_EINVAL;
+  if (mu && !mud) return RWKVQ_EINVAL;
+  rwkvq_prefill_op op;
+  op.W_desc = d; op.W_image_dev = W; op.mu_desc = mud; op.mu_image_dev = mu; op.X_bf16_dev = X; op.xprev0_bf16_dev = xprev0;
+  op.Y_dev = Y; op.workspace_dev = ws; op.workspace_bytes = ws_bytes;
+  return rwkvq_gemm_prefill_grouped(&op, 1, M, y_dtype, stream);
 }
 
 }  // extern "C"

@@ -161,3 +161,55 @@ def test_prefill_argument_errors():
     with pytest.raises(B.RwkvqError) as e:
         B.rwkvq_gemm_prefill(W.desc, W.dev, mu.desc, mu.dev, X, None, 4, Y, ws)
     assert e.value.status == 2
+
+
+def test_prefill_grouped_products_of_mixed_formats_and_lengths():
+    """One persistent launch over five products that differ in format, contraction length, row count and
+    token-shift use: every output equals the oracle's, and the single-product call gives the same bits."""
+    M = 300
+    specs = [("sq", 384, 1024, True), ("vq6", 256, 512, True), ("vq8", 512, 768, False), ("sq", 48, 384, True),
+             ("sq", 640, 2048, False)]
+    prods, entries = [], []
+    for i, (fmt, oc, ic, has_mu) in enumerate(specs):
+        W = (H.pack_sq(H.random_sq_codes(400 + i, oc, ic)) if fmt == "sq"
+             else H.pack_vq(H.random_vq_codes(410 + i, oc, ic, 6 if fmt == "vq6" else 8), 6 if fmt == "vq6" else 8))
+        mu = H.pack_mu(H.random_mu_codes(420 + i, ic)) if has_mu else None
+        Xv, Xd = _bf16(inputs.gen_activation(430 + i, M, ic, n_outliers=8))
+        p0v, p0d = (None, None)
+        if has_mu and i % 2 == 0:
+            p0v, p0d = _bf16(inputs.gen_activation(440 + i, 1, ic, n_outliers=8))
+            p0v, p0d = p0v.reshape(-1), p0d.reshape(-1)
+        Y = torch.full((M, oc), float("nan"), dtype=torch.float32, device="cuda")
+        ws = torch.empty(B.rwkvq_prefill_workspace_bytes(W.desc, M, has_mu), dtype=torch.uint8, device="cuda")
+        ws.fill_(0xCD)
+        prods.append((W, mu, Xv, Xd, p0v, p0d, Y))
+        entries.append(dict(desc=W.desc, W=W.dev, mu_desc=None if mu is None else mu.desc, mu=None if mu is None else mu.dev,
+                            X=Xd, xprev0=p0d, Y=Y, workspace=ws))
+    for _ in range(2):      # the scheduling word is cleared by every call
+        B.rwkvq_gemm_prefill_grouped(entries, M)
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 0
+    for (W, mu, Xv, Xd, p0v, p0d, Y) in prods:
+        xm = _reference(W, mu, Xv, p0v)
+        ref, tol = orc.gemv(W.w_hat, xm), orc.tolerance(W.w_hat, xm)
+        y = Y.cpu().numpy().astype(np.float64)
+        assert np.isfinite(y).all() and (np.abs(y - ref) <= tol).all()
+        single = _run(W, mu, Xd, p0d, M)
+        assert torch.equal(single, Y)
+
+
+def test_prefill_grouped_rejects_bad_groups():
+    W = H.pack_sq(H.random_sq_codes(450, 256, 512))
+    M = 64
+    _, Xd = _bf16(inputs.gen_activation(451, M, 512, n_outliers=8))
+    Y = torch.zeros((M, 256), dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.rwkvq_prefill_workspace_bytes(W.desc, M, False), dtype=torch.uint8, device="cuda")
+    e = dict(desc=W.desc, W=W.dev, X=Xd, Y=Y, workspace=ws)
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_gemm_prefill_grouped([e, dict(e)], M)                 # shared output and workspace
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_gemm_prefill_grouped([dict(e, workspace=ws[:1024])], M)      # workspace too small
+    with pytest.raises(B.RwkvqError):
+        B.rwkvq_gemm_prefill_grouped([e] * 17, M)
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 0
