@@ -9,13 +9,13 @@
 // Output tiles of 128 weight rows (one chunk row of the packed image) x 256 tokens are handed out
 // by an atomic ticket, longest contraction first, so tiles of different products balance:
 //   * a producer thread draws the ticket, publishes the tile to the other roles through a small
-//     queue, and streams packed chunks (12-17 KB per 256 columns, two slots) and activation tiles
-//     (32 KB per 64 columns, three stages) into shared memory with cp.async.bulk + mbarrier
-//     transactions;
+//     queue, and streams activation tiles (32 KB per 64 columns, four stages) into shared memory
+//     with cp.async.bulk + mbarrier transactions; a second producer thread streams the packed
+//     chunks (12-17 KB per 256 columns, as many slots as fit: two to four);
 //   * sixteen dequantisation warps in two groups (group g takes the 64-column blocks of parity g,
 //     one warp per 16-row record) turn packed codes into bf16, exactly bf16_rne of the fp32
 //     rounding of s * (q - z) or of the codebook entry, and store them in the K-major
-//     128-byte-swizzled layout, a ring of four tiles; a proxy fence hands them to the tensor core;
+//     128-byte-swizzled layout, a ring of three tiles; a proxy fence hands them to the tensor core;
 //   * one thread issues tcgen05.mma (A = weights 128 x 16, B = activations 256 x 16, fp32
 //     accumulators in tensor memory: two stages of 256 columns) and commits to mbarriers;
 //   * four epilogue warps read an accumulator stage with tcgen05.ld (lane = weight row, so a warp
@@ -43,16 +43,16 @@ int* device_status_ptr();  // api_misc.cu
 namespace pf {
 
 constexpr int kTileTokens = 256, kTileRows = 128, kKBlock = 64;
-constexpr int kXStages = 3, kWStages = 4;   // rings: activation tiles (32 KB); dequantised weight tiles (16 KB)
+constexpr int kXStages = 4, kWStages = 3;   // rings: activation tiles (32 KB); dequantised weight tiles (16 KB)
 constexpr uint32_t kXTileBytes = kTileTokens * kKBlock * 2;   // 32 KB: activations of one stage
 constexpr uint32_t kWTileBytes = kTileRows * kKBlock * 2;     // 16 KB: dequantised weights of one stage
-constexpr uint32_t kPackedSlot = 8 * 2048 + 1024;             // the largest chunk (VQ, 8-bit) + its codebook
-constexpr int kPackedSlots = 2;
+constexpr int kMaxPackedSlots = 4;                            // packed chunk (+ codebook) slots: as many as fit, at least two
 constexpr int kTileQueue = 4;                                 // tiles the producer may run ahead of the slowest role
 constexpr uint32_t kCtrlBytes = 1024;
-constexpr uint32_t kSmemBytes = kCtrlBytes + kXStages * kXTileBytes + kWStages * kWTileBytes + kPackedSlots * kPackedSlot + 1024;  // + alignment slack
+constexpr uint32_t kFixedSmemBytes = kCtrlBytes + kXStages * kXTileBytes + kWStages * kWTileBytes + 1024;  // + alignment slack
+constexpr uint32_t kMaxSmemBytes = 232448;                    // per-CTA limit of the architecture
 constexpr int kRecordWarps = 8, kDequantGroups = 2, kDequantWarps = kRecordWarps * kDequantGroups, kEpilogueWarps = 4;
-constexpr int kThreads = 32 * (2 + kDequantWarps + kEpilogueWarps);
+constexpr int kThreads = 32 * (3 + kDequantWarps + kEpilogueWarps);   // + activation producer, tensor-core issue, chunk producer
 constexpr uint32_t kPollLimit = 1u << 22;
 constexpr uint32_t kTmemCols = 512;                           // two accumulator stages of kTileTokens columns
 constexpr int kMaxGroup = 16;                                 // products per launch
@@ -210,6 +210,8 @@ struct GroupArgs {
   PrefillArgs p[kMaxGroup];          // longest contraction first
   int tile_start[kMaxGroup + 1];     // tickets of product i: tile_start[i] .. tile_start[i + 1] - 1
   int n, M, MT, y_dtype;
+  int n_slots;                       // packed chunk slots in use (2 .. kMaxPackedSlots)
+  uint32_t slot_bytes;               // bytes per slot: the largest chunk + codebook of the group, 128-byte multiple
   unsigned* ticket;                  // cleared before the launch
   int* status;
 };
@@ -217,7 +219,7 @@ struct GroupArgs {
 enum { PF_SQ3 = 0, PF_VQ6 = 1, PF_VQ8 = 2 };
 
 struct Ctrl {
-  uint64_t cfull[kPackedSlots], cempty[kPackedSlots];
+  uint64_t cfull[kMaxPackedSlots], cempty[kMaxPackedSlots];
   uint64_t xfull[kXStages], xempty[kXStages], wready[kWStages], wfree[kWStages];
   uint64_t accfull[2], accempty[2];
   uint64_t tqfull[kTileQueue], tqempty[kTileQueue];
@@ -294,7 +296,9 @@ __device__ __forceinline__ void vq_store_block(const uint32_t (&w)[2 * BITS], in
   }
 }
 
-// Ticket -> product index; the tile within the product is ticket - tile_start[product].
+// Ticket -> product index.  The tile within the product is ticket - tile_start[product], token tile
+// major (chunk row = tile % MB, token tile = tile / MB): CTAs that run at the same time read the
+// same few activation tiles from L2.
 __device__ __forceinline__ int product_of(const GroupArgs& ga, int ticket) {
   int p = 0;
   while (p + 1 < ga.n && ticket >= ga.tile_start[p + 1]) ++p;
@@ -351,16 +355,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
   uint8_t* xring = smem + kCtrlBytes;                        // [kXStages] activation tiles
   uint8_t* wring = xring + kXStages * kXTileBytes;           // [kWStages] dequantised weight tiles
-  uint8_t* packed = wring + kWStages * kWTileBytes;          // [kPackedSlots] chunk | codebook
+  uint8_t* packed = wring + kWStages * kWTileBytes;          // [n_slots] chunk | codebook
+  const uint32_t n_slots = (uint32_t)ga.n_slots, slot_bytes = ga.slot_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abortp = &ctrl->abort_flag;
   const int total = ga.tile_start[ga.n];
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kPackedSlots; ++s) { mbar_init(&ctrl->cfull[s], 1); mbar_init(&ctrl->cempty[s], kDequantWarps); }
+    for (int s = 0; s < kMaxPackedSlots; ++s) { mbar_init(&ctrl->cfull[s], 1); mbar_init(&ctrl->cempty[s], kDequantWarps); }
     for (int s = 0; s < kXStages; ++s) { mbar_init(&ctrl->xfull[s], 1); mbar_init(&ctrl->xempty[s], 1); }
     for (int s = 0; s < kWStages; ++s) { mbar_init(&ctrl->wready[s], kRecordWarps); mbar_init(&ctrl->wfree[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->accfull[s], 1); mbar_init(&ctrl->accempty[s], kEpilogueWarps); }
-    for (int s = 0; s < kTileQueue; ++s) { mbar_init(&ctrl->tqfull[s], 1); mbar_init(&ctrl->tqempty[s], 1 + kDequantWarps + kEpilogueWarps); }
+    for (int s = 0; s < kTileQueue; ++s) { mbar_init(&ctrl->tqfull[s], 1); mbar_init(&ctrl->tqempty[s], 2 + kDequantWarps + kEpilogueWarps); }
     ctrl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -371,9 +376,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
   const uint32_t tmem_base = ctrl->tmem_base;
 
   if (warp == 0) {
-    // ---- producer ------------------------------------------------------------------------------
+    // ---- activation producer: draws the tickets and streams the activation tiles ---------------------
     if (lane == 0) {
-      uint32_t tq = 0, ck = 0, kb_iter = 0;
+      uint32_t tq = 0, kb_iter = 0;
       bool ok = true;
       while (ok) {
         const int slot = (int)(tq % kTileQueue);
@@ -387,29 +392,43 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
         if (g < 0) break;
         const int pi = product_of(ga, g);
         const PrefillArgs& a = ga.p[pi];
-        const int local = g - ga.tile_start[pi], cr = local / ga.MT, mt = local % ga.MT;
-        for (int kt = 0; kt < a.KT && ok; ++kt, ++ck) {
-          const int c = (int)(ck % kPackedSlots);
-          ok = mbar_wait(&ctrl->cempty[c], ((ck / kPackedSlots) & 1u) ^ 1u, abortp, ga.status);
+        const int mt = (g - ga.tile_start[pi]) / a.MB, KB = a.KB;
+        const uint8_t* src = a.xtiles + (size_t)mt * KB * kXTileBytes;
+        for (int kb = 0; kb < KB && ok; ++kb, ++kb_iter) {
+          const int st = (int)(kb_iter % kXStages);
+          ok = mbar_wait(&ctrl->xempty[st], ((kb_iter / kXStages) & 1u) ^ 1u, abortp, ga.status);
           if (!ok) break;
-          uint8_t* slot_base = packed + (size_t)c * kPackedSlot;
-          mbar_arrive_expect_tx(&ctrl->cfull[c], a.chunk_bytes + a.cb_bytes);
-          bulk_g2s(slot_base, a.payload + (size_t)(cr * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->cfull[c]);
-          if (a.cb_bytes) bulk_g2s(slot_base + a.chunk_bytes, a.aux + (size_t)((cr >> 1) * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->cfull[c]);
-          for (int q = 0; q < 4 && ok; ++q, ++kb_iter) {
-            const int st = (int)(kb_iter % kXStages);
-            ok = mbar_wait(&ctrl->xempty[st], ((kb_iter / kXStages) & 1u) ^ 1u, abortp, ga.status);
-            if (!ok) break;
-            mbar_arrive_expect_tx(&ctrl->xfull[st], kXTileBytes);
-            bulk_g2s(xring + (size_t)st * kXTileBytes, a.xtiles + ((size_t)mt * a.KB + (kt * 4 + q)) * kXTileBytes, kXTileBytes, &ctrl->xfull[st]);
-          }
+          mbar_arrive_expect_tx(&ctrl->xfull[st], kXTileBytes);
+          bulk_g2s(xring + (size_t)st * kXTileBytes, src + (size_t)kb * kXTileBytes, kXTileBytes, &ctrl->xfull[st]);
         }
       }
       // do not leave while copies issued by this thread may still be landing
       for (uint32_t i = (kb_iter > kXStages ? kb_iter - kXStages : 0); i < kb_iter; ++i)
         for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->xfull[i % kXStages], (i / kXStages) & 1u)) break;
-      for (uint32_t i = (ck > kPackedSlots ? ck - kPackedSlots : 0); i < ck; ++i)
-        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->cfull[i % kPackedSlots], (i / kPackedSlots) & 1u)) break;
+    }
+  } else if (warp == 2 + kDequantWarps + kEpilogueWarps) {
+    // ---- chunk producer: streams the packed chunks (and codebooks) as far ahead as the slots allow ----
+    if (lane == 0) {
+      uint32_t tq = 0, ck = 0;
+      bool ok = true;
+      while (ok) {
+        const int g = next_tile(ctrl, tq, false, 0, abortp, ga.status);
+        if (g < 0) break;
+        const int pi = product_of(ga, g);
+        const PrefillArgs& a = ga.p[pi];
+        const int cr = (g - ga.tile_start[pi]) % a.MB;
+        for (int kt = 0; kt < a.KT && ok; ++kt, ++ck) {
+          const uint32_t c = ck % n_slots;
+          ok = mbar_wait(&ctrl->cempty[c], ((ck / n_slots) & 1u) ^ 1u, abortp, ga.status);
+          if (!ok) break;
+          uint8_t* slot_base = packed + (size_t)c * slot_bytes;
+          mbar_arrive_expect_tx(&ctrl->cfull[c], a.chunk_bytes + a.cb_bytes);
+          bulk_g2s(slot_base, a.payload + (size_t)(cr * a.KT + kt) * a.chunk_bytes, a.chunk_bytes, &ctrl->cfull[c]);
+          if (a.cb_bytes) bulk_g2s(slot_base + a.chunk_bytes, a.aux + (size_t)((cr >> 1) * a.KT + kt) * a.cb_bytes, a.cb_bytes, &ctrl->cfull[c]);
+        }
+      }
+      for (uint32_t i = (ck > n_slots ? ck - n_slots : 0); i < ck; ++i)
+        for (uint32_t it = 0; it < kPollLimit; ++it) if (mbar_try_wait(&ctrl->cfull[i % n_slots], (i / n_slots) & 1u)) break;
     }
   } else if (warp == 1) {
     // ---- tensor-core issue -----------------------------------------------------------------------
@@ -456,10 +475,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
       const int fmt = a.fmt, KT = a.KT;
       const uint32_t chunk_bytes = a.chunk_bytes, rec_bytes = a.rec_bytes;
       for (int kt = 0; kt < KT && ok; ++kt, ++ck, kb0 += 4) {
-        const int c = (int)(ck % kPackedSlots);
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->cfull[c], (ck / kPackedSlots) & 1u, abortp, ga.status));
+        const uint32_t c = ck % n_slots;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->cfull[c], (ck / n_slots) & 1u, abortp, ga.status));
         if (!ok) break;
-        const uint8_t* slot_base = packed + (size_t)c * kPackedSlot;
+        const uint8_t* slot_base = packed + (size_t)c * slot_bytes;
         const uint8_t* rec = slot_base + (size_t)dw * rec_bytes;
         const uint32_t* cb = reinterpret_cast<const uint32_t*>(slot_base + chunk_bytes);
         uint32_t w[16];
@@ -483,7 +502,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
         if (!early && ok && lane == 0) mbar_arrive(&ctrl->cempty[c]);
       }
     }
-  } else {
+  } else if (warp < 2 + kDequantWarps + kEpilogueWarps) {
     // ---- epilogue: warp quarter qd reads lanes 32 qd .. 32 qd + 31 (weight rows) of an accumulator stage ----
     const int qd = warp & 3;
     uint32_t tq = 0, tile_iter = 0;
@@ -493,7 +512,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
       if (g < 0) break;
       const int pi = product_of(ga, g);
       const PrefillArgs& a = ga.p[pi];
-      const int local = g - ga.tile_start[pi], cr = local / ga.MT, mt = local % ga.MT;
+      const int local = g - ga.tile_start[pi], cr = local % a.MB, mt = local / a.MB;
       const uint32_t as = tile_iter & 1u;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(&ctrl->accfull[as], (tile_iter >> 1) & 1u, abortp, ga.status));
       if (!ok) break;
@@ -642,6 +661,12 @@ rwkvq_status rwkvq_gemm_prefill_grouped(const rwkvq_prefill_op* ops, int n_ops, 
     if (total > 0x3FFFFFFF) return RWKVQ_EUNSUPPORTED;
   }
   ga.tile_start[n_ops] = (int)total;
+  uint32_t slot = 0;
+  for (int i = 0; i < n_ops; ++i) slot = std::max(slot, (ga.p[i].chunk_bytes + ga.p[i].cb_bytes + 127u) & ~127u);
+  ga.slot_bytes = slot;
+  ga.n_slots = (int)std::min<uint32_t>(pf::kMaxPackedSlots, (pf::kMaxSmemBytes - pf::kFixedSmemBytes) / slot);
+  if (ga.n_slots < 2) return RWKVQ_EUNSUPPORTED;
+  const uint32_t smem_bytes = pf::kFixedSmemBytes + (uint32_t)ga.n_slots * slot;
   const HostProduct& first = hp[order[0]];
   ga.ticket = reinterpret_cast<unsigned*>(first.ws + (size_t)MT * first.a.KB * pf::kXTileBytes);
   cudaError_t e = cudaMemsetAsync(ga.ticket, 0, sizeof(unsigned), s);
@@ -658,10 +683,10 @@ rwkvq_status rwkvq_gemm_prefill_grouped(const rwkvq_prefill_op* ops, int n_ops, 
   if (e != cudaSuccess) return cuda_status(e);
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  e = cudaFuncSetAttribute(pf::prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pf::kSmemBytes);
+  e = cudaFuncSetAttribute(pf::prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pf::kMaxSmemBytes);
   if (e != cudaSuccess) return cuda_status(e);
   const int grid = total < sms ? (int)total : sms;
-  pf::prefill_kernel<<<grid, pf::kThreads, pf::kSmemBytes, s>>>(ga);
+  pf::prefill_kernel<<<grid, pf::kThreads, smem_bytes, s>>>(ga);
   return cuda_status(cudaGetLastError());
 }
 
