@@ -75,6 +75,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(2000u) : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase (1 = complete).  Several tests issued back to back overlap their
+// latencies; a blocking try_wait would hold the thread, and with it the tensor-core issue, until
+// the phase completes or its time limit passes.
+__device__ __forceinline__ uint32_t mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok;
+}
 // Bounded wait: false after kPollLimit polls (status word set) or once another role has given up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   for (uint32_t it = 0; it < kPollLimit; ++it) {
@@ -445,12 +454,36 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
         if (!ok) break;
         tc_fence_after();
         const uint32_t acc = tmem_base + as * (uint32_t)kTileTokens;
+        // The operands of a block are ready when its activation stage has landed and its weight
+        // stage has been written.  The two phases are tested together, and those of the next block
+        // are tested before this block's instructions are issued, so that the tests' latencies
+        // overlap each other and the issue: tested one after the other with blocking waits, the
+        // waits and the six instructions of a block took longer than the tensor core needs for it.
+        bool ready = false;
         for (int kb = 0; kb < KB && ok; ++kb, ++kb_iter) {
           const int xst = (int)(kb_iter % kXStages), wst = (int)(kb_iter % kWStages);
-          ok = mbar_wait(&ctrl->xfull[xst], (kb_iter / kXStages) & 1u, abortp, ga.status) &&
-               mbar_wait(&ctrl->wready[wst], (kb_iter / kWStages) & 1u, abortp, ga.status);
+          const uint32_t xph = (kb_iter / kXStages) & 1u, wph = (kb_iter / kWStages) & 1u;
+          for (uint32_t it = 0; !ready; ++it) {
+            const uint32_t r0 = mbar_test(&ctrl->xfull[xst], xph);
+            const uint32_t r1 = mbar_test(&ctrl->wready[wst], wph);
+            ready = (r0 & r1) != 0u;
+            if (ready) break;
+            if ((it & 63u) == 63u && *abortp) { ok = false; break; }
+            if (it >= kPollLimit) {
+              *abortp = 1;
+              atomicExch(ga.status, (int)RWKVQ_ETIMEOUT);
+              ok = false;
+              break;
+            }
+          }
           if (!ok) break;
           tc_fence_after();
+          uint32_t n0 = 0u, n1 = 0u;
+          if (kb + 1 < KB) {
+            const uint32_t nk = kb_iter + 1u;
+            n0 = mbar_test(&ctrl->xfull[nk % kXStages], (nk / kXStages) & 1u);
+            n1 = mbar_test(&ctrl->wready[nk % kWStages], (nk / kWStages) & 1u);
+          }
           const uint32_t xs = smem_u32(xring + (size_t)xst * kXTileBytes);
           const uint32_t wa = smem_u32(wring + (size_t)wst * kWTileBytes);
 #pragma unroll
@@ -458,6 +491,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const __grid_const
             umma_bf16(acc, smem_desc_sw128(wa + k * 32), smem_desc_sw128(xs + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
           umma_commit(&ctrl->wfree[wst]);
           umma_commit(&ctrl->xempty[xst]);
+          ready = (n0 & n1) != 0u;
         }
         if (ok) umma_commit(&ctrl->accfull[as]);
         ++tile_iter;
