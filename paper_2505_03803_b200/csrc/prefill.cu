@@ -171,39 +171,60 @@ __device__ __forceinline__ uint32_t vec_index(const uint8_t* stream, int p, int 
   return (v >> (bitpos & 7u)) & ((1u << bits) - 1u);
 }
 
-// One thread per 8 consecutive columns of one (padded) token row.
+// One block per operand tile (256 tokens x 64 columns).  A thread owns 8 columns (one 16-byte vector)
+// and a run of kMixRun consecutive tokens: it decodes its four mu pairs once, reads each row's vector
+// once (the previous token's comes from the previous iteration) and writes 16 bytes per token into the
+// tile's swizzled rows; the eight threads of a row read and write 128 contiguous bytes.
+constexpr int kMixRun = 8;
+static_assert(kTileTokens == 32 * kMixRun, "a block of 256 threads covers one tile");
 __global__ void __launch_bounds__(256) prefill_mix_kernel(const __nv_bfloat16* X, const __nv_bfloat16* xprev0, const uint8_t* mu,
                                                           const uint8_t* mu_aux, int mu_bits, int M, int ic, int KB, int MT,
                                                           uint8_t* tiles) {
-  const long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int vec_per_row = KB * 8;
-  if (v >= (long long)MT * kTileTokens * vec_per_row) return;
-  const int t = (int)(v / vec_per_row), c = (int)(v % vec_per_row) * 8;
-  uint4 out = make_uint4(0u, 0u, 0u, 0u);
-  if (t < M && c < ic) {
-    const uint4 xr = *reinterpret_cast<const uint4*>(X + (size_t)t * ic + c);
-    out = xr;
-    if (mu) {
-      uint4 pr = make_uint4(0u, 0u, 0u, 0u);
-      if (t > 0) pr = *reinterpret_cast<const uint4*>(X + (size_t)(t - 1) * ic + c);
-      else if (xprev0) pr = *reinterpret_cast<const uint4*>(xprev0 + c);
-      const uint32_t xs[4] = {xr.x, xr.y, xr.z, xr.w}, ps[4] = {pr.x, pr.y, pr.z, pr.w};
-      uint32_t os[4];
+  const int kb = (int)(blockIdx.x % (unsigned)KB), mt = (int)(blockIdx.x / (unsigned)KB);
+  if (mt >= MT) return;
+  const int cx = threadIdx.x & 7, ty = threadIdx.x >> 3;
+  const int c = kb * kKBlock + cx * 8, r0 = ty * kMixRun, t0 = mt * kTileTokens + r0;
+  uint8_t* tile = tiles + ((size_t)mt * KB + kb) * kXTileBytes;
+  const bool col_ok = c < ic;
+  uint4 xr[kMixRun + 1];     // [0] = the token before the run
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const uint32_t mw = reinterpret_cast<const uint32_t*>(mu_aux)[vec_index(mu, (c >> 1) + k, mu_bits)];
-        const float2 mf = __half22float2(*reinterpret_cast<const __half2*>(&mw));
-        const float2 xf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&xs[k]));
-        const float2 pf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ps[k]));
-        const __nv_bfloat162 o = __floats2bfloat162_rn(fmaf(pf.x - xf.x, mf.x, xf.x), fmaf(pf.y - xf.y, mf.y, xf.y));
-        os[k] = *reinterpret_cast<const uint32_t*>(&o);
-      }
-      out = make_uint4(os[0], os[1], os[2], os[3]);
+  for (int i = 0; i <= kMixRun; ++i) {
+    const int t = t0 + i - 1;
+    xr[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (col_ok && t < M && (i > 0 || mu != nullptr)) {
+      if (t >= 0) xr[i] = *reinterpret_cast<const uint4*>(X + (size_t)t * ic + c);
+      else if (xprev0) xr[i] = *reinterpret_cast<const uint4*>(xprev0 + c);
     }
   }
-  const int mt = t / kTileTokens, r = t % kTileTokens, kb = c / kKBlock;
-  uint8_t* tile = tiles + ((size_t)mt * KB + kb) * kXTileBytes;
-  *reinterpret_cast<uint4*>(tile + sw128_offset((uint32_t)r, (uint32_t)(c % kKBlock))) = out;
+  float2 mf[4];
+  if (mu && col_ok) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t mw = reinterpret_cast<const uint32_t*>(mu_aux)[vec_index(mu, (c >> 1) + k, mu_bits)];
+      mf[k] = __half22float2(*reinterpret_cast<const __half2*>(&mw));
+    }
+  }
+#pragma unroll
+  for (int i = 1; i <= kMixRun; ++i) {
+    const int t = t0 + i - 1;
+    uint4 out = make_uint4(0u, 0u, 0u, 0u);
+    if (col_ok && t < M) {
+      out = xr[i];
+      if (mu) {
+        const uint32_t xs[4] = {xr[i].x, xr[i].y, xr[i].z, xr[i].w}, ps[4] = {xr[i - 1].x, xr[i - 1].y, xr[i - 1].z, xr[i - 1].w};
+        uint32_t os[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float2 xf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&xs[k]));
+          const float2 pf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ps[k]));
+          const __nv_bfloat162 o = __floats2bfloat162_rn(fmaf(pf.x - xf.x, mf[k].x, xf.x), fmaf(pf.y - xf.y, mf[k].y, xf.y));
+          os[k] = *reinterpret_cast<const uint32_t*>(&o);
+        }
+        out = make_uint4(os[0], os[1], os[2], os[3]);
+      }
+    }
+    *reinterpret_cast<uint4*>(tile + sw128_offset((uint32_t)(r0 + i - 1), (uint32_t)(cx * 8))) = out;
+  }
 }
 
 struct PrefillArgs {          // one product of the group
@@ -708,8 +729,7 @@ rwkvq_status rwkvq_gemm_prefill_grouped(const rwkvq_prefill_op* ops, int n_ops, 
   // pre-pass per product
   for (int i = 0; i < n_ops; ++i) {
     const HostProduct& h = hp[i];
-    const long long nvec = (long long)MT * pf::kTileTokens * h.a.KB * 8;
-    pf::prefill_mix_kernel<<<(unsigned)((nvec + 255) / 256), 256, 0, s>>>(
+    pf::prefill_mix_kernel<<<(unsigned)(MT * h.a.KB), 256, 0, s>>>(
         static_cast<const __nv_bfloat16*>(h.X), static_cast<const __nv_bfloat16*>(h.xprev0), h.mup, h.mua, h.mu_bits, M, h.a.ic,
         h.a.KB, MT, h.ws);
   }
