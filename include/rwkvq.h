@@ -125,6 +125,43 @@ rwkvq_status rwkvq_proxy_select(const void* const* w_fp16_dev, const int* oc, co
                                 size_t workspace_bytes, void* stream);
 
 /*
+ * The same proxy for weights of other types and at finer granularity (Section 4.1 evaluates one
+ * matrix at a time; the paper's limitations paragraph names finer granularity as future work).
+ *
+ * rwkvq_proxy_select_bf16: as rwkvq_proxy_select for bfloat16 matrices (the sort of Eq. 5 as a
+ * counting sort over the 65 536 bfloat16 patterns); same workspace size and errors.
+ *
+ * rwkvq_proxy_select_f32: one fp32 matrix resident on the device; the sort of Eq. 5 is the CUDA
+ * toolkit's radix sort, the gaps are reduced in fp64 in a fixed order.  workspace_dev:
+ * rwkvq_proxy_f32_workspace_bytes(oc, ic) bytes (two key arrays and the sort's scratch),
+ * 256-byte aligned.  Pc_host/Pf_host/phi_host: one value each.
+ *
+ * rwkvq_proxy_segments: P_c, P_f and Eq. 18 for every seg_rows x seg_cols tile of one matrix
+ * (dtype RWKVQ_F16, RWKVQ_BF16 or RWKVQ_F32, row-major [oc][ic] on the device): seg_rows = 1,
+ * seg_cols = ic is channel level, 256 x 256 the block of a VQ codebook; tiles at the right and
+ * bottom edges are smaller.  A tile is sorted by one thread block in shared memory, so it may hold
+ * at most 65 536 elements (16-bit types) or 32 768 (fp32): EUNSUPPORTED beyond.  Results are
+ * written tile-row major: index (r / seg_rows) * ceil(ic / seg_cols) + c / seg_cols; a tile with
+ * fewer than two elements, or constant, yields +inf (VQ).  workspace_dev:
+ * rwkvq_proxy_segments_workspace_bytes() bytes, 16-byte aligned.
+ * All three synchronize `stream` before returning.  Errors: EINVAL, EALIGN, ENOMEM,
+ * EUNSUPPORTED, ENONFINITE (the affected results are +inf), ECUDA.
+ */
+rwkvq_status rwkvq_proxy_select_bf16(const void* const* w_bf16_dev, const int* oc, const int* ic,
+                                     int n_mats, int K, double tau_c, double tau_f, double* Pc_host,
+                                     double* Pf_host, int* phi_host, void* workspace_dev,
+                                     size_t workspace_bytes, void* stream);
+size_t rwkvq_proxy_f32_workspace_bytes(int oc, int ic);
+rwkvq_status rwkvq_proxy_select_f32(const void* w_f32_dev, int oc, int ic, int K, double tau_c,
+                                    double tau_f, double* Pc_host, double* Pf_host, int* phi_host,
+                                    void* workspace_dev, size_t workspace_bytes, void* stream);
+size_t rwkvq_proxy_segments_workspace_bytes(int oc, int ic, int seg_rows, int seg_cols);
+rwkvq_status rwkvq_proxy_segments(const void* w_dev, int dtype, int oc, int ic, int seg_rows,
+                                  int seg_cols, int K, double tau_c, double tau_f, double* Pc_host,
+                                  double* Pf_host, int* phi_host, void* workspace_dev,
+                                  size_t workspace_bytes, void* stream);
+
+/*
  * The statistics of the normalised gaps G' (Eq. 6) that the ablation of Section 5.3 tries in the
  * proxy's place, from the same histogram pass: for each matrix stats_host[5*m + {0,1,2,3,4}] =
  * variance, coefficient of variation, range, mean absolute deviation of G' and its information

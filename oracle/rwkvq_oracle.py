@@ -278,6 +278,25 @@ def proxy(w: np.ndarray, K: int = 4):
     return pc, pf
 
 
+def proxy_segments(w: np.ndarray, seg_rows: int, seg_cols: int, K: int = 4):
+    """The proxy of Section 4.1 applied to every seg_rows x seg_cols tile of a matrix instead of
+    the whole matrix (the paper's limitations paragraph: finer granularity than one decision per
+    matrix): tile (i, j) covers rows i*seg_rows.. and columns j*seg_cols.., smaller at the right
+    and bottom edges; a tile with fewer than two elements has no gaps and returns (inf, inf).
+    Returns (P_c, P_f) arrays of shape [ceil(oc / seg_rows), ceil(ic / seg_cols)]."""
+    w = np.asarray(w, dtype=np.float64)
+    oc, ic = w.shape
+    gy, gx = -(-oc // seg_rows), -(-ic // seg_cols)
+    pc = np.full((gy, gx), math.inf)
+    pf = np.full((gy, gx), math.inf)
+    for i in range(gy):
+        for j in range(gx):
+            t = w[i * seg_rows:(i + 1) * seg_rows, j * seg_cols:(j + 1) * seg_cols]
+            if t.size >= 2:
+                pc[i, j], pf[i, j] = proxy(t, K)
+    return pc, pf
+
+
 def proxy_taylor_signed(w: np.ndarray, K: int) -> float:
     """Signed Taylor sum of Eq. 14/15: sum_k (-1)^k v_k M_k (approximates P_c near uniform)."""
     flat = np.sort(np.asarray(w, dtype=np.float64).reshape(-1))

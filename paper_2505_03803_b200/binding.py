@@ -67,7 +67,8 @@ EXPORTS = [
     "rwkvq_step_run_host", "rwkvq_step_plan_release", "rwkvq_step_set_wait", "rwkvq_step_plan_cover",
     "rwkvq_prefill_workspace_bytes", "rwkvq_gemm_prefill", "rwkvq_gemm_prefill_grouped", "rwkvq_dequant", "rwkvq_device_status",
     "rwkvq_status_str", "rwkvq_last_cuda_error",
-    "rwkvq_proxy_family", "rwkvq_tau_for_fraction", "rwkvq_tau_largest_gap", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
+    "rwkvq_proxy_family", "rwkvq_proxy_select_bf16", "rwkvq_proxy_f32_workspace_bytes", "rwkvq_proxy_select_f32",
+    "rwkvq_proxy_segments_workspace_bytes", "rwkvq_proxy_segments", "rwkvq_tau_for_fraction", "rwkvq_tau_largest_gap", "rwkvq_quant_error_workspace_bytes", "rwkvq_quant_error",
     "rwkvq_desc_for", "rwkvq_quantize_workspace_bytes", "rwkvq_quantize_dev", "rwkvq_calib_representative",
     "rwkvq_quantize_dev_async", "rwkvq_quantize_check",
 ]
@@ -116,6 +117,15 @@ def lib() -> C.CDLL:
         L.rwkvq_proxy_family.argtypes = [C.POINTER(vp), C.POINTER(i32), C.POINTER(i32), i32, C.POINTER(dbl), vp, sz, vp]
         L.rwkvq_tau_for_fraction.argtypes = [C.POINTER(dbl), i32, dbl, C.POINTER(dbl)]
         L.rwkvq_tau_largest_gap.argtypes = [C.POINTER(dbl), i32, C.POINTER(dbl)]
+    if hasattr(L, "rwkvq_proxy_segments"):
+        L.rwkvq_proxy_select_bf16.argtypes = L.rwkvq_proxy_select.argtypes
+        L.rwkvq_proxy_f32_workspace_bytes.argtypes = [i32, i32]
+        L.rwkvq_proxy_f32_workspace_bytes.restype = sz
+        L.rwkvq_proxy_select_f32.argtypes = [vp, i32, i32, i32, dbl, dbl, C.POINTER(dbl), C.POINTER(dbl), C.POINTER(i32), vp, sz, vp]
+        L.rwkvq_proxy_segments_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.rwkvq_proxy_segments_workspace_bytes.restype = sz
+        L.rwkvq_proxy_segments.argtypes = [vp, i32, i32, i32, i32, i32, i32, dbl, dbl, C.POINTER(dbl), C.POINTER(dbl),
+                                           C.POINTER(i32), vp, sz, vp]
     if hasattr(L, "rwkvq_quant_error"):
         L.rwkvq_quant_error_workspace_bytes.argtypes = [C.POINTER(Desc)]
         L.rwkvq_quant_error_workspace_bytes.restype = sz
@@ -328,6 +338,46 @@ def rwkvq_proxy_select(mats, K: int, tau_c: float, tau_f: float, workspace, stre
                                     _dev_ptr(workspace), workspace.numel() * workspace.element_size(),
                                     _stream_ptr(stream)), "rwkvq_proxy_select")
     return pc, pf, phi
+
+
+def _torch_dtype_code(t):
+    import torch
+    return {torch.float32: RWKVQ_F32, torch.float16: RWKVQ_F16, torch.bfloat16: RWKVQ_BF16}[t.dtype]
+
+
+def rwkvq_proxy_select_typed(w, K: int, tau_c: float, tau_f: float, stream=None):
+    """P_c, P_f and phi of ONE matrix (CUDA tensor [oc, ic], float16, bfloat16 or float32) as floats / int:
+    rwkvq_proxy_select, rwkvq_proxy_select_bf16 or rwkvq_proxy_select_f32 by the tensor's type."""
+    import torch
+    oc, ic = int(w.shape[0]), int(w.shape[1])
+    pc, pf, phi = C.c_double(), C.c_double(), C.c_int()
+    if w.dtype == torch.float32:
+        ws = torch.empty(int(lib().rwkvq_proxy_f32_workspace_bytes(oc, ic)), dtype=torch.uint8, device=w.device)
+        _check(lib().rwkvq_proxy_select_f32(_dev_ptr(w), oc, ic, K, tau_c, tau_f, C.byref(pc), C.byref(pf), C.byref(phi),
+                                            _dev_ptr(ws), ws.numel(), _stream_ptr(stream)), "rwkvq_proxy_select_f32")
+    else:
+        ws = torch.empty(rwkvq_proxy_workspace_bytes(1), dtype=torch.uint8, device=w.device)
+        fn = lib().rwkvq_proxy_select if w.dtype == torch.float16 else lib().rwkvq_proxy_select_bf16
+        ptrs, ocs, ics = (C.c_void_p * 1)(w.data_ptr()), (C.c_int * 1)(oc), (C.c_int * 1)(ic)
+        _check(fn(ptrs, ocs, ics, 1, K, tau_c, tau_f, C.byref(pc), C.byref(pf), C.byref(phi), _dev_ptr(ws), ws.numel(),
+                  _stream_ptr(stream)), "rwkvq_proxy_select (typed)")
+    return float(pc.value), float(pf.value), int(phi.value)
+
+
+def rwkvq_proxy_segments(w, seg_rows: int, seg_cols: int, K: int, tau_c: float, tau_f: float, stream=None):
+    """rwkvq_proxy_segments on a CUDA tensor [oc, ic] (float16, bfloat16 or float32).  Returns (P_c, P_f, phi)
+    numpy arrays of shape [ceil(oc / seg_rows), ceil(ic / seg_cols)]."""
+    import torch
+    oc, ic = int(w.shape[0]), int(w.shape[1])
+    sr, sc = min(seg_rows, oc), min(seg_cols, ic)
+    gy, gx = (oc + sr - 1) // sr, (ic + sc - 1) // sc
+    pc, pf, phi = np.empty(gy * gx, np.float64), np.empty(gy * gx, np.float64), np.empty(gy * gx, np.int32)
+    ws = torch.empty(max(256, int(lib().rwkvq_proxy_segments_workspace_bytes(oc, ic, sr, sc))), dtype=torch.uint8, device=w.device)
+    _check(lib().rwkvq_proxy_segments(_dev_ptr(w), _torch_dtype_code(w), oc, ic, seg_rows, seg_cols, K, tau_c, tau_f,
+                                      pc.ctypes.data_as(C.POINTER(C.c_double)), pf.ctypes.data_as(C.POINTER(C.c_double)),
+                                      phi.ctypes.data_as(C.POINTER(C.c_int)), _dev_ptr(ws), ws.numel(), _stream_ptr(stream)),
+           "rwkvq_proxy_segments")
+    return pc.reshape(gy, gx), pf.reshape(gy, gx), phi.reshape(gy, gx)
 
 
 def rwkvq_proxy_family(mats, workspace, stream=None):

@@ -43,21 +43,24 @@ __device__ __forceinline__ unsigned key_of(unsigned bits) {
   const unsigned mag = bits & 0x7FFFu;
   return (bits & 0x8000u) ? 0x8000u - mag : 0x8000u + mag;
 }
-__device__ __forceinline__ double value_of_key(unsigned key) {
+// bf16 != 0: the 16 bits are a bfloat16 pattern (same sign-magnitude order, other exponent width)
+__device__ __forceinline__ double value_of_key(unsigned key, int bf16 = 0) {
   const unsigned short bits = key >= 0x8000u ? (unsigned short)(key - 0x8000u) : (unsigned short)(0x8000u | (0x8000u - key));
+  if (bf16) return (double)__uint_as_float((unsigned)bits << 16);
   return (double)__half2float(__ushort_as_half(bits));
 }
 
-__device__ __forceinline__ void count_one(unsigned bits, unsigned* sh, unsigned* hist, int* nonfinite) {
-  if ((bits & 0x7C00u) == 0x7C00u) { *nonfinite = 1; return; }
+__device__ __forceinline__ void count_one(unsigned bits, unsigned* sh, unsigned* hist, int* nonfinite, unsigned expmask) {
+  if ((bits & expmask) == expmask) { *nonfinite = 1; return; }
   const unsigned key = key_of(bits);
   const unsigned rel = key - (unsigned)kHotBase;
   if (rel < (unsigned)kHotBins) atomicAdd(&sh[rel], 1u);
   else atomicAdd(&hist[key], 1u);
 }
 
-__global__ void __launch_bounds__(1024, 1) proxy_hist_kernel(const __half* w, unsigned long long n, unsigned* hist, ProxyResult* res) {
+__global__ void __launch_bounds__(1024, 1) proxy_hist_kernel(const __half* w, unsigned long long n, unsigned* hist, ProxyResult* res, int bf16) {
   extern __shared__ unsigned sh[];
+  const unsigned expmask = bf16 ? 0x7F80u : 0x7C00u;
   for (int j = threadIdx.x; j < kHotBins; j += blockDim.x) sh[j] = 0u;
   __syncthreads();
   int bad = 0;
@@ -69,13 +72,13 @@ __global__ void __launch_bounds__(1024, 1) proxy_hist_kernel(const __half* w, un
     const unsigned ws[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      count_one(ws[k] & 0xFFFFu, sh, hist, &bad);
-      count_one(ws[k] >> 16, sh, hist, &bad);
+      count_one(ws[k] & 0xFFFFu, sh, hist, &bad, expmask);
+      count_one(ws[k] >> 16, sh, hist, &bad, expmask);
     }
   }
   if (blockIdx.x == 0) {
     for (unsigned long long i = nvec * 8 + threadIdx.x; i < n; i += blockDim.x)
-      count_one((unsigned)__half_as_ushort(w[i]), sh, hist, &bad);
+      count_one((unsigned)__half_as_ushort(w[i]), sh, hist, &bad, expmask);
   }
   if (bad) res->nonfinite = 1;
   __syncthreads();
@@ -86,7 +89,7 @@ __global__ void __launch_bounds__(1024, 1) proxy_hist_kernel(const __half* w, un
 }
 
 // One block of 1024 threads per matrix; thread t owns keys [64t, 64t+64).
-__global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* hist_all, ProxyResult* res_all, int K) {
+__global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* hist_all, ProxyResult* res_all, int K, int bf16) {
   const unsigned* hist = hist_all + (size_t)blockIdx.x * kBins;
   ProxyResult* res = res_all + blockIdx.x;
   __shared__ int s_last[1024];
@@ -125,7 +128,7 @@ __global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* h
     }
     return;
   }
-  const double R = value_of_key((unsigned)mx) - value_of_key((unsigned)mn);
+  const double R = value_of_key((unsigned)mx, bf16) - value_of_key((unsigned)mn, bf16);
   const double n = (double)(N - 1);
   double acc[8];  // [0] = sum g' ln g', [k-1] = sum t^k for k = 2..8
 #pragma unroll
@@ -135,7 +138,7 @@ __global__ void __launch_bounds__(1024, 1) proxy_reduce_kernel(const unsigned* h
   for (int k = k0; k < k0 + 64; ++k) {
     if (hist[k] == 0u) continue;
     if (prev >= 0) {
-      const double gp = (value_of_key((unsigned)k) - value_of_key((unsigned)prev)) / R;
+      const double gp = (value_of_key((unsigned)k, bf16) - value_of_key((unsigned)prev, bf16)) / R;
       acc[0] += gp * log(gp);
       const double tt = n * gp - 1.0;
       double pw = tt;
@@ -203,7 +206,7 @@ size_t rwkvq_proxy_workspace_bytes(int n_mats) {
 }
 
 static rwkvq_status run_proxy(const void* const* w, const int* oc, const int* ic, int n_mats, int K, void* ws,
-                              size_t ws_bytes, void* stream, std::vector<ProxyResult>* out) {
+                              size_t ws_bytes, void* stream, std::vector<ProxyResult>* out, int bf16 = 0) {
   if (!w || !oc || !ic || n_mats <= 0) return RWKVQ_EINVAL;
   if (K < 2 || K > 8) return RWKVQ_EINVAL;
   if (!ws || ws_bytes < rwkvq_proxy_workspace_bytes(n_mats)) return RWKVQ_ENOMEM;
@@ -227,9 +230,9 @@ static rwkvq_status run_proxy(const void* const* w, const int* oc, const int* ic
     unsigned long long blocks = (n / 8 + 1023) / 1024;
     if (blocks < 1) blocks = 1;
     if (blocks > (unsigned long long)sms) blocks = sms;
-    proxy_hist_kernel<<<(unsigned)blocks, 1024, smem, s>>>(static_cast<const __half*>(w[m]), n, hist + (size_t)m * kBins, res + m);
+    proxy_hist_kernel<<<(unsigned)blocks, 1024, smem, s>>>(static_cast<const __half*>(w[m]), n, hist + (size_t)m * kBins, res + m, bf16);
   }
-  proxy_reduce_kernel<<<n_mats, 1024, 0, s>>>(hist, res, K);
+  proxy_reduce_kernel<<<n_mats, 1024, 0, s>>>(hist, res, K, bf16);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_status(e);
   out->resize(n_mats);
@@ -247,6 +250,20 @@ rwkvq_status rwkvq_proxy_select(const void* const* w, const int* oc, const int* 
   if (!Pc || !Pf || !phi) return RWKVQ_EINVAL;
   std::vector<ProxyResult> host;
   const rwkvq_status st = run_proxy(w, oc, ic, n_mats, K, ws, ws_bytes, stream, &host);
+  if (st != RWKVQ_OK && st != RWKVQ_ENONFINITE) return st;
+  for (int m = 0; m < n_mats; ++m) {
+    Pc[m] = host[m].pc; Pf[m] = host[m].pf;
+    phi[m] = (host[m].pc < tau_c && host[m].pf < tau_f) ? RWKVQ_SQ : RWKVQ_VQ;   // Eq. 18, strict <
+  }
+  return st;
+}
+
+rwkvq_status rwkvq_proxy_select_bf16(const void* const* w, const int* oc, const int* ic, int n_mats, int K,
+                                     double tau_c, double tau_f, double* Pc, double* Pf, int* phi, void* ws,
+                                     size_t ws_bytes, void* stream) {
+  if (!Pc || !Pf || !phi) return RWKVQ_EINVAL;
+  std::vector<ProxyResult> host;
+  const rwkvq_status st = run_proxy(w, oc, ic, n_mats, K, ws, ws_bytes, stream, &host, 1);
   if (st != RWKVQ_OK && st != RWKVQ_ENONFINITE) return st;
   for (int m = 0; m < n_mats; ++m) {
     Pc[m] = host[m].pc; Pf[m] = host[m].pf;

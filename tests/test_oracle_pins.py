@@ -455,3 +455,30 @@ def test_bf16_rounding_ties_to_even():
     vals = np.array([1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7 + 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -3.0])
     out = orc.bf16_rne(vals)
     assert [float(v) for v in out] == [1.0, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7, -3.0]
+
+
+def test_proxy_segments_closed_forms_per_tile():
+    """Per-tile proxy: a tile that is an equispaced ramp (in any order) has P_c = P_f = 0 exactly up to
+    rounding, a tile of two clusters has P_c > 0, a constant tile and a one-element tile give inf; the tile
+    grid is ragged at the edges."""
+    rng = np.random.default_rng(5)
+    w = np.zeros((5, 7))
+    w[0:2, 0:3] = rng.permutation(np.arange(6.0)).reshape(2, 3) * 0.25 - 1.0      # ramp
+    w[0:2, 3:6] = np.array([[0.0, 0.001, 0.002], [5.0, 5.001, 5.002]])            # two clusters
+    w[0:2, 6:7] = np.array([[1.0], [3.0]])                                        # two elements: one gap, g' = 1
+    w[2:4, 0:3] = 2.5                                                             # constant
+    w[2:4, 3:6] = rng.standard_normal((2, 3))
+    w[4:5, 6:7] = 9.0                                                             # single element
+    pc, pf = orc.proxy_segments(w, 2, 3, K=4)
+    assert pc.shape == (3, 3)
+    assert abs(pc[0, 0]) < 1e-12 and abs(pf[0, 0]) < 1e-12
+    assert pc[0, 1] > 0.5 and pf[0, 1] > 0.0
+    # n = 1: P_c = ln 1 - 0 = 0 and delta = 0
+    assert pc[0, 2] == 0.0 and pf[0, 2] == 0.0
+    assert np.isinf(pc[1, 0]) and np.isinf(pf[1, 0])
+    assert np.isinf(pc[2, 2]) and np.isinf(pf[2, 2])
+    a, b = orc.proxy(w[2:4, 3:6], 4)
+    assert pc[1, 1] == a and pf[1, 1] == b
+    # whole matrix as one tile = the matrix-level proxy
+    pcm, pfm = orc.proxy_segments(w, 5, 7, K=4)
+    assert (pcm[0, 0], pfm[0, 0]) == orc.proxy(w, 4)
