@@ -225,8 +225,47 @@ rwkvq_status rwkvq_gemv_static(const rwkvq_desc* W_desc, const void* W_image_dev
                                const void* mu_image_dev, const void* x_fp16_dev, const void* xprev_fp16_dev,
                                int B, void* y_dev, int y_dtype, void* stream);
 
+/*
+ * Where a product of a decode step takes its input row x[b][0..ic) from, when it is not a plain
+ * fp16 buffer: the element-wise operators that sit between the projections of an RWKV block
+ * (Appendix A.1).  The step computes them once per stage, after the barrier that completes the
+ * stage before, in fp32, rounds x to fp16 and then applies the token-shift mix (if mu is given).
+ *   RWKVQ_IN_BUFFER  x = x_fp16_dev (the plain case; every other field below is ignored).
+ *   RWKVQ_IN_WKV     x = sigmoid(src) * wkv (Eq. 24) with src = r, and wkv of Eq. 23 from k_f32,
+ *                    v_f32 (outputs of earlier products, [B][ic] fp32) and the running history
+ *                    sums.  The sums are kept scaled by a running exponent for range:
+ *                    state_a = e^{-p} * sum f(i) v_i, state_b = e^{-p} * sum f(i), state_p = p,
+ *                    each [B][ic] fp32, updated in place for the next token (start a sequence
+ *                    with a = b = 0, p = -1e30).  u_f32, w_f32: [ic] bonus and decay (the history
+ *                    decays by e^{-w} per token).
+ *   RWKVQ_IN_RELU2   x = max(src, 0)^2 (Eq. 27) with src = k'.
+ *   RWKVQ_IN_F32     x = src, or sigmoid(gate_f32) * src when gate_f32 != NULL (Eq. 27: the
+ *                    block's output as the next block's input), src / gate [B][ic] fp32.
+ * xprev_out_fp16 (any kind, may be NULL): receives this token's x (before the mix), [B][ic]
+ * fp16; it may be the very buffer xprev_fp16_dev points to (each element is read, then written,
+ * by one thread), which makes the previous-token state advance by itself from step to step.  A
+ * buffer that is updated this way must belong to ONE product.
+ * All pointers are device memory, 16-byte aligned, owned by the caller.
+ */
+typedef enum { RWKVQ_IN_BUFFER = 0, RWKVQ_IN_WKV = 1, RWKVQ_IN_RELU2 = 2, RWKVQ_IN_F32 = 3 } rwkvq_input_kind;
+typedef struct {
+  int32_t kind;               /* rwkvq_input_kind */
+  int32_t reserved;
+  const float* src_f32;
+  const float* k_f32;
+  const float* v_f32;
+  float* state_a;
+  float* state_b;
+  float* state_p;
+  const float* u_f32;
+  const float* w_f32;
+  const float* gate_f32;
+  void* xprev_out_fp16;
+} rwkvq_input_xform;
+
 /* One product of a decode step (same meaning as the rwkvq_gemv arguments).  `stage` orders the
- * step: every product of stage s is complete before any activation of stage s+1 is read. */
+ * step: every product of stage s is complete before any activation of stage s+1 is read.
+ * `in` all zero = the input is x_fp16_dev; otherwise x_fp16_dev may be NULL (see above). */
 typedef struct {
   rwkvq_desc W_desc;
   const void* W_image_dev;
@@ -237,6 +276,7 @@ typedef struct {
   void* y_dev;
   int32_t stage;
   int32_t y_dtype;
+  rwkvq_input_xform in;
 } rwkvq_gemv_op;
 
 /*

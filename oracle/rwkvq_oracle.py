@@ -19,7 +19,9 @@ Passages followed (RWKVQuant, arXiv 2505.03803):
   * selection rule phi                   -- Section 4.1, Eq. 18
   * other statistics of G' (ablation)    -- Section 5.3 (Variance, CV, Range, MAD, IE); thresholds for a
                                             target SQ share -- Section 5.1
-  * token shift mix and projections      -- Appendix A.1, Eqs. 20-22, 24-26
+  * token shift mix and projections      -- Appendix A.1, Eqs. 20-22, 24-27
+  * WKV, sigmoid gates, squared ReLU     -- Appendix A.1, Eq. 23 (wkv), Eq. 24 (sigma(r) * wkv),
+                                            Eq. 27 (sigma(r') * (W'_v . max(k', 0)^2))
   * weighted loss for element-wise mu    -- Section 4.2, Eq. 19 (weighted k-means; representative X by
                                             percentile clipping before the mean)
 
@@ -395,3 +397,55 @@ def tolerance(w_hat: np.ndarray, x_mix: np.ndarray, rel: float = 2e-3) -> np.nda
     wn = np.sqrt((np.asarray(w_hat, dtype=np.float64) ** 2).sum(axis=1))
     xn = np.sqrt((np.asarray(x_mix, dtype=np.float64) ** 2).sum(axis=1))
     return rel * xn[:, None] * wn[None, :]
+
+
+def sigmoid(x: np.ndarray) -> np.ndarray:
+    """sigma(x) = 1 / (1 + exp(-x)), float64."""
+    return 1.0 / (1.0 + np.exp(-np.asarray(x, dtype=np.float64)))
+
+
+def wkv_literal(ks: np.ndarray, vs: np.ndarray, u: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """Eq. 23 written out for the LAST token of a history: ks, vs are [T, d] (tokens 1..T = t),
+
+        wkv_t = ( sum_{i<t} f(i) * v_i + exp(u + k_t) * v_t ) / ( sum_{i<t} f(i) + exp(u + k_t) ),
+        f(i)  = exp( -(t - 1 - i) * w + k_i ),
+
+    element-wise over the d channels, float64.  Returns [d]."""
+    ks, vs = np.asarray(ks, dtype=np.float64), np.asarray(vs, dtype=np.float64)
+    u, w = np.asarray(u, dtype=np.float64), np.asarray(w, dtype=np.float64)
+    t = ks.shape[0]
+    num = np.exp(u + ks[t - 1]) * vs[t - 1]
+    den = np.exp(u + ks[t - 1])
+    for i in range(1, t):                       # token numbers 1 .. t-1
+        f = np.exp(-(t - 1 - i) * w + ks[i - 1])
+        num = num + f * vs[i - 1]
+        den = den + f
+    return num / den
+
+
+def wkv_step(a: np.ndarray, b: np.ndarray, k: np.ndarray, v: np.ndarray, u: np.ndarray, w: np.ndarray):
+    """One token of Eq. 23 as a recurrence over the two history sums a_{t-1} = sum_{i<t} f(i) v_i and
+    b_{t-1} = sum_{i<t} f(i):  wkv_t = (a + e^{u+k} v) / (b + e^{u+k});  the sums for the next token are
+    a' = e^{-w} a + e^{k} v,  b' = e^{-w} b + e^{k}  (every f(i) gains the factor e^{-w}, token t joins
+    with f = e^{k_t}).  All arrays [B, d] or [d], float64.  Returns (wkv, a', b')."""
+    a, b, k, v = (np.asarray(z, dtype=np.float64) for z in (a, b, k, v))
+    u, w = np.asarray(u, dtype=np.float64), np.asarray(w, dtype=np.float64)
+    e = np.exp(u + k)
+    wkv = (a + e * v) / (b + e)
+    return wkv, np.exp(-w) * a + np.exp(k) * v, np.exp(-w) * b + np.exp(k)
+
+
+def time_mix_gate(r: np.ndarray, wkv: np.ndarray) -> np.ndarray:
+    """Input of the output projection, Eq. 24: sigma(r) * wkv."""
+    return sigmoid(r) * np.asarray(wkv, dtype=np.float64)
+
+
+def relu_squared(k: np.ndarray) -> np.ndarray:
+    """Input of the channel-mix value projection, Eq. 27: max(k', 0)^2."""
+    return np.maximum(np.asarray(k, dtype=np.float64), 0.0) ** 2
+
+
+def channel_mix_gate(r: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """Output of channel mixing, Eq. 27: sigma(r') * y with y = W'_v . max(k', 0)^2."""
+    return sigmoid(r) * np.asarray(y, dtype=np.float64)
+

@@ -48,10 +48,19 @@ class Desc(C.Structure):
                 ("stream_bytes", C.c_uint64)]
 
 
+RWKVQ_IN_BUFFER, RWKVQ_IN_WKV, RWKVQ_IN_RELU2, RWKVQ_IN_F32 = 0, 1, 2, 3
+
+
+class InputXform(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("reserved", C.c_int32), ("src_f32", C.c_void_p), ("k_f32", C.c_void_p),
+                ("v_f32", C.c_void_p), ("state_a", C.c_void_p), ("state_b", C.c_void_p), ("state_p", C.c_void_p),
+                ("u_f32", C.c_void_p), ("w_f32", C.c_void_p), ("gate_f32", C.c_void_p), ("xprev_out_fp16", C.c_void_p)]
+
+
 class GemvOp(C.Structure):
     _fields_ = [("W_desc", Desc), ("W_image_dev", C.c_void_p), ("mu_desc", Desc), ("mu_image_dev", C.c_void_p),
                 ("x_fp16_dev", C.c_void_p), ("xprev_fp16_dev", C.c_void_p), ("y_dev", C.c_void_p),
-                ("stage", C.c_int32), ("y_dtype", C.c_int32)]
+                ("stage", C.c_int32), ("y_dtype", C.c_int32), ("in_", InputXform)]
 
 
 class PrefillOp(C.Structure):
@@ -421,7 +430,8 @@ def rwkvq_quant_error(w, desc: Desc, W_image, stream=None) -> float:
 
 
 def make_ops(entries):
-    """Array of GemvOp from dicts {desc, W, mu_desc, mu, x, xprev, y, stage} (torch tensors)."""
+    """Array of GemvOp from dicts {desc, W, mu_desc, mu, x, xprev, y, stage[, in]} (torch tensors; "in" is a
+    dict describing an rwkvq_input_xform)."""
     import torch
     arr = (GemvOp * len(entries))()
     for i, e in enumerate(entries):
@@ -435,7 +445,15 @@ def make_ops(entries):
         else:
             o.mu_image_dev = None
             o.xprev_fp16_dev = None
-        o.x_fp16_dev = e["x"].data_ptr()
+        o.x_fp16_dev = None if e.get("x") is None else e["x"].data_ptr()
+        xf = e.get("in")
+        if xf:      # {"kind": RWKVQ_IN_*, "src": .., "k": .., "v": .., "state_a": .., ..., "gate": .., "xprev_out": ..}
+            o.in_.kind = int(xf.get("kind", RWKVQ_IN_BUFFER))
+            for field, key in (("src_f32", "src"), ("k_f32", "k"), ("v_f32", "v"), ("state_a", "state_a"),
+                               ("state_b", "state_b"), ("state_p", "state_p"), ("u_f32", "u"), ("w_f32", "w"),
+                               ("gate_f32", "gate"), ("xprev_out_fp16", "xprev_out")):
+                t = xf.get(key)
+                setattr(o.in_, field, None if t is None else t.data_ptr())
         o.y_dev = e["y"].data_ptr()
         o.stage = e["stage"]
         o.y_dtype = RWKVQ_F32 if e["y"].dtype == torch.float32 else RWKVQ_F16

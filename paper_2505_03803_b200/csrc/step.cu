@@ -94,12 +94,15 @@ static_assert(sizeof(StepEvent) == 64, "event descriptor size");
 
 // One product's share of a stage's pre-pass: where its inputs are and where x_mix (fp16 rows of
 // ic_pad columns, zero beyond ic) and the per-group sums ([group][3][nbp] floats) go.
-struct StepMixOp {           // 64 bytes
+struct StepMixOp {           // 144 bytes
   uint64_t x, xprev, mu, mu_aux, dst_x, dst_sums;
   uint32_t ic, ic_pad;
-  uint16_t mu_bits, mu_entries, sums, pad;
+  uint16_t mu_bits, mu_entries, sums, kind;     // kind: rwkvq_input_kind
+  // element-wise operator in front of the product (rwkvq_input_xform): fp32 sources [B][ic], state, parameters
+  uint64_t src, k, v, state_a, state_b, state_p, u, w;   // src doubles as the gate's operand; `k` holds the gate for RWKVQ_IN_F32
+  uint64_t xprev_out, pad;
 };
-static_assert(sizeof(StepMixOp) == 64, "pre-pass descriptor size");
+static_assert(sizeof(StepMixOp) == 144, "pre-pass descriptor size");
 
 constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGroups, kStagerWarps = 3;
 constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
@@ -221,7 +224,6 @@ struct Ctrl {
                              // stage that the barrier closes.  Per barrier, not one running total: consumer
                              // warps of a CTA without work in the coming stages may run any number of
                              // stages ahead of the stagers.
-  uint32_t cdone;            // running total of stage reports of the consumer warps (two-batch-block launches)
   int abort_flag;
   int poll_limit;            // must follow abort_flag (poll_limit_of)
 };
@@ -239,19 +241,23 @@ __device__ __forceinline__ void stage_report(Ctrl* ctrl, const StepArgs& a, uint
   const uint32_t old = smem_add_acq_rel(&ctrl->stage_cnt[b >> 2], 1u << sh);
   if (((old >> sh) & 0xFFu) == (uint32_t)kConsumerWarps) red_release_gpu(a.counter + b, 1u);
 }
-// Where the consumer warps are the busy role (two batch blocks per record) they only add to one
-// running total, and a stager thread, which has nothing else to do at that point, waits (bounded)
-// for the sixteen reports of the stage and arrives: the release, which waits for the CTA's
-// outstanding reductions, and the bookkeeping of a barrier number stay off the consumer warps.
-__device__ __forceinline__ void stage_report_total(Ctrl* ctrl) {
-  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(&ctrl->cdone)), "r"(1u) : "memory");
+// Where the consumer warps are the busy role (two batch blocks per record) they only count
+// themselves in, and a stager thread, which has nothing else to do at that point, waits (bounded)
+// for the sixteen reports of THIS barrier and arrives: the release, which waits for the CTA's
+// outstanding reductions, stays off the consumer warps.  The count is per barrier (the 8-bit
+// fields of stage_cnt): a warp without work in the next stages runs ahead through their events,
+// so a running total over all stages would reach sixteen times the stage number while warps of
+// this stage are still adding to the outputs.
+__device__ __forceinline__ void stage_report_total(Ctrl* ctrl, uint32_t b) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(&ctrl->stage_cnt[b >> 2])), "r"(1u << (8u * (b & 3u))) : "memory");
 }
 __device__ __forceinline__ bool stage_wait_total_and_arrive(Ctrl* ctrl, const StepArgs& a, uint32_t b, volatile int* abort_flag) {
   const uint32_t limit = poll_limit_of(abort_flag) << 4;
+  const uint32_t sh = 8u * (b & 3u);
   for (uint32_t it = 0; it < limit; ++it) {
     uint32_t v;
-    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&ctrl->cdone)) : "memory");
-    if (v >= (uint32_t)kConsumerWarps * b) { red_release_gpu(a.counter + b, 1u); return true; }
+    asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&ctrl->stage_cnt[b >> 2])) : "memory");
+    if (((v >> sh) & 0xFFu) >= (uint32_t)kConsumerWarps) { red_release_gpu(a.counter + b, 1u); return true; }
     if ((it & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -338,6 +344,61 @@ __device__ __forceinline__ float pair_sum(uint32_t r) {
 
 constexpr int kStageUnroll = 4;
 
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+  const __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+// Eight consecutive inputs of a product from the element-wise operator in front of it (Appendix A.1
+// Eqs. 23, 24, 27), rounded to fp16.  e0: index of the first element in the [B][ic] fp32 arrays,
+// col: its column (index into the per-channel parameters).  `commit` false (a lane that repeats
+// another lane's group to keep the half-warp whole): the recurrence state is not written.
+__device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int col, bool commit) {
+  float s[8];
+  {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(op.src) + e0));
+    const float4 c = __ldcg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(op.src) + e0 + 4));
+    s[0] = a.x; s[1] = a.y; s[2] = a.z; s[3] = a.w; s[4] = c.x; s[5] = c.y; s[6] = c.z; s[7] = c.w;
+  }
+  float o[8];
+  if (op.kind == RWKVQ_IN_RELU2) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { const float m = fmaxf(s[i], 0.f); o[i] = m * m; }
+  } else if (op.kind == RWKVQ_IN_F32) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = s[i];
+    if (op.k) {      // gate
+      const float* g = reinterpret_cast<const float*>(op.k) + e0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[i] *= sigmoidf_(__ldcg(g + i));
+    }
+  } else {           // RWKVQ_IN_WKV
+    const float* kp = reinterpret_cast<const float*>(op.k) + e0;
+    const float* vp = reinterpret_cast<const float*>(op.v) + e0;
+    float* sa = reinterpret_cast<float*>(op.state_a) + e0;
+    float* sb = reinterpret_cast<float*>(op.state_b) + e0;
+    float* sp = reinterpret_cast<float*>(op.state_p) + e0;
+    const float* up = reinterpret_cast<const float*>(op.u) + col;
+    const float* wp = reinterpret_cast<const float*>(op.w) + col;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // the history sums are stored as a = e^{-p} sum f v, b = e^{-p} sum f; every exponential below has
+      // a non-positive argument
+      const float k = __ldcg(kp + i), vv = __ldcg(vp + i), a = __ldcg(sa + i), bb = __ldcg(sb + i), p = __ldcg(sp + i);
+      const float uk = __ldg(up + i) + k;
+      const float q = fmaxf(p, uk);
+      const float e1 = expf(p - q), e2 = expf(uk - q);
+      const float wkv = (e1 * a + e2 * vv) / (e1 * bb + e2);
+      o[i] = sigmoidf_(s[i]) * wkv;
+      const float pw = p - __ldg(wp + i);
+      const float q2 = fmaxf(pw, k);
+      const float f1 = expf(pw - q2), f2 = expf(k - q2);
+      if (commit) { sa[i] = f1 * a + f2 * vv; sb[i] = f1 * bb + f2; sp[i] = q2; }
+    }
+  }
+  return make_uint4(pack_half2(o[0], o[1]), pack_half2(o[2], o[3]), pack_half2(o[4], o[5]), pack_half2(o[6], o[7]));
+}
+
 // This CTA's share of a stage's pre-pass.  A half-warp takes one (product, batch row, 128-column
 // group) at a time: it loads x (and x_prev, and decodes mu_hat), mixes, rounds to fp16, stores the
 // 128 values to the product's pre-pass rows and reduces the three sums of the group with shuffles.
@@ -360,22 +421,29 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
     const int col = grp * 128 + l16 * 8;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (col < (int)op.ic) {
-      v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + (size_t)b * op.ic + col));
-      if (op.mu) {
-        const uint4 pr = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.xprev) + (size_t)b * op.ic + col));
-        const uint32_t bits = op.mu_bits, mask = (1u << bits) - 1u;
-        // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
-        const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
-        const uint32_t* w = reinterpret_cast<const uint32_t*>(op.mu) + (byte >> 2);
-        const uint32_t sh = (byte & 3u) * 8u;
-        const uint32_t wlo = __ldg(w);
-        const uint32_t whi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
-        const uint32_t f = __funnelshift_r(wlo, whi, sh);
-        const uint32_t* cb = reinterpret_cast<const uint32_t*>(op.mu_aux);
-        v.x = mix2(v.x, pr.x, __ldg(cb + (f & mask)));
-        v.y = mix2(v.y, pr.y, __ldg(cb + ((f >> bits) & mask)));
-        v.z = mix2(v.z, pr.z, __ldg(cb + ((f >> (2 * bits)) & mask)));
-        v.w = mix2(v.w, pr.w, __ldg(cb + ((f >> (3 * bits)) & mask)));
+      const size_t e0 = (size_t)b * op.ic + col;          // first of this lane's eight elements
+      if (op.kind == RWKVQ_IN_BUFFER) v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + e0));
+      else v = xform_input(op, e0, col, valid);
+      if (op.xprev_out || op.mu) {
+        // previous token's input: read for the mix, then (where asked) replaced by this token's
+        uint4 pr = make_uint4(0u, 0u, 0u, 0u);
+        if (op.mu) pr = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.xprev) + e0));
+        if (op.xprev_out && valid) *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(op.xprev_out) + e0) = v;
+        if (op.mu) {
+          const uint32_t bits = op.mu_bits, mask = (1u << bits) - 1u;
+          // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
+          const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
+          const uint32_t* w = reinterpret_cast<const uint32_t*>(op.mu) + (byte >> 2);
+          const uint32_t sh = (byte & 3u) * 8u;
+          const uint32_t wlo = __ldg(w);
+          const uint32_t whi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+          const uint32_t f = __funnelshift_r(wlo, whi, sh);
+          const uint32_t* cb = reinterpret_cast<const uint32_t*>(op.mu_aux);
+          v.x = mix2(v.x, pr.x, __ldg(cb + (f & mask)));
+          v.y = mix2(v.y, pr.y, __ldg(cb + ((f >> bits) & mask)));
+          v.z = mix2(v.z, pr.z, __ldg(cb + ((f >> (2 * bits)) & mask)));
+          v.w = mix2(v.w, pr.w, __ldg(cb + ((f >> (3 * bits)) & mask)));
+        }
       }
     }
     if (valid) *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(a.scratch + op.dst_x) + (size_t)b * op.ic_pad + col) = v;
@@ -667,7 +735,8 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
   auto arrive_stage = [&]() {
     __syncwarp();
     if constexpr (NB == 2) {
-      if (lane == 0 && !dead) stage_report_total(ctrl);
+      if (lane == 0 && !dead) stage_report_total(ctrl, next_bar);
+      ++next_bar;
     } else {
       if (lane == 0 && !dead) stage_report(ctrl, a, next_bar);
       ++next_bar;
@@ -840,7 +909,6 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
     for (int s = 0; s < a.n_slots; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], kGroupWarps); }
     for (int b = 0; b < 4; ++b) { mbar_init(&ctrl->xfull[b], kStagerWarps); mbar_init(&ctrl->xempty[b], kConsumerWarps); }
     for (int k = 0; k < 64; ++k) ctrl->stage_cnt[k] = 0u;
-    ctrl->cdone = 0u;
     ctrl->abort_flag = 0;
     ctrl->poll_limit = (int)a.poll_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -898,14 +966,31 @@ static rwkvq_status validate_ops(const rwkvq_gemv_op* ops, int n_ops, int B) {
     rwkvq_status st = check_matrix_desc(&o.W_desc);
     if (st != RWKVQ_OK) return st;
     if (o.W_desc.oc == 1) return RWKVQ_ESHAPE;
-    if (!o.W_image_dev || !o.x_fp16_dev || !o.y_dev) return RWKVQ_EINVAL;
+    if (!o.W_image_dev || !o.y_dev) return RWKVQ_EINVAL;
+    const rwkvq_input_xform& in = o.in;
+    if (in.kind == RWKVQ_IN_BUFFER) {
+      if (!o.x_fp16_dev) return RWKVQ_EINVAL;
+    } else {
+      if (in.kind != RWKVQ_IN_WKV && in.kind != RWKVQ_IN_RELU2 && in.kind != RWKVQ_IN_F32) return RWKVQ_EINVAL;
+      if (!in.src_f32 || !aligned16(in.src_f32)) return in.src_f32 ? RWKVQ_EALIGN : RWKVQ_EINVAL;
+      if (in.kind == RWKVQ_IN_WKV) {
+        const void* need[] = {in.k_f32, in.v_f32, in.state_a, in.state_b, in.state_p, in.u_f32, in.w_f32};
+        for (const void* q : need) {
+          if (!q) return RWKVQ_EINVAL;
+          if (!aligned16(q)) return RWKVQ_EALIGN;
+        }
+      }
+      if (in.kind == RWKVQ_IN_F32 && in.gate_f32 && !aligned16(in.gate_f32)) return RWKVQ_EALIGN;
+      if (o.W_desc.ic % 8) return RWKVQ_ESHAPE;
+    }
+    if (in.xprev_out_fp16 && !aligned16(in.xprev_out_fp16)) return RWKVQ_EALIGN;
     if ((o.mu_image_dev == nullptr) != (o.xprev_fp16_dev == nullptr)) return RWKVQ_EINVAL;
     if (o.mu_image_dev) {
       st = check_vector_desc(&o.mu_desc, o.W_desc.ic);
       if (st != RWKVQ_OK) return st;
       if (!aligned16(o.mu_image_dev) || !aligned16(o.xprev_fp16_dev)) return RWKVQ_EALIGN;
     }
-    if (!aligned16(o.W_image_dev) || !aligned16(o.x_fp16_dev) || !aligned16(o.y_dev)) return RWKVQ_EALIGN;
+    if (!aligned16(o.W_image_dev) || (o.x_fp16_dev && !aligned16(o.x_fp16_dev)) || !aligned16(o.y_dev)) return RWKVQ_EALIGN;
     if (o.y_dtype != RWKVQ_F32) return RWKVQ_EUNSUPPORTED;   // partial sums are added with fp32 atomics
     if (i > 0 && o.stage < ops[i - 1].stage) return RWKVQ_EINVAL;
   }
@@ -936,7 +1021,10 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   info->smem_bytes = fixed + (uint32_t)ns * info->slot_bytes;
   info->P = P; info->B = B; info->NB = B <= 8 ? 1 : 2;
   info->poll_limit = kDefaultPollLimit; info->wait_skew = 0;
-  const bool mix = B >= 4;     // see StepArgs::mix
+  bool any_xform = false;
+  for (int i = 0; i < n_ops; ++i) any_xform = any_xform || ops[i].in.kind != RWKVQ_IN_BUFFER || ops[i].in.xprev_out_fp16 != nullptr;
+  // see StepArgs::mix; the element-wise operators in front of a product exist in the stage pre-pass only
+  const bool mix = B >= 4 || any_xform;
   const uint32_t xbuf_bytes = mix && B <= 8 ? XBufs<true, 1>::kBytes : XBufs<false, 1>::kBytes;
   info->mix = mix ? 1 : 0;
   const uint32_t nbp = (uint32_t)((B + 1) & ~1);
@@ -1146,6 +1234,14 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
           m.mu_aux = (uint64_t)(uintptr_t)(mi + vector_aux_offset(&op.mu_desc));
           m.mu_bits = (uint16_t)op.mu_desc.bits; m.mu_entries = (uint16_t)op.mu_desc.entries;
         }
+        m.kind = (uint16_t)op.in.kind;
+        m.src = (uint64_t)(uintptr_t)op.in.src_f32;
+        m.k = (uint64_t)(uintptr_t)(op.in.kind == RWKVQ_IN_F32 ? op.in.gate_f32 : op.in.k_f32);
+        m.v = (uint64_t)(uintptr_t)op.in.v_f32;
+        m.state_a = (uint64_t)(uintptr_t)op.in.state_a; m.state_b = (uint64_t)(uintptr_t)op.in.state_b;
+        m.state_p = (uint64_t)(uintptr_t)op.in.state_p;
+        m.u = (uint64_t)(uintptr_t)op.in.u_f32; m.w = (uint64_t)(uintptr_t)op.in.w_f32;
+        m.xprev_out = (uint64_t)(uintptr_t)op.in.xprev_out_fp16;
         m.dst_x = mix_x_off[o]; m.dst_sums = mix_sums_off[o];
         m.ic = (uint32_t)op.W_desc.ic; m.ic_pad = (uint32_t)op.W_desc.ic_pad;
         m.sums = op.W_desc.method == RWKVQ_SQ ? 1 : 0;

@@ -482,3 +482,44 @@ def test_proxy_segments_closed_forms_per_tile():
     # whole matrix as one tile = the matrix-level proxy
     pcm, pfm = orc.proxy_segments(w, 5, 7, K=4)
     assert (pcm[0, 0], pfm[0, 0]) == orc.proxy(w, 4)
+
+
+def test_wkv_recurrence_equals_the_literal_sums_and_closed_forms():
+    """Eq. 23: the two-sum recurrence reproduces the written-out sums token by token; first token gives v;
+    with no decay and no bonus the result is the softmax(k)-weighted mean of v; a huge decay keeps the previous and the current token only."""
+    rng = np.random.default_rng(9)
+    T, d = 7, 5
+    ks, vs = rng.standard_normal((T, d)), rng.standard_normal((T, d))
+    u, w = rng.standard_normal(d) * 0.5, rng.uniform(0.1, 1.5, d)
+    a, b = np.zeros(d), np.zeros(d)
+    for t in range(1, T + 1):
+        wkv, a, b = orc.wkv_step(a, b, ks[t - 1], vs[t - 1], u, w)
+        ref = orc.wkv_literal(ks[:t], vs[:t], u, w)
+        assert np.allclose(wkv, ref, rtol=1e-12, atol=1e-14)
+        if t == 1:
+            assert np.allclose(wkv, vs[0], rtol=1e-14)
+    # w = 0, u = 0: every token weighs exp(k_i) -> softmax-weighted mean over the history
+    z = np.zeros(d)
+    got = orc.wkv_literal(ks, vs, z, z)
+    p = np.exp(ks) / np.exp(ks).sum(axis=0)
+    assert np.allclose(got, (p * vs).sum(axis=0), rtol=1e-12)
+    # very large decay: f(i) keeps only i = t - 1 (its exponent carries no multiple of w), so the result
+    # mixes the previous and the current token with weights e^{k_{t-1}} and e^{u + k_t}
+    e_prev, e_cur = np.exp(ks[-2]), np.exp(u + ks[-1])
+    assert np.allclose(orc.wkv_literal(ks, vs, u, np.full(d, 700.0)), (e_prev * vs[-2] + e_cur * vs[-1]) / (e_prev + e_cur),
+                       rtol=1e-12)
+    # hand-worked: one channel, two tokens, k = 0, u = 0, w = ln 2: wkv_2 = (v1 + v2) / 2 ... f(1) = exp(0) = 1
+    one = orc.wkv_literal(np.zeros((2, 1)), np.array([[2.0], [6.0]]), np.zeros(1), np.array([math.log(2.0)]))
+    assert np.allclose(one, [4.0])
+    # three tokens: f(1) = exp(-w) = 1/2, f(2) = 1: (0.5*2 + 1*6 + 1*10) / (0.5 + 1 + 1)
+    three = orc.wkv_literal(np.zeros((3, 1)), np.array([[2.0], [6.0], [10.0]]), np.zeros(1), np.array([math.log(2.0)]))
+    assert np.allclose(three, [17.0 / 2.5])
+
+
+def test_gates_closed_forms():
+    assert orc.sigmoid(np.array([0.0]))[0] == 0.5
+    x = np.array([-3.0, 0.5, 2.0])
+    assert np.allclose(orc.sigmoid(x) + orc.sigmoid(-x), 1.0)
+    assert np.array_equal(orc.relu_squared(np.array([-2.0, 0.0, 3.0])), np.array([0.0, 0.0, 9.0]))
+    assert np.allclose(orc.time_mix_gate(np.zeros(3), x), 0.5 * x)
+    assert np.allclose(orc.channel_mix_gate(np.full(3, 50.0), x), x)
