@@ -241,6 +241,14 @@ rwkvq_status rwkvq_gemv_static(const rwkvq_desc* W_desc, const void* W_image_dev
  *   RWKVQ_IN_RELU2   x = max(src, 0)^2 (Eq. 27) with src = k'.
  *   RWKVQ_IN_F32     x = src, or sigmoid(gate_f32) * src when gate_f32 != NULL (Eq. 27: the
  *                    block's output as the next block's input), src / gate [B][ic] fp32.
+ * flags & RWKVQ_INF_RMSNORM (RWKVQ_IN_F32 only, ic a multiple of 64): the row is divided by its root
+ * mean square, x = v / sqrt(mean_j v[b][j]^2 + 1e-6) with v = src (* sigmoid(gate)).  The appendix
+ * prints no normalisation, but a chain of its blocks does not keep its activations in range
+ * without one (the squared ReLU makes magnitudes collapse or blow up within a few blocks); the
+ * models the paper quantizes normalise at exactly these two places, the inputs of time mixing and
+ * of channel mixing.  No learned weight or bias: use scale_f32 for a gain.
+ * scale_f32 (kinds other than RWKVQ_IN_BUFFER, may be NULL): one float in device memory, read at run
+ * time, that multiplies the operator's result before it is rounded to fp16.
  * xprev_out_fp16 (any kind, may be NULL): receives this token's x (before the mix), [B][ic]
  * fp16; it may be the very buffer xprev_fp16_dev points to (each element is read, then written,
  * by one thread), which makes the previous-token state advance by itself from step to step.  A
@@ -248,9 +256,10 @@ rwkvq_status rwkvq_gemv_static(const rwkvq_desc* W_desc, const void* W_image_dev
  * All pointers are device memory, 16-byte aligned, owned by the caller.
  */
 typedef enum { RWKVQ_IN_BUFFER = 0, RWKVQ_IN_WKV = 1, RWKVQ_IN_RELU2 = 2, RWKVQ_IN_F32 = 3 } rwkvq_input_kind;
+#define RWKVQ_INF_RMSNORM 1   /* RWKVQ_IN_F32 only */
 typedef struct {
   int32_t kind;               /* rwkvq_input_kind */
-  int32_t reserved;
+  int32_t flags;              /* RWKVQ_INF_* */
   const float* src_f32;
   const float* k_f32;
   const float* v_f32;
@@ -261,6 +270,7 @@ typedef struct {
   const float* w_f32;
   const float* gate_f32;
   void* xprev_out_fp16;
+  const float* scale_f32;     /* one float on the device, or NULL */
 } rwkvq_input_xform;
 
 /* One product of a decode step (same meaning as the rwkvq_gemv arguments).  `stage` orders the

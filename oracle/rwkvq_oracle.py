@@ -449,3 +449,12 @@ def channel_mix_gate(r: np.ndarray, y: np.ndarray) -> np.ndarray:
     """Output of channel mixing, Eq. 27: sigma(r') * y with y = W'_v . max(k', 0)^2."""
     return sigmoid(r) * np.asarray(y, dtype=np.float64)
 
+
+def rms_normalize(x: np.ndarray, eps: float = 1e-6) -> np.ndarray:
+    """Row-wise x / sqrt(mean(x^2) + eps), float64.  Not printed in the paper's appendix: the chained-block
+    workload normalises the inputs of time mixing and of channel mixing this way (the places where the
+    models the paper quantizes normalise), because a chain of the printed blocks alone does not keep its
+    activations in range."""
+    x = np.asarray(x, dtype=np.float64)
+    return x / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps)
+

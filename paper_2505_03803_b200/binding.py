@@ -49,12 +49,13 @@ class Desc(C.Structure):
 
 
 RWKVQ_IN_BUFFER, RWKVQ_IN_WKV, RWKVQ_IN_RELU2, RWKVQ_IN_F32 = 0, 1, 2, 3
+RWKVQ_INF_RMSNORM = 1
 
 
 class InputXform(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("reserved", C.c_int32), ("src_f32", C.c_void_p), ("k_f32", C.c_void_p),
+    _fields_ = [("kind", C.c_int32), ("flags", C.c_int32), ("src_f32", C.c_void_p), ("k_f32", C.c_void_p),
                 ("v_f32", C.c_void_p), ("state_a", C.c_void_p), ("state_b", C.c_void_p), ("state_p", C.c_void_p),
-                ("u_f32", C.c_void_p), ("w_f32", C.c_void_p), ("gate_f32", C.c_void_p), ("xprev_out_fp16", C.c_void_p)]
+                ("u_f32", C.c_void_p), ("w_f32", C.c_void_p), ("gate_f32", C.c_void_p), ("xprev_out_fp16", C.c_void_p), ("scale_f32", C.c_void_p)]
 
 
 class GemvOp(C.Structure):
@@ -449,9 +450,10 @@ def make_ops(entries):
         xf = e.get("in")
         if xf:      # {"kind": RWKVQ_IN_*, "src": .., "k": .., "v": .., "state_a": .., ..., "gate": .., "xprev_out": ..}
             o.in_.kind = int(xf.get("kind", RWKVQ_IN_BUFFER))
+            o.in_.flags = RWKVQ_INF_RMSNORM if xf.get("rmsnorm") else 0
             for field, key in (("src_f32", "src"), ("k_f32", "k"), ("v_f32", "v"), ("state_a", "state_a"),
                                ("state_b", "state_b"), ("state_p", "state_p"), ("u_f32", "u"), ("w_f32", "w"),
-                               ("gate_f32", "gate"), ("xprev_out_fp16", "xprev_out")):
+                               ("gate_f32", "gate"), ("xprev_out_fp16", "xprev_out"), ("scale_f32", "scale")):
                 t = xf.get(key)
                 setattr(o.in_, field, None if t is None else t.data_ptr())
         o.y_dev = e["y"].data_ptr()

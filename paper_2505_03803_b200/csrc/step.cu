@@ -97,10 +97,10 @@ static_assert(sizeof(StepEvent) == 64, "event descriptor size");
 struct StepMixOp {           // 144 bytes
   uint64_t x, xprev, mu, mu_aux, dst_x, dst_sums;
   uint32_t ic, ic_pad;
-  uint16_t mu_bits, mu_entries, sums, kind;     // kind: rwkvq_input_kind
+  uint16_t mu_bits, mu_entries, sums, kind;     // kind: rwkvq_input_kind | 0x100 when the row is RMS-normalised
   // element-wise operator in front of the product (rwkvq_input_xform): fp32 sources [B][ic], state, parameters
   uint64_t src, k, v, state_a, state_b, state_p, u, w;   // src doubles as the gate's operand; `k` holds the gate for RWKVQ_IN_F32
-  uint64_t xprev_out, pad;
+  uint64_t xprev_out, scale;         // scale: device address of one float that multiplies the operator's result (0 = none)
 };
 static_assert(sizeof(StepMixOp) == 144, "pre-pass descriptor size");
 
@@ -353,7 +353,7 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
 // Eqs. 23, 24, 27), rounded to fp16.  e0: index of the first element in the [B][ic] fp32 arrays,
 // col: its column (index into the per-channel parameters).  `commit` false (a lane that repeats
 // another lane's group to keep the half-warp whole): the recurrence state is not written.
-__device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int col, bool commit) {
+__device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int col, bool commit, float rstd) {
   float s[8];
   {
     const float4 a = __ldcg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(op.src) + e0));
@@ -361,10 +361,11 @@ __device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int
     s[0] = a.x; s[1] = a.y; s[2] = a.z; s[3] = a.w; s[4] = c.x; s[5] = c.y; s[6] = c.z; s[7] = c.w;
   }
   float o[8];
-  if (op.kind == RWKVQ_IN_RELU2) {
+  const int kind = op.kind & 0xFF;
+  if (kind == RWKVQ_IN_RELU2) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) { const float m = fmaxf(s[i], 0.f); o[i] = m * m; }
-  } else if (op.kind == RWKVQ_IN_F32) {
+  } else if (kind == RWKVQ_IN_F32) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) o[i] = s[i];
     if (op.k) {      // gate
@@ -372,6 +373,8 @@ __device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int
 #pragma unroll
       for (int i = 0; i < 8; ++i) o[i] *= sigmoidf_(__ldcg(g + i));
     }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] *= rstd;
   } else {           // RWKVQ_IN_WKV
     const float* kp = reinterpret_cast<const float*>(op.k) + e0;
     const float* vp = reinterpret_cast<const float*>(op.v) + e0;
@@ -396,7 +399,34 @@ __device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int
       if (commit) { sa[i] = f1 * a + f2 * vv; sb[i] = f1 * bb + f2; sp[i] = q2; }
     }
   }
+  if (op.scale) {
+    const float gsc = __ldcg(reinterpret_cast<const float*>(op.scale));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] *= gsc;
+  }
   return make_uint4(pack_half2(o[0], o[1]), pack_half2(o[2], o[3]), pack_half2(o[4], o[5]), pack_half2(o[6], o[7]));
+}
+
+// 1 / sqrt(mean over the row of v^2 + 1e-6), v = src (* sigmoid(gate)): the sixteen lanes of a half-warp
+// read row b of the fp32 source(s) together.  Items that follow one another in a half-warp mostly share
+// the row, so the caller keeps the last result.
+// Called by whole warps (the shuffles name all 32 lanes); a half-warp with `active` false reads nothing.
+__device__ __forceinline__ float row_rstd(const StepMixOp& op, int b, int l16, bool active) {
+  const float* src = reinterpret_cast<const float*>(op.src) + (size_t)b * op.ic;
+  const float* gate = op.k ? reinterpret_cast<const float*>(op.k) + (size_t)b * op.ic : nullptr;
+  float acc = 0.f;
+  for (uint32_t c = (uint32_t)l16 * 4u; active && c < op.ic; c += 64u) {
+    float4 v = __ldcg(reinterpret_cast<const float4*>(src + c));
+    if (gate) {
+      const float4 g = __ldcg(reinterpret_cast<const float4*>(gate + c));
+      v.x *= sigmoidf_(g.x); v.y *= sigmoidf_(g.y); v.z *= sigmoidf_(g.z); v.w *= sigmoidf_(g.w);
+    }
+    acc += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  __syncwarp();
+#pragma unroll
+  for (int d = 8; d > 0; d >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, d);
+  return rsqrtf(acc / (float)op.ic + 1e-6f);
 }
 
 // This CTA's share of a stage's pre-pass.  A half-warp takes one (product, batch row, 128-column
@@ -408,6 +438,9 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
   const StepMixOp* ops = a.mixops + ev.arrd.op_first;
   const int n_ops = (int)ev.arrd.op_count;
   const int nbp = (a.B + 1) & ~1;
+  uint64_t stat_src = 0;     // row whose statistic this half-warp computed last
+  int stat_b = -1;
+  float stat_rstd = 1.f;
   for (uint32_t g0 = lo + 2u * (uint32_t)(stid >> 5); g0 < hi; g0 += 2u * (uint32_t)kStagerWarps) {
     const uint32_t gi = g0 + (uint32_t)(lane >> 4);
     const bool valid = gi < hi;
@@ -419,11 +452,23 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
     const uint32_t ng = op.ic_pad >> 7;
     const int b = (int)(r / ng), grp = (int)(r % ng);
     const int col = grp * 128 + l16 * 8;
+    float rstd = 1.f;
+    {
+      // the two half-warps of a warp hold different items: the statistic is computed by the whole warp
+      // whenever either half needs a new one
+      const bool norm = (op.kind & 0x100) != 0;
+      const bool want = norm && (stat_src != op.src || stat_b != b);
+      if (__any_sync(0xFFFFFFFFu, want)) {
+        const float r = row_rstd(op, b, l16, want);
+        if (want) { stat_rstd = r; stat_src = op.src; stat_b = b; }
+      }
+      if (norm) rstd = stat_rstd;
+    }
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (col < (int)op.ic) {
       const size_t e0 = (size_t)b * op.ic + col;          // first of this lane's eight elements
       if (op.kind == RWKVQ_IN_BUFFER) v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + e0));
-      else v = xform_input(op, e0, col, valid);
+      else v = xform_input(op, e0, col, valid, rstd);
       if (op.xprev_out || op.mu) {
         // previous token's input: read for the mix, then (where asked) replaced by this token's
         uint4 pr = make_uint4(0u, 0u, 0u, 0u);
@@ -981,6 +1026,8 @@ static rwkvq_status validate_ops(const rwkvq_gemv_op* ops, int n_ops, int B) {
         }
       }
       if (in.kind == RWKVQ_IN_F32 && in.gate_f32 && !aligned16(in.gate_f32)) return RWKVQ_EALIGN;
+      if (in.flags & ~RWKVQ_INF_RMSNORM) return RWKVQ_EINVAL;
+      if ((in.flags & RWKVQ_INF_RMSNORM) && (in.kind != RWKVQ_IN_F32 || o.W_desc.ic % 64)) return RWKVQ_EUNSUPPORTED;
       if (o.W_desc.ic % 8) return RWKVQ_ESHAPE;
     }
     if (in.xprev_out_fp16 && !aligned16(in.xprev_out_fp16)) return RWKVQ_EALIGN;
@@ -1234,7 +1281,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
           m.mu_aux = (uint64_t)(uintptr_t)(mi + vector_aux_offset(&op.mu_desc));
           m.mu_bits = (uint16_t)op.mu_desc.bits; m.mu_entries = (uint16_t)op.mu_desc.entries;
         }
-        m.kind = (uint16_t)op.in.kind;
+        m.kind = (uint16_t)(op.in.kind | ((op.in.kind == RWKVQ_IN_F32 && (op.in.flags & RWKVQ_INF_RMSNORM)) ? 0x100 : 0));
         m.src = (uint64_t)(uintptr_t)op.in.src_f32;
         m.k = (uint64_t)(uintptr_t)(op.in.kind == RWKVQ_IN_F32 ? op.in.gate_f32 : op.in.k_f32);
         m.v = (uint64_t)(uintptr_t)op.in.v_f32;
@@ -1242,6 +1289,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
         m.state_p = (uint64_t)(uintptr_t)op.in.state_p;
         m.u = (uint64_t)(uintptr_t)op.in.u_f32; m.w = (uint64_t)(uintptr_t)op.in.w_f32;
         m.xprev_out = (uint64_t)(uintptr_t)op.in.xprev_out_fp16;
+        m.scale = (uint64_t)(uintptr_t)op.in.scale_f32;
         m.dst_x = mix_x_off[o]; m.dst_sums = mix_sums_off[o];
         m.ic = (uint32_t)op.W_desc.ic; m.ic_pad = (uint32_t)op.W_desc.ic_pad;
         m.sums = op.W_desc.method == RWKVQ_SQ ? 1 : 0;

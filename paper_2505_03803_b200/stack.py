@@ -278,3 +278,144 @@ def from_name(name: str, batch: int | None = None, **kw) -> Stack:
     b = spec["batches"][0] if batch is None else batch
     return Stack(spec["d"], spec["h"], kw.pop("layers", spec["layers"]), spec["entries"], b,
                  n_outliers=spec["outliers"], tag=name, **kw)
+
+
+class BlockOp:
+    __slots__ = ("layer", "name", "oc", "ic", "method", "desc", "image", "mu_desc", "mu_image", "y", "stage", "xform",
+                 "x", "xprev", "blob", "mu_blob")
+
+
+class BlockStack:
+    """`layers` RWKV blocks as Appendix A.1 writes them, chained: per block the time-mixing projections R, K,
+    V (token-shift mix each), the WKV recurrence and sigmoid gate in front of O (Eqs. 23-24), the channel-mixing
+    projections cm_k and cm_r (token-shift mix each, input = O's output), the squared ReLU in front of cm_v
+    (Eq. 27); the next block's input is sigmoid(cm_r) * cm_v.  Every element-wise operator runs inside the
+    persistent decode step (rwkvq_input_xform), so the four stages of a block are real data dependencies.
+    The paper's block has no gate matrix and prints neither norms nor residual connections: none here.
+    Without a normalisation the squared ReLU makes the activations of a chain of blocks collapse to zero
+    or overflow within a few blocks (measured: zero by the third block, or NaN by the eighth), so the
+    inputs of time mixing (from the second block on) and of channel mixing are divided by their root
+    mean square (RWKVQ_INF_RMSNORM), the places where the models the paper quantizes normalise.
+    Weights, method selection and quantization as in Stack (drawn and quantized on the device)."""
+
+    def __init__(self, d: int, h: int, layers: int, entries: int, batch: int, n_outliers: int = 8,
+                 heavy_fraction: float = 0.1, tag: str = "block", device: str = "cuda", kmeans_iters: int = 10,
+                 weight_scale: float = 1.0):
+        self.d, self.h, self.layers, self.batch, self.device, self.tag = d, h, layers, batch, device, tag
+        self.n_outliers = n_outliers
+        vq_bits = 6 if entries == 64 else 8
+        names = (("R", d, d, True, 0), ("K", d, d, True, 0), ("V", d, d, True, 0), ("O", d, d, False, 1),
+                 ("cm_k", h, d, True, 2), ("cm_r", d, d, True, 2), ("cm_v", d, h, False, 3))
+        t0 = time.time()
+        raw, pcs = {}, []
+        for l in range(layers):
+            mats = []
+            for (name, oc, ic, has_mu, stage) in names:
+                seed = inputs.seed_of(tag, l, name)
+                kind = inputs.weight_kind(seed, heavy_fraction)
+                w = gen_weight_device(seed, oc, ic, kind, device)
+                if weight_scale != 1.0:
+                    w = (w.float() * weight_scale).to(torch.float16)
+                raw[(l, name)] = (w, seed)
+                mats.append(w)
+            ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(mats)), dtype=torch.uint8, device=device)
+            pc, _, _ = B.rwkvq_proxy_select(mats, 4, math.inf, math.inf, ws)
+            pcs.extend(float(v) for v in pc)
+        self.tau_c = B.rwkvq_tau_largest_gap(np.array(pcs))
+        z32 = lambda *s: torch.zeros(s, dtype=torch.float32, device=device)
+        z16 = lambda *s: torch.zeros(s, dtype=torch.float16, device=device)
+        self.x0 = z16(batch, d)
+        self.x0_host = torch.zeros((batch, d), dtype=torch.float16).pin_memory()
+        self.ops: list[BlockOp] = []
+        self.states = []
+        gen = torch.Generator(device=device).manual_seed(inputs.seed_of(tag, "wkv") & 0x7FFFFFFF)
+        prev = None
+        k = 0
+        for l in range(layers):
+            ws = torch.empty(B.rwkvq_proxy_workspace_bytes(len(names)), dtype=torch.uint8, device=device)
+            _, _, phi = B.rwkvq_proxy_select([raw[(l, n[0])][0] for n in names], 4, self.tau_c, math.inf, ws)
+            y = {}
+            st = dict(a=z32(batch, d), b=z32(batch, d), p=torch.full((batch, d), -1e30, dtype=torch.float32, device=device),
+                      u=torch.randn(d, generator=gen, device=device) * 0.3,
+                      w=torch.rand(d, generator=gen, device=device) * 0.95 + 0.05)
+            self.states.append(st)
+            layer_ops = {}
+            for (name, oc, ic, has_mu, stage), p in zip(names, phi):
+                w, seed = raw.pop((l, name))
+                method = int(p)
+                blob = _device_blob(w, oc, ic, method, 3 if method == B.RWKVQ_SQ else vq_bits, kmeans_iters, seed)
+                o = BlockOp()
+                o.layer, o.name, o.oc, o.ic, o.method, o.blob = l, name, oc, ic, method, blob
+                o.desc, o.image = blob.desc, blob._image
+                o.mu_desc = o.mu_image = o.mu_blob = o.xprev = o.x = None
+                if has_mu:
+                    mu = torch.from_numpy(inputs.gen_mu(seed ^ 0xABCD, ic)).to(device)
+                    o.mu_blob = _device_blob(mu, 1, ic, B.RWKVQ_VQ, vq_bits, kmeans_iters, seed + 1)
+                    o.mu_desc, o.mu_image = o.mu_blob.desc, o.mu_blob._image
+                    o.xprev = z16(batch, ic)                 # this product's previous-token input, advanced by the step
+                o.y = z32(batch, oc)
+                o.stage = 4 * l + stage
+                y[name] = o.y
+                layer_ops[name] = o
+                self.ops.append(o)
+                k += 1
+            for name in ("R", "K", "V"):
+                o = layer_ops[name]
+                if prev is None:
+                    o.x, o.xform = self.x0, dict(kind=B.RWKVQ_IN_BUFFER, xprev_out=o.xprev)
+                else:
+                    o.xform = dict(kind=B.RWKVQ_IN_F32, src=prev[1], gate=prev[0], xprev_out=o.xprev, rmsnorm=True)
+            layer_ops["O"].xform = dict(kind=B.RWKVQ_IN_WKV, src=y["R"], k=y["K"], v=y["V"], state_a=st["a"], state_b=st["b"],
+                                        state_p=st["p"], u=st["u"], w=st["w"])
+            for name in ("cm_k", "cm_r"):
+                layer_ops[name].xform = dict(kind=B.RWKVQ_IN_F32, src=y["O"], xprev_out=layer_ops[name].xprev, rmsnorm=True)
+            layer_ops["cm_v"].xform = dict(kind=B.RWKVQ_IN_RELU2, src=y["cm_k"])
+            prev = (y["cm_r"], y["cm_v"])
+        self.out_r, self.out_v = prev
+        self.out_host = torch.zeros((2, batch, d), dtype=torch.float32).pin_memory()
+        self.ops.sort(key=lambda o: o.stage)
+        self.n_weights = sum(o.oc * o.ic for o in self.ops)
+        self.stream_bytes = sum(int(o.desc.stream_bytes) + (int(o.mu_desc.stream_bytes) if o.mu_desc is not None else 0)
+                                for o in self.ops)
+        # fp32 outputs written once and read once or twice by the next stage, fp16 previous-token states, WKV state
+        self.act_bytes = (sum(batch * o.oc * 4 * 2 + (batch * o.ic * 2 * 2 if o.xprev is not None else 0) for o in self.ops)
+                          + layers * batch * d * 4 * 6)
+        self.n_sq = sum(1 for o in self.ops if o.method == B.RWKVQ_SQ)
+        self.n_stages = 4 * layers
+        self.setup_s = time.time() - t0
+        entries_ = [dict(desc=o.desc, W=o.image, mu_desc=o.mu_desc, mu=o.mu_image, x=o.x, xprev=o.xprev, y=o.y, stage=o.stage,
+                         **{"in": o.xform}) for o in self.ops]
+        ops_arr = B.make_ops(entries_)
+        nbytes = B.rwkvq_step_plan_bytes(ops_arr, batch)
+        if nbytes == 0:
+            raise RuntimeError("rwkvq_step_plan_bytes returned 0 (plan rejected)")
+        self._plan = torch.zeros(nbytes, dtype=torch.uint8, device=device)
+        B.rwkvq_step_plan(ops_arr, batch, self._plan)
+        torch.cuda.synchronize()
+
+    def reset_state(self):
+        """Start of a sequence: empty WKV history, zero previous-token inputs."""
+        for st in self.states:
+            st["a"].zero_(); st["b"].zero_(); st["p"].fill_(-1e30)
+        for o in self.ops:
+            if o.xprev is not None:
+                o.xprev.zero_()
+
+    def set_token(self, seed: int):
+        """A fresh seeded token (fp16 activations with outlier channels) in the pinned host buffer."""
+        self.x0_host.copy_(torch.from_numpy(inputs.gen_activation(seed, self.batch, self.d, self.n_outliers).astype(np.float16)))
+
+    def run_step(self, stream=None):
+        """One token through every block: one persistent launch; the input is whatever x0 holds."""
+        B.rwkvq_step_run(self._plan, stream)
+
+    def run_step_host(self, stream=None):
+        """The token comes from pinned host memory and the last block's cm_r / cm_v outputs (whose gated
+        product is the model's hidden state, Eq. 27) go back to it; the caller synchronizes."""
+        self.x0.copy_(self.x0_host, non_blocking=True)
+        B.rwkvq_step_run(self._plan, stream)
+        self.out_host[0].copy_(self.out_r, non_blocking=True)
+        self.out_host[1].copy_(self.out_v, non_blocking=True)
+
+    def host_codes(self, op: BlockOp):
+        return op.blob.export_codes(), (op.mu_blob.export_codes() if op.mu_blob is not None else None)

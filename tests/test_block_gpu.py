@@ -56,23 +56,24 @@ def _build(d, h, layers, Bn, seed):
         xs = {n: z16(Bn, d) for n in mu}                      # previous-token input, one per product
         st = {"a": z32(Bn, d), "b": z32(Bn, d), "p": torch.full((Bn, d), -1e30, dtype=torch.float32, device=dev),
               "u": torch.from_numpy((rng.standard_normal(d) * 0.3).astype(np.float32)).to(dev),
-              "w": torch.from_numpy(rng.uniform(0.05, 1.0, d).astype(np.float32)).to(dev)}
+              "w": torch.from_numpy(rng.uniform(0.05, 1.0, d).astype(np.float32)).to(dev),
+              "gain": torch.full((1,), 0.5 + 0.25 * l, dtype=torch.float32, device=dev)}
         blk = dict(m=m, mu=mu, y=y, xs=xs, st=st, prev=prev)
         for n in ("R", "K", "V"):
             if prev is None:
                 xin = dict(kind=B.RWKVQ_IN_BUFFER, xprev_out=xs[n])
                 e = dict(x=x0)
             else:
-                xin = dict(kind=B.RWKVQ_IN_F32, src=prev[1], gate=prev[0], xprev_out=xs[n])
+                xin = dict(kind=B.RWKVQ_IN_F32, src=prev[1], gate=prev[0], xprev_out=xs[n], rmsnorm=True)
                 e = dict(x=None)
             e.update(desc=m[n].desc, W=m[n].dev, mu_desc=mu[n].desc, mu=mu[n].dev, xprev=xs[n], y=y[n], stage=4 * l, **{"in": xin})
             entries.append(e)
         entries.append(dict(desc=m["O"].desc, W=m["O"].dev, x=None, y=y["O"], stage=4 * l + 1,
                             **{"in": dict(kind=B.RWKVQ_IN_WKV, src=y["R"], k=y["K"], v=y["V"], state_a=st["a"], state_b=st["b"],
-                                          state_p=st["p"], u=st["u"], w=st["w"])}))
+                                          state_p=st["p"], u=st["u"], w=st["w"], scale=st["gain"])}))
         for n in ("cK", "cR"):
             entries.append(dict(desc=m[n].desc, W=m[n].dev, mu_desc=mu[n].desc, mu=mu[n].dev, x=None, xprev=xs[n], y=y[n],
-                                stage=4 * l + 2, **{"in": dict(kind=B.RWKVQ_IN_F32, src=y["O"], xprev_out=xs[n])}))
+                                stage=4 * l + 2, **{"in": dict(kind=B.RWKVQ_IN_F32, src=y["O"], xprev_out=xs[n], rmsnorm=(n == "cK"))}))
         entries.append(dict(desc=m["cV"].desc, W=m["cV"].dev, x=None, y=y["cV"], stage=4 * l + 3,
                             **{"in": dict(kind=B.RWKVQ_IN_RELU2, src=y["cK"])}))
         prev = (y["cR"], y["cV"])
@@ -114,7 +115,7 @@ def test_block_chain_matches_oracle_token_by_token(Bn):
             if blk["prev"] is None:
                 x_t = x_host.astype(np.float64)
             else:
-                x_t = _f16(orc.channel_mix_gate(_np(blk["prev"][0]), _np(blk["prev"][1])))
+                x_t = _f16(orc.rms_normalize(orc.channel_mix_gate(_np(blk["prev"][0]), _np(blk["prev"][1]))))
             for n in ("R", "K", "V"):
                 _check_product(f"token {token} layer {l} {n}", m[n], orc.token_shift(x_t, bf["xs"][n], mu[n].mu_hat), y[n])
                 got_state = _np(blk["xs"][n])
@@ -123,13 +124,14 @@ def test_block_chain_matches_oracle_token_by_token(Bn):
             a_true, b_true = bf["a"] * np.exp(bf["p"]), bf["b"] * np.exp(bf["p"])
             u, w = _np(st["u"]), _np(st["w"])
             wkv, a_new, b_new = orc.wkv_step(a_true, b_true, _np(y["K"]), _np(y["V"]), u, w)
-            _check_product(f"token {token} layer {l} O", m["O"], _f16(orc.time_mix_gate(_np(y["R"]), wkv)), y["O"])
+            gain = float(st["gain"][0])
+            _check_product(f"token {token} layer {l} O", m["O"], _f16(gain * orc.time_mix_gate(_np(y["R"]), wkv)), y["O"])
             ga, gb = _np(st["a"]) * np.exp(_np(st["p"])), _np(st["b"]) * np.exp(_np(st["p"]))
             # fp32 recurrence: relative to the magnitudes that are added (the numerator sum can cancel)
             a_scale = np.exp(-w) * np.abs(a_true) + np.exp(_np(y["K"])) * np.abs(_np(y["V"]))
             assert (np.abs(ga - a_new) <= 2e-5 * a_scale + 1e-30).all() and np.allclose(gb, b_new, rtol=2e-5, atol=1e-30)
-            x_c = _f16(_np(y["O"]))
-            for n in ("cK", "cR"):
+            for n in ("cK", "cR"):       # cm_k reads the normalised output of time mixing, cm_r the plain one
+                x_c = _f16(orc.rms_normalize(_np(y["O"]))) if n == "cK" else _f16(_np(y["O"]))
                 _check_product(f"token {token} layer {l} {n}", m[n], orc.token_shift(x_c, bf["xs"][n], mu[n].mu_hat), y[n])
                 assert (np.abs(_np(blk["xs"][n]) - x_c) <= 2.0 ** -10 * np.abs(x_c) + 1e-7).all()
             _check_product(f"token {token} layer {l} cV", m["cV"], _f16(orc.relu_squared(_np(y["cK"]))), y["cV"])
@@ -148,7 +150,7 @@ def test_block_first_token_and_argument_checks():
     torch.cuda.synchronize()
     blk = blocks[0]
     y = blk["y"]
-    _check_product("first token O", blk["m"]["O"], _f16(orc.sigmoid(_np(y["R"])) * _np(y["V"])), y["O"])
+    _check_product("first token O", blk["m"]["O"], _f16(0.5 * orc.sigmoid(_np(y["R"])) * _np(y["V"])), y["O"])
     B.rwkvq_step_plan_release(plan)
     # a WKV input without its state, and an unknown kind, are refused before anything is planned
     bad = [dict(e) for e in entries]

@@ -523,3 +523,13 @@ def test_gates_closed_forms():
     assert np.array_equal(orc.relu_squared(np.array([-2.0, 0.0, 3.0])), np.array([0.0, 0.0, 9.0]))
     assert np.allclose(orc.time_mix_gate(np.zeros(3), x), 0.5 * x)
     assert np.allclose(orc.channel_mix_gate(np.full(3, 50.0), x), x)
+
+
+def test_rms_normalize_closed_forms():
+    x = np.array([[3.0, -3.0, 3.0, -3.0], [0.5, 0.0, 0.0, 0.0]])
+    y = orc.rms_normalize(x, eps=0.0)
+    assert np.allclose(y[0], [1.0, -1.0, 1.0, -1.0]) and np.allclose(y[1], [2.0, 0.0, 0.0, 0.0])
+    z = np.random.default_rng(2).standard_normal((3, 64))
+    n = orc.rms_normalize(z, eps=0.0)
+    assert np.allclose((n * n).mean(axis=1), 1.0) and np.allclose(orc.rms_normalize(7.5 * z, eps=0.0), n)
+    assert np.array_equal(orc.rms_normalize(np.zeros((1, 8))), np.zeros((1, 8)))      # eps keeps a zero row finite
