@@ -79,6 +79,7 @@ def parse_args(argv=None):
                          "generator on the device (default: device with --quantizer device, else host)")
     ap.add_argument("--no-configs", action="store_true", help="skip the configs map (the other stacks)")
     ap.add_argument("--no-proxy", action="store_true", help="skip the proxy leg")
+    ap.add_argument("--no-block", action="store_true", help="skip the chained-block leg")
     ap.add_argument("--no-quantize", action="store_true", help="skip the device-quantizer leg (one 7B-class layer)")
     return ap.parse_args(argv)
 
@@ -483,6 +484,59 @@ def quantize_leg(reps: int = 5):
                    "weights_per_s": oc * ic / (vq_ms * 1e-3)}}
 
 
+def block_leg(configs=(("c3_7b", 1), ("c4_14b", 16)), max_steps=300):
+    """Whole blocks with their element-wise operators inside the same persistent launch (Appendix A.1 Eqs.
+    20-27: token shift, R/K/V, WKV recurrence and sigmoid gate, O, channel-mix K/R, squared ReLU, V, output
+    gate; plus the root-mean-square normalisation the chain needs), so that every stage reads what the stage
+    before wrote: tokens/s of the chain of blocks, one token per sequence per step.  The matrix set is the
+    appendix's (no gate matrix), the shapes and depth those of the named stack."""
+    import torch
+    from paper_2505_03803_b200 import binding as B
+    from paper_2505_03803_b200 import inputs, stack as stack_mod
+    peak, kind = measured_hbm_peak()
+    out = {}
+    for (wl, batch) in configs:
+        sp = inputs.STACKS[wl]
+        st = stack_mod.BlockStack(sp["d"], sp["h"], sp["layers"], sp["entries"], batch, n_outliers=sp["outliers"], tag=wl)
+        st.set_token(11)
+        for _ in range(3):
+            st.run_step_host()
+        torch.cuda.synchronize()
+        K = int(min(max_steps, max(20, 1500.0 / max(0.05, st.stream_bytes / 2.0e9))))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            st.run_step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / K
+        stream = torch.cuda.current_stream()
+        e0.record()
+        for _ in range(K):
+            st.run_step_host(stream)
+            stream.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_e2e = e0.elapsed_time(e1) / K
+        if B.rwkvq_device_status() != 0:
+            raise SystemExit("bench.py: a device-side wait timed out in the block leg")
+        finite = bool(torch.isfinite(st.out_v).all())
+        alg = st.stream_bytes + st.act_bytes
+        gbs = alg / (ms * 1e-3) / 1e9
+        out[f"{wl}_b{batch}"] = {
+            "tokens_per_s": batch / (ms * 1e-3), "ms_per_step": ms, "steps": K, "matrices": len(st.ops), "sq_matrices": st.n_sq,
+            "stages": st.n_stages, "packed_bytes_per_step": st.stream_bytes, "activation_bytes_per_step": st.act_bytes,
+            "outputs_finite": finite, "setup_s": round(st.setup_s, 1),
+            "e2e": {"value": batch / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(st.x0_host.numel() * 2),
+                    "d2h_bytes_per_step": int(st.out_host.numel() * 4)},
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                         "peak_kind": f"of {kind}", "kernel": "step_kernel", "algorithmic_bytes_per_launch": alg}}
+        del st
+        torch.cuda.empty_cache()
+    return {"workload": "chain of RWKV blocks (7 projections per block, element-wise operators fused into the step), "
+                        "one token per sequence per step", "configs": out}
+
+
 # ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
@@ -665,6 +719,7 @@ def run_ours(args):
     prefill = prefill_leg() if world == 1 and not args.no_prefill else None
     quantize = quantize_leg() if world == 1 and not args.no_quantize else None
     proxy = proxy_leg(with_oracle=not args.no_cpu_baseline) if world == 1 and not args.no_proxy else None
+    block = block_leg() if world == 1 and whole and not args.no_block else None
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -681,7 +736,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": head["config"],
         "roofline": head["roofline"], "cpu_baseline": cpu, "e2e": head["e2e"], "clocks": head["clocks"],
         "gpu_launches": head["gpu_launches"], "hbm_gbs": head["roofline"]["achieved"],
-        "configs": configs, "prefill": prefill, "quantize": quantize, "proxy": proxy,
+        "configs": configs, "prefill": prefill, "quantize": quantize, "proxy": proxy, "block": block,
     }
     print(json.dumps(line), flush=True)
     if world > 1:

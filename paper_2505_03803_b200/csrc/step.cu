@@ -438,7 +438,55 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
   const StepMixOp* ops = a.mixops + ev.arrd.op_first;
   const int n_ops = (int)ev.arrd.op_count;
   const int nbp = (a.B + 1) & ~1;
-  uint64_t stat_src = 0;     // row whose statistic this half-warp computed last
+  // Row statistics first: the rows of normalised inputs that this CTA's items fall in (a few: the items
+  // are consecutive groups of consecutive rows) are reduced by all stager threads together, 1.5 KB per
+  // round of loads, into a small table; rows beyond the table are reduced by the half-warp that meets them.
+  constexpr int kRowTable = 8;
+  __shared__ float s_rstd[kRowTable];
+  __shared__ float s_part[kStagerWarps];
+  __shared__ uint32_t s_row_end[kRowTable];      // first item behind the row of each entry
+  int n_rows = 0;
+  {
+    uint32_t r = lo;
+    while (r < hi && n_rows < kRowTable) {
+      uint32_t rr = r;
+      int k = 0;
+      uint32_t icp = __ldg(&ops[0].ic_pad);
+      while (k + 1 < n_ops && rr >= (uint32_t)a.B * (icp >> 7)) { rr -= (uint32_t)a.B * (icp >> 7); ++k; icp = __ldg(&ops[k].ic_pad); }
+      const StepMixOp op = ops[k];
+      const uint32_t ng = op.ic_pad >> 7;
+      const int b = (int)(rr / ng);
+      float rstd = 1.f;
+      if (op.kind & 0x100) {
+        const float* src = reinterpret_cast<const float*>(op.src) + (size_t)b * op.ic;
+        const float* gate = op.k ? reinterpret_cast<const float*>(op.k) + (size_t)b * op.ic : nullptr;
+        float acc = 0.f;
+#pragma unroll 4
+        for (uint32_t c = (uint32_t)stid * 4u; c < op.ic; c += (uint32_t)kStagerThreads * 4u) {
+          float4 v = __ldcg(reinterpret_cast<const float4*>(src + c));
+          if (gate) {
+            const float4 g = __ldcg(reinterpret_cast<const float4*>(gate + c));
+            v.x *= sigmoidf_(g.x); v.y *= sigmoidf_(g.y); v.z *= sigmoidf_(g.z); v.w *= sigmoidf_(g.w);
+          }
+          acc += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, d);
+        if (lane == 0) s_part[stid >> 5] = acc;
+        named_bar_sync(5, kStagerThreads);
+        float tot = 0.f;
+#pragma unroll
+        for (int wdx = 0; wdx < kStagerWarps; ++wdx) tot += s_part[wdx];
+        rstd = rsqrtf(tot / (float)op.ic + 1e-6f);
+        named_bar_sync(5, kStagerThreads);      // s_part is reused by the next row
+      }
+      r += ng - rr % ng;                         // first item of the next row
+      if (stid == 0) { s_rstd[n_rows] = rstd; s_row_end[n_rows] = r; }
+      ++n_rows;
+    }
+    named_bar_sync(5, kStagerThreads);
+  }
+  uint64_t stat_src = 0;     // row whose statistic this half-warp computed last (rows beyond the table)
   int stat_b = -1;
   float stat_rstd = 1.f;
   for (uint32_t g0 = lo + 2u * (uint32_t)(stid >> 5); g0 < hi; g0 += 2u * (uint32_t)kStagerWarps) {
@@ -457,12 +505,16 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
       // the two half-warps of a warp hold different items: the statistic is computed by the whole warp
       // whenever either half needs a new one
       const bool norm = (op.kind & 0x100) != 0;
-      const bool want = norm && (stat_src != op.src || stat_b != b);
+      const uint32_t item = valid ? gi : lo;
+      int idx = 0;
+      while (idx < n_rows && item >= s_row_end[idx]) ++idx;
+      const bool tabled = idx < n_rows;
+      const bool want = norm && !tabled && (stat_src != op.src || stat_b != b);
       if (__any_sync(0xFFFFFFFFu, want)) {
-        const float r = row_rstd(op, b, l16, want);
-        if (want) { stat_rstd = r; stat_src = op.src; stat_b = b; }
+        const float rs = row_rstd(op, b, l16, want);
+        if (want) { stat_rstd = rs; stat_src = op.src; stat_b = b; }
       }
-      if (norm) rstd = stat_rstd;
+      if (norm) rstd = tabled ? s_rstd[idx] : stat_rstd;
     }
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (col < (int)op.ic) {

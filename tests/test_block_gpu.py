@@ -159,3 +159,43 @@ def test_block_first_token_and_argument_checks():
     bad = [dict(e) for e in entries]
     bad[6] = dict(bad[6], **{"in": dict(kind=9, src=y["cK"])})
     assert B.rwkvq_step_plan_bytes(B.make_ops(bad), Bn) == 0
+
+
+def _decode(st, op):
+    codes, mu_codes = st.host_codes(op)
+    w_hat = orc.sq_decode(codes["q"], codes["scale"], codes["zero"]) if op.method == B.RWKVQ_SQ else orc.vq_decode(codes["codebook"], codes["q"])
+    mu_hat = orc.mu_decode(mu_codes["codebook"], mu_codes["q"]) if mu_codes is not None else None
+    return w_hat, mu_hat
+
+
+@pytest.mark.parametrize("batch", [1, 16])
+def test_chained_blocks_at_7b_width_sampled(batch):
+    """The chain bench.py times (BlockStack), two blocks of the 7B-class width: after two tokens, one product of
+    every kind of input operator is recomputed by the oracle from the values the GPU holds upstream."""
+    from paper_2505_03803_b200 import stack as stack_mod
+    st = stack_mod.BlockStack(4096, 14336, 2, 64, batch, n_outliers=8, tag="c3_7b", kmeans_iters=2)
+    by = {(o.layer, o.name): o for o in st.ops}
+    for token in range(2):
+        st.set_token(50 + token)
+        prev_R1 = _np(by[(1, "R")].xprev)
+        prev_ck0 = _np(by[(0, "cm_k")].xprev)
+        a0, b0, p0 = (_np(st.states[0][k]) for k in ("a", "b", "p"))
+        st.run_step_host()
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+    y = {k: _np(o.y) for k, o in by.items()}
+    assert all(np.isfinite(v).all() for v in y.values())
+    # block 1, R: gated and normalised output of block 0 (Eq. 27), token-shift mix with the token before
+    w_hat, mu_hat = _decode(st, by[(1, "R")])
+    x_t = _f16(orc.rms_normalize(orc.channel_mix_gate(y[(0, "cm_r")], y[(0, "cm_v")])))
+    _check_product("block 1 R", type("M", (), {"w_hat": w_hat}), orc.token_shift(x_t, prev_R1, mu_hat), by[(1, "R")].y)
+    # block 0, O: WKV (Eq. 23) from the history before the second token, sigmoid gate (Eq. 24)
+    w_hat, _ = _decode(st, by[(0, "O")])
+    wkv, _, _ = orc.wkv_step(a0 * np.exp(p0), b0 * np.exp(p0), y[(0, "K")], y[(0, "V")], _np(st.states[0]["u"]), _np(st.states[0]["w"]))
+    _check_product("block 0 O", type("M", (), {"w_hat": w_hat}), _f16(orc.time_mix_gate(y[(0, "R")], wkv)), by[(0, "O")].y)
+    # block 0, cm_k: normalised output of time mixing with its own token shift; cm_v: squared ReLU (Eq. 27)
+    w_hat, mu_hat = _decode(st, by[(0, "cm_k")])
+    x_c = _f16(orc.rms_normalize(y[(0, "O")]))
+    _check_product("block 0 cm_k", type("M", (), {"w_hat": w_hat}), orc.token_shift(x_c, prev_ck0, mu_hat), by[(0, "cm_k")].y)
+    w_hat, _ = _decode(st, by[(1, "cm_v")])
+    _check_product("block 1 cm_v", type("M", (), {"w_hat": w_hat}), _f16(orc.relu_squared(y[(1, "cm_k")])), by[(1, "cm_v")].y)
