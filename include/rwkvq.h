@@ -12,7 +12,7 @@
  * Method references are to RWKVQuant (arXiv 2505.03803): scalar quantization
  * Section 3.2 Eq. 2, vector quantization Section 3.2 Eq. 3, coarse-to-fine proxy
  * Section 4.1 Eqs. 5-18, element-wise (token-shift) weights Section 4.2 and
- * Appendix A.1 Eqs. 20-26.
+ * Appendix A.1 Eqs. 20-27.
  */
 #ifndef RWKVQ_H_
 #define RWKVQ_H_
@@ -343,7 +343,7 @@ rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const 
 /*
  * Prefill product Y[t][i] = sum_j bf16(w_hat[i][j]) * x_mix[t][j] for M tokens, bf16 x bf16 ->
  * fp32 on the tensor cores (the dense contraction of the path: Appendix A.1, the projections of
- * Eqs. 21-24 applied to a whole sequence).  bf16(w_hat) is the decoded weight (the fp32 rounding
+ * Eqs. 20-22 and 24-27 applied to a whole sequence).  bf16(w_hat) is the decoded weight (the fp32 rounding
  * of s*(q-z), or the fp16 codebook entry) rounded to nearest even.  x_mix[t] = X[t] +
  * (X[t-1] - X[t]) (.) mu_hat (Eq. 20), with X[-1] = xprev0 (zeros if NULL); mu NULL = no mix.
  * X_bf16_dev: [M][ic] row-major; Y_dev: [M][oc] row-major, F32 or BF16; all device pointers,

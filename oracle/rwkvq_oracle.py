@@ -388,7 +388,7 @@ def prefill_prev(X: np.ndarray, x_prev0: np.ndarray | None) -> np.ndarray:
 
 
 def gemv(w_hat: np.ndarray, x_mix: np.ndarray) -> np.ndarray:
-    """y[b, i] = sum_j w_hat[i, j] * x_mix[b, j] in float64 (the W.(...) products of Eqs. 20-26)."""
+    """y[b, i] = sum_j w_hat[i, j] * x_mix[b, j] in float64 (the W.(...) products of Eqs. 20-22 and 24-27)."""
     return np.asarray(x_mix, dtype=np.float64) @ np.asarray(w_hat, dtype=np.float64).T
 
 
