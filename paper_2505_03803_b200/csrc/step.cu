@@ -19,6 +19,13 @@
 //     every input fragment shared by the two records.  Partial sums go to y with fp32 atomics at
 //     the end of a run along K.
 //
+// For batches of four and more, and whenever a product's input is an element-wise operator on
+// earlier outputs (rwkvq_input_xform: the WKV recurrence and sigmoid gate of Appendix A.1 Eqs. 23-24,
+// the squared ReLU and output gate of Eq. 27, optionally a root-mean-square normalisation), the
+// inputs of a stage are not built per CTA: after the stage barrier all CTAs together compute the
+// stage's x_mix once (mix_slice: a half-warp per 128-column group) into a scratch region of the plan,
+// publish it through a second barrier, and every CTA fetches its segments with bulk copies.
+//
 // The host plans the step once: every stage's units are dealt WHOLE to the CTAs, row of tiles by
 // row of tiles where that balances (each row gets a number of CTAs by greedy cost per CTA), else at
 // their cost midpoints, small stages in eighths of a unit (one warp's records); the plan is a per-CTA
@@ -446,7 +453,9 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
   __shared__ float s_part[kStagerWarps];
   __shared__ uint32_t s_row_end[kRowTable];      // first item behind the row of each entry
   int n_rows = 0;
-  {
+  bool any_norm = false;
+  for (int k = 0; k < n_ops; ++k) any_norm = any_norm || (__ldg(&ops[k].kind) & 0x100) != 0;
+  if (any_norm) {
     uint32_t r = lo;
     while (r < hi && n_rows < kRowTable) {
       uint32_t rr = r;
