@@ -484,7 +484,7 @@ def quantize_leg(reps: int = 5):
                    "weights_per_s": oc * ic / (vq_ms * 1e-3)}}
 
 
-def block_leg(configs=(("c3_7b", 1), ("c4_14b", 16)), max_steps=300):
+def block_leg(configs=(("c3_7b", 1), ("c4_14b", 16)), max_steps=300, steps=None):
     """Whole blocks with their element-wise operators inside the same persistent launch (Appendix A.1 Eqs.
     20-27: token shift, R/K/V, WKV recurrence and sigmoid gate, O, channel-mix K/R, squared ReLU, V, output
     gate; plus the root-mean-square normalisation the chain needs), so that every stage reads what the stage
@@ -502,7 +502,7 @@ def block_leg(configs=(("c3_7b", 1), ("c4_14b", 16)), max_steps=300):
         for _ in range(3):
             st.run_step_host()
         torch.cuda.synchronize()
-        K = int(min(max_steps, max(20, 1500.0 / max(0.05, st.stream_bytes / 2.0e9))))
+        K = steps if steps is not None else int(min(max_steps, max(20, 1500.0 / max(0.05, st.stream_bytes / 2.0e9))))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(K):
@@ -719,7 +719,7 @@ def run_ours(args):
     prefill = prefill_leg() if world == 1 and not args.no_prefill else None
     quantize = quantize_leg() if world == 1 and not args.no_quantize else None
     proxy = proxy_leg(with_oracle=not args.no_cpu_baseline) if world == 1 and not args.no_proxy else None
-    block = block_leg() if world == 1 and whole and not args.no_block else None
+    block = block_leg(steps=args.steps) if world == 1 and whole and not args.no_block else None
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:

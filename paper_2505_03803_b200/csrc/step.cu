@@ -101,15 +101,22 @@ static_assert(sizeof(StepEvent) == 64, "event descriptor size");
 
 // One product's share of a stage's pre-pass: where its inputs are and where x_mix (fp16 rows of
 // ic_pad columns, zero beyond ic) and the per-group sums ([group][3][nbp] floats) go.
-struct StepMixOp {           // 144 bytes
+struct StepMixOp {           // 64 bytes
   uint64_t x, xprev, mu, mu_aux, dst_x, dst_sums;
   uint32_t ic, ic_pad;
-  uint16_t mu_bits, mu_entries, sums, kind;     // kind: rwkvq_input_kind | 0x100 when the row is RMS-normalised
-  // element-wise operator in front of the product (rwkvq_input_xform): fp32 sources [B][ic], state, parameters
-  uint64_t src, k, v, state_a, state_b, state_p, u, w;   // src doubles as the gate's operand; `k` holds the gate for RWKVQ_IN_F32
+  // kind: rwkvq_input_kind | 0x100 when the row is RMS-normalised | 0x200 when this token's input is stored
+  // (xprev_out) | 0x400 on the first product of a stage in which some input is normalised; any non-zero kind
+  // has a StepMixX beside it
+  uint16_t mu_bits, mu_entries, sums, kind;
+};
+static_assert(sizeof(StepMixOp) == 64, "pre-pass descriptor size");
+// Element-wise operator in front of the product (rwkvq_input_xform): fp32 sources [B][ic], state,
+// parameters.  Kept apart so that the pre-pass of plain products reads 64 bytes per item as before.
+struct StepMixX {            // 80 bytes
+  uint64_t src, k, v, state_a, state_b, state_p, u, w;   // `k` holds the gate for RWKVQ_IN_F32
   uint64_t xprev_out, scale;         // scale: device address of one float that multiplies the operator's result (0 = none)
 };
-static_assert(sizeof(StepMixOp) == 144, "pre-pass descriptor size");
+static_assert(sizeof(StepMixX) == 80, "pre-pass operator descriptor size");
 
 constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGroups, kStagerWarps = 3;
 constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
@@ -141,6 +148,7 @@ struct StepArgs {
   // barrier per stage (counter[n_stages + 1 + s]), and fetched into the segment buffers with bulk copies.
   int mix;
   const StepMixOp* mixops;    // dst_x / dst_sums are offsets into `scratch`
+  const StepMixX* mixx;       // parallel to mixops
   uint8_t* scratch;
 };
 
@@ -360,7 +368,7 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
 // Eqs. 23, 24, 27), rounded to fp16.  e0: index of the first element in the [B][ic] fp32 arrays,
 // col: its column (index into the per-channel parameters).  `commit` false (a lane that repeats
 // another lane's group to keep the half-warp whole): the recurrence state is not written.
-__device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int col, bool commit, float rstd) {
+__device__ __forceinline__ uint4 xform_input(const StepMixOp& mo, const StepMixX& op, size_t e0, int col, bool commit, float rstd) {
   float s[8];
   {
     const float4 a = __ldcg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(op.src) + e0));
@@ -368,7 +376,7 @@ __device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int
     s[0] = a.x; s[1] = a.y; s[2] = a.z; s[3] = a.w; s[4] = c.x; s[5] = c.y; s[6] = c.z; s[7] = c.w;
   }
   float o[8];
-  const int kind = op.kind & 0xFF;
+  const int kind = mo.kind & 0xFF;
   if (kind == RWKVQ_IN_RELU2) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) { const float m = fmaxf(s[i], 0.f); o[i] = m * m; }
@@ -418,9 +426,9 @@ __device__ __forceinline__ uint4 xform_input(const StepMixOp& op, size_t e0, int
 // read row b of the fp32 source(s) together.  Items that follow one another in a half-warp mostly share
 // the row, so the caller keeps the last result.
 // Called by whole warps (the shuffles name all 32 lanes); a half-warp with `active` false reads nothing.
-__device__ __forceinline__ float row_rstd(const StepMixOp& op, int b, int l16, bool active) {
-  const float* src = reinterpret_cast<const float*>(op.src) + (size_t)b * op.ic;
-  const float* gate = op.k ? reinterpret_cast<const float*>(op.k) + (size_t)b * op.ic : nullptr;
+__device__ __forceinline__ float row_rstd(const StepMixOp& op, const StepMixX& ox, int b, int l16, bool active) {
+  const float* src = reinterpret_cast<const float*>(ox.src) + (size_t)b * op.ic;
+  const float* gate = ox.k ? reinterpret_cast<const float*>(ox.k) + (size_t)b * op.ic : nullptr;
   float acc = 0.f;
   for (uint32_t c = (uint32_t)l16 * 4u; active && c < op.ic; c += 64u) {
     float4 v = __ldcg(reinterpret_cast<const float4*>(src + c));
@@ -453,9 +461,7 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
   __shared__ float s_part[kStagerWarps];
   __shared__ uint32_t s_row_end[kRowTable];      // first item behind the row of each entry
   int n_rows = 0;
-  bool any_norm = false;
-  for (int k = 0; k < n_ops; ++k) any_norm = any_norm || (__ldg(&ops[k].kind) & 0x100) != 0;
-  if (any_norm) {
+  if (__ldg(&ops[0].kind) & 0x400) {      // the planner marks the first product of a stage that has a normalised input
     uint32_t r = lo;
     while (r < hi && n_rows < kRowTable) {
       uint32_t rr = r;
@@ -467,8 +473,9 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
       const int b = (int)(rr / ng);
       float rstd = 1.f;
       if (op.kind & 0x100) {
-        const float* src = reinterpret_cast<const float*>(op.src) + (size_t)b * op.ic;
-        const float* gate = op.k ? reinterpret_cast<const float*>(op.k) + (size_t)b * op.ic : nullptr;
+        const StepMixX ox = a.mixx[ev.arrd.op_first + k];
+        const float* src = reinterpret_cast<const float*>(ox.src) + (size_t)b * op.ic;
+        const float* gate = ox.k ? reinterpret_cast<const float*>(ox.k) + (size_t)b * op.ic : nullptr;
         float acc = 0.f;
 #pragma unroll 4
         for (uint32_t c = (uint32_t)stid * 4u; c < op.ic; c += (uint32_t)kStagerThreads * 4u) {
@@ -509,8 +516,11 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
     const uint32_t ng = op.ic_pad >> 7;
     const int b = (int)(r / ng), grp = (int)(r % ng);
     const int col = grp * 128 + l16 * 8;
+    StepMixX ox;
+    if (op.kind) ox = a.mixx[ev.arrd.op_first + k];
+    else { ox.src = ox.k = ox.xprev_out = ox.scale = 0; }
     float rstd = 1.f;
-    {
+    if (op.kind & 0x100) {
       // the two half-warps of a warp hold different items: the statistic is computed by the whole warp
       // whenever either half needs a new one
       const bool norm = (op.kind & 0x100) != 0;
@@ -518,23 +528,23 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
       int idx = 0;
       while (idx < n_rows && item >= s_row_end[idx]) ++idx;
       const bool tabled = idx < n_rows;
-      const bool want = norm && !tabled && (stat_src != op.src || stat_b != b);
+      const bool want = norm && !tabled && (stat_src != ox.src || stat_b != b);
       if (__any_sync(0xFFFFFFFFu, want)) {
-        const float rs = row_rstd(op, b, l16, want);
-        if (want) { stat_rstd = rs; stat_src = op.src; stat_b = b; }
+        const float rs = row_rstd(op, ox, b, l16, want);
+        if (want) { stat_rstd = rs; stat_src = ox.src; stat_b = b; }
       }
       if (norm) rstd = tabled ? s_rstd[idx] : stat_rstd;
     }
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (col < (int)op.ic) {
       const size_t e0 = (size_t)b * op.ic + col;          // first of this lane's eight elements
-      if (op.kind == RWKVQ_IN_BUFFER) v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + e0));
-      else v = xform_input(op, e0, col, valid, rstd);
-      if (op.xprev_out || op.mu) {
+      if ((op.kind & 0xFF) == RWKVQ_IN_BUFFER) v = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.x) + e0));
+      else v = xform_input(op, ox, e0, col, valid, rstd);
+      if (ox.xprev_out || op.mu) {
         // previous token's input: read for the mix, then (where asked) replaced by this token's
         uint4 pr = make_uint4(0u, 0u, 0u, 0u);
         if (op.mu) pr = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(op.xprev) + e0));
-        if (op.xprev_out && valid) *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(op.xprev_out) + e0) = v;
+        if (ox.xprev_out && valid) *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(ox.xprev_out) + e0) = v;
         if (op.mu) {
           const uint32_t bits = op.mu_bits, mask = (1u << bits) - 1u;
           // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
@@ -1040,7 +1050,7 @@ struct PlanInfo {
   unsigned abort_epoch; // value of the abort epoch when the counters were last known good
   uint32_t poll_limit, wait_skew;
   uint32_t slot_bytes, replica_bytes, smem_bytes;
-  size_t off_unit_off, off_event_off, off_units, off_events, off_counter, off_mixops, off_scratch, total_bytes;
+  size_t off_unit_off, off_event_off, off_units, off_events, off_counter, off_mixops, off_mixx, off_scratch, total_bytes;
   uint32_t n_units, n_events, n_barriers;
 };
 
@@ -1324,6 +1334,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   // previous stage, and with it every copy out of the region, has finished everywhere)
   std::vector<uint64_t> mix_x_off(n_ops, 0), mix_sums_off(n_ops, 0);
   std::vector<StepMixOp> mixops(mix ? n_ops : 0);
+  std::vector<StepMixX> mixx(mix ? n_ops : 0);
   uint64_t scratch_bytes = 0;
   if (mix) {
     for (int st_i = 0; st_i < n_stages; ++st_i) {
@@ -1342,19 +1353,25 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
           m.mu_aux = (uint64_t)(uintptr_t)(mi + vector_aux_offset(&op.mu_desc));
           m.mu_bits = (uint16_t)op.mu_desc.bits; m.mu_entries = (uint16_t)op.mu_desc.entries;
         }
-        m.kind = (uint16_t)(op.in.kind | ((op.in.kind == RWKVQ_IN_F32 && (op.in.flags & RWKVQ_INF_RMSNORM)) ? 0x100 : 0));
-        m.src = (uint64_t)(uintptr_t)op.in.src_f32;
-        m.k = (uint64_t)(uintptr_t)(op.in.kind == RWKVQ_IN_F32 ? op.in.gate_f32 : op.in.k_f32);
-        m.v = (uint64_t)(uintptr_t)op.in.v_f32;
-        m.state_a = (uint64_t)(uintptr_t)op.in.state_a; m.state_b = (uint64_t)(uintptr_t)op.in.state_b;
-        m.state_p = (uint64_t)(uintptr_t)op.in.state_p;
-        m.u = (uint64_t)(uintptr_t)op.in.u_f32; m.w = (uint64_t)(uintptr_t)op.in.w_f32;
-        m.xprev_out = (uint64_t)(uintptr_t)op.in.xprev_out_fp16;
-        m.scale = (uint64_t)(uintptr_t)op.in.scale_f32;
+        m.kind = (uint16_t)(op.in.kind | ((op.in.kind == RWKVQ_IN_F32 && (op.in.flags & RWKVQ_INF_RMSNORM)) ? 0x100 : 0) |
+                            (op.in.xprev_out_fp16 ? 0x200 : 0));
+        StepMixX& mx = mixx[o];
+        std::memset(&mx, 0, sizeof(mx));
+        mx.src = (uint64_t)(uintptr_t)op.in.src_f32;
+        mx.k = (uint64_t)(uintptr_t)(op.in.kind == RWKVQ_IN_F32 ? op.in.gate_f32 : op.in.k_f32);
+        mx.v = (uint64_t)(uintptr_t)op.in.v_f32;
+        mx.state_a = (uint64_t)(uintptr_t)op.in.state_a; mx.state_b = (uint64_t)(uintptr_t)op.in.state_b;
+        mx.state_p = (uint64_t)(uintptr_t)op.in.state_p;
+        mx.u = (uint64_t)(uintptr_t)op.in.u_f32; mx.w = (uint64_t)(uintptr_t)op.in.w_f32;
+        mx.xprev_out = (uint64_t)(uintptr_t)op.in.xprev_out_fp16;
+        mx.scale = (uint64_t)(uintptr_t)op.in.scale_f32;
         m.dst_x = mix_x_off[o]; m.dst_sums = mix_sums_off[o];
         m.ic = (uint32_t)op.W_desc.ic; m.ic_pad = (uint32_t)op.W_desc.ic_pad;
         m.sums = op.W_desc.method == RWKVQ_SQ ? 1 : 0;
       }
+      bool stage_norm = false;
+      for (int o = stage_ranges[st_i].first; o < stage_ranges[st_i].second; ++o) stage_norm = stage_norm || (mixops[o].kind & 0x100);
+      if (stage_norm) mixops[stage_ranges[st_i].first].kind |= 0x400;
       scratch_bytes = std::max(scratch_bytes, off);
     }
   }
@@ -1467,6 +1484,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   info->off_events = off; off += round_up_sz(all_events.size() * sizeof(StepEvent), 256);
   info->off_counter = off; off += round_up_sz((size_t)info->n_barriers * 4, 256);
   info->off_mixops = off; off += round_up_sz(mixops.size() * sizeof(StepMixOp), 256);
+  info->off_mixx = off; off += round_up_sz(mixx.size() * sizeof(StepMixX), 256);
   info->off_scratch = off; off += round_up_sz((size_t)scratch_bytes, 256);
   info->total_bytes = off;
   if (out) {
@@ -1476,6 +1494,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     if (!all_units.empty()) memcpy(out->data() + info->off_units, all_units.data(), all_units.size() * sizeof(StepUnit));
     memcpy(out->data() + info->off_events, all_events.data(), all_events.size() * sizeof(StepEvent));
     if (!mixops.empty()) memcpy(out->data() + info->off_mixops, mixops.data(), mixops.size() * sizeof(StepMixOp));
+    if (!mixx.empty()) memcpy(out->data() + info->off_mixx, mixx.data(), mixx.size() * sizeof(StepMixX));
   }
   return RWKVQ_OK;
 }
@@ -1545,6 +1564,7 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
   if (!a.status) return RWKVQ_ECUDA;
   a.B = info.B; a.n_slots = info.n_slots; a.n_stages = info.n_stages;
   a.mix = info.mix; a.mixops = reinterpret_cast<const StepMixOp*>(p + info.off_mixops);
+  a.mixx = reinterpret_cast<const StepMixX*>(p + info.off_mixx);
   a.scratch = const_cast<uint8_t*>(p) + info.off_scratch;
   a.slot_bytes = info.slot_bytes; a.replica_bytes = info.replica_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
