@@ -429,6 +429,21 @@ def proxy_leg(reps: int = 10, with_oracle: bool = True):
             "matrices": rows}
 
 
+def vq_alu_roofline(oc, ic, entries, iters, ms, sm_mhz=1965.0, sms=148):
+    """vq_kmeans_kernel against the fp32 instruction rate: an assignment pass evaluates, per (2-D vector,
+    centre) pair, two subtractions, a multiply, a fused multiply-add and a compare-and-keep = 5 thread
+    instructions; k-means++ seeding makes `entries` such passes against one new centre each (5 instructions per
+    vector and pass) and every Lloyd iteration one pass against all centres.  Peak = 128 fp32 lanes per SM per
+    clock at the maximum SM clock.  Centre updates, the scans of the seeding and the final fp64 assignment are
+    not counted, so the fraction is a lower bound on how busy the lanes are."""
+    vectors = oc * ic // 2
+    work = 5.0 * vectors * entries * (iters + 1)          # iterations against all centres + the seeding passes
+    achieved = work / (ms * 1e-3) / 1e12
+    peak = sms * 128 * sm_mhz * 1e6 / 1e12
+    return {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "T thread-instructions/s", "frac": achieved / peak,
+            "traffic": None, "kernel": "vq_kmeans_kernel"}
+
+
 def quantize_leg(reps: int = 5):
     """The device quantizers on one 7B-class layer: every projection scalar-quantized (Eq. 2) from fp16
     weights resident on the device, timed over the layer, and one 4096 x 4096 matrix vector-quantized
@@ -481,7 +496,7 @@ def quantize_leg(reps: int = 5):
                          "timed": "eight rwkvq_quantize_dev_async calls and one rwkvq_quantize_check (a stream "
                                   "synchronization) per layer"},
             "vq": {"matrix": f"{oc}x{ic}, 64 entries, 10 Lloyd iterations", "ms": vq_ms, "tiles": (oc // 256) * (ic // 256),
-                   "weights_per_s": oc * ic / (vq_ms * 1e-3)}}
+                   "weights_per_s": oc * ic / (vq_ms * 1e-3), "roofline": vq_alu_roofline(oc, ic, 64, 10, vq_ms)}}
 
 
 def block_leg(configs=(("c3_7b", 1), ("c4_14b", 16)), max_steps=300, steps=None):
