@@ -122,6 +122,11 @@ constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGrou
 constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
 constexpr int kGroupThreads = kGroupWarps * 32;
 constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
+// Registers per thread after the re-division at kernel entry: 4 consumer warpgroups and 1 warpgroup of
+// stagers + producer must fit the 96 x kThreads the launch reserved.
+constexpr int kConsumerRegs = 104, kStagerRegs = 64;
+static_assert(kConsumerWarps % 4 == 0 && (kStagerWarps + 1) == 4, "register re-division works on warpgroups of four warps");
+static_assert(kConsumerRegs * kConsumerThreads + kStagerRegs * 128 <= 96 * kThreads, "register re-division exceeds the launch's pool");
 constexpr int kMaxSlots = 12;
 constexpr uint32_t kCtrlBytes = 1024, kXBufTotal = 49152, kMuScratch = 1024;
 // Input-segment buffers: two of 24 KB when the CTA mixes its own inputs (the segment carries a mu row and
@@ -1033,6 +1038,17 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   const uint32_t u0 = a.unit_off[blockIdx.x], u1 = a.unit_off[blockIdx.x + 1];
   const uint32_t e0 = a.event_off[blockIdx.x], e1 = a.event_off[blockIdx.x + 1];
   const int warp = threadIdx.x >> 5;
+  // The launch gives every thread 96 registers.  With one batch block the last warpgroup (stagers and
+  // producer) hands part of its share back and the four consumer warpgroups take it: their record
+  // routine then keeps everything in registers.  With two batch blocks eight more registers do not
+  // end the consumers' spills, and the stagers' pre-pass needs its 96.
+  if constexpr (NB == 1) {
+    if (warp < kConsumerWarps) {
+      asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" :: "n"(kConsumerRegs));
+    } else {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" :: "n"(kStagerRegs));
+    }
+  }
   if (warp < kConsumerWarps) {
     consumer_role<NB, MIX>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
   } else if (warp < kConsumerWarps + kStagerWarps) {
