@@ -373,7 +373,7 @@ def prefill_leg(reps: int = 10, M: int = 2048):
     ms, flops, tf, n_sq, n = out["hybrid"]
     assert 0 < n_sq < n
     return {"workload": f"one 7B-class layer (8 projections, d=4096 h=14336), M={M} tokens, hybrid SQ/VQ-64, bf16 x bf16 -> fp32",
-            "ms_per_layer": ms, "flop_per_layer": flops, "launches_per_layer": n + 1, "sq_matrices": n_sq,
+            "ms_per_layer": ms, "flop_per_layer": flops, "launches_per_layer": 2, "sq_matrices": n_sq,
             "formats": hybrid,
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
                          "traffic": None, "peak_kind": f"of {kind} (burst)", "kernel": "prefill_kernel",

@@ -177,10 +177,34 @@ __device__ __forceinline__ uint32_t vec_index(const uint8_t* stream, int p, int 
 // tile's swizzled rows; the eight threads of a row read and write 128 contiguous bytes.
 constexpr int kMixRun = 8;
 static_assert(kTileTokens == 32 * kMixRun, "a block of 256 threads covers one tile");
-__global__ void __launch_bounds__(256) prefill_mix_kernel(const __nv_bfloat16* X, const __nv_bfloat16* xprev0, const uint8_t* mu,
-                                                          const uint8_t* mu_aux, int mu_bits, int M, int ic, int KB, int MT,
-                                                          uint8_t* tiles) {
-  const int kb = (int)(blockIdx.x % (unsigned)KB), mt = (int)(blockIdx.x / (unsigned)KB);
+struct MixProduct {
+  const __nv_bfloat16* X;
+  const __nv_bfloat16* xprev0;
+  const uint8_t* mu;
+  const uint8_t* mu_aux;
+  uint8_t* tiles;
+  int mu_bits, ic, KB;
+};
+
+struct MixArgs {
+  MixProduct p[kMaxGroup];
+  unsigned block_start[kMaxGroup + 1];   // first block of each product; [n] = grid size
+  int n, M, MT;
+};
+
+// One launch mixes the operands of every product of the group: block -> (product, token tile, column block).
+__global__ void __launch_bounds__(256) prefill_mix_kernel(const __grid_constant__ MixArgs ma) {
+  int pi = 0;
+  while (pi + 1 < ma.n && blockIdx.x >= ma.block_start[pi + 1]) ++pi;
+  const MixProduct& mp = ma.p[pi];
+  const __nv_bfloat16* X = mp.X;
+  const __nv_bfloat16* xprev0 = mp.xprev0;
+  const uint8_t* mu = mp.mu;
+  const uint8_t* mu_aux = mp.mu_aux;
+  uint8_t* tiles = mp.tiles;
+  const int mu_bits = mp.mu_bits, ic = mp.ic, KB = mp.KB, M = ma.M, MT = ma.MT;
+  const unsigned blk = blockIdx.x - ma.block_start[pi];
+  const int kb = (int)(blk % (unsigned)KB), mt = (int)(blk / (unsigned)KB);
   if (mt >= MT) return;
   const int cx = threadIdx.x & 7, ty = threadIdx.x >> 3;
   const int c = kb * kKBlock + cx * 8, r0 = ty * kMixRun, t0 = mt * kTileTokens + r0;
@@ -726,13 +750,22 @@ rwkvq_status rwkvq_gemm_prefill_grouped(const rwkvq_prefill_op* ops, int n_ops, 
   ga.ticket = reinterpret_cast<unsigned*>(first.ws + (size_t)MT * first.a.KB * pf::kXTileBytes);
   cudaError_t e = cudaMemsetAsync(ga.ticket, 0, sizeof(unsigned), s);
   if (e != cudaSuccess) return cuda_status(e);
-  // pre-pass per product
+  // pre-pass: the operands of all products in one launch, in the order the tiles will be dealt
+  pf::MixArgs ma;
+  memset(&ma, 0, sizeof(ma));
+  ma.n = n_ops; ma.M = M; ma.MT = MT;
+  unsigned long long mix_blocks = 0;
   for (int i = 0; i < n_ops; ++i) {
-    const HostProduct& h = hp[i];
-    pf::prefill_mix_kernel<<<(unsigned)(MT * h.a.KB), 256, 0, s>>>(
-        static_cast<const __nv_bfloat16*>(h.X), static_cast<const __nv_bfloat16*>(h.xprev0), h.mup, h.mua, h.mu_bits, M, h.a.ic,
-        h.a.KB, MT, h.ws);
+    const HostProduct& h = hp[order[i]];
+    pf::MixProduct& mp = ma.p[i];
+    mp.X = static_cast<const __nv_bfloat16*>(h.X); mp.xprev0 = static_cast<const __nv_bfloat16*>(h.xprev0);
+    mp.mu = h.mup; mp.mu_aux = h.mua; mp.tiles = h.ws; mp.mu_bits = h.mu_bits; mp.ic = h.a.ic; mp.KB = h.a.KB;
+    ma.block_start[i] = (unsigned)mix_blocks;
+    mix_blocks += (unsigned long long)MT * (unsigned long long)h.a.KB;
+    if (mix_blocks > 0x7FFFFFFFull) return RWKVQ_EUNSUPPORTED;
   }
+  ma.block_start[n_ops] = (unsigned)mix_blocks;
+  pf::prefill_mix_kernel<<<(unsigned)mix_blocks, 256, 0, s>>>(ma);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_status(e);
   int dev = 0, sms = 148;
