@@ -118,15 +118,30 @@ struct StepMixX {            // 80 bytes
 };
 static_assert(sizeof(StepMixX) == 80, "pre-pass operator descriptor size");
 
-constexpr int kGroupWarps = 8, kGroups = 2, kConsumerWarps = kGroupWarps * kGroups, kStagerWarps = 3;
-constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
-constexpr int kGroupThreads = kGroupWarps * 32;
-constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
-// Registers per thread after the re-division at kernel entry: 4 consumer warpgroups and 1 warpgroup of
-// stagers + producer must fit the 96 x kThreads the launch reserved.
-constexpr int kConsumerRegs = 104, kStagerRegs = 64;
-static_assert(kConsumerWarps % 4 == 0 && (kStagerWarps + 1) == 4, "register re-division works on warpgroups of four warps");
-static_assert(kConsumerRegs * kConsumerThreads + kStagerRegs * 128 <= 96 * kThreads, "register re-division exceeds the launch's pool");
+constexpr int kGroupWarps = 8, kGroupThreads = kGroupWarps * 32;
+// Thread layout of a CTA, by the number of batch blocks NB a record is multiplied with.
+//   NB = 1 (B <= 8): two consumer groups of eight warps, three stager warps, one producer warp: 640 threads,
+//     96 registers each at launch, re-divided at entry (consumers kConsumerRegs, the last warpgroup
+//     kStagerRegs).
+//   NB = 2 (B > 8): the record routine wants about 150 registers, which sixteen consumer warps cannot have,
+//     and eight warps that keep everything in registers outrun sixteen that spill: ONE consumer group,
+//     seven stager warps (the stage pre-pass is theirs), one producer: 512 threads, 128 registers at
+//     launch, re-divided to 168 for the two consumer warpgroups and 88 for the other two.
+template <int NB> struct Shape {
+  static constexpr int kGroups = NB == 2 ? 1 : 2;
+  static constexpr int kStagerWarps = NB == 2 ? 7 : 3;
+  static constexpr int kConsumerWarps = kGroupWarps * kGroups;
+  static constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
+  static constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
+  static constexpr int kLaunchRegs = NB == 2 ? 128 : 96;
+  static constexpr int kConsumerRegs = NB == 2 ? 168 : 104, kStagerRegs = NB == 2 ? 88 : 64;
+  static_assert(kConsumerWarps % 4 == 0 && (kStagerWarps + 1) % 4 == 0, "register re-division works on warpgroups of four warps");
+  static_assert(kConsumerRegs * kConsumerThreads + kStagerRegs * (kStagerThreads + 32) <= kLaunchRegs * kThreads,
+                "register re-division exceeds the launch's pool");
+  static_assert(kLaunchRegs * kThreads <= 65536, "register file");
+};
+constexpr int groups_of(int NB) { return NB == 2 ? 1 : 2; }
+constexpr int threads_of(int NB) { return NB == 2 ? Shape<2>::kThreads : Shape<1>::kThreads; }
 constexpr int kMaxSlots = 12;
 constexpr uint32_t kCtrlBytes = 1024, kXBufTotal = 49152, kMuScratch = 1024;
 // Input-segment buffers: two of 24 KB when the CTA mixes its own inputs (the segment carries a mu row and
@@ -256,10 +271,11 @@ constexpr uint32_t kMaxBarriers = 256;   // barriers that close a stage (8-bit c
 // after everything every party did before reporting (the consumers' reductions into y, the
 // stagers' clearing of the next outputs): block-level synchronisation followed by one thread's
 // release, the pattern of a cooperative grid barrier.
+template <int NB>
 __device__ __forceinline__ void stage_report(Ctrl* ctrl, const StepArgs& a, uint32_t b) {
   const uint32_t sh = 8u * (b & 3u);
   const uint32_t old = smem_add_acq_rel(&ctrl->stage_cnt[b >> 2], 1u << sh);
-  if (((old >> sh) & 0xFFu) == (uint32_t)kConsumerWarps) red_release_gpu(a.counter + b, 1u);
+  if (((old >> sh) & 0xFFu) == (uint32_t)Shape<NB>::kConsumerWarps) red_release_gpu(a.counter + b, 1u);
 }
 // Where the consumer warps are the busy role (two batch blocks per record) they only count
 // themselves in, and a stager thread, which has nothing else to do at that point, waits (bounded)
@@ -271,13 +287,14 @@ __device__ __forceinline__ void stage_report(Ctrl* ctrl, const StepArgs& a, uint
 __device__ __forceinline__ void stage_report_total(Ctrl* ctrl, uint32_t b) {
   asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(&ctrl->stage_cnt[b >> 2])), "r"(1u << (8u * (b & 3u))) : "memory");
 }
+template <int NB>
 __device__ __forceinline__ bool stage_wait_total_and_arrive(Ctrl* ctrl, const StepArgs& a, uint32_t b, volatile int* abort_flag) {
   const uint32_t limit = poll_limit_of(abort_flag) << 4;
   const uint32_t sh = 8u * (b & 3u);
   for (uint32_t it = 0; it < limit; ++it) {
     uint32_t v;
     asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&ctrl->stage_cnt[b >> 2])) : "memory");
-    if (((v >> sh) & 0xFFu) >= (uint32_t)kConsumerWarps) { red_release_gpu(a.counter + b, 1u); return true; }
+    if (((v >> sh) & 0xFFu) >= (uint32_t)Shape<NB>::kConsumerWarps) { red_release_gpu(a.counter + b, 1u); return true; }
     if ((it & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -452,7 +469,9 @@ __device__ __forceinline__ float row_rstd(const StepMixOp& op, const StepMixX& o
 // This CTA's share of a stage's pre-pass.  A half-warp takes one (product, batch row, 128-column
 // group) at a time: it loads x (and x_prev, and decodes mu_hat), mixes, rounds to fp16, stores the
 // 128 values to the product's pre-pass rows and reduces the three sums of the group with shuffles.
+template <int NB>
 __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
+  constexpr int kStagerWarps = Shape<NB>::kStagerWarps, kStagerThreads = Shape<NB>::kStagerThreads;
   const int lane = stid & 31, l16 = lane & 15;
   const uint32_t lo = ev.arr.grp_lo, hi = ev.arr.grp_hi;
   const StepMixOp* ops = a.mixops + ev.arrd.op_first;
@@ -601,7 +620,8 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
 template <bool MIX, int NB>
 __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_t* xbufs, uint32_t* mucb,
                             uint32_t e0, uint32_t e1) {
-  const int stid = threadIdx.x - kConsumerThreads;
+  constexpr int kStagerThreads = Shape<NB>::kStagerThreads;
+  const int stid = threadIdx.x - Shape<NB>::kConsumerThreads;
   const int lane = stid & 31;
   volatile int* abortp = &ctrl->abort_flag;
   uint32_t nseg = 0;          // segments staged so far
@@ -622,8 +642,8 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       // before it: arrive directly.  Otherwise report; the last of the seventeen parties arrives.
       if (stid == 0) {
         if (ev.barrier == 0u) red_release_gpu(a.counter, 1u);
-        else if constexpr (NB == 2) ok = stage_wait_total_and_arrive(ctrl, a, ev.barrier, abortp);
-        else stage_report(ctrl, a, ev.barrier);
+        else if constexpr (NB == 2) ok = stage_wait_total_and_arrive<NB>(ctrl, a, ev.barrier, abortp);
+        else stage_report<NB>(ctrl, a, ev.barrier);
       }
       if constexpr (MIX) {
         // once the barrier opens, do this CTA's share of the new stage's pre-pass and publish it
@@ -637,7 +657,7 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
           }
           ok = named_bar_and(6, kStagerThreads, ok);   // thread 0's acquire precedes every thread's loads of x
           if (!ok) break;
-          mix_slice(a, ev, stid);
+          mix_slice<NB>(a, ev, stid);
           named_bar_sync(4, kStagerThreads);           // every thread's pre-pass stores precede thread 0's release
           if (stid == 0) red_release_gpu(a.counter + (uint32_t)a.n_stages + 1u + ev.barrier, 1u);
         }
@@ -835,6 +855,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
                               uint32_t unit_base, uint32_t n_units, uint32_t ev_base, uint32_t n_events) {
   bool dead = false;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kGroups = Shape<NB>::kGroups;
   const int grp = warp >> 3, w = warp & 7;
   const int g = lane >> 2, t = lane & 3;
   volatile int* abortp = &ctrl->abort_flag;
@@ -859,7 +880,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
       if (lane == 0 && !dead) stage_report_total(ctrl, next_bar);
       ++next_bar;
     } else {
-      if (lane == 0 && !dead) stage_report(ctrl, a, next_bar);
+      if (lane == 0 && !dead) stage_report<NB>(ctrl, a, next_bar);
       ++next_bar;
     }
   };
@@ -1020,7 +1041,8 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
 }
 
 template <int NB, bool MIX>
-__global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(Shape<NB>::kThreads, 1) step_kernel(const StepArgs a) {
+  constexpr int kConsumerWarps = Shape<NB>::kConsumerWarps, kStagerWarps = Shape<NB>::kStagerWarps;
   extern __shared__ __align__(128) uint8_t smem[];
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem);
   uint8_t* xbufs = smem + kCtrlBytes + (size_t)a.n_slots * a.slot_bytes;
@@ -1038,16 +1060,13 @@ __global__ void __launch_bounds__(kThreads, 1) step_kernel(const StepArgs a) {
   const uint32_t u0 = a.unit_off[blockIdx.x], u1 = a.unit_off[blockIdx.x + 1];
   const uint32_t e0 = a.event_off[blockIdx.x], e1 = a.event_off[blockIdx.x + 1];
   const int warp = threadIdx.x >> 5;
-  // The launch gives every thread 96 registers.  With one batch block the last warpgroup (stagers and
-  // producer) hands part of its share back and the four consumer warpgroups take it: their record
-  // routine then keeps everything in registers.  With two batch blocks eight more registers do not
-  // end the consumers' spills, and the stagers' pre-pass needs its 96.
-  if constexpr (NB == 1) {
-    if (warp < kConsumerWarps) {
-      asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" :: "n"(kConsumerRegs));
-    } else {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" :: "n"(kStagerRegs));
-    }
+  // Registers are re-divided at entry (see Shape): the warpgroups of stagers and producer hand part of
+  // their share back and the consumer warpgroups take it, so that the record routine keeps everything
+  // in registers.
+  if (warp < kConsumerWarps) {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" :: "n"(Shape<NB>::kConsumerRegs));
+  } else {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" :: "n"(Shape<NB>::kStagerRegs));
   }
   if (warp < kConsumerWarps) {
     consumer_role<NB, MIX>(a, smem, ctrl, xbufs, replicas, u0, u1 - u0, e0, e1 - e0);
@@ -1141,6 +1160,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     else if (ops[i].W_desc.bits == 6) has_vq6 = true;
     else has_vq8 = true;
   }
+  const int kGroups = groups_of(B <= 8 ? 1 : 2);   // consumer groups per CTA: they take a CTA's units in turn
   uint32_t data_max = 0;
   if (has_sq) data_max = std::max(data_max, 2u * 8u * RWKVQ_SQ_RECORD_BYTES);
   if (has_vq6) data_max = std::max(data_max, 2u * 8u * 1536u + 256u);
@@ -1401,7 +1421,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     const size_t n = L.size();
     // a group accumulates along K in registers while its consecutive units stay on the same rows
     for (size_t i = 0; i < n; ++i) {
-      const size_t j = i + kGroups;
+      const size_t j = i + (size_t)kGroups;
       const bool same_run = j < n && L[j].stage == L[i].stage && L[j].op == L[i].op && L[j].tr == L[i].tr &&
                             L[j].w0 == L[i].w0 && L[j].w1 == L[i].w1;
       if (!same_run) L[i].u.flags |= UF_FLUSH;
@@ -1461,7 +1481,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       all_events.push_back(cta_arrivals[c][s + 1]);
     }
     // what each group has to pass between its consecutive segments, and after its last unit of a stage
-    uint32_t prev_ev[kGroups] = {0, 0};
+    uint32_t prev_ev[2] = {0, 0};
     const StepEvent* evs = all_events.data() + event_off[c];
     const uint32_t n_ev = (uint32_t)(all_events.size() - event_off[c]);
     std::vector<uint32_t> arr_idx(n_stages, 0);
@@ -1597,7 +1617,7 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
   if (e != cudaSuccess) return cuda_status(e);
   void* params[] = {&a};
   // Cooperative launch: all CTAs must be resident at once because they meet at the stage barrier.
-  e = cudaLaunchCooperativeKernel(fn, dim3(info.P), dim3(kThreads), params, info.smem_bytes, s);
+  e = cudaLaunchCooperativeKernel(fn, dim3(info.P), dim3(threads_of(info.NB)), params, info.smem_bytes, s);
   if (e != cudaSuccess) {   // this run will never arrive: have the next one clear the counters
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     auto it = g_plans.find(plan_dev);
