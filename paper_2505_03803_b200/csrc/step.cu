@@ -466,6 +466,59 @@ __device__ __forceinline__ float row_rstd(const StepMixOp& op, const StepMixX& o
   return rsqrtf(acc / (float)op.ic + 1e-6f);
 }
 
+// A load whose value is not needed: it brings the sector into this SM's L1.
+__device__ __forceinline__ void touch_global(const void* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(reinterpret_cast<uintptr_t>(p) & ~static_cast<uintptr_t>(3)));
+}
+
+// Everything mix_slice will read that does not depend on the stage before -- the products' descriptors,
+// the mu_hat codes of this CTA's items and the codebook entries they select -- is read once ahead of
+// time, while the consumer warps are still busy with the current stage, so that behind the barrier the
+// chain of dependent loads (descriptor -> codes -> codebook) hits in L1 and only x itself comes from L2.
+template <int NB>
+__device__ void mix_warm(const StepArgs& a, const StepEvent& ev, int stid) {
+  constexpr int kStagerWarps = Shape<NB>::kStagerWarps;
+  const int lane = stid & 31, l16 = lane & 15;
+  const uint32_t lo = ev.arr.grp_lo, hi = ev.arr.grp_hi;
+  const StepMixOp* ops = a.mixops + ev.arrd.op_first;
+  const int n_ops = (int)ev.arrd.op_count;
+  if (lo >= hi) return;
+  touch_global(reinterpret_cast<const uint8_t*>(ops) + 32);
+  for (uint32_t g0 = lo + 2u * (uint32_t)(stid >> 5); g0 < hi; g0 += 2u * (uint32_t)kStagerWarps) {
+    const uint32_t gi = g0 + (uint32_t)(lane >> 4);
+    uint32_t r = gi < hi ? gi : lo;
+    int k = 0;
+    uint32_t icp = __ldg(&ops[0].ic_pad);
+    while (k + 1 < n_ops && r >= (uint32_t)a.B * (icp >> 7)) { r -= (uint32_t)a.B * (icp >> 7); ++k; icp = __ldg(&ops[k].ic_pad); }
+    const StepMixOp* op = ops + k;
+    touch_global(op);                                            // both 32-byte sectors of the descriptor
+    touch_global(reinterpret_cast<const uint8_t*>(op) + 32);
+    const uint64_t mu = __ldg(&op->mu);
+    const uint32_t kind = __ldg(&op->kind);
+    if (kind) {
+      const uint8_t* ox = reinterpret_cast<const uint8_t*>(a.mixx + ev.arrd.op_first + k);
+      touch_global(ox); touch_global(ox + 32); touch_global(ox + 64); touch_global(ox + 76);
+    }
+    const uint32_t ic = __ldg(&op->ic);
+    const int col = (int)(r % (icp >> 7)) * 128 + l16 * 8;
+    if (mu && col < (int)ic) {
+      const uint32_t bits = __ldg(&op->mu_bits), mask = (1u << bits) - 1u;
+      const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(mu) + (byte >> 2);
+      const uint32_t sh = (byte & 3u) * 8u;
+      const uint32_t wlo = __ldg(w);
+      const uint32_t whi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+      const uint32_t f = __funnelshift_r(wlo, whi, sh);
+      const uint32_t* cb = reinterpret_cast<const uint32_t*>(__ldg(&op->mu_aux));
+      touch_global(cb + (f & mask));
+      touch_global(cb + ((f >> bits) & mask));
+      touch_global(cb + ((f >> (2 * bits)) & mask));
+      touch_global(cb + ((f >> (3 * bits)) & mask));
+    }
+  }
+}
+
 // This CTA's share of a stage's pre-pass.  A half-warp takes one (product, batch row, 128-column
 // group) at a time: it loads x (and x_prev, and decodes mu_hat), mixes, rounds to fp16, stores the
 // 128 values to the product's pre-pass rows and reduces the three sums of the group with shuffles.
@@ -630,6 +683,9 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
   for (uint32_t ei = e0; ei < e1; ++ei) {
     const StepEvent ev = *reinterpret_cast<const StepEvent*>(reinterpret_cast<const uint8_t*>(a.events) + (size_t)ei * 64);
     if (ev.kind == EV_ARRIVE) {
+      if constexpr (MIX) {
+        if (ev.barrier < (uint32_t)a.n_stages) mix_warm<NB>(a, ev, stid);
+      }
 #pragma unroll
       for (int k = 0; k < 3; ++k) {
         float* z = reinterpret_cast<float*>(ev.arr.zptr[k]);
@@ -824,18 +880,12 @@ __device__ __forceinline__ void sq_group_words(const uint8_t* rec, int lane, uin
   }
 }
 
-// One 128-column group of the two records of a warp.  With one batch block (B <= 8) the input
-// fragments are loaded once and shared by both records; with two blocks that costs more
-// registers than a thread has, so the records are taken one after the other.
+// One 128-column group of the two records of a warp: the input fragments are loaded once and shared
+// by both records, whose tensor-core chains run interleaved.
 template <int NB, int GRP>
 __device__ __forceinline__ void sq_pair(const uint32_t (&wa)[6], const uint32_t (&wb)[6], const uint4 sza, const uint4 szb,
                                         bool has_b, const XLane& xl, float (&acca)[NB][4], float (&accb)[NB][4]) {
-  if constexpr (NB == 1) {
-    sq_group_mma2<NB, GRP>(wa, wb, sza, szb, has_b, xl, acca, accb);
-  } else {
-    sq_group_mma<NB, GRP>(wa, GRP == 0 ? sza.x : sza.y, GRP == 0 ? sza.z : sza.w, xl, acca);
-    if (has_b) sq_group_mma<NB, GRP>(wb, GRP == 0 ? szb.x : szb.y, GRP == 0 ? szb.z : szb.w, xl, accb);
-  }
+  sq_group_mma2<NB, GRP>(wa, wb, sza, szb, has_b, xl, acca, accb);
 }
 
 template <int BITS, int NB, int HALF>
