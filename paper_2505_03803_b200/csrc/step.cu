@@ -105,8 +105,9 @@ struct StepMixOp {           // 64 bytes
   uint64_t x, xprev, mu, mu_aux, dst_x, dst_sums;
   uint32_t ic, ic_pad;
   // kind: rwkvq_input_kind | 0x100 when the row is RMS-normalised | 0x200 when this token's input is stored
-  // (xprev_out) | 0x400 on the first product of a stage in which some input is normalised; any non-zero kind
-  // has a StepMixX beside it
+  // (xprev_out) | 0x400 on the first product of a stage in which some input is normalised | 0x800 on the first
+  // product of a stage whose inputs are all plain buffers; a kind with any of the low ten bits set has a
+  // StepMixX beside it
   uint16_t mu_bits, mu_entries, sums, kind;
 };
 static_assert(sizeof(StepMixOp) == 64, "pre-pass descriptor size");
@@ -538,7 +539,87 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
   __shared__ float s_part[kStagerWarps];
   __shared__ uint32_t s_row_end[kRowTable];      // first item behind the row of each entry
   int n_rows = 0;
-  if (__ldg(&ops[0].kind) & 0x400) {      // the planner marks the first product of a stage that has a normalised input
+  const uint32_t stage_kind = __ldg(&ops[0].kind);
+  if (stage_kind & 0x800) {
+    // Stage of plain inputs (no operator, no normalisation): a quarter-warp per item, sixteen columns per
+    // lane, so that a CTA's share is done in one round of loads.
+    const int l8 = lane & 7;
+    for (uint32_t g0 = lo + 4u * (uint32_t)(stid >> 5); g0 < hi; g0 += 4u * (uint32_t)kStagerWarps) {
+      const uint32_t gi = g0 + (uint32_t)(lane >> 3);
+      const bool valid = gi < hi;
+      uint32_t r = valid ? gi : lo;
+      int k = 0;
+      uint32_t icp = __ldg(&ops[0].ic_pad);
+      while (k + 1 < n_ops && r >= (uint32_t)a.B * (icp >> 7)) { r -= (uint32_t)a.B * (icp >> 7); ++k; icp = __ldg(&ops[k].ic_pad); }
+      const StepMixOp op = ops[k];
+      const uint32_t ng = op.ic_pad >> 7;
+      const int b = (int)(r / ng), grp = (int)(r % ng);
+      const int col = grp * 128 + l8 * 16;
+      const size_t e0 = (size_t)b * op.ic + col;
+      const bool in0 = col < (int)op.ic, in1 = col + 8 < (int)op.ic;
+      uint4 v[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+      uint4 pr[2] = {v[0], v[0]};
+      uint32_t f[2] = {0u, 0u};
+      const __half* xs = reinterpret_cast<const __half*>(op.x) + e0;
+      if (in0) v[0] = __ldcg(reinterpret_cast<const uint4*>(xs));
+      if (in1) v[1] = __ldcg(reinterpret_cast<const uint4*>(xs + 8));
+      if (op.mu) {
+        const __half* ps = reinterpret_cast<const __half*>(op.xprev) + e0;
+        if (in0) pr[0] = __ldcg(reinterpret_cast<const uint4*>(ps));
+        if (in1) pr[1] = __ldcg(reinterpret_cast<const uint4*>(ps + 8));
+        const uint32_t bits = op.mu_bits;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h == 0 ? in0 : in1) {
+            // four indices = 4*bits bits starting at a byte boundary (col/2 is a multiple of 4)
+            const uint32_t byte = (uint32_t)((col + 8 * h) >> 1) * bits >> 3;
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(op.mu) + (byte >> 2);
+            const uint32_t sh = (byte & 3u) * 8u;
+            const uint32_t wlo = __ldg(w);
+            const uint32_t whi = (sh + 4u * bits > 32u) ? __ldg(w + 1) : 0u;
+            f[h] = __funnelshift_r(wlo, whi, sh);
+          }
+        }
+        const uint32_t mask = (1u << bits) - 1u;
+        const uint32_t* cb = reinterpret_cast<const uint32_t*>(op.mu_aux);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h == 0 ? in0 : in1) {
+            v[h].x = mix2(v[h].x, pr[h].x, __ldg(cb + (f[h] & mask)));
+            v[h].y = mix2(v[h].y, pr[h].y, __ldg(cb + ((f[h] >> bits) & mask)));
+            v[h].z = mix2(v[h].z, pr[h].z, __ldg(cb + ((f[h] >> (2 * bits)) & mask)));
+            v[h].w = mix2(v[h].w, pr[h].w, __ldg(cb + ((f[h] >> (3 * bits)) & mask)));
+          }
+        }
+      }
+      if (valid) {
+        __half* dst = reinterpret_cast<__half*>(a.scratch + op.dst_x) + (size_t)b * op.ic_pad + col;
+        *reinterpret_cast<uint4*>(dst) = v[0];
+        *reinterpret_cast<uint4*>(dst + 8) = v[1];
+      }
+      // both vectors of a lane lie in one 16-column span of a triple: the same two bias values
+      const int o = (16 * l8) & 63;
+      const float pa = pair_sum(v[0].x) + pair_sum(v[0].z) + pair_sum(v[1].x) + pair_sum(v[1].z);
+      const float pb = pair_sum(v[0].y) + pair_sum(v[0].w) + pair_sum(v[1].y) + pair_sum(v[1].w);
+      float sx = pa + pb;
+      float t0 = fmaf((float)rwkvq_sq_bias(o, 0), pa, (float)rwkvq_sq_bias(o + 2, 0) * pb);
+      float t1 = fmaf((float)rwkvq_sq_bias(o, 1), pa, (float)rwkvq_sq_bias(o + 2, 1) * pb);
+#pragma unroll
+      for (int d = 4; d > 0; d >>= 1) {
+        sx += __shfl_xor_sync(0xFFFFFFFFu, sx, d);
+        t0 += __shfl_xor_sync(0xFFFFFFFFu, t0, d);
+        t1 += __shfl_xor_sync(0xFFFFFFFFu, t1, d);
+      }
+      if (valid && l8 == 0 && op.sums) {
+        float* gs = reinterpret_cast<float*>(a.scratch + op.dst_sums);
+        gs[(grp * 3 + 0) * nbp + b] = sx;
+        gs[(grp * 3 + 1) * nbp + b] = t0;
+        gs[(grp * 3 + 2) * nbp + b] = t1;
+      }
+    }
+    return;
+  }
+  if (stage_kind & 0x400) {      // the planner marks the first product of a stage that has a normalised input
     uint32_t r = lo;
     while (r < hi && n_rows < kRowTable) {
       uint32_t rr = r;
@@ -1458,6 +1539,9 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
       bool stage_norm = false;
       for (int o = stage_ranges[st_i].first; o < stage_ranges[st_i].second; ++o) stage_norm = stage_norm || (mixops[o].kind & 0x100);
       if (stage_norm) mixops[stage_ranges[st_i].first].kind |= 0x400;
+      bool stage_plain = true;
+      for (int o = stage_ranges[st_i].first; o < stage_ranges[st_i].second; ++o) stage_plain = stage_plain && mixops[o].kind == 0;
+      if (stage_plain) mixops[stage_ranges[st_i].first].kind |= 0x800;
       scratch_bytes = std::max(scratch_bytes, off);
     }
   }
