@@ -473,6 +473,20 @@ __device__ __forceinline__ void touch_global(const void* p) {
   asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(reinterpret_cast<uintptr_t>(p) & ~static_cast<uintptr_t>(3)));
 }
 
+// Asks for the line to be brought into L2 (the point of coherence: a later write by another CTA, reduction
+// or plain store, is seen by the load that follows).
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" :: "l"(p));
+}
+
+// A pre-pass descriptor through the read-only path, so that the copy read ahead by mix_warm is found in L1.
+__device__ __forceinline__ StepMixOp load_mixop(const StepMixOp* p) {
+  union { StepMixOp op; uint4 q[4]; } u;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) u.q[i] = __ldg(reinterpret_cast<const uint4*>(p) + i);
+  return u.op;
+}
+
 // Everything mix_slice will read that does not depend on the stage before -- the products' descriptors,
 // the mu_hat codes of this CTA's items and the codebook entries they select -- is read once ahead of
 // time, while the consumer warps are still busy with the current stage, so that behind the barrier the
@@ -502,7 +516,15 @@ __device__ void mix_warm(const StepArgs& a, const StepEvent& ev, int stid) {
       touch_global(ox); touch_global(ox + 32); touch_global(ox + 64); touch_global(ox + 76);
     }
     const uint32_t ic = __ldg(&op->ic);
-    const int col = (int)(r % (icp >> 7)) * 128 + l16 * 8;
+    const uint32_t ng = icp >> 7;
+    const int col = (int)(r % ng) * 128 + l16 * 8;
+    // Inputs that no earlier stage of this step writes (the first products' x, every x_prev) are still in
+    // HBM: ask for them now.  Inputs an earlier stage writes are in L2 already and the request is void.
+    if ((kind & 0xFFu) == RWKVQ_IN_BUFFER && col < (int)ic && (l16 & 1) == 0) {
+      const size_t e0 = (size_t)(r / ng) * ic + col;
+      prefetch_l2(reinterpret_cast<const __half*>(__ldg(&op->x)) + e0);
+      if (mu) prefetch_l2(reinterpret_cast<const __half*>(__ldg(&op->xprev)) + e0);
+    }
     if (mu && col < (int)ic) {
       const uint32_t bits = __ldg(&op->mu_bits), mask = (1u << bits) - 1u;
       const uint32_t byte = (uint32_t)(col >> 1) * bits >> 3;
@@ -551,7 +573,7 @@ __device__ void mix_slice(const StepArgs& a, const StepEvent& ev, int stid) {
       int k = 0;
       uint32_t icp = __ldg(&ops[0].ic_pad);
       while (k + 1 < n_ops && r >= (uint32_t)a.B * (icp >> 7)) { r -= (uint32_t)a.B * (icp >> 7); ++k; icp = __ldg(&ops[k].ic_pad); }
-      const StepMixOp op = ops[k];
+      const StepMixOp op = load_mixop(ops + k);
       const uint32_t ng = op.ic_pad >> 7;
       const int b = (int)(r / ng), grp = (int)(r % ng);
       const int col = grp * 128 + l8 * 16;
