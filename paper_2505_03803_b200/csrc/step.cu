@@ -1002,6 +1002,24 @@ __device__ __forceinline__ void vq_pair(const uint32_t (&wa)[2 * BITS], const ui
   }
 }
 
+// c[k] of the four lanes whose row index g differs in its two low bits (lanes 4 apart) -> lane i (= g & 3)
+// ends with element i of lanes g & ~3 ... (g & ~3) + 3, in that order.  All lanes of the warp call it.
+__device__ __forceinline__ void transpose4_lanes(float (&c)[4], int i) {
+  const bool hi = (i & 2) != 0, lo = (i & 1) != 0;
+  const float s0 = hi ? c[0] : c[2], s1 = hi ? c[1] : c[3];
+  const float r0 = __shfl_xor_sync(0xFFFFFFFFu, s0, 8), r1 = __shfl_xor_sync(0xFFFFFFFFu, s1, 8);
+  // element 2*hi + {0, 1} of source lanes j1 = 0, 1
+  const float a00 = hi ? r0 : c[0], a01 = hi ? r1 : c[1];
+  const float a10 = hi ? c[2] : r0, a11 = hi ? c[3] : r1;
+  const float q0 = lo ? a00 : a01, q1 = lo ? a10 : a11;
+  const float p0 = __shfl_xor_sync(0xFFFFFFFFu, q0, 4), p1 = __shfl_xor_sync(0xFFFFFFFFu, q1, 4);
+  c[0] = lo ? p0 : a00;  c[1] = lo ? a01 : p0;
+  c[2] = lo ? p1 : a10;  c[3] = lo ? a11 : p1;
+}
+__device__ __forceinline__ void red_add_v4(float* p, const float (&v)[4]) {
+  asm volatile("red.global.v4.f32.add [%0], {%1, %2, %3, %4};" :: "l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+}
+
 // Consumer warp `w` of group `grp`: units grp, grp + 2, ... of the CTA's list.
 template <int NB, bool MIX>
 __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, const uint8_t* xbufs, uint8_t* replicas,
@@ -1117,6 +1135,28 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
       const uint32_t col = u->xcol0;
       const XLane xl = make_xlane(xb + (size_t)col * 2, xstride,
                                   reinterpret_cast<const float*>(xb + u->gs_off) + (size_t)(col >> 7) * 3 * nbp, nbp, a.B, lane);
+      if constexpr (NB == 2) {
+        // Registers suffice for the whole record pair: take all of it, free the slot, then run both
+        // 128-column groups as one stretch of code (eight tensor-core chains for the scheduler to interleave).
+        uint32_t wa0[6], wb0[6], wa1[6], wb1[6];
+        uint4 sza = make_uint4(0, 0, 0, 0), szb = sza;
+        if (active) {
+          sq_group_words<0>(ra, lane, wa0);
+          sq_group_words<1>(ra, lane, wa1);
+          sza = *reinterpret_cast<const uint4*>(ra + RWKVQ_SQ_CODE_BYTES + g * 16);
+          if (has_b) {
+            sq_group_words<0>(rbp, lane, wb0);
+            sq_group_words<1>(rbp, lane, wb1);
+            szb = *reinterpret_cast<const uint4*>(rbp + RWKVQ_SQ_CODE_BYTES + g * 16);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->empty[slot]);
+        if (active) {
+          sq_pair<NB, 0>(wa0, wb0, sza, szb, has_b, xl, acca, accb);
+          sq_pair<NB, 1>(wa1, wb1, sza, szb, has_b, xl, acca, accb);
+        }
+      } else {
       uint32_t wa[6], wb[6];
       uint4 sza = make_uint4(0, 0, 0, 0), szb = sza;
       if (active) {
@@ -1133,6 +1173,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctrl->empty[slot]);     // the rest of the records is in registers: free the slot
       if (active) sq_pair<NB, 1>(wa, wb, sza, szb, has_b, xl, acca, accb);
+      }
     } else {
       // replicate the tile's codebook for conflict-free lookups (the eight warps of the group)
       const uint32_t E = u->entries;
@@ -1169,6 +1210,25 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
     }
     if (flags & UF_FLUSH) {
       if (active) {
+        if ((oc & 3u) == 0u && (reinterpret_cast<uintptr_t>(y) & 15u) == 0u) {
+          // Four lanes that share t hold a 4 x 4 block (rows 4J .. 4J+3 of one row half x the accumulator's four
+          // elements): transposed, every lane owns four consecutive rows of ONE batch column and adds them
+          // with a single 16-byte reduction instead of four scattered ones.
+          const int i = g & 3;
+          const uint32_t rbase = row0 + (uint32_t)w * 16u + 8u * (uint32_t)(i >> 1) + (uint32_t)(g & ~3);
+#pragma unroll
+          for (int n = 0; n < NB; ++n) {
+            const int b = n * 8 + 2 * t + (i & 1);
+            float va[4] = {acca[n][0], acca[n][1], acca[n][2], acca[n][3]};
+            transpose4_lanes(va, i);
+            if (b < a.B && rbase < oc) red_add_v4(y + (size_t)b * oc + rbase, va);
+            if (has_b) {                      // warp-uniform
+              float vb[4] = {accb[n][0], accb[n][1], accb[n][2], accb[n][3]};
+              transpose4_lanes(vb, i);
+              if (b < a.B && rbase + 128u < oc) red_add_v4(y + (size_t)b * oc + rbase + 128u, vb);
+            }
+          }
+        } else {
 #pragma unroll
         for (int n = 0; n < NB; ++n)
 #pragma unroll
@@ -1178,6 +1238,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
             if (b < a.B && row < oc) atomicAdd(y + (size_t)b * oc + row, acca[n][k]);
             if (b < a.B && has_b && row + 128u < oc) atomicAdd(y + (size_t)b * oc + row + 128u, accb[n][k]);
           }
+        }
       }
 #pragma unroll
       for (int n = 0; n < NB; ++n)
