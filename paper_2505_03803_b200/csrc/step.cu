@@ -8,16 +8,17 @@
 //   * a producer warp streams packed weights from HBM into a ring of shared-memory slots with
 //     bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts).  Weights never depend
 //     on activations, so the stream runs ahead across products and across stage boundaries;
-//   * three stager warps build the fp16 input x_mix = x + (x_prev - x) (.) mu_hat (Appendix A.1
+//   * the stager warps (three, or seven for batches above 8: Shape) build the fp16 input x_mix = x + (x_prev - x) (.) mu_hat (Appendix A.1
 //     Eq. 20) of the next run of units in one of two shared-memory buffers.  What does not depend
 //     on the previous stage (mu_hat, x_prev) is prepared before the grid-wide stage barrier; the
 //     stagers also clear the next stage's outputs and post this CTA's arrival at the barrier;
-//   * sixteen consumer warps in two groups of eight.  A unit is a 256-row x 256-column tile (two
-//     128-row chunks of the packed image); the groups take the CTA's units alternately, so one
-//     group computes while the other waits, flushes or synchronises.  Warp w of a group owns rows
+//   * consumer warps in groups of eight (two groups; one for batches above 8, whose record routine
+//     needs the registers of two).  A unit is a 256-row x 256-column tile (two 128-row chunks of the
+//     packed image); the groups take the CTA's units alternately, so one group computes while the
+//     other waits, flushes or synchronises.  Warp w of a group owns rows
 //     16w..16w+15 of both chunks and runs the m16n8k16 tensor-core steps of gemv_core.cuh with
-//     every input fragment shared by the two records.  Partial sums go to y with fp32 atomics at
-//     the end of a run along K.
+//     every input fragment shared by the two records.  Partial sums go to y with fp32 reductions
+//     (16 bytes per lane after a transpose among lanes) at the end of a run along K.
 //
 // For batches of four and more, and whenever a product's input is an element-wise operator on
 // earlier outputs (rwkvq_input_xform: the WKV recurrence and sigmoid gate of Appendix A.1 Eqs. 23-24,
@@ -255,8 +256,8 @@ __device__ __forceinline__ uint32_t smem_add_acq_rel(uint32_t* p, uint32_t v) {
 struct Ctrl {
   uint64_t full[kMaxSlots], empty[kMaxSlots];
   uint64_t xfull[4], xempty[4];
-  uint32_t stage_cnt[64];    // one 8-bit count per grid barrier (four per word): how many of the seventeen
-                             // parties of this CTA (sixteen consumer warps, the stagers) have reported the
+  uint32_t stage_cnt[64];    // one 8-bit count per grid barrier (four per word): how many of the parties
+                             // of this CTA (every consumer warp, and the stagers as one) have reported the
                              // stage that the barrier closes.  Per barrier, not one running total: consumer
                              // warps of a CTA without work in the coming stages may run any number of
                              // stages ahead of the stagers.
@@ -266,7 +267,7 @@ struct Ctrl {
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block");
 constexpr uint32_t kMaxBarriers = 256;   // barriers that close a stage (8-bit counts in Ctrl::stage_cnt)
 
-// One of the seventeen parties of grid barrier `b` reports that its part of the stage the barrier
+// One of the parties of grid barrier `b` (each consumer warp, the stagers as one) reports that its part of the stage the barrier
 // closes is done; whoever reports last posts the CTA's arrival.  The count is an acquire-release
 // read-modify-write at CTA scope and the arrival a GPU-scope release, so the arrival is ordered
 // after everything every party did before reporting (the consumers' reductions into y, the
@@ -280,10 +281,10 @@ __device__ __forceinline__ void stage_report(Ctrl* ctrl, const StepArgs& a, uint
 }
 // Where the consumer warps are the busy role (two batch blocks per record) they only count
 // themselves in, and a stager thread, which has nothing else to do at that point, waits (bounded)
-// for the sixteen reports of THIS barrier and arrives: the release, which waits for the CTA's
+// for the consumer warps' reports of THIS barrier and arrives: the release, which waits for the CTA's
 // outstanding reductions, stays off the consumer warps.  The count is per barrier (the 8-bit
 // fields of stage_cnt): a warp without work in the next stages runs ahead through their events,
-// so a running total over all stages would reach sixteen times the stage number while warps of
+// so a running total over all stages would reach its value for this stage while warps of
 // this stage are still adding to the outputs.
 __device__ __forceinline__ void stage_report_total(Ctrl* ctrl, uint32_t b) {
   asm volatile("red.release.cta.shared::cta.add.u32 [%0], %1;" ::"r"(smem_u32(&ctrl->stage_cnt[b >> 2])), "r"(1u << (8u * (b & 3u))) : "memory");
@@ -798,7 +799,7 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
       ok = named_bar_and(4, kStagerThreads, ok);
       if (!ok) break;
       // The stagers' part of the stage is done.  Barrier 0 (the clearing pass) has no consumer work
-      // before it: arrive directly.  Otherwise report; the last of the seventeen parties arrives.
+      // before it: arrive directly.  Otherwise report; the last party to report arrives.
       if (stid == 0) {
         if (ev.barrier == 0u) red_release_gpu(a.counter, 1u);
         else if constexpr (NB == 2) ok = stage_wait_total_and_arrive<NB>(ctrl, a, ev.barrier, abortp);
@@ -994,12 +995,7 @@ __device__ __forceinline__ void sq_pair(const uint32_t (&wa)[6], const uint32_t 
 template <int BITS, int NB, int HALF>
 __device__ __forceinline__ void vq_pair(const uint32_t (&wa)[2 * BITS], const uint32_t (&wb)[2 * BITS], const uint32_t* cb_lane,
                                         const XLane& xl, float (&acca)[NB][4], float (&accb)[NB][4]) {
-  if constexpr (NB == 1) {
-    vq_half_mma2<BITS, NB, HALF>(wa, wb, cb_lane, xl, acca, accb);
-  } else {
-    vq_record_mma<BITS, NB, 8 * HALF, 8 * HALF + 8>(wa, cb_lane, xl, acca);
-    vq_record_mma<BITS, NB, 8 * HALF, 8 * HALF + 8>(wb, cb_lane, xl, accb);
-  }
+  vq_half_mma2<BITS, NB, HALF>(wa, wb, cb_lane, xl, acca, accb);
 }
 
 // c[k] of the four lanes whose row index g differs in its two low bits (lanes 4 apart) -> lane i (= g & 3)
@@ -1037,7 +1033,7 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
     for (int k = 0; k < 4; ++k) acca[n][k] = accb[n][k] = 0.f;
   // Every consumer warp walks the CTA's event list in order -- it reports each stage it leaves and
   // passes through each input segment, used or not -- so that the phases of the shared barriers
-  // advance in step for all sixteen warps.
+  // advance in step for all consumer warps.
   int held = -1;              // input segment this warp currently holds
   uint32_t seg_next = 0;      // number of segment events passed so far
   uint32_t cur_ev = 0;        // last event processed (event 0 is the clearing arrival: nothing to do)
@@ -1484,7 +1480,11 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
     // get a stage's VQ matrix do not finish last.
     auto cost_of = [&](const HostUnit& h) -> uint64_t {
       const uint64_t recs = (h.u.bytes0 + h.u.bytes1) / h.u.rec_bytes;
-      const uint64_t wgt = !(h.u.flags & UF_VQ) ? 20u : (h.u.flags & UF_BITS8) ? 25u : 29u;
+      // in twentieths of an SQ record; the table lookups weigh more the more batch columns a record meets
+      // (whole-step times of all-SQ against all-VQ-64 stacks less the per-stage chain: 1.4 at B = 1,
+      // 1.6 at B = 8, 2.0 at B = 16)
+      const uint64_t vq6 = B > 8 ? 40u : B >= 4 ? 32u : 29u, vq8 = B > 8 ? 34u : B >= 4 ? 28u : 25u;
+      const uint64_t wgt = !(h.u.flags & UF_VQ) ? 20u : (h.u.flags & UF_BITS8) ? vq8 : vq6;
       return recs * wgt * 64u;
     };
     // A consumer group spends about the same time on a piece of a unit as on a whole unit (the
