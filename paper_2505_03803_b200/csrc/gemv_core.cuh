@@ -239,11 +239,16 @@ template <int NB, int GRP>
 __device__ __forceinline__ void sq_group_mma2(const uint32_t (&wa)[6], const uint32_t (&wb)[6], const uint4 sza,
                                               const uint4 szb, bool has_b, const XLane& xl, float (&acca)[NB][4],
                                               float (&accb)[NB][4]) {
+  // The tensor-core chains start at -Bx_h, the bias the extracted halves carry, instead of at zero:
+  // what they end with is sum(q x) of the group.
+  const uint8_t* gsp = xl.gs + (size_t)(GRP * 3) * xl.gstride;
   float ca[NB][4], cb[NB][4];
 #pragma unroll
   for (int n = 0; n < NB; ++n) {
-    ca[n][0] = ca[n][1] = ca[n][2] = ca[n][3] = 0.f;
-    cb[n][0] = cb[n][1] = cb[n][2] = cb[n][3] = 0.f;
+    const float2 b0 = *reinterpret_cast<const float2*>(gsp + xl.gstride + n * 32);
+    const float2 b1 = *reinterpret_cast<const float2*>(gsp + 2 * xl.gstride + n * 32);
+    ca[n][0] = cb[n][0] = -b0.x; ca[n][1] = cb[n][1] = -b0.y;
+    ca[n][2] = cb[n][2] = -b1.x; ca[n][3] = cb[n][3] = -b1.y;
   }
 #pragma unroll
   for (int ti = 0; ti < 2; ++ti) {
@@ -279,20 +284,17 @@ __device__ __forceinline__ void sq_group_mma2(const uint32_t (&wa)[6], const uin
   const float2 sa1 = __half22float2(*reinterpret_cast<const __half2*>(&a_hi));
   const float2 sb0 = __half22float2(*reinterpret_cast<const __half2*>(&b_lo));
   const float2 sb1 = __half22float2(*reinterpret_cast<const __half2*>(&b_hi));
-  const uint8_t* gsp = xl.gs + (size_t)(GRP * 3) * xl.gstride;
 #pragma unroll
   for (int n = 0; n < NB; ++n) {
     const float2 sx = *reinterpret_cast<const float2*>(gsp + n * 32);
-    const float2 b0 = *reinterpret_cast<const float2*>(gsp + xl.gstride + n * 32);
-    const float2 b1 = *reinterpret_cast<const float2*>(gsp + 2 * xl.gstride + n * 32);
-    acca[n][0] = fmaf(sa0.x, fmaf(-sa0.y, sx.x, ca[n][0] - b0.x), acca[n][0]);
-    acca[n][1] = fmaf(sa0.x, fmaf(-sa0.y, sx.y, ca[n][1] - b0.y), acca[n][1]);
-    acca[n][2] = fmaf(sa1.x, fmaf(-sa1.y, sx.x, ca[n][2] - b1.x), acca[n][2]);
-    acca[n][3] = fmaf(sa1.x, fmaf(-sa1.y, sx.y, ca[n][3] - b1.y), acca[n][3]);
-    accb[n][0] = fmaf(sb0.x, fmaf(-sb0.y, sx.x, cb[n][0] - b0.x), accb[n][0]);
-    accb[n][1] = fmaf(sb0.x, fmaf(-sb0.y, sx.y, cb[n][1] - b0.y), accb[n][1]);
-    accb[n][2] = fmaf(sb1.x, fmaf(-sb1.y, sx.x, cb[n][2] - b1.x), accb[n][2]);
-    accb[n][3] = fmaf(sb1.x, fmaf(-sb1.y, sx.y, cb[n][3] - b1.y), accb[n][3]);
+    acca[n][0] = fmaf(sa0.x, fmaf(-sa0.y, sx.x, ca[n][0]), acca[n][0]);
+    acca[n][1] = fmaf(sa0.x, fmaf(-sa0.y, sx.y, ca[n][1]), acca[n][1]);
+    acca[n][2] = fmaf(sa1.x, fmaf(-sa1.y, sx.x, ca[n][2]), acca[n][2]);
+    acca[n][3] = fmaf(sa1.x, fmaf(-sa1.y, sx.y, ca[n][3]), acca[n][3]);
+    accb[n][0] = fmaf(sb0.x, fmaf(-sb0.y, sx.x, cb[n][0]), accb[n][0]);
+    accb[n][1] = fmaf(sb0.x, fmaf(-sb0.y, sx.y, cb[n][1]), accb[n][1]);
+    accb[n][2] = fmaf(sb1.x, fmaf(-sb1.y, sx.x, cb[n][2]), accb[n][2]);
+    accb[n][3] = fmaf(sb1.x, fmaf(-sb1.y, sx.y, cb[n][3]), accb[n][3]);
   }
 }
 
