@@ -1206,10 +1206,11 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
     }
     if (flags & UF_FLUSH) {
       if (active) {
-        if ((oc & 3u) == 0u && (reinterpret_cast<uintptr_t>(y) & 15u) == 0u) {
+        {
           // Four lanes that share t hold a 4 x 4 block (rows 4J .. 4J+3 of one row half x the accumulator's four
           // elements): transposed, every lane owns four consecutive rows of ONE batch column and adds them
-          // with a single 16-byte reduction instead of four scattered ones.
+          // with a single 16-byte reduction instead of four scattered ones.  The plan accepts only outputs
+          // that start on a 16-byte boundary, and the format only row counts that are multiples of 16.
           const int i = g & 3;
           const uint32_t rbase = row0 + (uint32_t)w * 16u + 8u * (uint32_t)(i >> 1) + (uint32_t)(g & ~3);
 #pragma unroll
@@ -1223,16 +1224,6 @@ __device__ void consumer_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, cons
               transpose4_lanes(vb, i);
               if (b < a.B && rbase + 128u < oc) red_add_v4(y + (size_t)b * oc + rbase + 128u, vb);
             }
-          }
-        } else {
-#pragma unroll
-        for (int n = 0; n < NB; ++n)
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint32_t row = row0 + (uint32_t)w * 16u + (uint32_t)g + 8u * (uint32_t)(k >> 1);
-            const int b = n * 8 + 2 * t + (k & 1);
-            if (b < a.B && row < oc) atomicAdd(y + (size_t)b * oc + row, acca[n][k]);
-            if (b < a.B && has_b && row + 128u < oc) atomicAdd(y + (size_t)b * oc + row + 128u, accb[n][k]);
           }
         }
       }

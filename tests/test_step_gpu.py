@@ -179,3 +179,33 @@ def test_bounded_waits_run_out_and_the_plan_recovers():
             torch.cuda.synchronize()
             assert B.rwkvq_device_status() == 0
             _check(ops, Bn)
+
+
+@pytest.mark.parametrize("Bn", [1, 8, 16])
+def test_step_output_rows_end_inside_a_unit(Bn):
+    """Row counts that end inside a 256-row unit (272 = one unit and one record) and inside a 128-row chunk
+    (144): the 16-byte reductions of the flush stop at the last row; nothing beyond the outputs is written.
+    An output that does not start on a 16-byte boundary is refused by the plan."""
+    ops = []
+    for k, (oc, ic) in enumerate([(272, 384), (144, 640), (256, 512), (272, 384)]):
+        W = H.pack_sq(H.random_sq_codes(900 + 10 * Bn + k, oc, ic)) if k != 2 else H.pack_vq(H.random_vq_codes(900 + 10 * Bn + k, oc, ic, 6), 6)
+        mu = H.pack_mu(H.random_mu_codes(950 + 10 * Bn + k, ic, 6), 6) if k % 2 == 0 else None
+        x, xp = inputs.gen_activation_pair(990 + 10 * Bn + k, Bn, ic, n_outliers=4)
+        x16, xp16 = x.astype(np.float16), xp.astype(np.float16)
+        buf = torch.full((Bn * oc + 8,), float("nan"), dtype=torch.float32, device="cuda")
+        y = buf[4:4 + Bn * oc].view(Bn, oc)
+        ops.append(dict(W=W, mu=mu, x16=x16, xp16=xp16, stage=k // 2, xd=torch.from_numpy(x16).cuda(),
+                        xpd=torch.from_numpy(xp16).cuda() if mu is not None else None, y=y, buf=buf))
+    plan = _plan(ops, Bn)
+    for _ in range(2):
+        B.rwkvq_step_run(plan)
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        _check(ops, Bn)
+    for e in ops:      # nothing outside the outputs was touched
+        assert torch.isnan(e["buf"][:4]).all() and torch.isnan(e["buf"][4 + e["y"].numel():]).all()
+    e = ops[0]
+    bad = e["buf"][1:1 + Bn * e["W"].oc].view(Bn, e["W"].oc)
+    arr = B.make_ops([dict(desc=e["W"].desc, W=e["W"].dev, mu_desc=e["mu"].desc, mu=e["mu"].dev, x=e["xd"], xprev=e["xpd"],
+                           y=bad, stage=0)])
+    assert B.rwkvq_step_plan_bytes(arr, Bn) == 0
