@@ -330,11 +330,19 @@ rwkvq_status rwkvq_step_set_wait(const void* plan_dev, uint32_t poll_limit, uint
 rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, int n_ctas,
                                    uint32_t* counts_host, size_t n_counts, uint32_t* cta_items_host);
 /*
- * The same step for callers whose activations live in host memory: copies act_bytes from act_host
- * to act_dev (the device buffer the plan's x / x_prev pointers lie in), runs the step, and copies
- * y_bytes from y_dev (the buffer the plan's outputs lie in) to y_host, all asynchronously on
- * `stream` in that order; the caller synchronizes the stream before reading y_host.  Host buffers
- * should be page-locked, otherwise the copies serialize with the host.  A size of 0 skips that copy.
+ * The same step for callers whose activations live in host memory: act_bytes are copied from act_host
+ * to act_dev (the device buffer the plan's x / x_prev pointers lie in), the step runs, and y_bytes are
+ * copied from y_dev (the buffer the plan's outputs lie in) to y_host.  Everything is ordered behind what
+ * `stream` already holds, and `stream` ends behind all of it: the caller synchronizes `stream` before
+ * reading y_host or changing act_host.  Small steps (less than 16 MB of copies) run the three parts one
+ * after the other on `stream`.  Larger ones overlap them: the activations are copied in chunks of 4 MB
+ * on a stream of the library's own while the step is already running (its input stages wait, bounded,
+ * for the chunk that holds what they are about to read), and the outputs are copied, on another stream,
+ * stage by stage as soon as the stage barrier that completes them has been passed, provided the stages'
+ * outputs lie one behind the other inside [y_dev, y_dev + y_bytes) (otherwise in one piece at the end).
+ * The bytes that reach y_host are those of the plain order.  Host buffers should be page-locked,
+ * otherwise the copies serialize with the host.  A size of 0 skips that copy.  Calls on different
+ * streams of one device are serialized by the library.  Errors: as rwkvq_step_run, ECUDA.
  */
 rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const void* act_host,
                                  void* act_dev, size_t act_bytes, const void* y_dev, void* y_host,

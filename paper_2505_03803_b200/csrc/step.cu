@@ -32,6 +32,7 @@
 // their cost midpoints, small stages in eighths of a unit (one warp's records); the plan is a per-CTA
 // list of 128-byte unit descriptors plus a list of 64-byte input events (segments and barrier
 // arrivals).
+#include <cuda.h>           // types of the stream memory operations (no driver symbol is linked)
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -172,6 +173,13 @@ struct StepArgs {
   const StepMixOp* mixops;    // dst_x / dst_sums are offsets into `scratch`
   const StepMixX* mixx;       // parallel to mixops
   uint8_t* scratch;
+  // Host-buffer runs (rwkvq_step_run_host): the activations arrive in chunks of 2^in_shift bytes while
+  // the step is already running; after chunk i the copy stream stores in_base + i + 1 in *in_flag.
+  // Whoever reads inputs inside [in_lo, in_hi) first waits for the chunk that holds their last byte.
+  // in_flag == nullptr: the inputs are resident.
+  const unsigned* in_flag;
+  unsigned in_base, in_shift;
+  uint64_t in_lo, in_hi;
 };
 
 // ---- mbarrier / bulk-copy wrappers ------------------------------------------------------------
@@ -239,6 +247,11 @@ __device__ __forceinline__ void bulk_g2s_plain(void* dst_smem, const void* src, 
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+__device__ __forceinline__ unsigned ld_acquire_sys(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -297,6 +310,21 @@ __device__ __forceinline__ bool stage_wait_total_and_arrive(Ctrl* ctrl, const St
     uint32_t v;
     asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&ctrl->stage_cnt[b >> 2])) : "memory");
     if (((v >> sh) & 0xFFu) >= (uint32_t)Shape<NB>::kConsumerWarps) { red_release_gpu(a.counter + b, 1u); return true; }
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicExch(a.status, (int)RWKVQ_ETIMEOUT);
+  return false;
+}
+
+// One thread: wait (bounded) until the chunk that holds byte `last` (the address of the last input byte
+// about to be read) has arrived.  Addresses outside the arriving range are resident already.
+__device__ __forceinline__ bool wait_inputs(const StepArgs& a, uint64_t last, volatile int* abort_flag) {
+  if (!a.in_flag || last < a.in_lo || last >= a.in_hi) return true;
+  const unsigned need = a.in_base + (unsigned)((last - a.in_lo) >> a.in_shift) + 1u;
+  const uint32_t limit = a.poll_limit << 2;
+  for (uint32_t it = 0; it < limit; ++it) {
+    if ((int)(ld_acquire_sys(a.in_flag) - need) >= 0) return true;
     if ((it & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -814,6 +842,18 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
             while ((int)(ld_acquire_gpu(a.counter + ev.barrier) - (a.target + a.wait_skew)) < 0) {
               if (++it >= (a.poll_limit << 2) || *abortp) { *abortp = 1; atomicExch(a.status, (int)RWKVQ_ETIMEOUT); ok = false; break; }
             }
+            if (ok && a.in_flag) {
+              // the last input byte any product of the coming stage reads (x and x_prev, [B][ic] fp16 each)
+              const StepMixOp* mo = a.mixops + ev.arrd.op_first;
+              uint64_t last = 0;
+              for (uint32_t k = 0; k < ev.arrd.op_count; ++k) {
+                const uint64_t span = (uint64_t)a.B * __ldg(&mo[k].ic) * 2u - 1u;
+                const uint64_t px = __ldg(&mo[k].x), pp = __ldg(&mo[k].xprev);
+                if (px >= a.in_lo && px < a.in_hi) last = max(last, px + span);
+                if (pp >= a.in_lo && pp < a.in_hi) last = max(last, pp + span);
+              }
+              if (last) ok = wait_inputs(a, last, abortp);
+            }
           }
           ok = named_bar_and(6, kStagerThreads, ok);   // thread 0's acquire precedes every thread's loads of x
           if (!ok) break;
@@ -869,6 +909,14 @@ __device__ void stager_role(const StepArgs& a, uint8_t* smem, Ctrl* ctrl, uint8_
     const int total = a.B * nvr;
     const int nbp = (a.B + 1) & ~1;
     uint8_t* murow = xb + (size_t)ev.mu_off16 * 16;
+    if (a.in_flag) {      // uniform: host-buffer run
+      if (ok && stid == 0) {
+        const uint64_t span = ((uint64_t)(a.B - 1) * (uint64_t)ic + (uint64_t)min(ic, col0 + (int)ev.segd.ncols)) * 2u - 1u;
+        ok = wait_inputs(a, (uint64_t)(uintptr_t)x + span, abortp);
+        if (ok && mu) ok = wait_inputs(a, (uint64_t)(uintptr_t)xp + span, abortp);
+      }
+      ok = named_bar_and(5, kStagerThreads, ok);
+    }
     if (ok && mu) {
       for (int e = stid; e < (int)ev.segd.mu_entries; e += kStagerThreads) mucb[e] = __ldg(reinterpret_cast<const uint32_t*>(ev.seg.mu_aux) + e);
       named_bar_sync(5, kStagerThreads);
@@ -1288,6 +1336,7 @@ struct PlanInfo {
   uint32_t slot_bytes, replica_bytes, smem_bytes;
   size_t off_unit_off, off_event_off, off_units, off_events, off_counter, off_mixops, off_mixx, off_scratch, total_bytes;
   uint32_t n_units, n_events, n_barriers;
+  std::vector<uint64_t> y_lo, y_hi;   // per stage: device address range its products write (host-buffer runs)
 };
 
 static std::mutex g_plan_mutex;
@@ -1776,12 +1825,40 @@ rwkvq_status rwkvq_step_plan(const rwkvq_gemv_op* ops, int n_ops, int B, void* p
   if (e != cudaSuccess) return cuda_status(e);
   info.runs = 0;
   info.abort_epoch = abort_epoch();   // the image just copied holds zeroed counters
+  for (int i = 0; i < n_ops; ++i) {
+    if (i == 0 || ops[i].stage != ops[i - 1].stage) { info.y_lo.push_back(~0ull); info.y_hi.push_back(0ull); }
+    const uint64_t lo = (uint64_t)(uintptr_t)ops[i].y_dev, hi = lo + (uint64_t)B * (uint64_t)ops[i].W_desc.oc * 4u;
+    info.y_lo.back() = std::min(info.y_lo.back(), lo);
+    info.y_hi.back() = std::max(info.y_hi.back(), hi);
+  }
   std::lock_guard<std::mutex> lock(g_plan_mutex);
   g_plans[plan_dev] = info;
   return RWKVQ_OK;
 }
 
-rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+// Inputs that arrive while the step runs (see StepArgs::in_flag), and what the caller needs back to
+// order its output copies behind the stage barriers.
+struct HostRun {
+  const unsigned* in_flag = nullptr;
+  unsigned in_base = 0, in_shift = 0;
+  uint64_t in_lo = 0, in_hi = 0;
+  // out
+  unsigned* counter = nullptr;
+  unsigned target = 0;
+  PlanInfo info;
+};
+
+// Every arrival counter that is short of `target` (a run that gave up) is raised to it, so that
+// nothing ordered behind a counter waits for ever and the next run starts from a consistent state.
+__global__ void step_finish_kernel(unsigned* counter, int n, unsigned target) {
+  const int k = (int)(blockIdx.x * blockDim.x + threadIdx.x);
+  if (k < n && (int)(counter[k] - target) < 0) counter[k] = target;
+}
+
+rwkvq_status step_run_impl(const void* plan_dev, size_t plan_bytes, void* stream, HostRun* hr) {
   if (!plan_dev) return RWKVQ_EINVAL;
   PlanInfo info;
   bool clear_counters = false;
@@ -1814,6 +1891,11 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   a.target = info.runs * (unsigned)info.P;
   a.poll_limit = info.poll_limit; a.wait_skew = info.wait_skew;
+  a.in_flag = nullptr; a.in_base = 0; a.in_shift = 0; a.in_lo = 0; a.in_hi = 0;
+  if (hr) {
+    a.in_flag = hr->in_flag; a.in_base = hr->in_base; a.in_shift = hr->in_shift; a.in_lo = hr->in_lo; a.in_hi = hr->in_hi;
+    hr->counter = a.counter; hr->target = a.target; hr->info = info;
+  }
   cudaError_t e = cudaSuccess;
   if (clear_counters) {
     e = cudaMemsetAsync(a.counter, 0, round_up_sz((size_t)info.n_barriers * 4, 256), s);
@@ -1831,7 +1913,18 @@ rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* strea
     auto it = g_plans.find(plan_dev);
     if (it != g_plans.end()) it->second.abort_epoch = abort_epoch() - 1u;
   }
+  if (e == cudaSuccess && hr) {
+    step_finish_kernel<<<(info.n_barriers + 255u) / 256u, 256, 0, s>>>(a.counter, (int)info.n_barriers, a.target);
+    e = cudaGetLastError();
+  }
   return cuda_status(e);
+}
+}  // namespace
+
+extern "C" {
+
+rwkvq_status rwkvq_step_run(const void* plan_dev, size_t plan_bytes, void* stream) {
+  return step_run_impl(plan_dev, plan_bytes, stream, nullptr);
 }
 
 rwkvq_status rwkvq_step_plan_release(const void* plan_dev) {
@@ -1901,9 +1994,54 @@ rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, i
   return RWKVQ_OK;
 }
 
-rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const void* act_host, void* act_dev,
-                                 size_t act_bytes, const void* y_dev, void* y_host, size_t y_bytes, void* stream) {
-  if ((act_bytes && (!act_host || !act_dev)) || (y_bytes && (!y_dev || !y_host))) return RWKVQ_EINVAL;
+}  // extern "C"
+
+namespace {
+// Streams, events and the arrival word of host-buffer runs, one set per device.  The stream memory
+// operations come from the driver through the runtime's entry-point query (no link to the driver library).
+typedef CUresult (*StreamValueFn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+struct HostPipe {
+  bool tried = false, ok = false;
+  cudaStream_t h2d = nullptr, d2h = nullptr;
+  cudaEvent_t start = nullptr, h2d_done = nullptr, d2h_done = nullptr;
+  unsigned* flag = nullptr;      // device word: chunks arrived so far, over all runs
+  unsigned chunks = 0;           // the host's copy of its final value after the last run enqueued
+  StreamValueFn wait_value = nullptr, write_value = nullptr;
+};
+std::mutex g_pipe_mutex;
+std::unordered_map<int, HostPipe> g_pipes;
+constexpr unsigned kChunkShift = 22;                 // activations arrive in chunks of 4 MB
+constexpr size_t kOutGroupBytes = (size_t)2 << 20;   // outputs leave in groups of whole stages of at least 2 MB
+
+HostPipe* host_pipe() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  HostPipe& hp = g_pipes[dev];
+  if (hp.tried) return hp.ok ? &hp : nullptr;
+  hp.tried = true;
+  cudaDriverEntryPointQueryResult q1, q2;
+  void *f1 = nullptr, *f2 = nullptr;
+  if (cudaGetDriverEntryPoint("cuStreamWaitValue32", &f1, cudaEnableDefault, &q1) != cudaSuccess || q1 != cudaDriverEntryPointSuccess || !f1) return nullptr;
+  if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &f2, cudaEnableDefault, &q2) != cudaSuccess || q2 != cudaDriverEntryPointSuccess || !f2) return nullptr;
+  hp.wait_value = reinterpret_cast<StreamValueFn>(f1);
+  hp.write_value = reinterpret_cast<StreamValueFn>(f2);
+  if (cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  if (cudaEventCreateWithFlags(&hp.h2d_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  if (cudaEventCreateWithFlags(&hp.d2h_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  if (cudaMalloc(&hp.flag, 256) != cudaSuccess) return nullptr;
+  if (cudaMemset(hp.flag, 0, 256) != cudaSuccess) return nullptr;
+  // one write and one wait that is already satisfied: if the driver refuses either, stay on the plain path
+  if (hp.write_value(hp.h2d, (CUdeviceptr)(uintptr_t)hp.flag, 0u, 0u) != CUDA_SUCCESS) return nullptr;
+  if (hp.wait_value(hp.h2d, (CUdeviceptr)(uintptr_t)hp.flag, 0u, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS) return nullptr;
+  if (cudaStreamSynchronize(hp.h2d) != cudaSuccess) return nullptr;
+  hp.ok = true;
+  return &hp;
+}
+
+rwkvq_status run_host_plain(const void* plan_dev, size_t plan_bytes, const void* act_host, void* act_dev, size_t act_bytes,
+                            const void* y_dev, void* y_host, size_t y_bytes, void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (act_bytes) {
     cudaError_t e = cudaMemcpyAsync(act_dev, act_host, act_bytes, cudaMemcpyHostToDevice, s);
@@ -1916,6 +2054,77 @@ rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const 
     if (e != cudaSuccess) return cuda_status(e);
   }
   return RWKVQ_OK;
+}
+}  // namespace
+
+extern "C" {
+
+rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const void* act_host, void* act_dev,
+                                 size_t act_bytes, const void* y_dev, void* y_host, size_t y_bytes, void* stream) {
+  if ((act_bytes && (!act_host || !act_dev)) || (y_bytes && (!y_dev || !y_host))) return RWKVQ_EINVAL;
+  // Small steps: the copies are short and the plain order (copy in, run, copy out on one stream) is best.
+  if (act_bytes + y_bytes < ((size_t)4 << kChunkShift))
+    return run_host_plain(plan_dev, plan_bytes, act_host, act_dev, act_bytes, y_dev, y_host, y_bytes, stream);
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe* hp = host_pipe();
+  if (!hp) return run_host_plain(plan_dev, plan_bytes, act_host, act_dev, act_bytes, y_dev, y_host, y_bytes, stream);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // Both side streams start behind everything already enqueued on the caller's stream.
+  cudaError_t e = cudaEventRecord(hp->start, s);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hp->h2d, hp->start, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hp->d2h, hp->start, 0);
+  if (e != cudaSuccess) return cuda_status(e);
+  // Activations: chunk by chunk on the copy stream; the word counts the chunks that have arrived.
+  HostRun hr;
+  const size_t chunk = (size_t)1 << kChunkShift;
+  const unsigned n_in = (unsigned)((act_bytes + chunk - 1) >> kChunkShift);
+  if (n_in) {
+    hr.in_flag = hp->flag; hr.in_base = hp->chunks; hr.in_shift = kChunkShift;
+    hr.in_lo = (uint64_t)(uintptr_t)act_dev; hr.in_hi = hr.in_lo + act_bytes;
+    for (unsigned i = 0; i < n_in; ++i) {
+      const size_t off = (size_t)i << kChunkShift, len = std::min(chunk, act_bytes - off);
+      e = cudaMemcpyAsync(static_cast<uint8_t*>(act_dev) + off, static_cast<const uint8_t*>(act_host) + off, len, cudaMemcpyHostToDevice, hp->h2d);
+      if (e != cudaSuccess) break;
+      if (hp->write_value(hp->h2d, (CUdeviceptr)(uintptr_t)hp->flag, hp->chunks + i + 1u, 0u) != CUDA_SUCCESS) { e = cudaErrorUnknown; break; }
+    }
+    // Whatever happened, the word reaches its final value, so that no stager waits for a chunk in vain.
+    if (e != cudaSuccess) hp->write_value(hp->h2d, (CUdeviceptr)(uintptr_t)hp->flag, hp->chunks + n_in, 0u);
+    hp->chunks += n_in;
+    if (e != cudaSuccess) { cudaStreamSynchronize(hp->h2d); return cuda_status(e); }
+  }
+  // The step itself, on the caller's stream, at once: its stagers wait for the chunks they read.
+  rwkvq_status st = step_run_impl(plan_dev, plan_bytes, stream, &hr);
+  if (st != RWKVQ_OK) { cudaStreamSynchronize(hp->h2d); return st; }
+  // Outputs: stage by stage behind the stage barriers (the arrival counters of the plan), in groups of
+  // whole stages, as long as the stages' outputs lie one behind the other in [y_dev, y_dev + y_bytes).
+  if (y_bytes) {
+    const PlanInfo& info = hr.info;
+    const uint64_t y0 = (uint64_t)(uintptr_t)y_dev, y1 = y0 + y_bytes;
+    bool ordered = !info.y_lo.empty();
+    uint64_t prev = y0;
+    for (size_t k = 0; k < info.y_lo.size() && ordered; ++k) {
+      if (info.y_lo[k] < prev || info.y_hi[k] > y1 || info.y_hi[k] < info.y_lo[k]) ordered = false;
+      prev = info.y_hi[k];
+    }
+    const int n_st = info.n_stages;
+    size_t done = 0;                               // bytes of the output buffer already handed to copies
+    for (int k = 0; k < n_st && e == cudaSuccess; ++k) {
+      const bool last = k + 1 == n_st;
+      const size_t upto = last || !ordered ? (last ? y_bytes : done) : (size_t)(info.y_hi[k] - y0);
+      if (!last && upto - done < kOutGroupBytes) continue;
+      if (upto == done) continue;
+      // barrier k + 1 closes stage k: every CTA has arrived behind its reductions into these outputs
+      if (hp->wait_value(hp->d2h, (CUdeviceptr)(uintptr_t)(hr.counter + (k + 1)), hr.target, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS) { e = cudaErrorUnknown; break; }
+      e = cudaMemcpyAsync(static_cast<uint8_t*>(y_host) + done, static_cast<const uint8_t*>(y_dev) + done, upto - done, cudaMemcpyDeviceToHost, hp->d2h);
+      done = upto;
+    }
+  }
+  // The caller's stream ends behind both side streams: synchronizing it covers the whole step.
+  if (e == cudaSuccess) e = cudaEventRecord(hp->h2d_done, hp->h2d);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(s, hp->h2d_done, 0);
+  if (e == cudaSuccess) e = cudaEventRecord(hp->d2h_done, hp->d2h);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(s, hp->d2h_done, 0);
+  return cuda_status(e);
 }
 
 }  // extern "C"

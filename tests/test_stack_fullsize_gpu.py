@@ -62,3 +62,38 @@ def _check_step(st, name):
     # every output of every product was written (none left at its cleared value by accident): spot-check norms
     for op in st.ops[:: max(1, n // 16)]:
         assert float(op.y.abs().sum()) > 0.0
+
+
+@pytest.mark.parametrize("name,batch", [("c3_7b", 8), ("c3_7b", 1), ("c4_14b", 16)])
+def test_host_buffer_step_overlaps_copies_without_changing_results(name, batch):
+    """rwkvq_step_run_host at sizes where the activations arrive in chunks while the step runs and the
+    outputs leave stage by stage: the host gets exactly what the device holds at the end of the step
+    (no output copied before its stage was complete), and the step has read the NEW activations (none
+    read before its chunk arrived): fresh inputs through the host path against the same inputs copied
+    to the device first and a resident run."""
+    st = stack_mod.from_name(name, batch=batch, distinct_layers=2, kmeans_iters=2, quantizer="device", weights="device")
+    st.plan_step()
+    st.run_step()
+    torch.cuda.synchronize()
+    g = torch.Generator().manual_seed(1234 + batch)
+    halves = st.act_host.view(torch.float16)
+    for rep in range(3):
+        # new activations on the host only; the device arena keeps the old ones until the call copies them
+        halves.copy_((torch.randn(halves.numel(), generator=g) * 0.5).to(torch.float16))
+        st.y_host.zero_()
+        st.run_step_host()
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        assert torch.equal(st.y_host, st.y_arena.cpu())
+        assert torch.equal(st.act_arena.cpu(), st.act_host)
+        y_host = st.y_host.view(torch.float32).clone()
+        st.run_step()                       # resident run on the same (now copied) activations
+        torch.cuda.synchronize()
+        y_dev = st.y_arena.cpu().view(torch.float32)
+        # the two runs differ only in the order of the fp32 reductions into y
+        scale = float(y_dev.abs().max())
+        assert float((y_host - y_dev).abs().max()) <= 1e-4 * scale
+    op = st.ops[len(st.ops) // 2]
+    ref, tol = _oracle_product(st, op)
+    y = op.y.double().cpu().numpy()
+    assert (np.abs(y - ref) <= tol).all()
