@@ -97,3 +97,27 @@ def test_host_buffer_step_overlaps_copies_without_changing_results(name, batch):
     ref, tol = _oracle_product(st, op)
     y = op.y.double().cpu().numpy()
     assert (np.abs(y - ref) <= tol).all()
+
+
+def test_host_buffer_step_that_gives_up_releases_its_output_copies():
+    """A host-buffer run whose stage barriers can never open (wait_skew) with a small poll limit: the
+    kernel gives up by itself (ETIMEOUT), the output copies that were ordered behind the barriers are
+    released all the same, the caller's synchronize returns, and the next run is correct again."""
+    st = stack_mod.from_name("c3_7b", batch=8, distinct_layers=2, kmeans_iters=2, quantizer="device", weights="device")
+    st.plan_step()
+    st.run_step_host()
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 0
+    good = st.y_host.clone()
+    B.rwkvq_step_set_wait(st._plan, poll_limit=2000, wait_skew=1)
+    st.run_step_host()
+    torch.cuda.synchronize()
+    assert B.rwkvq_device_status() == 8          # RWKVQ_ETIMEOUT; reading it clears the word
+    B.rwkvq_step_set_wait(st._plan, poll_limit=0, wait_skew=0)
+    for _ in range(2):
+        st.y_host.zero_()
+        st.run_step_host()
+        torch.cuda.synchronize()
+        assert B.rwkvq_device_status() == 0
+        a, b = st.y_host.view(torch.float32), good.view(torch.float32)
+        assert float((a - b).abs().max()) <= 1e-4 * float(b.abs().max())
