@@ -555,15 +555,17 @@ def block_leg(configs=(("c3_7b", 1), ("c4_14b", 16)), max_steps=300, steps=None)
 # ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
-def build_stack(args, workload, batch):
+def build_stack(args, workload, batch, force_method=None, distinct_layers=None):
     from paper_2505_03803_b200 import binding as B
     from paper_2505_03803_b200 import inputs, stack as stack_mod
     sp = inputs.STACKS[workload]
-    force = None if args.force_method is None else (B.RWKVQ_SQ if args.force_method == "sq" else B.RWKVQ_VQ)
+    fm = force_method or args.force_method
+    force = None if fm is None else (B.RWKVQ_SQ if fm == "sq" else B.RWKVQ_VQ)
     weights = args.weights or ("device" if args.quantizer == "device" else "host")
     t0 = time.time()
     st = stack_mod.Stack(sp["d"], sp["h"], sp["layers"], sp["entries"], batch, n_outliers=sp["outliers"],
-                         tag=workload, device="cuda", distinct_layers=args.distinct_layers, force_method=force,
+                         tag=workload, device="cuda", distinct_layers=args.distinct_layers if distinct_layers is None else distinct_layers,
+                         force_method=force,
                          quantizer=args.quantizer, weights=weights)
     st.bench_setup_s = time.time() - t0
     return st
@@ -731,6 +733,22 @@ def run_ours(args):
         del st
         torch.cuda.empty_cache()
 
+    # each format alone on the headline stack, so that neither hides behind the mix (two distinct layers,
+    # reused: the set-up of 488 k-means matrices is not what is timed; 180 MB of images still exceed L2)
+    formats = None
+    if whole and world == 1 and not args.no_configs and args.force_method is None:
+        formats = {}
+        for fm in ("sq", "vq"):
+            st = build_stack(args, workload, batch, force_method=fm, distinct_layers=2)
+            k, w = default_steps(st, args)
+            r = measure_stack(st, args, workload, min(k, 200), w, 1, None, gpu_id, with_e2e=False)
+            formats["all_" + fm] = {"tokens_per_s": r["value"], "ms_per_step": r["ms_per_step"], "steps": r["steps"],
+                                    "roofline": r["roofline"], "clocks": r["clocks"],
+                                    "packed_bytes_per_step": r["config"]["packed_bytes_per_step"],
+                                    "distinct_layers": 2}
+            del st
+            torch.cuda.empty_cache()
+
     prefill = prefill_leg() if world == 1 and not args.no_prefill else None
     quantize = quantize_leg() if world == 1 and not args.no_quantize else None
     proxy = proxy_leg(with_oracle=not args.no_cpu_baseline) if world == 1 and not args.no_proxy else None
@@ -751,7 +769,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "f16", "data": "synthetic", "config": head["config"],
         "roofline": head["roofline"], "cpu_baseline": cpu, "e2e": head["e2e"], "clocks": head["clocks"],
         "gpu_launches": head["gpu_launches"], "hbm_gbs": head["roofline"]["achieved"],
-        "configs": configs, "prefill": prefill, "quantize": quantize, "proxy": proxy, "block": block,
+        "configs": configs, "formats": formats, "prefill": prefill, "quantize": quantize, "proxy": proxy, "block": block,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
