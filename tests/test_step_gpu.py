@@ -110,21 +110,29 @@ def test_step_rejects_bad_plans():
     assert B.rwkvq_step_plan_bytes(arr, 1) == 0   # fp16 outputs are not supported by the step launch
 
 
-def test_step_run_host_matches_oracle():
+@pytest.mark.parametrize("Bn,layout", [(4, "packed"), (4, "spread"), (16, "spread"), (1, "spread"), (8, "reversed")])
+def test_step_run_host_matches_oracle(Bn, layout):
     """rwkvq_step_run_host (the call behind the benchmark's end-to-end figure): activations come from
-    pinned host memory, results go back to pinned host memory, compared with the oracle there."""
-    Bn = 4
-    ops = _build_ops(512, 1280, 2, Bn, 6, seed=91)
+    pinned host memory, results go back to pinned host memory, compared with the oracle there.
+    "packed": small arenas, the copies run before and after the step.  "spread": the same products
+    3 MB apart in arenas of tens of MB, so that the activations arrive in several chunks while the step
+    runs and the outputs leave in several groups behind their stage barriers.  "reversed": outputs laid
+    out against the order of the stages, which the call must answer with one copy at the end."""
+    ops = _build_ops(512, 1280, 2, Bn, 6, seed=91 + Bn)
     # one arena for the activations and one for the outputs, as the stack runner lays them out
+    gap = 0 if layout == "packed" else 3 << 20
     def al(n):
-        return (n + 255) // 256 * 256
+        return (n + 255) // 256 * 256 + gap
     act_off, y_off, slots = 0, 0, []
     for e in ops:
         xo = act_off; act_off += al(e["x16"].nbytes)
         po = None
         if e["mu"] is not None:
             po = act_off; act_off += al(e["xp16"].nbytes)
-        slots.append((xo, po, y_off)); y_off += al(Bn * e["W"].oc * 4)
+        slots.append([xo, po, y_off]); y_off += al(Bn * e["W"].oc * 4)
+    if layout == "reversed":
+        for sl, e in zip(slots, ops):
+            sl[2] = y_off - sl[2] - al(Bn * e["W"].oc * 4)
     act_host = torch.zeros(act_off, dtype=torch.uint8).pin_memory()
     y_host = torch.zeros(y_off, dtype=torch.uint8).pin_memory()
     act_dev = torch.zeros(act_off, dtype=torch.uint8, device="cuda")
