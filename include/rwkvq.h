@@ -342,7 +342,8 @@ rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, i
  * outputs lie one behind the other inside [y_dev, y_dev + y_bytes) (otherwise in one piece at the end).
  * The bytes that reach y_host are those of the plain order.  Host buffers should be page-locked,
  * otherwise the copies serialize with the host.  A size of 0 skips that copy.  Calls on different
- * streams of one device are serialized by the library.  Errors: as rwkvq_step_run, ECUDA.
+ * streams of one device are serialized by the library.  The environment variable RWKVQ_HOST_OVERLAP=0
+ * (read at every call) keeps every step on the plain order.  Errors: as rwkvq_step_run, ECUDA.
  */
 rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const void* act_host,
                                  void* act_dev, size_t act_bytes, const void* y_dev, void* y_host,

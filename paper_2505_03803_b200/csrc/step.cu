@@ -36,6 +36,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <unordered_map>
@@ -2063,7 +2064,8 @@ rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const 
                                  size_t act_bytes, const void* y_dev, void* y_host, size_t y_bytes, void* stream) {
   if ((act_bytes && (!act_host || !act_dev)) || (y_bytes && (!y_dev || !y_host))) return RWKVQ_EINVAL;
   // Small steps: the copies are short and the plain order (copy in, run, copy out on one stream) is best.
-  if (act_bytes + y_bytes < ((size_t)4 << kChunkShift))
+  const char* ov = std::getenv("RWKVQ_HOST_OVERLAP");      // "0": always the plain order
+  if ((ov && ov[0] == '0') || act_bytes + y_bytes < ((size_t)4 << kChunkShift))
     return run_host_plain(plan_dev, plan_bytes, act_host, act_dev, act_bytes, y_dev, y_host, y_bytes, stream);
   std::lock_guard<std::mutex> lock(g_pipe_mutex);
   HostPipe* hp = host_pipe();
