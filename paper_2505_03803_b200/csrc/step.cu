@@ -2077,6 +2077,8 @@ rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const 
   if (e == cudaSuccess) e = cudaStreamWaitEvent(hp->d2h, hp->start, 0);
   if (e != cudaSuccess) return cuda_status(e);
   // Activations: chunk by chunk on the copy stream; the word counts the chunks that have arrived.
+  // They are enqueued BEFORE the launch: streams share a limited number of hardware queues, and a copy
+  // enqueued behind the running step in the same queue would start only when the step, which waits for it, ends.
   HostRun hr;
   const size_t chunk = (size_t)1 << kChunkShift;
   const unsigned n_in = (unsigned)((act_bytes + chunk - 1) >> kChunkShift);
