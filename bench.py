@@ -635,7 +635,7 @@ def measure_stack(st, args, workload, K, W, world, dist, gpu_id, with_e2e=True):
     if with_e2e and args.mode == "step":
         e2e_ms = e2e_region()
         e2e_copies = "plain order" if os.environ.get("RWKVQ_HOST_OVERLAP", "")[:1] == "0" else \
-            "overlapped with the step where the step copies 16 MB or more"
+            "overlapped with the step where the step copies 8 MB or more"
         if world == 1 and status == 0 and e2e_copies != "plain order" and B.rwkvq_device_status() != 0:
             # the overlapped host-buffer step gave up on a bounded wait: measure the plain order instead
             print("bench.py: the overlapped host-buffer step timed out; end-to-end figure taken in the plain order",

@@ -334,7 +334,7 @@ rwkvq_status rwkvq_step_plan_cover(const rwkvq_gemv_op* ops, int n_ops, int B, i
  * to act_dev (the device buffer the plan's x / x_prev pointers lie in), the step runs, and y_bytes are
  * copied from y_dev (the buffer the plan's outputs lie in) to y_host.  Everything is ordered behind what
  * `stream` already holds, and `stream` ends behind all of it: the caller synchronizes `stream` before
- * reading y_host or changing act_host.  Small steps (less than 16 MB of copies) run the three parts one
+ * reading y_host or changing act_host.  Small steps (less than 8 MB of copies) run the three parts one
  * after the other on `stream`.  Larger ones overlap them: the activations are copied in chunks of 4 MB
  * on a stream of the library's own while the step is already running (its input stages wait, bounded,
  * for the chunk that holds what they are about to read), and the outputs are copied, on another stream,

@@ -2013,6 +2013,7 @@ std::mutex g_pipe_mutex;
 std::unordered_map<int, HostPipe> g_pipes;
 constexpr unsigned kChunkShift = 22;                 // activations arrive in chunks of 4 MB
 constexpr size_t kOutGroupBytes = (size_t)2 << 20;   // outputs leave in groups of whole stages of at least 2 MB
+constexpr size_t kOverlapMinBytes = (size_t)8 << 20; // steps that copy less run the plain order
 
 HostPipe* host_pipe() {
   int dev = 0;
@@ -2065,7 +2066,7 @@ rwkvq_status rwkvq_step_run_host(const void* plan_dev, size_t plan_bytes, const 
   if ((act_bytes && (!act_host || !act_dev)) || (y_bytes && (!y_dev || !y_host))) return RWKVQ_EINVAL;
   // Small steps: the copies are short and the plain order (copy in, run, copy out on one stream) is best.
   const char* ov = std::getenv("RWKVQ_HOST_OVERLAP");      // "0": always the plain order
-  if ((ov && ov[0] == '0') || act_bytes + y_bytes < ((size_t)4 << kChunkShift))
+  if ((ov && ov[0] == '0') || act_bytes + y_bytes < kOverlapMinBytes)
     return run_host_plain(plan_dev, plan_bytes, act_host, act_dev, act_bytes, y_dev, y_host, y_bytes, stream);
   std::lock_guard<std::mutex> lock(g_pipe_mutex);
   HostPipe* hp = host_pipe();
