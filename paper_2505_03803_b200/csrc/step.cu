@@ -130,7 +130,8 @@ constexpr int kGroupWarps = 8, kGroupThreads = kGroupWarps * 32;
 //   NB = 2 (B > 8): the record routine wants about 150 registers, which sixteen consumer warps cannot have,
 //     and eight warps that keep everything in registers outrun sixteen that spill: ONE consumer group,
 //     seven stager warps (the stage pre-pass is theirs), one producer: 512 threads, 128 registers at
-//     launch, re-divided to 168 for the two consumer warpgroups and 88 for the other two.
+//     launch, re-divided to 152 for the two consumer warpgroups (what their routine needs to keep
+//     everything in registers) and 104 for the other two (measured: 168 / 88 and 144 / 112 are slower).
 template <int NB> struct Shape {
   static constexpr int kGroups = NB == 2 ? 1 : 2;
   static constexpr int kStagerWarps = NB == 2 ? 7 : 3;
@@ -138,7 +139,7 @@ template <int NB> struct Shape {
   static constexpr int kConsumerThreads = kConsumerWarps * 32, kStagerThreads = kStagerWarps * 32;
   static constexpr int kThreads = kConsumerThreads + kStagerThreads + 32;
   static constexpr int kLaunchRegs = NB == 2 ? 128 : 96;
-  static constexpr int kConsumerRegs = NB == 2 ? 168 : 104, kStagerRegs = NB == 2 ? 88 : 64;
+  static constexpr int kConsumerRegs = NB == 2 ? 152 : 104, kStagerRegs = NB == 2 ? 104 : 64;
   static_assert(kConsumerWarps % 4 == 0 && (kStagerWarps + 1) % 4 == 0, "register re-division works on warpgroups of four warps");
   static_assert(kConsumerRegs * kConsumerThreads + kStagerRegs * (kStagerThreads + 32) <= kLaunchRegs * kThreads,
                 "register re-division exceeds the launch's pool");
