@@ -40,7 +40,7 @@ if ROOT not in sys.path:
 # stacks are beyond the size a capture should hold on the device).  The packed weights are read once
 # whatever the stack, so the traffic of a larger stack is this ratio times its algorithmic bytes.
 # None = no capture of the kernel as it stands.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0133    # 538.7 MB of DRAM traffic for 531.6 MB algorithmic
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0131    # 538.6 MB of DRAM traffic for 531.6 MB algorithmic
 
 HEADLINE = ("c4_14b", 16)
 CONFIGS = (("c2_1p6b", 1), ("c3_7b", 1), ("c3_7b", 8))
