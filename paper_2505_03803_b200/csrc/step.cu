@@ -148,11 +148,11 @@ template <int NB> struct Shape {
 constexpr int groups_of(int NB) { return NB == 2 ? 1 : 2; }
 constexpr int threads_of(int NB) { return NB == 2 ? Shape<2>::kThreads : Shape<1>::kThreads; }
 constexpr int kMaxSlots = 12;
-constexpr uint32_t kCtrlBytes = 1024, kXBufTotal = 49152, kMuScratch = 1024;
-// Input-segment buffers: two of 24 KB when the CTA mixes its own inputs (the segment carries a mu row and
-// is prepared ahead), four of 12 KB when segments are copied from the stage's pre-pass.
-// (up to 8 batch rows; larger batches keep two buffers, a 256-column tile of 16 rows being 9 KB).
-template <bool MIX, int NB> struct XBufs { static constexpr uint32_t kCount = (MIX && NB == 1) ? 4u : 2u, kBytes = kXBufTotal / kCount; };
+constexpr uint32_t kCtrlBytes = 1024, kXBufTotal = 65536, kMuScratch = 1024;
+// Input-segment buffers: two of 32 KB, one in use and one being filled.  Large segments matter more than
+// deep buffering (every hand-over of a segment costs all roles a pass through the barriers): four buffers
+// of a quarter the size, and buffers that cost the weight ring a slot or two, were measured and are slower.
+template <bool MIX, int NB> struct XBufs { static constexpr uint32_t kCount = 2u, kBytes = kXBufTotal / kCount; };
 constexpr uint32_t kSmemLimit = 232448;  // 227 KB
 constexpr uint32_t kDefaultPollLimit = 1u << 22;
 
@@ -1431,7 +1431,7 @@ static rwkvq_status build_plan(const rwkvq_gemv_op* ops, int n_ops, int B, int P
   for (int i = 0; i < n_ops; ++i) any_xform = any_xform || ops[i].in.kind != RWKVQ_IN_BUFFER || ops[i].in.xprev_out_fp16 != nullptr;
   // see StepArgs::mix; the element-wise operators in front of a product exist in the stage pre-pass only
   const bool mix = B >= 4 || any_xform;
-  const uint32_t xbuf_bytes = mix && B <= 8 ? XBufs<true, 1>::kBytes : XBufs<false, 1>::kBytes;
+  const uint32_t xbuf_bytes = XBufs<false, 1>::kBytes;
   info->mix = mix ? 1 : 0;
   const uint32_t nbp = (uint32_t)((B + 1) & ~1);
 
